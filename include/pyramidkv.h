@@ -1,0 +1,205 @@
+/*
+ * pyramidkv.h: C boundary of the B200 (sm_100a) PyramidKV prefill KV-cache
+ * compression library.
+ *
+ * The library implements one step of the paper (arXiv 2406.02069, Section 4.2):
+ * at the end of prefill, for each transformer layer, score every cached key by
+ * the attention it receives from the last alpha ("instruction") tokens, smooth
+ * the scores with a 1-D max pool, keep the k^l best positions per KV head under
+ * the pyramidal per-layer budget, always keep the alpha window tokens, and copy
+ * the survivors into a compact ragged K/V cache with a list of their original
+ * positions.
+ *
+ * Conventions that hold for every call
+ *   - C linkage; every function returns an int status (PKV_OK = 0) unless noted.
+ *   - "host" pointers are dereferenced on the CPU before the call returns;
+ *     "device" pointers are only touched by kernels enqueued on `stream`.
+ *   - The caller owns every buffer.  The library never allocates or frees
+ *     device memory, never synchronises the stream (except
+ *     pyramidkv_check_status), and enqueues all device work on `stream`
+ *     (a cudaStream_t passed as void*; NULL is the default stream).
+ *   - Arguments are validated before anything is enqueued; on an error status
+ *     other than PKV_ERR_CUDA no device work has been submitted by that call.
+ *   - Output sizes are pure functions of host-known values (the config, the
+ *     sequence lengths and the layer budget): nothing is read back from the
+ *     device to size a buffer.
+ *   - Sequences of a batch are independent; each has its own length n_b.
+ *     P_b = n_b - alpha is its prefix length.
+ *
+ * Tensor layout
+ *   K, V     [batch][H_kv][n_max][d]   element strides given per tensor
+ *   Q_win    [batch][H_q][alpha][d]    the queries of the last alpha positions
+ *   The head dimension is contiguous (stride 1) in every tensor; base pointers
+ *   and strides are multiples of 16 bytes.  Query head g belongs to KV head
+ *   g / (H_q / H_kv).
+ *
+ * Packed ragged output of one layer
+ *   Every KV head of sequence b keeps the same number of rows
+ *   c_b = pyramidkv_kept_count(cfg, k_layer, n_b).  Rows are packed sequence
+ *   after sequence, head after head:  head h of sequence b owns rows
+ *   [off_b + h*c_b, off_b + (h+1)*c_b)  with  off_b = H_kv * sum_{b'<b} c_{b'}.
+ *   `indices` holds one int32 per row (the row's original position in its
+ *   sequence, ascending inside a head, the alpha window positions last);
+ *   k_out / v_out hold the d elements of that row, contiguous.
+ */
+#ifndef PYRAMIDKV_H_
+#define PYRAMIDKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Status codes. */
+#define PKV_OK 0
+#define PKV_ERR_INVALID_ARG 1     /* null pointer, bad shape, bad length, even pool width ... */
+#define PKV_ERR_UNSUPPORTED 2     /* dtype / head_dim / pool kind / batch size not built */
+#define PKV_ERR_WORKSPACE 3       /* workspace too small or misaligned (256 bytes) */
+#define PKV_ERR_CUDA 4            /* a launch failed; the CUDA error is left for the caller */
+#define PKV_ERR_DEVICE_STATUS 5   /* a kernel recorded a failure in the workspace status word */
+
+#define PKV_DTYPE_FP32 0
+#define PKV_DTYPE_BF16 1
+
+#define PKV_POOL_MAX 0
+
+#define PKV_MAX_BATCH 64          /* sequences per call */
+
+typedef struct pkv_config {
+  int32_t num_layers;    /* m >= 1 */
+  int32_t num_q_heads;   /* H_q, a multiple of num_kv_heads */
+  int32_t num_kv_heads;  /* H_kv */
+  int32_t head_dim;      /* d: 64 or 128 */
+  int32_t window;        /* alpha >= 1: instruction tokens, always kept (Section 4.2.1) */
+  int32_t pool_kernel;   /* odd width of the score pooling, 1 = none (Section 4.2.2) */
+  int32_t pool_kind;     /* PKV_POOL_MAX */
+  int32_t dtype;         /* PKV_DTYPE_*: element type shared by K, V and Q_win */
+  int32_t avg_budget;    /* B: mean rows kept per layer and KV head, window rows included; >= alpha */
+  int32_t reserved;      /* must be 0 */
+  double  beta;          /* pyramid shape, >= 1 (Section 4.2.1); 1 = same size in every layer */
+} pkv_config;
+
+typedef struct pkv_tensor {
+  const void* ptr;       /* device */
+  int64_t stride_batch;  /* strides in elements */
+  int64_t stride_head;
+  int64_t stride_token;  /* >= head_dim; the head dimension itself has stride 1 */
+} pkv_tensor;
+
+/* Human-readable name of a status code (static string, never NULL). */
+const char* pyramidkv_strerror(int status);
+
+/*
+ * Per-layer budgets, Section 4.2.1 and Eq. 1.  Host only, no CUDA call.
+ * The alpha window tokens are set aside first, so the budget that the pyramid
+ * shares out is k_total = m * (B - alpha):
+ *     k^{m-1} = k_total / (beta * m),   k^0 = 2 * k_total / m - k^{m-1},
+ *     k^l = k^0 - (k^0 - k^{m-1}) * l / (m - 1).
+ * beta is snapped to the nearest multiple of 1/1024 and the schedule is
+ * evaluated in integers: every k^l is floored and the units lost to flooring go
+ * one each to layers 0, 1, ... so that the budgets are non-increasing and sum to
+ * k_total exactly.  m = 1 gives k^0 = k_total.
+ *   k_out  host, [num_layers]: rows of the prefix layer l may keep (window rows come on top).
+ * Errors: PKV_ERR_INVALID_ARG for a null pointer or a config outside the ranges above.
+ */
+int pyramidkv_layer_budgets(const pkv_config* cfg, int32_t* k_out);
+
+/*
+ * Rows each KV head of a sequence of seq_len tokens keeps in a layer whose
+ * budget is k_layer (Section 4.1: a budget k^l < n; Section 4.2.1: the window is
+ * kept in every layer).  Host only.
+ *   seq_len <= avg_budget      -> seq_len (the context fits: nothing is evicted)
+ *   otherwise                  -> min(k_layer, seq_len - alpha) + alpha
+ * Returns the count, or a negative status (-PKV_ERR_INVALID_ARG).
+ */
+int pyramidkv_kept_count(const pkv_config* cfg, int32_t k_layer, int32_t seq_len);
+
+/*
+ * Bytes of device scratch that any call below needs for up to `batch` sequences
+ * of at most `max_seq_len` tokens.  Host only.  Returns 0 for an invalid config.
+ * The workspace must be 256-byte aligned.  Its first 256 bytes hold a status
+ * word that kernels only ever set to non-zero; the caller zeroes those bytes once
+ * after allocation (the rest needs no initialisation).  Calls that share a
+ * workspace must be ordered on one stream.
+ */
+size_t pyramidkv_workspace_bytes(const pkv_config* cfg, int32_t batch, int32_t max_seq_len);
+
+/*
+ * Window attention scores, Section 4.2.2, Eq. 2 and Eq. 3.
+ * For query head g and window row j (absolute position P_b + j) the logits are
+ * q . k_i / sqrt(d) over the keys i <= P_b + j the row can see (causal), and
+ * A = softmax over those keys.  The score of prefix key i < P_b for KV head h is
+ *     s[h][i] = (1/G) * sum over the G query heads of the group, sum over j < alpha, of A[j][i].
+ * Inputs in fp32 or bf16; products and sums accumulate in fp32; scores are fp32.
+ *   q_win, k   device tensors (layout above)
+ *   seq_lens   host [batch], each alpha + 1 <= n_b
+ *   scores     device, [batch][H_kv][ld_scores] floats; the first P_b entries of a row are written
+ *   ld_scores  >= max_b P_b
+ *   workspace  device scratch, workspace_bytes >= pyramidkv_workspace_bytes(cfg, batch, max n_b)
+ * Errors: INVALID_ARG, UNSUPPORTED (dtype, head_dim, batch > PKV_MAX_BATCH), WORKSPACE, CUDA.
+ */
+int pyramidkv_score_window(const pkv_config* cfg, pkv_tensor q_win, pkv_tensor k,
+                           const int32_t* seq_lens, int32_t batch,
+                           float* scores, int64_t ld_scores,
+                           void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Pooling and selection, Section 4.2.2.  Per sequence and KV head:
+ * pooled[i] = max of scores[i + t] over |t| <= (pool_kernel - 1)/2 clipped to [0, P_b);
+ * the min(k_layer, P_b) positions with the largest pooled value are kept, ties
+ * going to the smaller position; kept positions are written in ascending order
+ * followed by the window positions P_b .. n_b - 1.  A sequence with
+ * n_b <= avg_budget keeps every position and its scores are not read.
+ *   scores     device, as written by pyramidkv_score_window
+ *   k_layer    >= 0, this layer's entry of pyramidkv_layer_budgets
+ *   indices    device int32, packed rows (layout above), sum_b H_kv * c_b entries
+ * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA.
+ */
+int pyramidkv_select_topk(const pkv_config* cfg, const float* scores, int64_t ld_scores,
+                          const int32_t* seq_lens, int32_t batch, int32_t k_layer,
+                          int32_t* indices,
+                          void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Eviction by gather (appendix on torch.gather: select indices, compute source
+ * addresses from the strides, write a new tensor).  Copies, bit for bit, row
+ * indices[r] of K and of V into row r of k_out and v_out.  Out of place: k_out
+ * and v_out must not overlap K or V.  v.ptr and v_out may both be NULL to move K only.
+ *   indices    device int32, packed rows as written by pyramidkv_select_topk
+ *   k_out,v_out device, [sum_b H_kv * c_b][d] elements of the config dtype, 16-byte aligned
+ * Errors: INVALID_ARG, UNSUPPORTED, CUDA.
+ */
+int pyramidkv_gather_compact(const pkv_config* cfg, pkv_tensor k, pkv_tensor v,
+                             const int32_t* indices, const int32_t* seq_lens, int32_t batch,
+                             int32_t k_layer, void* k_out, void* v_out, void* stream);
+
+/*
+ * The whole step for one layer (Section 4.2): scores, pool, top-k with the
+ * budget of `layer`, window retention, gather; the same results as the three
+ * calls above issued in order.
+ *   layer          0 <= layer < num_layers; its budget is taken from the Eq. 1 schedule
+ *   scores_or_null device [batch][H_kv][ld_scores] to receive the scores, or NULL
+ *                  (then ld_scores is ignored and scores live in the workspace)
+ * Errors: as above.
+ */
+int pyramidkv_compress_layer(const pkv_config* cfg, int32_t layer,
+                             pkv_tensor q_win, pkv_tensor k, pkv_tensor v,
+                             const int32_t* seq_lens, int32_t batch,
+                             void* k_out, void* v_out, int32_t* indices,
+                             float* scores_or_null, int64_t ld_scores,
+                             void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Synchronises `stream` and reads the workspace status word.  For tests and
+ * debugging.  Returns PKV_OK, PKV_ERR_DEVICE_STATUS (a kernel gave up on a
+ * bounded wait or saw an impossible state; *detail_or_null receives the word),
+ * or PKV_ERR_CUDA.
+ */
+int pyramidkv_check_status(const void* workspace, void* stream, uint32_t* detail_or_null);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PYRAMIDKV_H_ */

@@ -1,0 +1,170 @@
+// Window-score kernels on the plain fp32 pipes (Section 4.2.2, Eq. 2 and Eq. 3).
+//
+// These cover every dtype / shape the boundary admits (fp32 inputs, any window,
+// any group size) and are the path of small fp32 problems.  The tensor-core
+// kernels in pkv_score_tc.cuh take over for bf16 inputs when their shape rules hold.
+//
+// The score of a key mixes softmax rows that each have their own normaliser, so
+// the normalisers must be known before any score can be formed.  Three launches:
+//   rowstats    one thread per window row r = (query head g, window row j): running
+//               max and sum of exp over one chunk of keys     -> partial (max, sum)
+//   combine     merges the chunks of a (sequence, KV head)     -> lse2[r] = log2 sum_i 2^(x_ri)
+//   scores      one thread per key: s_i = sum_r 2^(x_ri - lse2[r] - log2 G)
+// with x_ri = q_r . k_i * log2(e) / sqrt(d); both sweeps form x with the same
+// sequence of operations, so the two agree bit for bit.
+#pragma once
+
+#include "pkv_common.cuh"
+
+namespace pkv {
+
+constexpr int kGenChunk = 256;       // keys per rowstats CTA
+constexpr int kGenKeyTile = 16;      // keys staged in shared memory at a time
+constexpr int kGenRowBlock = 256;    // window rows per rowstats CTA pass (= its thread count)
+constexpr int kGenScoreKeys = 128;   // keys (= threads) per scores CTA
+constexpr int kGenQRows = 32;        // window rows staged per pass in the scores kernel
+
+struct ScoreParams {
+  TensorView q, k;
+  SeqTable seq;
+  int32_t num_kv_heads, group, rows;     // rows = group * alpha
+  float scale_log2;                      // log2(e) / sqrt(d)
+  float2* partial;                       // [sum_b chunks_b][H_kv][rows] (max, sum) per chunk
+  float* lse2;                           // [batch][H_kv][rows]
+  float* scores;                         // [batch][H_kv][ld]
+  int64_t ld_scores;
+};
+
+// grid (total chunks, H_kv), block kGenRowBlock.
+template <typename T, int D>
+__global__ void __launch_bounds__(kGenRowBlock) rowstats_generic_kernel(const ScoreParams p) {
+  __shared__ __align__(16) float ktile[kGenKeyTile][D];
+  const int tile = blockIdx.x, h = blockIdx.y;
+  const int b = find_sequence(p.seq.stat_off, p.seq.batch, tile);
+  const int n = p.seq.n[b], alpha = p.seq.alpha, P = n - alpha;
+  const int key0 = (tile - p.seq.stat_off[b]) * kGenChunk;
+  const int key1 = min(n, key0 + kGenChunk);
+  const T* kbase = static_cast<const T*>(p.k.ptr) + b * p.k.sb + h * p.k.sh;
+
+  for (int r0 = 0; r0 < p.rows; r0 += kGenRowBlock) {
+    const int r = r0 + threadIdx.x;
+    const bool live = r < p.rows;
+    const int g = live ? r / alpha : 0, j = live ? r % alpha : 0;
+    const int last_visible = P + j;                  // row j sees keys 0 .. P + j
+    float qreg[D];
+    {
+      const T* qrow = static_cast<const T*>(p.q.ptr) + b * p.q.sb +
+                      static_cast<int64_t>(h * p.group + g) * p.q.sh + j * p.q.st;
+#pragma unroll
+      for (int c = 0; c < D; ++c) qreg[c] = live ? to_float(qrow[c]) : 0.f;
+    }
+    float m = -INFINITY, z = 0.f;
+    for (int t0 = key0; t0 < key1; t0 += kGenKeyTile) {
+      __syncthreads();
+      for (int e = threadIdx.x; e < kGenKeyTile * D; e += blockDim.x) {
+        const int kk = e / D, c = e % D;
+        const int i = t0 + kk;
+        ktile[kk][c] = i < key1 ? to_float(kbase[static_cast<int64_t>(i) * p.k.st + c]) : 0.f;
+      }
+      __syncthreads();
+      float x[kGenKeyTile];
+      float tmax = -INFINITY;
+#pragma unroll
+      for (int kk = 0; kk < kGenKeyTile; ++kk) {
+        float dot = 0.f;
+#pragma unroll
+        for (int c = 0; c < D; c += 4) {
+          const float4 kv = *reinterpret_cast<const float4*>(&ktile[kk][c]);
+          dot = fmaf(qreg[c], kv.x, dot);
+          dot = fmaf(qreg[c + 1], kv.y, dot);
+          dot = fmaf(qreg[c + 2], kv.z, dot);
+          dot = fmaf(qreg[c + 3], kv.w, dot);
+        }
+        const int i = t0 + kk;
+        x[kk] = (i < key1 && i <= last_visible) ? dot * p.scale_log2 : -INFINITY;
+        tmax = fmaxf(tmax, x[kk]);
+      }
+      if (tmax > -INFINITY) {
+        const float mn = fmaxf(m, tmax);
+        float acc = 0.f;
+#pragma unroll
+        for (int kk = 0; kk < kGenKeyTile; ++kk) acc += exp2f(x[kk] - mn);
+        z = z * exp2f(m - mn) + acc;                 // exp2f(-inf) = 0 on the first tile
+        m = mn;
+      }
+    }
+    if (live) p.partial[(static_cast<int64_t>(tile) * p.num_kv_heads + h) * p.rows + r] = make_float2(m, z);
+  }
+}
+
+// grid (H_kv, batch), block 256: merge the chunk partials of each window row.
+// extra_log2 = log2(G) folds the mean over the group's query heads into the normaliser.
+__global__ void __launch_bounds__(256) combine_stats_kernel(const ScoreParams p, float extra_log2) {
+  const int h = blockIdx.x, b = blockIdx.y;
+  const int t0 = p.seq.stat_off[b], t1 = p.seq.stat_off[b + 1];
+  for (int r = threadIdx.x; r < p.rows; r += blockDim.x) {
+    float m = -INFINITY;
+    for (int t = t0; t < t1; ++t)
+      m = fmaxf(m, p.partial[(static_cast<int64_t>(t) * p.num_kv_heads + h) * p.rows + r].x);
+    float z = 0.f;
+    for (int t = t0; t < t1; ++t) {
+      const float2 pz = p.partial[(static_cast<int64_t>(t) * p.num_kv_heads + h) * p.rows + r];
+      z += pz.y * exp2f(pz.x - m);
+    }
+    p.lse2[(static_cast<int64_t>(b) * p.num_kv_heads + h) * p.rows + r] = m + log2f(z) + extra_log2;
+  }
+}
+
+// grid (total prefix tiles, H_kv), block kGenScoreKeys: one thread per prefix key.
+template <typename T, int D>
+__global__ void __launch_bounds__(kGenScoreKeys) scores_generic_kernel(const ScoreParams p) {
+  __shared__ __align__(16) float qs[kGenQRows][D];
+  __shared__ float lse_s[kGenQRows];
+  const int tile = blockIdx.x, h = blockIdx.y;
+  const int b = find_sequence(p.seq.score_off, p.seq.batch, tile);
+  const int alpha = p.seq.alpha, P = p.seq.n[b] - alpha;
+  const int i = (tile - p.seq.score_off[b]) * kGenScoreKeys + threadIdx.x;
+  const bool live = i < P;
+  float kreg[D];
+  {
+    const T* krow = static_cast<const T*>(p.k.ptr) + b * p.k.sb + h * p.k.sh +
+                    static_cast<int64_t>(live ? i : 0) * p.k.st;
+#pragma unroll
+    for (int c = 0; c < D; ++c) kreg[c] = to_float(krow[c]);
+  }
+  float s = 0.f;
+  for (int r0 = 0; r0 < p.rows; r0 += kGenQRows) {
+    __syncthreads();
+    for (int e = threadIdx.x; e < kGenQRows * D; e += blockDim.x) {
+      const int rr = e / D, c = e % D, r = r0 + rr;
+      float v = 0.f;
+      if (r < p.rows) {
+        const int g = r / alpha, j = r % alpha;
+        v = to_float(static_cast<const T*>(p.q.ptr)[b * p.q.sb + static_cast<int64_t>(h * p.group + g) * p.q.sh +
+                                                     j * p.q.st + c]);
+      }
+      qs[rr][c] = v;
+    }
+    if (threadIdx.x < kGenQRows) {
+      const int r = r0 + threadIdx.x;
+      lse_s[threadIdx.x] = r < p.rows ? p.lse2[(static_cast<int64_t>(b) * p.num_kv_heads + h) * p.rows + r] : INFINITY;
+    }
+    __syncthreads();
+    const int rn = min(kGenQRows, p.rows - r0);
+    for (int rr = 0; rr < rn; ++rr) {
+      float dot = 0.f;
+#pragma unroll
+      for (int c = 0; c < D; c += 4) {
+        const float4 qv = *reinterpret_cast<const float4*>(&qs[rr][c]);
+        dot = fmaf(qv.x, kreg[c], dot);
+        dot = fmaf(qv.y, kreg[c + 1], dot);
+        dot = fmaf(qv.z, kreg[c + 2], dot);
+        dot = fmaf(qv.w, kreg[c + 3], dot);
+      }
+      s += exp2f(dot * p.scale_log2 - lse_s[rr]);
+    }
+  }
+  if (live) p.scores[(static_cast<int64_t>(b) * p.num_kv_heads + h) * p.ld_scores + i] = s;
+}
+
+}  // namespace pkv
