@@ -66,6 +66,7 @@ extern "C" {
 #define PKV_POOL_MAX 0
 
 #define PKV_MAX_BATCH 64          /* sequences per call */
+#define PKV_MAX_STAGES 8          /* kernels one pyramidkv_compress_layer call may launch */
 
 typedef struct pkv_config {
   int32_t num_layers;    /* m >= 1 */
@@ -190,6 +191,23 @@ int pyramidkv_compress_layer(const pkv_config* cfg, int32_t layer,
                              void* k_out, void* v_out, int32_t* indices,
                              float* scores_or_null, int64_t ld_scores,
                              void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Measuring aid; the paper has no counterpart.  Same arguments and results as
+ * pyramidkv_compress_layer, but a CUDA event is recorded after every kernel the
+ * call launches, the stream is synchronised, and the device time of each kernel
+ * is returned.  Creates and destroys CUDA events; not for use on a hot path.
+ *   stage_ms     host [PKV_MAX_STAGES]      milliseconds per kernel, in launch order
+ *   stage_names  host [PKV_MAX_STAGES][32]  NUL-terminated kernel names
+ *   num_stages   host                       kernels launched
+ */
+int pyramidkv_profile_layer(const pkv_config* cfg, int32_t layer,
+                            pkv_tensor q_win, pkv_tensor k, pkv_tensor v,
+                            const int32_t* seq_lens, int32_t batch,
+                            void* k_out, void* v_out, int32_t* indices,
+                            float* scores_or_null, int64_t ld_scores,
+                            void* workspace, size_t workspace_bytes, void* stream,
+                            float* stage_ms, char (*stage_names)[32], int32_t* num_stages);
 
 /*
  * Synchronises `stream` and reads the workspace status word.  For tests and

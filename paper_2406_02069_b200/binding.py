@@ -1,0 +1,216 @@
+"""ctypes binding of libpyramidkv.so: same names as the C boundary, argument marshalling only.
+
+Every step of the path runs in the library's CUDA kernels.  torch supplies device
+memory and the stream, nothing else.  There is no CPU fallback: if the library
+cannot be loaded the import of this module fails.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence
+
+import torch
+
+from . import build as _build
+
+PKV_OK = 0
+PKV_ERR_INVALID_ARG = 1
+PKV_ERR_UNSUPPORTED = 2
+PKV_ERR_WORKSPACE = 3
+PKV_ERR_CUDA = 4
+PKV_ERR_DEVICE_STATUS = 5
+PKV_MAX_BATCH = 64
+
+EXPORTS = ("pyramidkv_strerror", "pyramidkv_layer_budgets", "pyramidkv_kept_count",
+           "pyramidkv_workspace_bytes", "pyramidkv_score_window", "pyramidkv_select_topk",
+           "pyramidkv_gather_compact", "pyramidkv_compress_layer", "pyramidkv_profile_layer",
+           "pyramidkv_check_status")
+PKV_MAX_STAGES = 8
+
+
+class PkvConfig(ctypes.Structure):
+    _fields_ = [("num_layers", ctypes.c_int32), ("num_q_heads", ctypes.c_int32),
+                ("num_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32),
+                ("window", ctypes.c_int32), ("pool_kernel", ctypes.c_int32),
+                ("pool_kind", ctypes.c_int32), ("dtype", ctypes.c_int32),
+                ("avg_budget", ctypes.c_int32), ("reserved", ctypes.c_int32),
+                ("beta", ctypes.c_double)]
+
+
+class PkvTensor(ctypes.Structure):
+    _fields_ = [("ptr", ctypes.c_void_p), ("stride_batch", ctypes.c_int64),
+                ("stride_head", ctypes.c_int64), ("stride_token", ctypes.c_int64)]
+
+
+class PkvError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s: %s (status %d)" % (where, strerror(status), status))
+
+
+def _load() -> ctypes.CDLL:
+    path = _build.LIB
+    if not os.path.exists(path):
+        _build.build_library()
+    lib = ctypes.CDLL(path)
+    P, I32, I64, SZ = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
+    CFG = ctypes.POINTER(PkvConfig)
+    lib.pyramidkv_strerror.argtypes = [ctypes.c_int]
+    lib.pyramidkv_strerror.restype = ctypes.c_char_p
+    lib.pyramidkv_layer_budgets.argtypes = [CFG, P]
+    lib.pyramidkv_kept_count.argtypes = [CFG, I32, I32]
+    lib.pyramidkv_workspace_bytes.argtypes = [CFG, I32, I32]
+    lib.pyramidkv_workspace_bytes.restype = SZ
+    lib.pyramidkv_score_window.argtypes = [CFG, PkvTensor, PkvTensor, P, I32, P, I64, P, SZ, P]
+    lib.pyramidkv_select_topk.argtypes = [CFG, P, I64, P, I32, I32, P, P, SZ, P]
+    lib.pyramidkv_gather_compact.argtypes = [CFG, PkvTensor, PkvTensor, P, P, I32, I32, P, P, P]
+    lib.pyramidkv_compress_layer.argtypes = [CFG, I32, PkvTensor, PkvTensor, PkvTensor, P, I32, P, P, P, P, I64,
+                                             P, SZ, P]
+    lib.pyramidkv_profile_layer.argtypes = lib.pyramidkv_compress_layer.argtypes + [P, P, P]
+    lib.pyramidkv_check_status.argtypes = [P, P, P]
+    for name in EXPORTS:
+        if name not in ("pyramidkv_strerror", "pyramidkv_workspace_bytes"):
+            getattr(lib, name).restype = ctypes.c_int
+    return lib
+
+
+_lib = _load()
+
+
+def library_path() -> str:
+    return _build.LIB
+
+
+def strerror(status: int) -> str:
+    return _lib.pyramidkv_strerror(int(status)).decode()
+
+
+def make_config(*, num_layers: int, num_q_heads: int, num_kv_heads: int, head_dim: int, window: int,
+                pool_kernel: int, dtype: str, avg_budget: int, beta: float = 20.0, pool_kind: int = 0) -> PkvConfig:
+    code = {"fp32": 0, "bf16": 1, torch.float32: 0, torch.bfloat16: 1}[dtype]
+    return PkvConfig(num_layers, num_q_heads, num_kv_heads, head_dim, window, pool_kernel, pool_kind, code,
+                     avg_budget, 0, float(beta))
+
+
+def config_of(w) -> PkvConfig:
+    """Config of a workloads.Workload."""
+    return make_config(num_layers=w.num_layers, num_q_heads=w.num_q_heads, num_kv_heads=w.num_kv_heads,
+                       head_dim=w.head_dim, window=w.window, pool_kernel=w.pool_kernel, dtype=w.dtype,
+                       avg_budget=w.avg_budget, beta=w.beta)
+
+
+def _tensor(t: Optional[torch.Tensor]) -> PkvTensor:
+    """[batch][head][token][d] view -> pkv_tensor (no copy; the last dimension must be contiguous)."""
+    if t is None:
+        return PkvTensor(None, 0, 0, 0)
+    if t.dim() != 4 or t.stride(3) != 1:
+        raise ValueError("expected a [batch][head][token][d] tensor with a contiguous last dimension")
+    return PkvTensor(t.data_ptr(), t.stride(0), t.stride(1), t.stride(2))
+
+
+def _lens(seq_lens: Sequence[int]):
+    arr = (ctypes.c_int32 * len(seq_lens))(*[int(x) for x in seq_lens])
+    return arr, len(seq_lens)
+
+
+def _stream(stream: Optional[torch.cuda.Stream]) -> int:
+    return (stream or torch.cuda.current_stream()).cuda_stream
+
+
+def _check(status: int, where: str) -> None:
+    if status != PKV_OK:
+        raise PkvError(status, where)
+
+
+def layer_budgets(cfg: PkvConfig) -> List[int]:
+    out = (ctypes.c_int32 * max(1, cfg.num_layers))()
+    _check(_lib.pyramidkv_layer_budgets(ctypes.byref(cfg), out), "pyramidkv_layer_budgets")
+    return [int(x) for x in out[: cfg.num_layers]]
+
+
+def kept_count(cfg: PkvConfig, k_layer: int, seq_len: int) -> int:
+    c = _lib.pyramidkv_kept_count(ctypes.byref(cfg), int(k_layer), int(seq_len))
+    if c < 0:
+        raise PkvError(-c, "pyramidkv_kept_count")
+    return int(c)
+
+
+def workspace_bytes(cfg: PkvConfig, batch: int, max_seq_len: int) -> int:
+    return int(_lib.pyramidkv_workspace_bytes(ctypes.byref(cfg), int(batch), int(max_seq_len)))
+
+
+def new_workspace(cfg: PkvConfig, batch: int, max_seq_len: int, device="cuda") -> torch.Tensor:
+    """Allocates (with torch) and prepares a workspace: the status bytes are zeroed once."""
+    nbytes = workspace_bytes(cfg, batch, max_seq_len)
+    if nbytes == 0:
+        raise PkvError(PKV_ERR_INVALID_ARG, "pyramidkv_workspace_bytes")
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=device)
+    ws[:256].zero_()
+    return ws
+
+
+def total_rows(cfg: PkvConfig, k_layer: int, seq_lens: Sequence[int]) -> int:
+    return sum(cfg.num_kv_heads * kept_count(cfg, k_layer, n) for n in seq_lens)
+
+
+def score_window(cfg: PkvConfig, q_win: torch.Tensor, k: torch.Tensor, seq_lens: Sequence[int],
+                 scores: torch.Tensor, workspace: torch.Tensor, stream=None) -> None:
+    lens, batch = _lens(seq_lens)
+    _check(_lib.pyramidkv_score_window(ctypes.byref(cfg), _tensor(q_win), _tensor(k), lens, batch,
+                                       scores.data_ptr(), scores.stride(1), workspace.data_ptr(),
+                                       workspace.numel(), _stream(stream)), "pyramidkv_score_window")
+
+
+def select_topk(cfg: PkvConfig, scores: torch.Tensor, seq_lens: Sequence[int], k_layer: int,
+                indices: torch.Tensor, workspace: torch.Tensor, stream=None) -> None:
+    lens, batch = _lens(seq_lens)
+    _check(_lib.pyramidkv_select_topk(ctypes.byref(cfg), scores.data_ptr(), scores.stride(1), lens, batch,
+                                      int(k_layer), indices.data_ptr(), workspace.data_ptr(), workspace.numel(),
+                                      _stream(stream)), "pyramidkv_select_topk")
+
+
+def gather_compact(cfg: PkvConfig, k: torch.Tensor, v: Optional[torch.Tensor], indices: torch.Tensor,
+                   seq_lens: Sequence[int], k_layer: int, k_out: torch.Tensor, v_out: Optional[torch.Tensor],
+                   stream=None) -> None:
+    lens, batch = _lens(seq_lens)
+    _check(_lib.pyramidkv_gather_compact(ctypes.byref(cfg), _tensor(k), _tensor(v), indices.data_ptr(), lens, batch,
+                                         int(k_layer), k_out.data_ptr(),
+                                         v_out.data_ptr() if v_out is not None else None, _stream(stream)),
+           "pyramidkv_gather_compact")
+
+
+def compress_layer(cfg: PkvConfig, layer: int, q_win: torch.Tensor, k: torch.Tensor, v: torch.Tensor,
+                   seq_lens: Sequence[int], k_out: torch.Tensor, v_out: torch.Tensor, indices: torch.Tensor,
+                   workspace: torch.Tensor, scores: Optional[torch.Tensor] = None, stream=None) -> None:
+    lens, batch = _lens(seq_lens)
+    _check(_lib.pyramidkv_compress_layer(ctypes.byref(cfg), int(layer), _tensor(q_win), _tensor(k), _tensor(v), lens,
+                                         batch, k_out.data_ptr(), v_out.data_ptr(), indices.data_ptr(),
+                                         scores.data_ptr() if scores is not None else None,
+                                         scores.stride(1) if scores is not None else 0,
+                                         workspace.data_ptr(), workspace.numel(), _stream(stream)),
+           "pyramidkv_compress_layer")
+
+
+def profile_layer(cfg: PkvConfig, layer: int, q_win: torch.Tensor, k: torch.Tensor, v: torch.Tensor,
+                  seq_lens: Sequence[int], k_out: torch.Tensor, v_out: torch.Tensor, indices: torch.Tensor,
+                  workspace: torch.Tensor, stream=None):
+    """compress_layer with per-kernel device times: returns [(kernel name, milliseconds), ...]."""
+    lens, batch = _lens(seq_lens)
+    ms = (ctypes.c_float * PKV_MAX_STAGES)()
+    names = ((ctypes.c_char * 32) * PKV_MAX_STAGES)()
+    n = ctypes.c_int32(0)
+    _check(_lib.pyramidkv_profile_layer(ctypes.byref(cfg), int(layer), _tensor(q_win), _tensor(k), _tensor(v), lens,
+                                        batch, k_out.data_ptr(), v_out.data_ptr(), indices.data_ptr(), None, 0,
+                                        workspace.data_ptr(), workspace.numel(), _stream(stream), ms, names,
+                                        ctypes.byref(n)), "pyramidkv_profile_layer")
+    return [(names[i].value.decode(), float(ms[i])) for i in range(n.value)]
+
+
+def check_status(workspace: torch.Tensor, stream=None) -> int:
+    """Synchronises the stream; raises PkvError if a kernel flagged a failure."""
+    detail = ctypes.c_uint32(0)
+    st = _lib.pyramidkv_check_status(workspace.data_ptr(), _stream(stream), ctypes.byref(detail))
+    if st != PKV_OK:
+        raise PkvError(st, "pyramidkv_check_status (word 0x%x)" % detail.value)
+    return 0

@@ -1,0 +1,417 @@
+// Host side of the PyramidKV compression library: argument validation, the
+// budget schedule, workspace carving and kernel launches behind the C boundary
+// declared in include/pyramidkv.h.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+
+#include "pkv_common.cuh"
+#include "pkv_gather.cuh"
+#include "pkv_score_generic.cuh"
+#include "pkv_select.cuh"
+
+namespace pkv {
+namespace {
+
+constexpr size_t kAlign = 256;
+constexpr int kPartialChunk = 128;   // smallest key chunk any row-statistics kernel uses (sizes the workspace)
+
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+bool config_ok(const pkv_config* c) {
+  if (!c) return false;
+  if (c->num_layers < 1 || c->num_kv_heads < 1 || c->num_q_heads < 1) return false;
+  if (c->num_q_heads % c->num_kv_heads != 0) return false;
+  if (c->window < 1 || c->avg_budget < c->window) return false;
+  if (c->pool_kernel < 1 || (c->pool_kernel % 2) == 0) return false;
+  if (!(c->beta >= 1.0) || c->beta > 1.0e6) return false;
+  if (c->reserved != 0) return false;
+  return true;
+}
+
+int config_supported(const pkv_config* c) {
+  if (c->dtype != PKV_DTYPE_FP32 && c->dtype != PKV_DTYPE_BF16) return PKV_ERR_UNSUPPORTED;
+  if (c->head_dim != 64 && c->head_dim != 128) return PKV_ERR_UNSUPPORTED;
+  if (c->pool_kind != PKV_POOL_MAX) return PKV_ERR_UNSUPPORTED;
+  return PKV_OK;
+}
+
+// Eq. 1 in integers.  beta = bq / 1024.  With k_total = m (B - alpha):
+//   k^l = k_total * ((2 bq - 1024)(m - 1) - (2 bq - 2048) l) / (bq m (m - 1)),
+// floored; the units lost to flooring go to layers 0, 1, ...
+void budgets(const pkv_config* c, int32_t* out) {
+  const int m = c->num_layers;
+  const long long k_total = static_cast<long long>(m) * (c->avg_budget - c->window);
+  if (m == 1) { out[0] = static_cast<int32_t>(k_total); return; }
+  const long long bq = std::llround(c->beta * 1024.0);
+  const unsigned __int128 den = static_cast<unsigned __int128>(bq) * m * (m - 1);
+  long long given = 0;
+  for (int l = 0; l < m; ++l) {
+    // (2bq-1024)(m-1) >= (2bq-2048) l for l <= m-1, so the numerator is never negative
+    const unsigned __int128 num = static_cast<unsigned __int128>(2 * bq - 1024) * (m - 1) -
+                                  static_cast<unsigned __int128>(2 * bq - 2048) * l;
+    const long long kl = static_cast<long long>(static_cast<unsigned __int128>(k_total) * num / den);
+    out[l] = static_cast<int32_t>(kl);
+    given += kl;
+  }
+  for (int l = 0; given < k_total; ++l, ++given) out[l] += 1;
+}
+
+int kept_count(const pkv_config* c, int k_layer, int n) {
+  if (n <= c->avg_budget) return n;
+  const int prefix = n - c->window;
+  return (k_layer < prefix ? k_layer : prefix) + c->window;
+}
+
+struct Workspace {
+  uint32_t* status;
+  float* lse2;
+  float2* partial;
+  float* scores;
+  int64_t ld_scores;
+  size_t bytes;
+};
+
+// Carves the workspace for `batch` sequences of at most max_n tokens.  base may be null (sizing only).
+Workspace carve(const pkv_config* c, int batch, int max_n, void* base) {
+  Workspace w{};
+  char* p = static_cast<char*>(base);
+  size_t off = 0;
+  auto take = [&](size_t bytes) { char* r = p ? p + off : nullptr; off += align_up(bytes); return r; };
+  const size_t rows = static_cast<size_t>(c->num_q_heads / c->num_kv_heads) * c->window;
+  const size_t heads = static_cast<size_t>(batch) * c->num_kv_heads;
+  const size_t chunks = (static_cast<size_t>(max_n) + kPartialChunk - 1) / kPartialChunk;
+  w.status = reinterpret_cast<uint32_t*>(take(kAlign));
+  w.lse2 = reinterpret_cast<float*>(take(heads * rows * sizeof(float)));
+  w.partial = reinterpret_cast<float2*>(take(heads * chunks * rows * sizeof(float2)));
+  w.ld_scores = static_cast<int64_t>((static_cast<size_t>(max_n) + 63) / 64 * 64);
+  w.scores = reinterpret_cast<float*>(take(heads * w.ld_scores * sizeof(float)));
+  w.bytes = off;
+  return w;
+}
+
+// Validates the sequence lengths and fills the per-call table for budget k_layer.
+int build_table(const pkv_config* c, const int32_t* seq_lens, int batch, int k_layer, SeqTable* t, int* max_n,
+                int64_t* total_rows) {
+  if (!seq_lens || batch < 1 || k_layer < 0) return PKV_ERR_INVALID_ARG;
+  if (batch > PKV_MAX_BATCH) return PKV_ERR_UNSUPPORTED;
+  std::memset(t, 0, sizeof *t);
+  t->batch = batch;
+  t->alpha = c->window;
+  int64_t rows = 0;
+  int mx = 0;
+  for (int b = 0; b < batch; ++b) {
+    const int n = seq_lens[b];
+    if (n < c->window + 1) return PKV_ERR_INVALID_ARG;
+    t->n[b] = n;
+    t->count[b] = kept_count(c, k_layer, n);
+    t->row_off[b] = rows;
+    rows += static_cast<int64_t>(c->num_kv_heads) * t->count[b];
+    if (n > mx) mx = n;
+  }
+  *max_n = mx;
+  *total_rows = rows;
+  return PKV_OK;
+}
+
+bool tensor_ok(const pkv_tensor& t, int d, int elem_bytes) {
+  if (!t.ptr || t.stride_token < d) return false;
+  if (reinterpret_cast<uintptr_t>(t.ptr) % 16) return false;
+  const int64_t q = 16 / elem_bytes;
+  return t.stride_token % q == 0 && t.stride_head % q == 0 && t.stride_batch % q == 0;
+}
+
+TensorView view(const pkv_tensor& t) { return TensorView{t.ptr, t.stride_batch, t.stride_head, t.stride_token}; }
+
+int check_launch() { return cudaPeekAtLastError() == cudaSuccess ? PKV_OK : PKV_ERR_CUDA; }
+
+// Optional per-kernel timing (pyramidkv_profile_layer): when armed, an event is recorded after every launch.
+struct StageTimer {
+  cudaEvent_t ev[PKV_MAX_STAGES + 1];
+  const char* name[PKV_MAX_STAGES];
+  int n = 0;
+};
+thread_local StageTimer* g_timer = nullptr;
+
+void mark(cudaStream_t st, const char* name) {
+  if (!g_timer || g_timer->n >= PKV_MAX_STAGES) return;
+  g_timer->name[g_timer->n] = name;
+  cudaEventRecord(g_timer->ev[++g_timer->n], st);
+}
+
+// ---------------------------------------------------------------- scores
+template <typename T, int D>
+int launch_scores_generic(ScoreParams& sp, int batch, cudaStream_t st) {
+  int stat_tiles = 0, score_tiles = 0;
+  for (int b = 0; b < batch; ++b) {
+    sp.seq.stat_off[b] = stat_tiles;
+    sp.seq.score_off[b] = score_tiles;
+    stat_tiles += (sp.seq.n[b] + kGenChunk - 1) / kGenChunk;
+    score_tiles += (sp.seq.n[b] - sp.seq.alpha + kGenScoreKeys - 1) / kGenScoreKeys;
+  }
+  sp.seq.stat_off[batch] = stat_tiles;
+  sp.seq.score_off[batch] = score_tiles;
+  rowstats_generic_kernel<T, D><<<dim3(stat_tiles, sp.num_kv_heads), kGenRowBlock, 0, st>>>(sp);
+  mark(st, "rowstats_generic");
+  combine_stats_kernel<<<dim3(sp.num_kv_heads, batch), 256, 0, st>>>(sp, std::log2(static_cast<float>(sp.group)));
+  mark(st, "combine_stats");
+  scores_generic_kernel<T, D><<<dim3(score_tiles, sp.num_kv_heads), kGenScoreKeys, 0, st>>>(sp);
+  mark(st, "scores_generic");
+  return check_launch();
+}
+
+int run_scores(const pkv_config* c, const pkv_tensor& q, const pkv_tensor& k, const SeqTable& table, int batch,
+               float* scores, int64_t ld, const Workspace& w, cudaStream_t st) {
+  ScoreParams sp{};
+  sp.q = view(q);
+  sp.k = view(k);
+  sp.seq = table;
+  sp.num_kv_heads = c->num_kv_heads;
+  sp.group = c->num_q_heads / c->num_kv_heads;
+  sp.rows = sp.group * c->window;
+  sp.scale_log2 = static_cast<float>(1.4426950408889634 / std::sqrt(static_cast<double>(c->head_dim)));
+  sp.partial = w.partial;
+  sp.lse2 = w.lse2;
+  sp.scores = scores;
+  sp.ld_scores = ld;
+  if (c->dtype == PKV_DTYPE_FP32)
+    return c->head_dim == 64 ? launch_scores_generic<float, 64>(sp, batch, st)
+                             : launch_scores_generic<float, 128>(sp, batch, st);
+  return c->head_dim == 64 ? launch_scores_generic<__nv_bfloat16, 64>(sp, batch, st)
+                           : launch_scores_generic<__nv_bfloat16, 128>(sp, batch, st);
+}
+
+// ---------------------------------------------------------------- select
+int run_select(const pkv_config* c, const float* scores, int64_t ld, const SeqTable& table, int batch, int max_n,
+               int32_t* indices, const Workspace& w, cudaStream_t st) {
+  SelectParams sp{};
+  sp.scores = scores;
+  sp.ld_scores = ld;
+  sp.indices = indices;
+  sp.seq = table;
+  sp.num_kv_heads = c->num_kv_heads;
+  sp.pool_radius = (c->pool_kernel - 1) / 2;
+  sp.status = w.status;
+  const int max_p = max_n - c->window;
+  int cluster = 1;
+  while (cluster < kSelMaxCluster && (max_p + cluster - 1) / cluster > 8192) cluster *= 2;
+  const int slice = ((max_p + cluster - 1) / cluster + 31) & ~31;
+  sp.slice_cap = slice <= kSelSliceCap ? slice : 0;
+  const size_t smem = static_cast<size_t>(sp.slice_cap) * sizeof(uint32_t);
+  static bool attr_done[64] = {};  // the attribute is per device; setting it twice is harmless
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return PKV_ERR_CUDA;
+  if (dev >= 64 || !attr_done[dev]) {
+    if (cudaFuncSetAttribute(pool_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             kSelSliceCap * static_cast<int>(sizeof(uint32_t))) != cudaSuccess)
+      return PKV_ERR_CUDA;
+    if (dev < 64) attr_done[dev] = true;
+  }
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(cluster * c->num_kv_heads, batch);
+  cfg.blockDim = dim3(kSelThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = cluster;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, pool_select_kernel, sp) != cudaSuccess) return PKV_ERR_CUDA;
+  mark(st, "pool_select");
+  return check_launch();
+}
+
+// ---------------------------------------------------------------- gather
+int run_gather(const pkv_config* c, const pkv_tensor& k, const pkv_tensor& v, const int32_t* indices,
+               const SeqTable& table, int64_t total_rows, void* k_out, void* v_out, cudaStream_t st) {
+  GatherParams gp{};
+  gp.k = view(k);
+  gp.v = view(v);
+  gp.indices = indices;
+  gp.k_out = k_out;
+  gp.v_out = v_out;
+  gp.seq = table;
+  gp.num_kv_heads = c->num_kv_heads;
+  gp.elem_bytes = c->dtype == PKV_DTYPE_FP32 ? 4 : 2;
+  gp.pieces = c->head_dim * gp.elem_bytes / 16;
+  gp.total_rows = total_rows;
+  const int64_t threads = total_rows * gp.pieces;
+  if (threads == 0) return PKV_OK;
+  const unsigned blocks = static_cast<unsigned>((threads + kGatherThreads - 1) / kGatherThreads);
+  gather_rows_kernel<<<blocks, kGatherThreads, 0, st>>>(gp);
+  mark(st, "gather_rows");
+  return check_launch();
+}
+
+int workspace_check(const pkv_config* c, int batch, int max_n, void* ws, size_t ws_bytes, Workspace* out) {
+  if (!ws || reinterpret_cast<uintptr_t>(ws) % kAlign) return PKV_ERR_WORKSPACE;
+  *out = carve(c, batch, max_n, ws);
+  return out->bytes <= ws_bytes ? PKV_OK : PKV_ERR_WORKSPACE;
+}
+
+}  // namespace
+}  // namespace pkv
+
+using namespace pkv;
+
+extern "C" {
+
+const char* pyramidkv_strerror(int status) {
+  switch (status) {
+    case PKV_OK: return "ok";
+    case PKV_ERR_INVALID_ARG: return "invalid argument";
+    case PKV_ERR_UNSUPPORTED: return "unsupported dtype, head_dim, pool kind or batch size";
+    case PKV_ERR_WORKSPACE: return "workspace too small or misaligned";
+    case PKV_ERR_CUDA: return "CUDA launch failed";
+    case PKV_ERR_DEVICE_STATUS: return "a kernel recorded a failure in the workspace status word";
+    default: return "unknown status";
+  }
+}
+
+int pyramidkv_layer_budgets(const pkv_config* cfg, int32_t* k_out) {
+  if (!config_ok(cfg) || !k_out) return PKV_ERR_INVALID_ARG;
+  budgets(cfg, k_out);
+  return PKV_OK;
+}
+
+int pyramidkv_kept_count(const pkv_config* cfg, int32_t k_layer, int32_t seq_len) {
+  if (!config_ok(cfg) || k_layer < 0 || seq_len < cfg->window + 1) return -PKV_ERR_INVALID_ARG;
+  return kept_count(cfg, k_layer, seq_len);
+}
+
+size_t pyramidkv_workspace_bytes(const pkv_config* cfg, int32_t batch, int32_t max_seq_len) {
+  if (!config_ok(cfg) || batch < 1 || batch > PKV_MAX_BATCH || max_seq_len < cfg->window + 1) return 0;
+  return carve(cfg, batch, max_seq_len, nullptr).bytes;
+}
+
+int pyramidkv_score_window(const pkv_config* cfg, pkv_tensor q_win, pkv_tensor k, const int32_t* seq_lens,
+                           int32_t batch, float* scores, int64_t ld_scores, void* workspace,
+                           size_t workspace_bytes, void* stream) {
+  if (!config_ok(cfg)) return PKV_ERR_INVALID_ARG;
+  if (int rc = config_supported(cfg)) return rc;
+  const int eb = cfg->dtype == PKV_DTYPE_FP32 ? 4 : 2;
+  if (!tensor_ok(q_win, cfg->head_dim, eb) || !tensor_ok(k, cfg->head_dim, eb) || !scores) return PKV_ERR_INVALID_ARG;
+  SeqTable table;
+  int max_n;
+  int64_t rows;
+  if (int rc = build_table(cfg, seq_lens, batch, 0, &table, &max_n, &rows)) return rc;
+  if (ld_scores < max_n - cfg->window) return PKV_ERR_INVALID_ARG;
+  Workspace w;
+  if (int rc = workspace_check(cfg, batch, max_n, workspace, workspace_bytes, &w)) return rc;
+  return run_scores(cfg, q_win, k, table, batch, scores, ld_scores, w, static_cast<cudaStream_t>(stream));
+}
+
+int pyramidkv_select_topk(const pkv_config* cfg, const float* scores, int64_t ld_scores, const int32_t* seq_lens,
+                          int32_t batch, int32_t k_layer, int32_t* indices, void* workspace,
+                          size_t workspace_bytes, void* stream) {
+  if (!config_ok(cfg)) return PKV_ERR_INVALID_ARG;
+  if (int rc = config_supported(cfg)) return rc;
+  if (!scores || !indices) return PKV_ERR_INVALID_ARG;
+  SeqTable table;
+  int max_n;
+  int64_t rows;
+  if (int rc = build_table(cfg, seq_lens, batch, k_layer, &table, &max_n, &rows)) return rc;
+  if (ld_scores < max_n - cfg->window) return PKV_ERR_INVALID_ARG;
+  Workspace w;
+  if (int rc = workspace_check(cfg, batch, max_n, workspace, workspace_bytes, &w)) return rc;
+  return run_select(cfg, scores, ld_scores, table, batch, max_n, indices, w, static_cast<cudaStream_t>(stream));
+}
+
+int pyramidkv_gather_compact(const pkv_config* cfg, pkv_tensor k, pkv_tensor v, const int32_t* indices,
+                             const int32_t* seq_lens, int32_t batch, int32_t k_layer, void* k_out, void* v_out,
+                             void* stream) {
+  if (!config_ok(cfg)) return PKV_ERR_INVALID_ARG;
+  if (int rc = config_supported(cfg)) return rc;
+  const int eb = cfg->dtype == PKV_DTYPE_FP32 ? 4 : 2;
+  if (!tensor_ok(k, cfg->head_dim, eb) || !indices || !k_out) return PKV_ERR_INVALID_ARG;
+  if ((v.ptr == nullptr) != (v_out == nullptr)) return PKV_ERR_INVALID_ARG;
+  if (v.ptr && !tensor_ok(v, cfg->head_dim, eb)) return PKV_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(k_out) % 16 || reinterpret_cast<uintptr_t>(v_out) % 16) return PKV_ERR_INVALID_ARG;
+  SeqTable table;
+  int max_n;
+  int64_t rows;
+  if (int rc = build_table(cfg, seq_lens, batch, k_layer, &table, &max_n, &rows)) return rc;
+  return run_gather(cfg, k, v, indices, table, rows, k_out, v_out, static_cast<cudaStream_t>(stream));
+}
+
+int pyramidkv_compress_layer(const pkv_config* cfg, int32_t layer, pkv_tensor q_win, pkv_tensor k, pkv_tensor v,
+                             const int32_t* seq_lens, int32_t batch, void* k_out, void* v_out, int32_t* indices,
+                             float* scores_or_null, int64_t ld_scores, void* workspace, size_t workspace_bytes,
+                             void* stream) {
+  if (!config_ok(cfg)) return PKV_ERR_INVALID_ARG;
+  if (int rc = config_supported(cfg)) return rc;
+  if (layer < 0 || layer >= cfg->num_layers) return PKV_ERR_INVALID_ARG;
+  const int eb = cfg->dtype == PKV_DTYPE_FP32 ? 4 : 2;
+  if (!tensor_ok(q_win, cfg->head_dim, eb) || !tensor_ok(k, cfg->head_dim, eb) || !tensor_ok(v, cfg->head_dim, eb))
+    return PKV_ERR_INVALID_ARG;
+  if (!k_out || !v_out || !indices) return PKV_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(k_out) % 16 || reinterpret_cast<uintptr_t>(v_out) % 16) return PKV_ERR_INVALID_ARG;
+  int32_t k_layer;
+  {
+    // the schedule is O(m) integer work; small enough to redo per call
+    int32_t stack_buf[512];
+    int32_t* all = cfg->num_layers <= 512 ? stack_buf : new int32_t[cfg->num_layers];
+    budgets(cfg, all);
+    k_layer = all[layer];
+    if (all != stack_buf) delete[] all;
+  }
+  SeqTable table;
+  int max_n;
+  int64_t rows;
+  if (int rc = build_table(cfg, seq_lens, batch, k_layer, &table, &max_n, &rows)) return rc;
+  Workspace w;
+  if (int rc = workspace_check(cfg, batch, max_n, workspace, workspace_bytes, &w)) return rc;
+  float* scores = scores_or_null ? scores_or_null : w.scores;
+  const int64_t ld = scores_or_null ? ld_scores : w.ld_scores;
+  if (ld < max_n - cfg->window) return PKV_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // A batch in which no sequence is compressed needs no scores unless the caller asked for them.
+  bool any_compress = false;
+  for (int b = 0; b < batch; ++b) any_compress |= table.count[b] < table.n[b];
+  if (any_compress || scores_or_null)
+    if (int rc = run_scores(cfg, q_win, k, table, batch, scores, ld, w, st)) return rc;
+  if (int rc = run_select(cfg, scores, ld, table, batch, max_n, indices, w, st)) return rc;
+  return run_gather(cfg, k, v, indices, table, rows, k_out, v_out, st);
+}
+
+int pyramidkv_profile_layer(const pkv_config* cfg, int32_t layer, pkv_tensor q_win, pkv_tensor k, pkv_tensor v,
+                            const int32_t* seq_lens, int32_t batch, void* k_out, void* v_out, int32_t* indices,
+                            float* scores_or_null, int64_t ld_scores, void* workspace, size_t workspace_bytes,
+                            void* stream, float* stage_ms, char (*stage_names)[32], int32_t* num_stages) {
+  if (!stage_ms || !stage_names || !num_stages) return PKV_ERR_INVALID_ARG;
+  StageTimer timer;
+  for (auto& e : timer.ev)
+    if (cudaEventCreate(&e) != cudaSuccess) return PKV_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  cudaEventRecord(timer.ev[0], st);
+  g_timer = &timer;
+  int rc = pyramidkv_compress_layer(cfg, layer, q_win, k, v, seq_lens, batch, k_out, v_out, indices, scores_or_null,
+                                    ld_scores, workspace, workspace_bytes, stream);
+  g_timer = nullptr;
+  if (rc == PKV_OK && cudaStreamSynchronize(st) != cudaSuccess) rc = PKV_ERR_CUDA;
+  *num_stages = 0;
+  if (rc == PKV_OK) {
+    for (int i = 0; i < timer.n; ++i) {
+      cudaEventElapsedTime(&stage_ms[i], timer.ev[i], timer.ev[i + 1]);
+      std::snprintf(stage_names[i], 32, "%s", timer.name[i]);
+    }
+    *num_stages = timer.n;
+  }
+  for (auto& e : timer.ev) cudaEventDestroy(e);
+  return rc;
+}
+
+int pyramidkv_check_status(const void* workspace, void* stream, uint32_t* detail_or_null) {
+  if (!workspace) return PKV_ERR_INVALID_ARG;
+  uint32_t word = 0;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(&word, workspace, sizeof word, cudaMemcpyDeviceToHost, st) != cudaSuccess) return PKV_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return PKV_ERR_CUDA;
+  if (detail_or_null) *detail_or_null = word;
+  return word == 0 ? PKV_OK : PKV_ERR_DEVICE_STATUS;
+}
+
+}  // extern "C"

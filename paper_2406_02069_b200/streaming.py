@@ -1,0 +1,93 @@
+"""Whole-model drivers over the per-layer C-ABI call.
+
+`compress_model` runs every layer of a model whose K/V already live on the device.
+`compress_model_from_host` is the end-to-end form for callers whose prefill K/V
+sit in (pinned) host memory, e.g. an offloaded cache: each layer is copied to the
+device on a copy stream while the previous layer is being compressed, and the
+compact cache and its index list are copied back.  Both only marshal arguments
+and order streams; all arithmetic is in the library's kernels.
+"""
+from __future__ import annotations
+
+from typing import List, Optional, Sequence
+
+import torch
+
+from . import binding as pkv
+
+
+class LayerOutputs:
+    """Preallocated packed outputs of every layer of a model (device)."""
+
+    def __init__(self, cfg: pkv.PkvConfig, seq_lens: Sequence[int], dtype: torch.dtype, device="cuda"):
+        self.budgets = pkv.layer_budgets(cfg)
+        self.rows = [pkv.total_rows(cfg, kl, seq_lens) for kl in self.budgets]
+        self.k = [torch.empty(r, cfg.head_dim, dtype=dtype, device=device) for r in self.rows]
+        self.v = [torch.empty(r, cfg.head_dim, dtype=dtype, device=device) for r in self.rows]
+        self.idx = [torch.empty(r, dtype=torch.int32, device=device) for r in self.rows]
+
+
+def compress_model(cfg: pkv.PkvConfig, layers, seq_lens: Sequence[int], out: LayerOutputs,
+                   workspace: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """layers: sequence of objects with .q_win, .k, .v device tensors, one per layer."""
+    for l, x in enumerate(layers):
+        pkv.compress_layer(cfg, l, x.q_win, x.k, x.v, seq_lens, out.k[l], out.v[l], out.idx[l], workspace,
+                           stream=stream)
+
+
+class HostPipeline:
+    """Double-buffered host -> device -> host pipeline for one model shape."""
+
+    def __init__(self, cfg: pkv.PkvConfig, seq_lens: Sequence[int], q_shape, kv_shape, dtype: torch.dtype,
+                 device="cuda"):
+        self.cfg, self.seq_lens = cfg, list(seq_lens)
+        self.budgets = pkv.layer_budgets(cfg)
+        self.rows = [pkv.total_rows(cfg, kl, seq_lens) for kl in self.budgets]
+        max_rows = max(self.rows)
+        self.dev = [dict(q=torch.empty(q_shape, dtype=dtype, device=device),
+                         k=torch.empty(kv_shape, dtype=dtype, device=device),
+                         v=torch.empty(kv_shape, dtype=dtype, device=device),
+                         ko=torch.empty(max_rows, cfg.head_dim, dtype=dtype, device=device),
+                         vo=torch.empty(max_rows, cfg.head_dim, dtype=dtype, device=device),
+                         io=torch.empty(max_rows, dtype=torch.int32, device=device)) for _ in range(2)]
+        self.workspace = pkv.new_workspace(cfg, len(self.seq_lens), max(self.seq_lens), device)
+        self.copy_in = torch.cuda.Stream(device=device)
+        self.compute = torch.cuda.Stream(device=device)
+        self.copy_out = torch.cuda.Stream(device=device)
+        self.h2d_bytes = 0
+        self.d2h_bytes = 0
+
+    def run(self, host_layers, host_out) -> None:
+        """host_layers[l] has pinned .q_win/.k/.v; host_out[l] has pinned .k/.v/.idx sized rows[l]."""
+        m = self.cfg.num_layers
+        loaded = [torch.cuda.Event() for _ in range(m)]
+        computed = [torch.cuda.Event() for _ in range(m)]
+        drained = [torch.cuda.Event() for _ in range(m)]
+        self.h2d_bytes = self.d2h_bytes = 0
+        for l in range(m):
+            buf, src, dst, r = self.dev[l & 1], host_layers[l], host_out[l], self.rows[l]
+            with torch.cuda.stream(self.copy_in):
+                if l >= 2:
+                    self.copy_in.wait_event(computed[l - 2])      # buffer free once its layer was compressed
+                buf["q"].copy_(src.q_win, non_blocking=True)
+                buf["k"].copy_(src.k, non_blocking=True)
+                buf["v"].copy_(src.v, non_blocking=True)
+                loaded[l].record(self.copy_in)
+            self.h2d_bytes += sum(t.numel() * t.element_size() for t in (src.q_win, src.k, src.v))
+            with torch.cuda.stream(self.compute):
+                self.compute.wait_event(loaded[l])
+                if l >= 2:
+                    self.compute.wait_event(drained[l - 2])       # outputs of this buffer were copied out
+                pkv.compress_layer(self.cfg, l, buf["q"], buf["k"], buf["v"], self.seq_lens, buf["ko"], buf["vo"],
+                                   buf["io"], self.workspace, stream=self.compute)
+                computed[l].record(self.compute)
+            with torch.cuda.stream(self.copy_out):
+                self.copy_out.wait_event(computed[l])
+                dst.k.copy_(buf["ko"][:r], non_blocking=True)
+                dst.v.copy_(buf["vo"][:r], non_blocking=True)
+                dst.idx.copy_(buf["io"][:r], non_blocking=True)
+                drained[l].record(self.copy_out)
+            self.d2h_bytes += sum(t.numel() * t.element_size() for t in (dst.k, dst.v, dst.idx))
+        cur = torch.cuda.current_stream()
+        cur.wait_stream(self.copy_out)
+        cur.wait_stream(self.compute)

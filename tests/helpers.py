@@ -1,0 +1,49 @@
+"""Comparison protocol shared by the GPU parity tests."""
+import numpy as np
+import torch
+
+import oracle
+
+RTOL, ATOL = 2e-3, 1e-5     # score tolerance: |gpu - oracle| <= RTOL * |oracle| + ATOL (fp32)
+
+
+def assert_scores_close(got: np.ndarray, want: np.ndarray, what=""):
+    err = np.abs(got.astype(np.float64) - want.astype(np.float64))
+    bound = RTOL * np.abs(want.astype(np.float64)) + ATOL
+    bad = err > bound
+    if bad.any():
+        i = np.unravel_index(np.argmax(err - bound), err.shape)
+        raise AssertionError("%s scores differ at %s: got %r want %r (%d of %d outside tolerance)"
+                             % (what, i, got[i], want[i], int(bad.sum()), bad.size))
+
+
+def assert_indices_match(got_row: np.ndarray, want_row: np.ndarray, oracle_scores_row: np.ndarray, w: int,
+                         alpha: int, what=""):
+    """Kept lists of one (sequence, head): identical, or differing only where the oracle's pooled
+    score is within tolerance of the oracle's k-th pooled value (the threshold)."""
+    assert len(got_row) == len(want_row), what
+    # window block and ordering are exact requirements
+    assert np.array_equal(got_row[len(got_row) - alpha:], want_row[len(want_row) - alpha:]), what + " window block"
+    assert np.all(np.diff(got_row) > 0), what + " not strictly ascending"
+    if np.array_equal(got_row, want_row):
+        return True
+    P = oracle_scores_row.shape[0]
+    pooled = oracle.pool_max(oracle_scores_row, w).astype(np.float64)
+    k = len(want_row) - alpha
+    kth = np.sort(pooled)[::-1][k - 1]
+    diff = np.setxor1d(got_row[:k], want_row[:k])
+    assert diff.size > 0 and diff.max() < P
+    slack = RTOL * abs(kth) + ATOL
+    worst = np.max(np.abs(pooled[diff] - kth))
+    assert worst <= 2 * slack, "%s: index sets differ away from the threshold (|pooled - kth| = %g, slack %g)" % (
+        what, worst, slack)
+    return False
+
+
+def packed_rows(counts, num_kv_heads):
+    """Yield (b, h, slice) over the packed ragged layout."""
+    off = 0
+    for b, c in enumerate(counts):
+        for h in range(num_kv_heads):
+            yield b, h, slice(off + h * c, off + (h + 1) * c)
+        off += num_kv_heads * c

@@ -1,0 +1,230 @@
+"""GPU parity: every C-ABI call against the CPU oracle on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2406_02069_b200 as pkv
+from paper_2406_02069_b200 import binding, workloads
+from helpers import assert_indices_match, assert_scores_close, packed_rows
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+# Cases the oracle finishes in seconds; each spans several key tiles and a ragged tail.
+SCALED = [
+    workloads.TINY,
+    workloads.scaled(workloads.LLAMA2_7B, num_layers=2, seq_len=4096, name="llama2_7b_full_len"),
+    workloads.scaled(workloads.LLAMA3_8B, num_layers=2, seq_len=5000 + 37, name="llama3_8b_5k"),
+    workloads.scaled(workloads.LLAMA3_70B, num_layers=3, seq_len=3000 + 11, name="llama3_70b_3k"),
+    workloads.scaled(workloads.MISTRAL_RAGGED, num_layers=2, batch=3, name="mistral_b3"),
+    workloads.scaled(workloads.with_budget(workloads.MISTRAL_RAGGED, 2048), num_layers=1, batch=2, name="mistral_b2_2048"),
+]
+
+
+def small_lens(w):
+    """Shrink the ragged workload's lengths so the oracle stays fast, keeping them uneven."""
+    lens = w.seq_lens()
+    if w.name.startswith("mistral"):
+        lens = [300 + (n % 1777) for n in lens]
+    return lens
+
+
+def run_scores(w, cfg, x, lens):
+    ws = pkv.new_workspace(cfg, len(lens), max(lens), DEV)
+    ld = max(lens) - w.window + 5
+    scores = torch.full((len(lens), w.num_kv_heads, ld), -1.0, dtype=torch.float32, device=DEV)
+    pkv.score_window(cfg, x.q_win, x.k, lens, scores, ws)
+    pkv.check_status(ws)
+    return scores
+
+
+@pytest.mark.parametrize("w", SCALED, ids=lambda w: w.name)
+def test_scores_match_oracle(w):
+    cfg = pkv.config_of(w)
+    lens = small_lens(w)
+    for layer in range(w.num_layers):
+        x = workloads.make_layer(w, layer, device=DEV, seq_lens=lens)
+        scores = run_scores(w, cfg, x, lens).cpu().numpy()
+        qc, kc = x.q_win.cpu(), x.k.cpu()
+        for b, n in enumerate(lens):
+            want, mass = oracle.window_scores(qc[b], kc[b, :, :n])
+            got = scores[b, :, : n - w.window]
+            assert_scores_close(got, want, "%s layer %d seq %d" % (w.name, layer, b))
+            # mass invariant on the GPU result too: prefix scores + window mass = alpha
+            np.testing.assert_allclose(got.astype(np.float64).sum(axis=1) + mass, w.window, rtol=1e-3)
+            assert (scores[b, :, n - w.window:] == -1.0).all()        # nothing written past the prefix
+
+
+@pytest.mark.parametrize("P,k,w", [(1, 1, 1), (5, 2, 7), (33, 32, 3), (100, 0, 5), (100, 100, 5), (100, 250, 5),
+                                   (1000, 37, 7), (4064, 188, 7), (8193, 500, 7), (20000, 4, 7), (40000, 937, 7),
+                                   (131040, 188, 7), (70001, 2016, 1)])
+def test_select_is_bit_exact_on_oracle_scores(P, k, w):
+    """Selection alone: same scores in, identical index lists out, ties included."""
+    alpha, hkv, batch = 4, 3, 2
+    rng = np.random.default_rng(P * 7 + k)
+    # few distinct levels plus pooling plateaus: ties at the threshold are the normal case
+    levels = rng.integers(0, 50, size=(batch, hkv, P)).astype(np.float32) / 64.0
+    levels[0, 0] = rng.random(P).astype(np.float32)                 # one head with distinct values
+    if P > 10:
+        levels[1, 1] = 0.25                                         # one head all equal
+    cfg = pkv.make_config(num_layers=1, num_q_heads=hkv, num_kv_heads=hkv, head_dim=64, window=alpha, pool_kernel=w,
+                          dtype="fp32", avg_budget=alpha + k, beta=1.0)
+    lens = [P + alpha] * batch
+    ws = pkv.new_workspace(cfg, batch, P + alpha, DEV)
+    scores = torch.from_numpy(levels).to(DEV)
+    c = pkv.kept_count(cfg, k, P + alpha)
+    idx = torch.full((batch * hkv * c,), -7, dtype=torch.int32, device=DEV)
+    pkv.select_topk(cfg, scores, lens, k, idx, ws)
+    pkv.check_status(ws)
+    got = idx.cpu().numpy()
+    for b, h, rows in packed_rows([c] * batch, hkv):
+        if P + alpha <= alpha + k:
+            want = np.arange(P + alpha)
+        else:
+            want = np.concatenate([oracle.select_topk(oracle.pool_max(levels[b, h], w), k), np.arange(P, P + alpha)])
+        np.testing.assert_array_equal(got[rows], want.astype(np.int32), err_msg="b=%d h=%d" % (b, h))
+
+
+@pytest.mark.parametrize("dtype,d", [("bf16", 128), ("fp32", 64), ("bf16", 64), ("fp32", 128)])
+def test_gather_is_bit_exact(dtype, d):
+    hkv, alpha, B, kl = 3, 4, 40, 21
+    lens = [300, 77, 30, 129]                                        # 30 <= B: kept whole
+    cfg = pkv.make_config(num_layers=1, num_q_heads=hkv, num_kv_heads=hkv, head_dim=d, window=alpha, pool_kernel=3,
+                          dtype=dtype, avg_budget=B, beta=1.0)
+    g = torch.Generator(device="cpu").manual_seed(5)
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    n_max = max(lens)
+    # non-contiguous views: token stride wider than d, as a fused QKV buffer would give
+    kbuf = torch.randn(len(lens), hkv, n_max, 2 * d, generator=g).to(tdt).to(DEV)
+    k, v = kbuf[..., :d], kbuf[..., d:]
+    counts = [pkv.kept_count(cfg, kl, n) for n in lens]
+    rows = sum(c * hkv for c in counts)
+    idx_np = np.zeros(rows, dtype=np.int32)
+    rng = np.random.default_rng(1)
+    for b, h, sl in packed_rows(counts, hkv):
+        idx_np[sl] = np.sort(rng.choice(lens[b], size=counts[b], replace=False))
+    idx = torch.from_numpy(idx_np).to(DEV)
+    k_out = torch.zeros(rows, d, dtype=tdt, device=DEV)
+    v_out = torch.zeros(rows, d, dtype=tdt, device=DEV)
+    pkv.gather_compact(cfg, k, v, idx, lens, kl, k_out, v_out)
+    torch.cuda.synchronize()
+    for b, h, sl in packed_rows(counts, hkv):
+        sel = torch.from_numpy(idx_np[sl]).long().to(DEV)
+        assert torch.equal(k_out[sl], k[b, h, sel]) and torch.equal(v_out[sl], v[b, h, sel])
+    # K only
+    k_only = torch.zeros_like(k_out)
+    pkv.gather_compact(cfg, k, None, idx, lens, kl, k_only, None)
+    torch.cuda.synchronize()
+    assert torch.equal(k_only, k_out)
+
+
+@pytest.mark.parametrize("w", SCALED, ids=lambda w: w.name)
+def test_compress_layer_matches_oracle(w):
+    cfg = pkv.config_of(w)
+    lens = small_lens(w)
+    budgets = pkv.layer_budgets(cfg)
+    assert budgets == oracle.layer_budgets(w.num_layers, w.avg_budget, w.window, w.beta)
+    ws = pkv.new_workspace(cfg, len(lens), max(lens), DEV)
+    for layer in range(w.num_layers):
+        kl = budgets[layer]
+        x = workloads.make_layer(w, layer, device=DEV, seq_lens=lens)
+        rows = pkv.total_rows(cfg, kl, lens)
+        k_out = torch.empty(rows, w.head_dim, dtype=x.k.dtype, device=DEV)
+        v_out = torch.empty_like(k_out)
+        idx = torch.empty(rows, dtype=torch.int32, device=DEV)
+        pkv.compress_layer(cfg, layer, x.q_win, x.k, x.v, lens, k_out, v_out, idx, ws)   # scores in the workspace
+        pkv.check_status(ws)
+        ref = oracle.compress_batch(x.q_win.cpu(), x.k.cpu(), x.v.cpu(), lens, pool_kernel=w.pool_kernel,
+                                    avg_budget=w.avg_budget, k_layer=kl)
+        assert ref["indices"].shape[0] == rows
+        got_idx = idx.cpu().numpy()
+        identical = 0
+        for b, h, sl in packed_rows(ref["counts"], w.num_kv_heads):
+            same = assert_indices_match(got_idx[sl], ref["indices"][sl], ref["scores"][b][h], w.pool_kernel, w.window,
+                                        "%s layer %d b %d h %d" % (w.name, layer, b, h))
+            identical += bool(same)
+            # gathered rows must be the rows the GPU's own index list names, bit for bit
+            sel = idx[sl].long()
+            assert torch.equal(k_out[sl], x.k[b, h, sel]) and torch.equal(v_out[sl], x.v[b, h, sel])
+            if same:
+                assert torch.equal(k_out[sl].cpu(), ref["k_out"][sl]) and torch.equal(v_out[sl].cpu(), ref["v_out"][sl])
+            # planted sinks and needles survive wherever the budget has room for their pooled plateaus
+            planted = x.planted[b]
+            if kl >= w.pool_kernel * len(planted) and lens[b] > w.avg_budget:
+                assert set(planted) <= set(got_idx[sl].tolist()), "planted tokens evicted"
+        total = len(ref["counts"]) * w.num_kv_heads
+        assert identical >= 0.9 * total, "only %d of %d index lists identical" % (identical, total)
+
+
+def test_three_calls_equal_the_fused_call():
+    w = workloads.scaled(workloads.LLAMA3_8B, num_layers=2, seq_len=3000, name="l3_3k")
+    cfg = pkv.config_of(w)
+    lens = w.seq_lens()
+    kl = pkv.layer_budgets(cfg)[1]
+    x = workloads.make_layer(w, 1, device=DEV)
+    ws = pkv.new_workspace(cfg, 1, max(lens), DEV)
+    rows = pkv.total_rows(cfg, kl, lens)
+    outs = []
+    for fused in (True, False):
+        k_out = torch.empty(rows, w.head_dim, dtype=x.k.dtype, device=DEV)
+        v_out = torch.empty_like(k_out)
+        idx = torch.empty(rows, dtype=torch.int32, device=DEV)
+        scores = torch.zeros(1, w.num_kv_heads, max(lens), dtype=torch.float32, device=DEV)
+        if fused:
+            pkv.compress_layer(cfg, 1, x.q_win, x.k, x.v, lens, k_out, v_out, idx, ws, scores=scores)
+        else:
+            pkv.score_window(cfg, x.q_win, x.k, lens, scores, ws)
+            pkv.select_topk(cfg, scores, lens, kl, idx, ws)
+            pkv.gather_compact(cfg, x.k, x.v, idx, lens, kl, k_out, v_out)
+        pkv.check_status(ws)
+        outs.append((k_out, v_out, idx, scores))
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("n,B,alpha,G", [(9, 16, 8, 2), (9, 8, 8, 1), (40, 64, 8, 2), (64, 64, 8, 4), (65, 64, 8, 4),
+                                         (130, 16, 16, 1), (257, 40, 1, 3), (513, 100, 48, 2)])
+def test_edge_cases(n, B, alpha, G):
+    """Shortest contexts, contexts that fit the budget, window-only budgets, odd group sizes."""
+    hkv, d, w_pool, m = 2, 64, 5, 3
+    cfg = pkv.make_config(num_layers=m, num_q_heads=hkv * G, num_kv_heads=hkv, head_dim=d, window=alpha,
+                          pool_kernel=w_pool, dtype="fp32", avg_budget=B, beta=20.0)
+    g = torch.Generator(device="cpu").manual_seed(n * 3 + B)
+    q = torch.randn(1, hkv * G, alpha, d, generator=g)
+    k = torch.randn(1, hkv, n, d, generator=g)
+    v = torch.randn(1, hkv, n, d, generator=g)
+    ws = pkv.new_workspace(cfg, 1, n, DEV)
+    budgets = pkv.layer_budgets(cfg)
+    for layer, kl in enumerate(budgets):
+        c = pkv.kept_count(cfg, kl, n)
+        k_out = torch.empty(hkv * c, d, device=DEV)
+        v_out = torch.empty_like(k_out)
+        idx = torch.empty(hkv * c, dtype=torch.int32, device=DEV)
+        pkv.compress_layer(cfg, layer, q.to(DEV), k.to(DEV), v.to(DEV), [n], k_out, v_out, idx, ws)
+        pkv.check_status(ws)
+        ref = oracle.compress_layer(q[0], k[0], v[0], pool_kernel=w_pool, avg_budget=B, k_layer=kl)
+        assert ref["count"] == c
+        got = idx.cpu().numpy().reshape(hkv, c)
+        for h in range(hkv):
+            assert_indices_match(got[h], ref["kept"][h], ref["scores"][h], w_pool, alpha, "edge layer %d h %d" % (layer, h))
+            assert torch.equal(k_out.view(hkv, c, d)[h].cpu(), k[0, h, torch.from_numpy(got[h]).long()])
+        if n <= B:
+            assert (got == np.arange(n)).all()
+            assert torch.equal(k_out.cpu().view(hkv, n, d), k[0]) and torch.equal(v_out.cpu().view(hkv, n, d), v[0])
+
+
+def test_device_errors_are_reported_not_raised_as_faults():
+    """Bad arguments come back as status codes even with real device buffers."""
+    w = workloads.TINY
+    cfg = pkv.config_of(w)
+    x = workloads.make_layer(w, 0, device=DEV)
+    ws = pkv.new_workspace(cfg, 1, 512, DEV)
+    scores = torch.zeros(1, w.num_kv_heads, 100, dtype=torch.float32, device=DEV)      # ld too small
+    with pytest.raises(pkv.PkvError) as e:
+        pkv.score_window(cfg, x.q_win, x.k, [512], scores, ws)
+    assert e.value.status == binding.PKV_ERR_INVALID_ARG
+    with pytest.raises(pkv.PkvError) as e:
+        pkv.score_window(cfg, x.q_win, x.k, [512], torch.zeros(1, 2, 512, device=DEV), ws[:1024])
+    assert e.value.status == binding.PKV_ERR_WORKSPACE
+    pkv.check_status(ws)
