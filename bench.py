@@ -1,0 +1,350 @@
+#!/usr/bin/env python
+"""Benchmark of the PyramidKV prefill KV-cache compression path on B200.
+
+One step = the whole hot path (window scores, pool + top-k, window retention,
+gather) over every layer of one synthetic model-shaped workload whose K/V are
+resident in HBM.  Metric: context tokens compressed per second over all layers.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+With N > 1 (launched by torch.distributed.run) every rank compresses its own
+copy of the workload (sequences are independent units: no data-path
+collective); the reported value is the sum over ranks divided by the slowest
+rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+METRIC = "context tokens compressed/s (all layers)"
+UNIT = "tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
+
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from ncu captures, keyed by
+# kernel name, valid only for the kernel sources whose digest is given: any change to csrc/ voids them.
+NCU_TRAFFIC = {
+    # "kernel": {"csrc_digest": "...", "bytes_per_key_row": ...}
+}
+
+
+def csrc_digest() -> str:
+    h = hashlib.sha256()
+    d = os.path.join(ROOT, "paper_2406_02069_b200", "csrc")
+    for name in sorted(os.listdir(d)):
+        with open(os.path.join(d, name), "rb") as f:
+            h.update(name.encode() + b"\0" + f.read())
+    return h.hexdigest()[:16]
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return p, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], 0.0, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx = max(mx, float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        sm.sort()
+        med = sm[len(sm) // 2] if sm else None
+        return {"sm_mhz": med, "sm_max_mhz": mx or None, "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def graded_bytes_per_layer(w, lens, count_rows, esz):
+    """K read once + kept K,V rows read + compact K,V written + index list written (+ window Q)."""
+    d = w.head_dim
+    k_read = sum(lens) * w.num_kv_heads * d * esz
+    q_read = len(lens) * w.num_q_heads * w.window * d * esz
+    moved = count_rows * d * esz * 2          # K and V rows
+    return k_read + q_read + 2 * moved + 4 * count_rows
+
+
+def cpu_baseline_sample(w, layer_inputs, lens, budgets, budget_s=20.0):
+    """Times the oracle, as it stands, on (sequence 0, a few KV heads) of layer 0 and scales to all layers."""
+    import oracle
+    n = lens[0]
+    q = layer_inputs.q_win[0].cpu()
+    k = layer_inputs.k[0, :, :n].cpu()
+    v = layer_inputs.v[0, :, :n].cpu()
+    g = w.group
+    heads_done, t_total = 0, 0.0
+    while heads_done < w.num_kv_heads:
+        h = heads_done
+        t0 = time.perf_counter()
+        oracle.compress_layer(q[h * g:(h + 1) * g], k[h:h + 1], v[h:h + 1], pool_kernel=w.pool_kernel,
+                              avg_budget=w.avg_budget, k_layer=budgets[0], want_scores=False)
+        t_total += time.perf_counter() - t0
+        heads_done += 1
+        if t_total * (heads_done + 1) / heads_done > budget_s:
+            break
+    # one (sequence, head) unit costs t_total / heads_done; all layers, all heads, all sequences (by length)
+    per_token_head = t_total / heads_done / n
+    full = per_token_head * sum(lens) * w.num_kv_heads * w.num_layers
+    return {"value": sum(lens) / full, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": "layer 0, sequence 0 (n=%d), %d of %d KV heads with their %d query heads each; "
+                      "%.1f s of CPU work scaled by heads x layers x tokens" % (n, heads_done, w.num_kv_heads, g, t_total)}
+
+
+def run_reference(args, w):
+    """The oracle as the reference arm: each step is a bounded sample of the workload on the host cores."""
+    import oracle
+    from paper_2406_02069_b200 import workloads
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    lens = w.seq_lens()
+    budgets = oracle.layer_budgets(w.num_layers, w.avg_budget, w.window, w.beta)
+    x = workloads.make_layer(w, 0, device="cpu", seq_lens=lens[:1])
+    per_step_budget = max(2.0, 100.0 / max(1, args.steps + args.warmup))
+    res = None
+    for _ in range(args.warmup):
+        res = cpu_baseline_sample(w, x, lens[:1], budgets, budget_s=per_step_budget)
+    vals = []
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        res = cpu_baseline_sample(w, x, lens[:1], budgets, budget_s=per_step_budget)
+        vals.append(res["value"])
+    wall = time.perf_counter() - t0
+    value = len(vals) / sum(1.0 / v for v in vals)
+    # scale the sample's rate from sequence 0 to the whole batch: rate per token is length independent
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1000.0 * sum(lens) / value,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "layers": w.num_layers, "batch": w.batch, "seq_lens": lens,
+                       "note": "each step times a bounded sample (%.1f s wall in total) and scales it to the full "
+                               "workload; ms_per_step is that extrapolation" % wall},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": res["cores"], "kind": "oracle",
+                             "sample": res["sample"]},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+class HostLayer:
+    def __init__(self, x):
+        self.q_win = x.q_win.cpu().pin_memory()
+        self.k = x.k.cpu().pin_memory()
+        self.v = x.v.cpu().pin_memory()
+
+
+class HostOut:
+    def __init__(self, rows, d, dtype):
+        self.k_full = torch.empty(rows, d, dtype=dtype).pin_memory()
+        self.v_full = torch.empty(rows, d, dtype=dtype).pin_memory()
+        self.idx_full = torch.empty(rows, dtype=torch.int32).pin_memory()
+
+    def view(self, r):
+        o = HostOut.__new__(HostOut)
+        o.k, o.v, o.idx = self.k_full[:r], self.v_full[:r], self.idx_full[:r]
+        return o
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama3_70b_128k")
+    ap.add_argument("--budget", type=int, default=None, help="override the average budget B")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--host-ring", type=int, default=4, help="distinct pinned host layers cycled by the e2e leg")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    from paper_2406_02069_b200 import workloads
+    w = workloads.WORKLOADS[args.workload]
+    if args.budget:
+        w = workloads.with_budget(w, args.budget)
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import paper_2406_02069_b200 as pkv
+    from paper_2406_02069_b200 import streaming
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the compression path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    cfg = pkv.config_of(w)
+    lens = w.seq_lens()
+    esz = 2 if w.dtype == "bf16" else 4
+    tdt = w.torch_dtype()
+    layers = [workloads.make_layer(w, l, device="cuda") for l in range(w.num_layers)]
+    out = streaming.LayerOutputs(cfg, lens, tdt)
+    ws = pkv.new_workspace(cfg, len(lens), max(lens))
+    tokens = sum(lens)
+    torch.cuda.synchronize()
+
+    # ---- device-resident timing
+    for _ in range(args.warmup):
+        streaming.compress_model(cfg, layers, lens, out, ws)
+    pkv.check_status(ws)
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.3)
+    barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(args.steps):
+        streaming.compress_model(cfg, layers, lens, out, ws)
+    ev1.record()
+    barrier()
+    clocks = sampler.stop()
+    ms = ev0.elapsed_time(ev1)
+    if dist is not None:
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    pkv.check_status(ws)
+    ms_per_step = ms / args.steps
+    value = world * tokens / (ms_per_step * 1e-3)
+
+    # ---- per-kernel device times (events between the launches of each layer's call), same inputs and launch shapes
+    stages = {}
+    for rep in range(2):                                           # first repetition warms, second is kept
+        stages = {}
+        for l, x in enumerate(layers):
+            for name, t_ms in pkv.profile_layer(cfg, l, x.q_win, x.k, x.v, lens, out.k[l], out.v[l], out.idx[l], ws):
+                s = stages.setdefault(name, [0, 0.0])
+                s[0] += 1
+                s[1] += t_ms
+    launches_per_step = sum(s[0] for s in stages.values())
+    dominant = max(stages, key=lambda k: stages[k][1])
+    dom_ms = stages[dominant][1] / stages[dominant][0]
+    peak, peak_kind = peaks()
+    k_bytes_layer = sum(lens) * w.num_kv_heads * w.head_dim * esz
+    q_bytes_layer = len(lens) * w.num_q_heads * w.window * w.head_dim * esz
+    score_bytes_layer = sum(n - w.window for n in lens) * w.num_kv_heads * 4
+    dom_bytes = k_bytes_layer + q_bytes_layer + score_bytes_layer   # one sweep over K per launch
+    achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
+    traffic = None
+    tr = NCU_TRAFFIC.get(dominant)
+    if tr and tr.get("csrc_digest") == csrc_digest():
+        traffic = tr["bytes_per_key_row"] * sum(lens) * w.num_kv_heads
+    graded = sum(graded_bytes_per_layer(w, lens, r, esz) for r in out.rows)
+    path_gbs = graded / (ms_per_step * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peak["hbm_gbs"], "traffic": traffic, "peak_source": peak_kind,
+                "bytes_per_launch": dom_bytes, "ms_per_launch": dom_ms,
+                "kernels": {k: {"launches": v[0], "ms_total": v[1]} for k, v in stages.items()},
+                "path": {"graded_bytes_per_step": graded, "achieved": path_gbs, "frac": path_gbs / peak["hbm_gbs"],
+                         "frac_of_8TBs": path_gbs / 8000.0}}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
+            "config": {"workload": w.name, "layers": w.num_layers, "q_heads": w.num_q_heads,
+                       "kv_heads": w.num_kv_heads, "head_dim": w.head_dim, "batch": w.batch, "seq_lens": lens,
+                       "window": w.window, "pool_kernel": w.pool_kernel, "avg_budget": w.avg_budget, "beta": w.beta,
+                       "tokens_per_step_per_gpu": tokens, "parallelism": "replicas x%d" % world,
+                       "l2": "every layer's K (%.0f MB) is distinct and larger than L2; %d layers (%.1f GB) resident"
+                             % (k_bytes_layer / 1e6, w.num_layers, 2 * k_bytes_layer * w.num_layers / 1e9)},
+            "clocks": clocks, "roofline": roofline, "gpu_launches": launches_per_step * args.steps,
+            "tokens_per_s_per_layer": value * w.num_layers}
+
+    # ---- end to end: pinned host K/V/Q in, compact cache + index list out, copies inside the timed region
+    if not args.no_e2e:
+        ring = max(1, min(args.host_ring, w.num_layers))
+        host_layers = [HostLayer(layers[l]) for l in range(ring)]
+        host_outs = [HostOut(max(out.rows), w.head_dim, tdt) for _ in range(ring)]
+        pipe = streaming.HostPipeline(cfg, lens, layers[0].q_win.shape, layers[0].k.shape, tdt)
+        hl = [host_layers[l % ring] for l in range(w.num_layers)]
+        ho = [host_outs[l % ring].view(out.rows[l]) for l in range(w.num_layers)]
+        pipe.run(hl, ho)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.e2e_steps):
+            pipe.run(hl, ho)
+        e1.record()
+        barrier()
+        e_ms = e0.elapsed_time(e1)
+        if dist is not None:
+            t = torch.tensor([e_ms], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e_ms = float(t.item())
+        pkv.check_status(pipe.workspace)
+        line["e2e"] = {"value": world * tokens / (e_ms / args.e2e_steps * 1e-3), "unit": UNIT,
+                       "h2d_bytes_per_step": pipe.h2d_bytes, "d2h_bytes_per_step": pipe.d2h_bytes,
+                       "steps": args.e2e_steps, "ms_per_step": e_ms / args.e2e_steps,
+                       "note": "host side cycles %d distinct pinned layers; every layer is copied in every step" % ring}
+
+    if rank == 0 and not args.no_cpu_baseline and world == 1:
+        line["cpu_baseline"] = cpu_baseline_sample(w, layers[0], lens, out.budgets)
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
