@@ -59,6 +59,7 @@ extern "C" {
 #define PKV_ERR_WORKSPACE 3       /* workspace too small or misaligned (256 bytes) */
 #define PKV_ERR_CUDA 4            /* a launch failed; the CUDA error is left for the caller */
 #define PKV_ERR_DEVICE_STATUS 5   /* a kernel recorded a failure in the workspace status word */
+#define PKV_ERR_STATIC_SCRATCH 6  /* problem needs more than PKV_STATIC_SCRATCH_BYTES of built-in scratch */
 
 #define PKV_DTYPE_FP32 0
 #define PKV_DTYPE_BF16 1
@@ -67,6 +68,7 @@ extern "C" {
 
 #define PKV_MAX_BATCH 64          /* sequences per call */
 #define PKV_MAX_STAGES 8          /* kernels one pyramidkv_compress_layer call may launch */
+#define PKV_STATIC_SCRATCH_BYTES (8u << 20)  /* built-in scratch of pyramidkv_score_window_static: 8 MiB per GPU */
 
 typedef struct pkv_config {
   int32_t num_layers;    /* m >= 1 */
@@ -145,6 +147,35 @@ int pyramidkv_score_window(const pkv_config* cfg, pkv_tensor q_win, pkv_tensor k
                            const int32_t* seq_lens, int32_t batch,
                            float* scores, int64_t ld_scores,
                            void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * pyramidkv_score_window for callers that cannot allocate.  The paper has no
+ * counterpart: this is an integration aid.  Same inputs, same scores as
+ * pyramidkv_score_window, but no workspace argument: the kernels' scratch
+ * (per-chunk row statistics and the row normalisers) lives in an array of
+ * PKV_STATIC_SCRATCH_BYTES (8 MiB) that is built into the library, so the call
+ * and everything under it performs no cudaMalloc / cudaFree and needs no memory
+ * pool.  It is meant for code that is handed only its input and output buffers:
+ * an operator plugged into a serving engine that has already given all device
+ * memory to its own pool, or a section where an allocation (which may
+ * synchronise the whole device) is not acceptable.
+ *   - Every GPU on which the library is loaded holds the 8 MiB until the process ends.
+ *   - The problem must fit: the scratch grows with batch * H_kv * ceil(n_max / 128) *
+ *     (H_q / H_kv) * alpha * 8 bytes.  Larger problems are refused with
+ *     PKV_ERR_STATIC_SCRATCH before anything is enqueued; use pyramidkv_score_window
+ *     with a workspace for those.
+ *   - The first call made on a device looks up the array's device address
+ *     (cudaGetSymbolAddress) and caches it; make that first call outside any
+ *     stream capture.
+ *   - All calls on a device share the one array, which keeps the previous call's
+ *     contents.  The call clears the part that must start at zero itself, but two
+ *     calls whose kernels overlap on the GPU (different streams, no ordering
+ *     between them) race on it: order them on one stream or with events.
+ * Errors: INVALID_ARG, UNSUPPORTED, STATIC_SCRATCH, CUDA.
+ */
+int pyramidkv_score_window_static(const pkv_config* cfg, pkv_tensor q_win, pkv_tensor k,
+                                  const int32_t* seq_lens, int32_t batch,
+                                  float* scores, int64_t ld_scores, void* stream);
 
 /*
  * Pooling and selection, Section 4.2.2.  Per sequence and KV head:

@@ -20,12 +20,14 @@ PKV_ERR_UNSUPPORTED = 2
 PKV_ERR_WORKSPACE = 3
 PKV_ERR_CUDA = 4
 PKV_ERR_DEVICE_STATUS = 5
+PKV_ERR_STATIC_SCRATCH = 6
 PKV_MAX_BATCH = 64
+PKV_STATIC_SCRATCH_BYTES = 8 << 20
 
 EXPORTS = ("pyramidkv_strerror", "pyramidkv_layer_budgets", "pyramidkv_kept_count",
            "pyramidkv_workspace_bytes", "pyramidkv_score_window", "pyramidkv_select_topk",
            "pyramidkv_gather_compact", "pyramidkv_compress_layer", "pyramidkv_profile_layer",
-           "pyramidkv_check_status")
+           "pyramidkv_check_status", "pyramidkv_score_window_static")
 PKV_MAX_STAGES = 8
 
 
@@ -63,6 +65,7 @@ def _load() -> ctypes.CDLL:
     lib.pyramidkv_workspace_bytes.argtypes = [CFG, I32, I32]
     lib.pyramidkv_workspace_bytes.restype = SZ
     lib.pyramidkv_score_window.argtypes = [CFG, PkvTensor, PkvTensor, P, I32, P, I64, P, SZ, P]
+    lib.pyramidkv_score_window_static.argtypes = [CFG, PkvTensor, PkvTensor, P, I32, P, I64, P]
     lib.pyramidkv_select_topk.argtypes = [CFG, P, I64, P, I32, I32, P, P, SZ, P]
     lib.pyramidkv_gather_compact.argtypes = [CFG, PkvTensor, PkvTensor, P, P, I32, I32, P, P, P]
     lib.pyramidkv_compress_layer.argtypes = [CFG, I32, PkvTensor, PkvTensor, PkvTensor, P, I32, P, P, P, P, I64,
@@ -160,6 +163,20 @@ def score_window(cfg: PkvConfig, q_win: torch.Tensor, k: torch.Tensor, seq_lens:
     _check(_lib.pyramidkv_score_window(ctypes.byref(cfg), _tensor(q_win), _tensor(k), lens, batch,
                                        scores.data_ptr(), scores.stride(1), workspace.data_ptr(),
                                        workspace.numel(), _stream(stream)), "pyramidkv_score_window")
+
+
+def score_window_static(cfg: PkvConfig, q_win: torch.Tensor, k: torch.Tensor, seq_lens: Sequence[int],
+                        scores: torch.Tensor, stream=None) -> None:
+    """score_window without a workspace: scratch is the library's built-in 8 MiB array.
+
+    For callers that may not allocate device memory.  Problems that need more
+    scratch raise PkvError(PKV_ERR_STATIC_SCRATCH).  Calls on one device share the
+    array, so keep them ordered on a stream.
+    """
+    lens, batch = _lens(seq_lens)
+    _check(_lib.pyramidkv_score_window_static(ctypes.byref(cfg), _tensor(q_win), _tensor(k), lens, batch,
+                                              scores.data_ptr(), scores.stride(1), _stream(stream)),
+           "pyramidkv_score_window_static")
 
 
 def select_topk(cfg: PkvConfig, scores: torch.Tensor, seq_lens: Sequence[int], k_layer: int,

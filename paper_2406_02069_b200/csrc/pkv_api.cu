@@ -4,6 +4,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 
 #include "pkv_common.cuh"
 #include "pkv_gather.cuh"
@@ -267,6 +268,7 @@ const char* pyramidkv_strerror(int status) {
     case PKV_ERR_WORKSPACE: return "workspace too small or misaligned";
     case PKV_ERR_CUDA: return "CUDA launch failed";
     case PKV_ERR_DEVICE_STATUS: return "a kernel recorded a failure in the workspace status word";
+    case PKV_ERR_STATIC_SCRATCH: return "problem too large for the built-in scratch (PKV_STATIC_SCRATCH_BYTES)";
     default: return "unknown status";
   }
 }
@@ -415,3 +417,67 @@ int pyramidkv_check_status(const void* workspace, void* stream, uint32_t* detail
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------
+// Scoring without any caller-provided scratch.
+//
+// Some callers of pyramidkv_score_window cannot hand over a workspace because they
+// cannot allocate device memory at the point of the call: code that runs inside a
+// serving engine whose memory pool is already carved up, a plugin that is only given
+// its input and output tensors, or a latency-critical section in which cudaMalloc
+// (which may synchronise the device) is off limits.  For them the scratch of the
+// score kernels (chunk statistics and row normalisers) lives in the fixed array
+// below, which is part of the library image: every GPU that loads the library holds
+// PKV_STATIC_SCRATCH_BYTES of it until the process exits.
+//
+// In host code `g_static_scratch` only names the symbol; it is not a device address.
+// The address that kernels may use is looked up once per device with
+// cudaGetSymbolAddress, on the first call made while that device is current.
+static __device__ __align__(256) unsigned char g_static_scratch[PKV_STATIC_SCRATCH_BYTES];
+
+namespace {
+std::mutex g_static_mutex;
+void* g_static_ptr[64] = {};
+
+// Device address of the static scratch on the current device (nullptr on failure).
+void* static_scratch_address() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  if (!g_static_ptr[dev]) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess) return nullptr;
+    g_static_ptr[dev] = ptr;
+  }
+  return g_static_ptr[dev];
+}
+}  // namespace
+
+extern "C" int pyramidkv_score_window_static(const pkv_config* cfg, pkv_tensor q_win, pkv_tensor k,
+                                             const int32_t* seq_lens, int32_t batch, float* scores,
+                                             int64_t ld_scores, void* stream) {
+  if (!config_ok(cfg)) return PKV_ERR_INVALID_ARG;
+  if (int rc = config_supported(cfg)) return rc;
+  const int eb = cfg->dtype == PKV_DTYPE_FP32 ? 4 : 2;
+  if (!tensor_ok(q_win, cfg->head_dim, eb) || !tensor_ok(k, cfg->head_dim, eb) || !scores) return PKV_ERR_INVALID_ARG;
+  SeqTable table;
+  int max_n;
+  int64_t rows;
+  if (int rc = build_table(cfg, seq_lens, batch, 0, &table, &max_n, &rows)) return rc;
+  if (ld_scores < max_n - cfg->window) return PKV_ERR_INVALID_ARG;
+  // Scratch the score kernels need: everything the usual workspace holds ahead of its score buffer.
+  // (the score buffer is the workspace's last region and is supplied by the caller here)
+  const Workspace sizing = carve(cfg, batch, max_n, nullptr);
+  const size_t score_region =
+      align_up(static_cast<size_t>(batch) * cfg->num_kv_heads * sizing.ld_scores * sizeof(float));
+  const size_t need = sizing.bytes - score_region;
+  if (need > PKV_STATIC_SCRATCH_BYTES) return PKV_ERR_STATIC_SCRATCH;
+  void* base = static_scratch_address();
+  if (!base) return PKV_ERR_CUDA;
+  const Workspace w = carve(cfg, batch, max_n, base);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // The array keeps whatever the previous call left.  Only the status word has to start from zero;
+  // statistics and normalisers are fully rewritten before they are read.
+  if (cudaMemsetAsync(w.status, 0, kAlign, st) != cudaSuccess) return PKV_ERR_CUDA;
+  return run_scores(cfg, q_win, k, table, batch, scores, ld_scores, w, st);
+}
