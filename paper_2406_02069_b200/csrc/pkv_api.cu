@@ -3,12 +3,14 @@
 // declared in include/pyramidkv.h.
 #include <cmath>
 #include <cstdio>
+#include <algorithm>
 #include <cstring>
 #include <mutex>
 
 #include "pkv_common.cuh"
 #include "pkv_gather.cuh"
 #include "pkv_score_generic.cuh"
+#include "pkv_score_tc.cuh"
 #include "pkv_select.cuh"
 
 namespace pkv {
@@ -84,7 +86,7 @@ Workspace carve(const pkv_config* c, int batch, int max_n, void* base) {
   const size_t chunks = (static_cast<size_t>(max_n) + kPartialChunk - 1) / kPartialChunk;
   w.status = reinterpret_cast<uint32_t*>(take(kAlign));
   w.lse2 = reinterpret_cast<float*>(take(heads * rows * sizeof(float)));
-  w.partial = reinterpret_cast<float2*>(take(heads * chunks * rows * sizeof(float2)));
+  w.partial = reinterpret_cast<float2*>(take(heads * chunks * 2 * rows * sizeof(float2)));   // 2 slots per chunk
   w.ld_scores = static_cast<int64_t>((static_cast<size_t>(max_n) + 63) / 64 * 64);
   w.scores = reinterpret_cast<float*>(take(heads * w.ld_scores * sizeof(float)));
   w.bytes = off;
@@ -152,12 +154,137 @@ int launch_scores_generic(ScoreParams& sp, int batch, cudaStream_t st) {
   }
   sp.seq.stat_off[batch] = stat_tiles;
   sp.seq.score_off[batch] = score_tiles;
+  sp.slots_per_chunk = 1;
   rowstats_generic_kernel<T, D><<<dim3(stat_tiles, sp.num_kv_heads), kGenRowBlock, 0, st>>>(sp);
   mark(st, "rowstats_generic");
   combine_stats_kernel<<<dim3(sp.num_kv_heads, batch), 256, 0, st>>>(sp, std::log2(static_cast<float>(sp.group)));
   mark(st, "combine_stats");
   scores_generic_kernel<T, D><<<dim3(score_tiles, sp.num_kv_heads), kGenScoreKeys, 0, st>>>(sp);
   mark(st, "scores_generic");
+  return check_launch();
+}
+
+// ---------------------------------------------------------------- tensor-core scores
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = [] {
+    void* sym = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      sym = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(sym);
+  }();
+  return fn;
+}
+
+// Tensor map of a bf16 [batch][head][token][d] view: dims (d, token, head, batch), box (64, box_tok, box_head, 1),
+// 128-byte swizzle, zero fill outside the tensor.
+bool make_map(CUtensorMap* map, const pkv_tensor& t, int d, uint64_t tokens, uint64_t heads, uint64_t batch,
+              uint32_t box_tok, uint32_t box_head) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[4] = {static_cast<cuuint64_t>(d), tokens, heads, batch};
+  auto bytes = [](int64_t elems) { return static_cast<cuuint64_t>(elems > 0 ? elems : 8) * 2; };
+  const cuuint64_t strides[3] = {bytes(t.stride_token), bytes(t.stride_head), bytes(t.stride_batch)};
+  const cuuint32_t box[4] = {64, box_tok, box_head, 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(t.ptr), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool tc_eligible(const pkv_config* c) {
+  const int g = c->num_q_heads / c->num_kv_heads;
+  return c->dtype == PKV_DTYPE_BF16 && g * c->window <= kTcMaxRows && c->window <= 256 && g <= 256;
+}
+
+int device_sm_count() {
+  static int sms[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+  if (!sms[dev]) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+    sms[dev] = n;
+  }
+  return sms[dev];
+}
+
+template <int D>
+int launch_scores_tc(const pkv_config* c, const pkv_tensor& q, const pkv_tensor& k, ScoreParams& sp, int batch,
+                     int max_n, uint32_t* status, cudaStream_t st) {
+  const int sms = device_sm_count();
+  if (sms <= 0) return PKV_ERR_CUDA;
+  static bool attr_done[64] = {};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (!attr_done[dev]) {
+    if (cudaFuncSetAttribute(score_tc_kernel<D, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcSmem<D>::kTotal) !=
+            cudaSuccess ||
+        cudaFuncSetAttribute(score_tc_kernel<D, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcSmem<D>::kTotal) !=
+            cudaSuccess)
+      return PKV_ERR_CUDA;
+    attr_done[dev] = true;
+  }
+  alignas(64) CUtensorMap q_map, k_map;
+  if (!make_map(&q_map, q, D, c->window, c->num_q_heads, batch, c->window, sp.group) ||
+      !make_map(&k_map, k, D, max_n, c->num_kv_heads, batch, kTcTileKeys, 1))
+    return PKV_ERR_CUDA;
+
+  TcParams tp{};
+  tp.seq = sp.seq;
+  tp.num_kv_heads = sp.num_kv_heads;
+  tp.group = sp.group;
+  tp.rows = sp.rows;
+  tp.rows_pad = (sp.rows + 31) / 32 * 32;
+  tp.row_blocks = (sp.rows + 127) / 128;
+  tp.scale_log2 = sp.scale_log2;
+  tp.partial = sp.partial;
+  tp.lse2 = sp.lse2;
+  tp.scores = sp.scores;
+  tp.ld_scores = sp.ld_scores;
+  tp.status = status;
+  // Key tiles per work item: the largest power of two that still spreads the items evenly over the SMs.
+  auto items_for = [&](int ct, bool prefix) {
+    long long items = 0;
+    for (int b = 0; b < batch; ++b) {
+      const int keys = prefix ? sp.seq.n[b] - sp.seq.alpha : sp.seq.n[b];
+      const int tiles = (keys + kTcTileKeys - 1) / kTcTileKeys;
+      items += (tiles + ct - 1) / ct;
+    }
+    return items * sp.num_kv_heads;
+  };
+  int ct = 16;
+  for (; ct > 1; ct /= 2) {
+    const long long items = items_for(ct, false);
+    const long long waves = (items + sms - 1) / sms;
+    if (items >= sms && static_cast<double>(items) / static_cast<double>(waves * sms) >= 0.93) break;
+  }
+  tp.chunk_tiles = ct;
+  int stat_items = 0, score_items = 0;
+  for (int b = 0; b < batch; ++b) {
+    tp.seq.stat_off[b] = stat_items;
+    tp.seq.score_off[b] = score_items;
+    stat_items += ((sp.seq.n[b] + kTcTileKeys - 1) / kTcTileKeys + ct - 1) / ct;
+    score_items += ((sp.seq.n[b] - sp.seq.alpha + kTcTileKeys - 1) / kTcTileKeys + ct - 1) / ct;
+  }
+  tp.seq.stat_off[batch] = stat_items;
+  tp.seq.score_off[batch] = score_items;
+  sp.seq = tp.seq;
+  sp.slots_per_chunk = 2;
+
+  const int grid_a = static_cast<int>(std::min<long long>(sms, static_cast<long long>(stat_items) * sp.num_kv_heads));
+  const int grid_b = static_cast<int>(std::min<long long>(sms, static_cast<long long>(score_items) * sp.num_kv_heads));
+  score_tc_kernel<D, 0><<<grid_a, kTcThreads, TcSmem<D>::kTotal, st>>>(q_map, k_map, tp);
+  mark(st, "rowstats_tc");
+  combine_stats_kernel<<<dim3(sp.num_kv_heads, batch), 256, 0, st>>>(sp, std::log2(static_cast<float>(sp.group)));
+  mark(st, "combine_stats");
+  score_tc_kernel<D, 1><<<grid_b, kTcThreads, TcSmem<D>::kTotal, st>>>(q_map, k_map, tp);
+  mark(st, "scores_tc");
   return check_launch();
 }
 
@@ -175,6 +302,12 @@ int run_scores(const pkv_config* c, const pkv_tensor& q, const pkv_tensor& k, co
   sp.lse2 = w.lse2;
   sp.scores = scores;
   sp.ld_scores = ld;
+  if (tc_eligible(c)) {
+    int max_n = 0;
+    for (int b = 0; b < batch; ++b) max_n = std::max(max_n, table.n[b]);
+    return c->head_dim == 64 ? launch_scores_tc<64>(c, q, k, sp, batch, max_n, w.status, st)
+                             : launch_scores_tc<128>(c, q, k, sp, batch, max_n, w.status, st);
+  }
   if (c->dtype == PKV_DTYPE_FP32)
     return c->head_dim == 64 ? launch_scores_generic<float, 64>(sp, batch, st)
                              : launch_scores_generic<float, 128>(sp, batch, st);

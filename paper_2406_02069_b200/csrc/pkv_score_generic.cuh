@@ -29,7 +29,8 @@ struct ScoreParams {
   SeqTable seq;
   int32_t num_kv_heads, group, rows;     // rows = group * alpha
   float scale_log2;                      // log2(e) / sqrt(d)
-  float2* partial;                       // [sum_b chunks_b][H_kv][rows] (max, sum) per chunk
+  float2* partial;                       // [sum_b chunks_b][slots_per_chunk][H_kv][rows] (max, sum)
+  int32_t slots_per_chunk;               // partial slots each chunk writes (1 here, 2 for the tensor-core sweep)
   float* lse2;                           // [batch][H_kv][rows]
   float* scores;                         // [batch][H_kv][ld]
   int64_t ld_scores;
@@ -101,7 +102,7 @@ __global__ void __launch_bounds__(kGenRowBlock) rowstats_generic_kernel(const Sc
 // extra_log2 = log2(G) folds the mean over the group's query heads into the normaliser.
 __global__ void __launch_bounds__(256) combine_stats_kernel(const ScoreParams p, float extra_log2) {
   const int h = blockIdx.x, b = blockIdx.y;
-  const int t0 = p.seq.stat_off[b], t1 = p.seq.stat_off[b + 1];
+  const int t0 = p.seq.stat_off[b] * p.slots_per_chunk, t1 = p.seq.stat_off[b + 1] * p.slots_per_chunk;
   for (int r = threadIdx.x; r < p.rows; r += blockDim.x) {
     float m = -INFINITY;
     for (int t = t0; t < t1; ++t)

@@ -1,0 +1,477 @@
+// Window-score kernels on the sm_100a tensor cores (Section 4.2.2, Eq. 2 and Eq. 3), bf16 inputs.
+//
+// Two sweeps over K, because the score of a key sums softmax rows that each have
+// their own normaliser (known only after a whole row has been seen):
+//
+//   sweep A  D[row r][key i] = Q K^T   (A operand = window queries, B operand = key tile)
+//            TMEM lane = window row, so each epilogue thread owns one row and keeps its
+//            running max and sum of 2^x privately: no cross-thread reduction at all.
+//   sweep B  D[key i][row r] = K Q^T   (operands swapped)
+//            TMEM lane = key, so each epilogue thread owns one key and sums
+//            2^(x_ri - lse2_r) over the rows r, reading lse2 from shared memory.
+//
+// x = (q . k) * log2(e) / sqrt(d).  Operands arrive by TMA (no multicast) into
+// 128-byte-swizzled shared memory; tcgen05.mma accumulates in TMEM; epilogue warps
+// read TMEM with tcgen05.ld.  Warp roles: warp 0 = TMA producer, warp 1 = MMA
+// issuer and TMEM owner, warps 4..11 = epilogue.  CTAs are persistent: each takes
+// a contiguous range of (sequence, KV head, key chunk) work items.
+//
+// Every wait on an mbarrier is bounded.  A wait that runs out sets an abort flag in
+// shared memory and a status bit in the workspace; all roles then leave their loops,
+// the producer drains the copies it still has in flight, TMEM is released and the
+// kernel returns.
+#pragma once
+
+#include <cuda.h>
+
+#include "pkv_common.cuh"
+
+namespace pkv {
+
+constexpr int kTcThreads = 384;
+constexpr int kTcEpiWarp0 = 4;          // first epilogue warp
+constexpr int kTcEpiThreads = 256;
+constexpr int kTcTileKeys = 128;        // keys per MMA tile
+constexpr int kTcKStages = 4;           // shared-memory stages of K tiles
+constexpr int kTcMaxRows = 256;         // window rows (G * alpha) the tensor-core path takes
+constexpr uint32_t kTcSpinCap = 1u << 22;
+
+struct TcParams {
+  SeqTable seq;                 // stat_off / score_off count CHUNKS of chunk_tiles tiles
+  int32_t num_kv_heads, group, rows;      // rows = group * alpha (R)
+  int32_t rows_pad;             // R rounded up to 32
+  int32_t row_blocks;           // ceil(R / 128): M-blocks of sweep A
+  int32_t chunk_tiles;          // key tiles per work item
+  float scale_log2;             // log2(e) / sqrt(d)
+  float2* partial;              // sweep A out: [chunk][2][H_kv][R] (max, sum) in the log2 domain; the two
+                                // epilogue warp groups each write their own slot of a chunk
+  const float* lse2;            // sweep B in:  [batch][H_kv][R]
+  float* scores;                // sweep B out: [batch][H_kv][ld]
+  int64_t ld_scores;
+  uint32_t* status;
+};
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: polls without blocking, backs off after the first polls, and gives up after
+// kTcSpinCap polls (of the order of a second).  Returns false if it gave up, or if another
+// thread did (abort flag).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  for (uint32_t it = 0; it < kTcSpinCap; ++it) {
+    if (mbar_test(bar, parity)) return true;
+    if (it >= 64u) {
+      __nanosleep(100);
+      if ((it & 255u) == 255u && *abort_flag) return false;
+    }
+  }
+  *abort_flag = 1;
+  return false;
+}
+
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
+                                            int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+        "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+        "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// Shared-memory matrix descriptor of a K-major bf16 operand whose rows are 128 bytes wide and
+// stored with the 128-byte swizzle: 8-row groups are 1024 bytes apart.  `addr` is the byte address
+// of the first row, plus 32 bytes per 16-element step along the contraction dimension.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((addr & 0x3FFFFu) >> 4);          // start address
+  d |= static_cast<uint64_t>(1) << 16;                         // leading byte offset (unused with swizzle), 16 B
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;                 // stride byte offset: 1024 B between 8-row groups
+  d |= static_cast<uint64_t>(1) << 46;                         // descriptor version of this architecture
+  d |= static_cast<uint64_t>(2) << 61;                         // 128-byte swizzle
+  return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M x N tile.
+__device__ __forceinline__ uint32_t instr_desc_bf16(int M, int N) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(N >> 3) << 17) |
+         (static_cast<uint32_t>(M >> 4) << 24);
+}
+
+// Work item -> (sequence, head, chunk).  Items are ordered sequence, head, chunk.
+struct TcItem { int b, h, c, nchunks; };
+__device__ __forceinline__ TcItem tc_item(const int32_t* off, int batch, int heads, int id) {
+  int b = 0;
+  while (b + 1 < batch && id >= heads * off[b + 1]) ++b;
+  const int local = id - heads * off[b];
+  const int nc = off[b + 1] - off[b];
+  return TcItem{b, local / nc, local % nc, nc};
+}
+
+// Dynamic shared memory carve-up (bytes), all regions 1024-aligned.
+template <int D>
+struct TcSmem {
+  static constexpr int kHalves = D / 64;                       // 64-element (128-byte) column blocks
+  static constexpr int kQBytes = kTcMaxRows * D * 2;
+  static constexpr int kKStageBytes = kTcTileKeys * D * 2;
+  static constexpr int kQOff = 0;
+  static constexpr int kKOff = kQBytes;
+  static constexpr int kMiscOff = kKOff + kTcKStages * kKStageBytes;
+  static constexpr int kMiscBytes = 12288;                     // barriers, per-warp copies of lse2
+  static constexpr int kTotal = kMiscOff + kMiscBytes + 1024;  // + slack for manual 1024-byte alignment
+};
+
+// SWEEP 0 = row statistics (A), 1 = scores (B).
+template <int D, int SWEEP>
+__global__ void __launch_bounds__(kTcThreads, 1)
+score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
+                const TcParams p) {
+  using L = TcSmem<D>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* q_s = smem + L::kQOff;
+  uint8_t* k_s = smem + L::kKOff;
+  uint8_t* misc = smem + L::kMiscOff;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(misc);          // [0..3] k_full, [4..7] k_empty, [8..11] t_full,
+                                                               // [12..15] t_empty, [16] q_full, [17] q_empty
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 256);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 260);
+  float* lse_all = reinterpret_cast<float*>(misc + 1024);      // sweep B: [8 warps][256] lse2 of the current head
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t bar0 = smem_u32(bars);
+  auto k_full = [&](int s) { return bar0 + 8u * s; };
+  auto k_empty = [&](int s) { return bar0 + 8u * (4 + s); };
+  auto t_full = [&](int s) { return bar0 + 8u * (8 + s); };
+  auto t_empty = [&](int s) { return bar0 + 8u * (12 + s); };
+  const uint32_t q_full = bar0 + 8u * 16, q_empty = bar0 + 8u * 17;
+
+  // TMEM stages: sweep A holds row_blocks x 128 key columns per stage, sweep B rows_pad columns.
+  int stage_cols = SWEEP == 0 ? p.row_blocks * 128 : p.rows_pad;
+  if (stage_cols <= 32) stage_cols = 32; else if (stage_cols <= 64) stage_cols = 64;
+  else if (stage_cols <= 128) stage_cols = 128; else stage_cols = 256;
+  const int t_stages = min(4, 512 / stage_cols);
+
+  // ---- set-up
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kTcKStages; ++s) { mbar_init(k_full(s), 1); mbar_init(k_empty(s), 1); }
+    const uint32_t consumers = (SWEEP == 0 && p.row_blocks == 2) ? 8 : 4;   // epilogue warps that read one tile
+    for (int s = 0; s < 4; ++s) { mbar_init(t_full(s), 1); mbar_init(t_empty(s), consumers); }
+    mbar_init(q_full, 1);
+    mbar_init(q_empty, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  // rows of the Q tile beyond R stay zero for the whole kernel (TMA only ever writes R rows)
+  for (int i = threadIdx.x; i < L::kQBytes / 16; i += kTcThreads) reinterpret_cast<uint4*>(q_s)[i] = make_uint4(0, 0, 0, 0);
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  // ---- this CTA's contiguous range of work items
+  const int32_t* off = SWEEP == 0 ? p.seq.stat_off : p.seq.score_off;
+  const int total = p.num_kv_heads * off[p.seq.batch];
+  const int per = total / gridDim.x, rem = total % gridDim.x;
+  const int item0 = blockIdx.x * per + min(static_cast<int>(blockIdx.x), rem);
+  const int item1 = item0 + per + (static_cast<int>(blockIdx.x) < rem ? 1 : 0);
+  // keys an item of sequence b spans: sweep A covers all n keys, sweep B the prefix only
+  auto span_keys = [&](int b) { return SWEEP == 0 ? p.seq.n[b] : p.seq.n[b] - p.seq.alpha; };
+
+  if (warp == 0) {
+    // =========================================================== TMA producer
+    if (lane == 0) {
+      uint32_t it = 0, heads_loaded = 0;
+      int cur_b = -1, cur_h = -1;
+      bool ok = true;
+      for (int id = item0; id < item1 && ok; ++id) {
+        const TcItem w = tc_item(off, p.seq.batch, p.num_kv_heads, id);
+        if (w.b != cur_b || w.h != cur_h) {
+          if (heads_loaded > 0) ok = mbar_wait(q_empty, (heads_loaded - 1) & 1, abort_flag);
+          if (!ok) break;
+          mbar_expect_tx(q_full, static_cast<uint32_t>(p.rows) * D * 2);
+          for (int half = 0; half < L::kHalves; ++half)
+            tma_load_4d(smem_u32(q_s) + half * kTcMaxRows * 128, &q_map, q_full, half * 64, 0, w.h * p.group, w.b);
+          ++heads_loaded;
+          cur_b = w.b; cur_h = w.h;
+        }
+        const int keys = span_keys(w.b);
+        const int tile0 = w.c * p.chunk_tiles;
+        const int tile1 = min(tile0 + p.chunk_tiles, (keys + kTcTileKeys - 1) / kTcTileKeys);
+        for (int t = tile0; t < tile1 && ok; ++t, ++it) {
+          const int s = it % kTcKStages;
+          ok = mbar_wait(k_empty(s), ((it / kTcKStages) & 1) ^ 1, abort_flag);
+          if (!ok) break;
+          mbar_expect_tx(k_full(s), L::kKStageBytes);
+          for (int half = 0; half < L::kHalves; ++half)
+            tma_load_4d(smem_u32(k_s) + s * L::kKStageBytes + half * kTcTileKeys * 128, &k_map, k_full(s), half * 64,
+                        t * kTcTileKeys, w.h, w.b);
+        }
+      }
+      if (!ok) {
+        // drain: wait (bounded) for the copies still in flight before shared memory is given up
+        const uint32_t first = it > kTcKStages ? it - kTcKStages : 0;
+        for (uint32_t j = first; j < it; ++j)
+          for (uint32_t spin = 0; spin < (1u << 16) && !mbar_test(k_full(j % kTcKStages), (j / kTcKStages) & 1); ++spin)
+            __nanosleep(64);
+        if (heads_loaded > 0)
+          for (uint32_t spin = 0; spin < (1u << 16) && !mbar_test(q_full, (heads_loaded - 1) & 1); ++spin) __nanosleep(64);
+      }
+    }
+  } else if (warp == 1) {
+    // =========================================================== MMA issuer
+    if (lane == 0) {
+      uint32_t it = 0, heads_seen = 0;
+      int cur_b = -1, cur_h = -1;
+      bool ok = true;
+      const uint32_t idesc = SWEEP == 0 ? instr_desc_bf16(128, kTcTileKeys) : instr_desc_bf16(kTcTileKeys, p.rows_pad);
+      for (int id = item0; id < item1 && ok; ++id) {
+        const TcItem w = tc_item(off, p.seq.batch, p.num_kv_heads, id);
+        if (w.b != cur_b || w.h != cur_h) {
+          ok = mbar_wait(q_full, heads_seen & 1, abort_flag);
+          if (!ok) break;
+          ++heads_seen;
+          cur_b = w.b; cur_h = w.h;
+        }
+        // does the next item belong to another head?  then Q may be overwritten after this item's MMAs
+        bool last_of_head = id + 1 >= item1;
+        if (!last_of_head) {
+          const TcItem nx = tc_item(off, p.seq.batch, p.num_kv_heads, id + 1);
+          last_of_head = nx.b != w.b || nx.h != w.h;
+        }
+        const int keys = span_keys(w.b);
+        const int tile0 = w.c * p.chunk_tiles;
+        const int tile1 = min(tile0 + p.chunk_tiles, (keys + kTcTileKeys - 1) / kTcTileKeys);
+        for (int t = tile0; t < tile1 && ok; ++t, ++it) {
+          const int s = it % kTcKStages, ts = it % t_stages;
+          ok = mbar_wait(k_full(s), (it / kTcKStages) & 1, abort_flag) &&
+               mbar_wait(t_empty(ts), ((it / t_stages) & 1) ^ 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t k_addr = smem_u32(k_s) + s * L::kKStageBytes;
+          const uint32_t q_addr = smem_u32(q_s);
+          const uint32_t d_addr = tmem_base + ts * stage_cols;
+          if (SWEEP == 0) {
+            for (int mb = 0; mb < p.row_blocks; ++mb)
+#pragma unroll
+              for (int kk = 0; kk < D / 16; ++kk) {
+                const uint32_t qa = q_addr + (kk / 4) * kTcMaxRows * 128 + mb * 128 * 128 + (kk % 4) * 32;
+                const uint32_t ka = k_addr + (kk / 4) * kTcTileKeys * 128 + (kk % 4) * 32;
+                tc_mma_bf16(d_addr + mb * 128, smem_desc_sw128(qa), smem_desc_sw128(ka), idesc, kk > 0);
+              }
+          } else {
+#pragma unroll
+            for (int kk = 0; kk < D / 16; ++kk) {
+              const uint32_t qa = q_addr + (kk / 4) * kTcMaxRows * 128 + (kk % 4) * 32;
+              const uint32_t ka = k_addr + (kk / 4) * kTcTileKeys * 128 + (kk % 4) * 32;
+              tc_mma_bf16(d_addr, smem_desc_sw128(ka), smem_desc_sw128(qa), idesc, kk > 0);
+            }
+          }
+          tc_commit(k_empty(s));
+          tc_commit(t_full(ts));
+        }
+        if (ok && last_of_head) tc_commit(q_empty);
+      }
+    }
+  } else if (warp >= kTcEpiWarp0) {
+    // =========================================================== epilogue
+    const int e = warp - kTcEpiWarp0;
+    const int quarter = warp & 3;               // TMEM lanes 32*quarter .. +31 are this warp's
+    const int half = e >> 2;                    // which half of the work of a lane this warp takes
+    const int lane_row = quarter * 32 + lane;   // TMEM lane of this thread
+    const float c2 = p.scale_log2;
+    uint32_t it = 0;
+    int cur_b = -1, cur_h = -1;
+    bool ok = true;
+    for (int id = item0; id < item1 && ok; ++id) {
+      const TcItem w = tc_item(off, p.seq.batch, p.num_kv_heads, id);
+      const int n = p.seq.n[w.b], alpha = p.seq.alpha, P = n - alpha;
+      const int keys = span_keys(w.b);
+      const int tile0 = w.c * p.chunk_tiles;
+      const int tile1 = min(tile0 + p.chunk_tiles, (keys + kTcTileKeys - 1) / kTcTileKeys);
+      if (SWEEP == 0) {
+        // thread -> window row.  Two row blocks: each warp group owns one block and sees every tile.
+        // One row block: the groups take alternate tiles of the same 128 rows.  Either way each group
+        // writes its own partial slot, so no exchange between warps is needed.
+        const bool two = p.row_blocks == 2;
+        const int r = (two ? half * 128 : 0) + lane_row;
+        const int last_visible = P + (r % alpha);             // row (g, j) sees keys 0 .. P + j
+        float m = -INFINITY, z = 0.f;
+        for (int t = tile0; t < tile1 && ok; ++t, ++it) {
+          if (!two && static_cast<int>(it & 1u) != half) continue;   // the other group's tile
+          const int ts = it % t_stages;
+          ok = mbar_wait(t_full(ts), (it / t_stages) & 1, abort_flag);
+          ok = __all_sync(0xffffffffu, ok);                   // whole warp proceeds together or not at all
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + ts * stage_cols +
+                                 (two ? half * 128 : 0);
+          const int key_base = t * kTcTileKeys;
+          const bool masked = key_base + kTcTileKeys - 1 > P; // tile reaches into the window: per-element mask
+          for (int cg = 0; cg < kTcTileKeys; cg += 32) {
+            uint32_t v[32];
+            tc_ld32(taddr + cg, v);
+            tc_wait_ld();
+            if (!masked) {
+              float gm = __uint_as_float(v[0]);
+#pragma unroll
+              for (int j = 1; j < 32; ++j) gm = fmaxf(gm, __uint_as_float(v[j]));
+              const float mn = fmaxf(m, gm * c2);
+              z *= ex2(m - mn);
+              m = mn;
+              float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+              for (int j = 0; j < 32; j += 4) {
+                a0 += ex2(fmaf(__uint_as_float(v[j]), c2, -m));
+                a1 += ex2(fmaf(__uint_as_float(v[j + 1]), c2, -m));
+                a2 += ex2(fmaf(__uint_as_float(v[j + 2]), c2, -m));
+                a3 += ex2(fmaf(__uint_as_float(v[j + 3]), c2, -m));
+              }
+              z += (a0 + a1) + (a2 + a3);
+            } else {
+              float gm = -INFINITY;
+#pragma unroll
+              for (int j = 0; j < 32; ++j) {
+                const bool vis = key_base + cg + j <= last_visible;
+                const float x = vis ? __uint_as_float(v[j]) * c2 : -INFINITY;
+                v[j] = __float_as_uint(x);
+                gm = fmaxf(gm, x);
+              }
+              if (gm > -INFINITY) {
+                const float mn = fmaxf(m, gm);
+                z *= ex2(m - mn);
+                m = mn;
+                float a0 = 0.f;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) a0 += ex2(__uint_as_float(v[j]) - m);
+                z += a0;
+              }
+            }
+          }
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(t_empty(ts));
+        }
+        if (!ok) break;
+        if (r < p.rows) {
+          const int64_t chunk = off[w.b] + w.c;
+          float2* slot0 = p.partial + ((chunk * 2 + 0) * p.num_kv_heads + w.h) * p.rows;
+          float2* slot1 = p.partial + ((chunk * 2 + 1) * p.num_kv_heads + w.h) * p.rows;
+          if (two) {                                          // this group alone saw row r
+            slot0[r] = make_float2(m, z);
+            slot1[r] = make_float2(-INFINITY, 0.f);
+          } else {
+            (half == 0 ? slot0 : slot1)[r] = make_float2(m, z);
+          }
+        }
+      } else {
+        // thread -> key; the two warp groups take alternate tiles, each thread sums all rows of its key
+        float* lse_s = lse_all + e * 256;                     // this warp's private copy of lse2
+        if (w.b != cur_b || w.h != cur_h) {
+          __syncwarp();
+          const float* src = p.lse2 + (static_cast<int64_t>(w.b) * p.num_kv_heads + w.h) * p.rows;
+          for (int i = lane; i < 256; i += 32) lse_s[i] = i < p.rows ? src[i] : INFINITY;
+          __syncwarp();
+          cur_b = w.b; cur_h = w.h;
+        }
+        float* srow = p.scores + (static_cast<int64_t>(w.b) * p.num_kv_heads + w.h) * p.ld_scores;
+        for (int t = tile0; t < tile1 && ok; ++t, ++it) {
+          if (static_cast<int>(it & 1u) != half) continue;    // the other group's tile
+          const int ts = it % t_stages;
+          ok = mbar_wait(t_full(ts), (it / t_stages) & 1, abort_flag);
+          ok = __all_sync(0xffffffffu, ok);                   // whole warp proceeds together or not at all
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + ts * stage_cols;
+          float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+          for (int cg = 0; cg < p.rows_pad; cg += 32) {
+            uint32_t v[32];
+            tc_ld32(taddr + cg, v);
+            tc_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 32; j += 4) {
+              const float4 l4 = *reinterpret_cast<const float4*>(&lse_s[cg + j]);
+              a0 += ex2(fmaf(__uint_as_float(v[j]), c2, -l4.x));
+              a1 += ex2(fmaf(__uint_as_float(v[j + 1]), c2, -l4.y));
+              a2 += ex2(fmaf(__uint_as_float(v[j + 2]), c2, -l4.z));
+              a3 += ex2(fmaf(__uint_as_float(v[j + 3]), c2, -l4.w));
+            }
+          }
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(t_empty(ts));
+          const int i = t * kTcTileKeys + lane_row;
+          if (i < P) srow[i] = (a0 + a1) + (a2 + a3);
+        }
+        if (!ok) break;
+      }
+    }
+  }
+
+  // ---- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag) atomicOr(p.status, kStatusWaitExpired);
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+  }
+}
+
+}  // namespace pkv

@@ -56,6 +56,35 @@ def test_scores_match_oracle(w):
             assert (scores[b, :, n - w.window:] == -1.0).all()        # nothing written past the prefix
 
 
+@pytest.mark.parametrize("hq,hkv,alpha,d,lens", [
+    (3, 3, 8, 64, [700]),                 # R = 8, head_dim 64
+    (12, 4, 8, 64, [129, 1000, 136]),     # R = 24, ragged, one sequence barely longer than a tile
+    (8, 2, 48, 128, [2000, 333]),         # R = 192: two row blocks, padded
+    (16, 2, 32, 128, [1500]),             # R = 256
+    (4, 4, 1, 128, [300]),                # alpha = 1
+    (8, 1, 16, 128, [16 + 1, 16 + 128, 16 + 129]),   # prefix of 1, of one tile, of one tile + 1
+])
+def test_scores_bf16_shapes(hq, hkv, alpha, d, lens):
+    """Tensor-core score path over window sizes, group sizes, head dims and ragged tails."""
+    cfg = pkv.make_config(num_layers=1, num_q_heads=hq, num_kv_heads=hkv, head_dim=d, window=alpha, pool_kernel=3,
+                          dtype="bf16", avg_budget=alpha, beta=1.0)
+    g = torch.Generator(device="cpu").manual_seed(hq * 100 + alpha)
+    n_max = max(lens)
+    q = (torch.randn(len(lens), hq, alpha, d, generator=g) * 1.5).to(torch.bfloat16)
+    k = torch.randn(len(lens), hkv, n_max, d, generator=g).to(torch.bfloat16)
+    k[:, :, 0] *= 3.0
+    ws = pkv.new_workspace(cfg, len(lens), n_max, DEV)
+    scores = torch.full((len(lens), hkv, n_max), -1.0, dtype=torch.float32, device=DEV)
+    for rep in range(2):                                            # second run reuses the workspace
+        pkv.score_window(cfg, q.to(DEV), k.to(DEV), lens, scores, ws)
+        pkv.check_status(ws)
+    got = scores.cpu().numpy()
+    for b, n in enumerate(lens):
+        want, _ = oracle.window_scores(q[b], k[b, :, :n])
+        assert_scores_close(got[b, :, : n - alpha], want, "seq %d" % b)
+        assert (got[b, :, n - alpha:] == -1.0).all()
+
+
 @pytest.mark.parametrize("P,k,w", [(1, 1, 1), (5, 2, 7), (33, 32, 3), (100, 0, 5), (100, 100, 5), (100, 250, 5),
                                    (1000, 37, 7), (4064, 188, 7), (8193, 500, 7), (20000, 4, 7), (40000, 937, 7),
                                    (131040, 188, 7), (70001, 2016, 1)])
