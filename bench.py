@@ -200,6 +200,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama3_70b_128k")
     ap.add_argument("--budget", type=int, default=None, help="override the average budget B")
+    ap.add_argument("--layers", type=int, default=None, help="profile aid: only the first N layers (named in config)")
+    ap.add_argument("--seq-len", type=int, default=None, help="profile aid: override the sequence length")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--host-ring", type=int, default=4, help="distinct pinned host layers cycled by the e2e leg")
     ap.add_argument("--no-e2e", action="store_true")
@@ -211,6 +213,10 @@ def main():
     w = workloads.WORKLOADS[args.workload]
     if args.budget:
         w = workloads.with_budget(w, args.budget)
+    if args.layers or args.seq_len:
+        w = workloads.scaled(w, num_layers=args.layers, seq_len=args.seq_len,
+                             name="%s[layers=%s,seq_len=%s]" % (w.name, args.layers or w.num_layers,
+                                                                args.seq_len or w.seq_len_hi))
     if args.impl == "reference":
         run_reference(args, w)
         return

@@ -157,7 +157,7 @@ int launch_scores_generic(ScoreParams& sp, int batch, cudaStream_t st) {
   sp.slots_per_chunk = 1;
   rowstats_generic_kernel<T, D><<<dim3(stat_tiles, sp.num_kv_heads), kGenRowBlock, 0, st>>>(sp);
   mark(st, "rowstats_generic");
-  combine_stats_kernel<<<dim3(sp.num_kv_heads, batch), 256, 0, st>>>(sp, std::log2(static_cast<float>(sp.group)));
+  combine_stats_kernel<<<dim3((sp.rows + 31) / 32, sp.num_kv_heads, batch), 256, 0, st>>>(sp, std::log2(static_cast<float>(sp.group)));
   mark(st, "combine_stats");
   scores_generic_kernel<T, D><<<dim3(score_tiles, sp.num_kv_heads), kGenScoreKeys, 0, st>>>(sp);
   mark(st, "scores_generic");
@@ -281,7 +281,7 @@ int launch_scores_tc(const pkv_config* c, const pkv_tensor& q, const pkv_tensor&
   const int grid_b = static_cast<int>(std::min<long long>(sms, static_cast<long long>(score_items) * sp.num_kv_heads));
   score_tc_kernel<D, 0><<<grid_a, kTcThreads, TcSmem<D>::kTotal, st>>>(q_map, k_map, tp);
   mark(st, "rowstats_tc");
-  combine_stats_kernel<<<dim3(sp.num_kv_heads, batch), 256, 0, st>>>(sp, std::log2(static_cast<float>(sp.group)));
+  combine_stats_kernel<<<dim3((sp.rows + 31) / 32, sp.num_kv_heads, batch), 256, 0, st>>>(sp, std::log2(static_cast<float>(sp.group)));
   mark(st, "combine_stats");
   score_tc_kernel<D, 1><<<grid_b, kTcThreads, TcSmem<D>::kTotal, st>>>(q_map, k_map, tp);
   mark(st, "scores_tc");

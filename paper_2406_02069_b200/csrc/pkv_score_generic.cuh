@@ -98,21 +98,38 @@ __global__ void __launch_bounds__(kGenRowBlock) rowstats_generic_kernel(const Sc
   }
 }
 
-// grid (H_kv, batch), block 256: merge the chunk partials of each window row.
-// extra_log2 = log2(G) folds the mean over the group's query heads into the normaliser.
+// grid (ceil(rows / 32), H_kv, batch), block 256: merge the chunk partials of each window row.
+// Thread (rl, sg) = (tid % 32, tid / 32) takes row r0 + rl and every 8th partial slot starting at sg, so
+// a warp reads 32 consecutive rows of one slot (256 contiguous bytes); the 8 slot groups of a row are
+// merged through shared memory.  extra_log2 = log2(G) folds the mean over the group's query heads
+// into the normaliser.
 __global__ void __launch_bounds__(256) combine_stats_kernel(const ScoreParams p, float extra_log2) {
-  const int h = blockIdx.x, b = blockIdx.y;
+  __shared__ float sm[8][32], sz[8][32];
+  const int h = blockIdx.y, b = blockIdx.z;
+  const int rl = threadIdx.x & 31, sg = threadIdx.x >> 5;
+  const int r = blockIdx.x * 32 + rl;
   const int t0 = p.seq.stat_off[b] * p.slots_per_chunk, t1 = p.seq.stat_off[b + 1] * p.slots_per_chunk;
-  for (int r = threadIdx.x; r < p.rows; r += blockDim.x) {
-    float m = -INFINITY;
-    for (int t = t0; t < t1; ++t)
-      m = fmaxf(m, p.partial[(static_cast<int64_t>(t) * p.num_kv_heads + h) * p.rows + r].x);
-    float z = 0.f;
-    for (int t = t0; t < t1; ++t) {
+  float m = -INFINITY, z = 0.f;
+  if (r < p.rows) {
+    for (int t = t0 + sg; t < t1; t += 8) {
       const float2 pz = p.partial[(static_cast<int64_t>(t) * p.num_kv_heads + h) * p.rows + r];
-      z += pz.y * exp2f(pz.x - m);
+      if (pz.x > -INFINITY) {                      // (-inf, 0) marks a slot that saw no key of this row
+        const float mn = fmaxf(m, pz.x);
+        z = z * exp2f(m - mn) + pz.y * exp2f(pz.x - mn);
+        m = mn;
+      }
     }
-    p.lse2[(static_cast<int64_t>(b) * p.num_kv_heads + h) * p.rows + r] = m + log2f(z) + extra_log2;
+  }
+  sm[sg][rl] = m;
+  sz[sg][rl] = z;
+  __syncthreads();
+  if (sg == 0 && r < p.rows) {
+    float mm = -INFINITY;
+    for (int g = 0; g < 8; ++g) mm = fmaxf(mm, sm[g][rl]);
+    float zz = 0.f;
+    for (int g = 0; g < 8; ++g)
+      if (sm[g][rl] > -INFINITY) zz += sz[g][rl] * exp2f(sm[g][rl] - mm);
+    p.lse2[(static_cast<int64_t>(b) * p.num_kv_heads + h) * p.rows + r] = mm + log2f(zz) + extra_log2;
   }
 }
 

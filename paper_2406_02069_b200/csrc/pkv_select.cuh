@@ -4,11 +4,14 @@
 // split into contiguous slices, one per CTA of the cluster; each CTA pools its
 // slice (reading a halo of (w-1)/2 scores on both sides) and keeps the pooled
 // values in shared memory as order-preserving 32-bit keys.  The k-th largest key
-// is found by a most-significant-digit radix search (4 passes of 8 bits): every
-// CTA histograms its slice, the histograms are summed across the cluster through
-// distributed shared memory, and every CTA walks the summed histogram to the same
-// digit.  Ties at the threshold go to the smaller position, and kept positions
-// are written in ascending order, so the result is one canonical list:
+// is found by a most-significant-digit radix search in three passes (11, 11 and
+// 10 bits): every CTA histograms its slice, the histograms are summed across the
+// cluster through distributed shared memory, and every CTA walks the summed
+// histogram to the same digit.  While summing, a CTA also accumulates the
+// histograms of the CTAs that own earlier positions, which gives it, with no
+// further exchange, how many kept keys precede its slice.  Ties at the threshold
+// go to the smaller position and kept positions are written in ascending order,
+// so the result is one canonical list:
 //   kept = { i : key_i > T }  plus the leftmost (k - |{key > T}|) positions with key_i == T.
 // The alpha window positions are appended after them.
 //
@@ -52,15 +55,17 @@ __device__ __forceinline__ uint32_t pooled_key(const float* s, int i, int P, int
   return ordered_key(best);
 }
 
+constexpr int kSelBins = 2048;
+
 // grid (cluster * H_kv, batch), cluster (cluster, 1, 1), block kSelThreads,
 // dynamic shared memory slice_cap * 4 bytes.
 __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectParams p) {
   extern __shared__ __align__(16) uint32_t keys[];          // this CTA's pooled keys (if cached)
-  __shared__ uint32_t hist[2][256];                         // per-pass digit histogram (double buffered)
-  __shared__ uint32_t total[256];                           // histogram summed over the cluster
+  __shared__ uint32_t hist[2][kSelBins];                    // per-pass digit histogram (double buffered)
+  __shared__ uint32_t lower[kSelBins];                      // ... summed over the CTAs of lower rank only
+  __shared__ uint32_t warp_sum[kSelWarps];
   __shared__ uint32_t warp_gt[kSelWarps], warp_eq[kSelWarps];
-  __shared__ uint32_t cta_cnt[2];                           // (greater, equal) counts of this CTA
-  __shared__ uint32_t sel_digit, sel_above;
+  __shared__ uint32_t sel_digit, sel_above, lower_above;
 
   cg::cluster_group cluster = cg::this_cluster();
   const int C = cluster.dim_blocks().x;
@@ -92,60 +97,70 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
   auto key_at = [&](int i) -> uint32_t {
     return cached ? keys[i - lo] : pooled_key(s, i, P, p.pool_radius);
   };
-  for (int i = tid; i < 512; i += kSelThreads) (&hist[0][0])[i] = 0;
+  for (int i = tid; i < 2 * kSelBins; i += kSelThreads) (&hist[0][0])[i] = 0;
   __syncthreads();
 
   // ---- radix search for the k-th largest key
   uint32_t prefix = 0, mask = 0, remaining = k;
-  for (int pass = 0; pass < 4; ++pass) {
-    const int shift = 24 - 8 * pass;
+  uint32_t gt_before_cta = 0, eq_before_cta = 0;            // kept-candidate keys owned by lower-rank CTAs
+  for (int pass = 0; pass < 3; ++pass) {
+    const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
+    const uint32_t dmask = pass == 2 ? 1023u : 2047u;
     uint32_t* hcur = hist[pass & 1];
     for (int base = lo + warp * 32; base < hi; base += kSelThreads) {
       const int i = base + lane;
-      uint32_t digit = 256;                                 // 256 = does not take part
+      uint32_t digit = kSelBins;                            // kSelBins = does not take part
       if (i < hi) {
         const uint32_t key = key_at(i);
-        if ((key & mask) == prefix) digit = (key >> shift) & 255u;
+        if ((key & mask) == prefix) digit = (key >> shift) & dmask;
       }
       const uint32_t peers = __match_any_sync(0xffffffffu, digit);
-      if (digit < 256 && lane == __ffs(peers) - 1) atomicAdd(&hcur[digit], __popc(peers));
+      if (digit < kSelBins && lane == __ffs(peers) - 1) atomicAdd(&hcur[digit], __popc(peers));
     }
     cluster.sync();                                         // all histograms of this pass complete
-    if (tid < 256) {
-      uint32_t t = 0;
-      for (int c = 0; c < C; ++c) t += cluster.map_shared_rank(hcur, c)[tid];
-      total[tid] = t;
-      hist[(pass + 1) & 1][tid] = 0;                        // next pass's buffer: last read two syncs ago
+    // every thread owns two adjacent digits
+    uint32_t tot[2] = {0, 0}, low[2] = {0, 0};
+    for (int c = 0; c < C; ++c) {
+      const uint2 v = reinterpret_cast<const uint2*>(cluster.map_shared_rank(hcur, c))[tid];
+      tot[0] += v.x; tot[1] += v.y;
+      if (c < rank) { low[0] += v.x; low[1] += v.y; }
+    }
+    lower[2 * tid] = low[0]; lower[2 * tid + 1] = low[1];
+    reinterpret_cast<uint2*>(hist[(pass + 1) & 1])[tid] = make_uint2(0, 0);   // next pass's buffer
+    // keys in digits above this thread's pair: suffix sums inside the warp, then over warps
+    const uint32_t mine = tot[0] + tot[1];
+    uint32_t incl = mine;
+    for (int off = 1; off < 32; off <<= 1) {
+      const uint32_t v = __shfl_down_sync(0xffffffffu, incl, off);
+      if (lane + off < 32) incl += v;
+    }
+    if (lane == 0) warp_sum[warp] = incl;
+    if (tid == 0) lower_above = 0;
+    __syncthreads();
+    uint32_t higher = incl - mine;
+    for (int w2 = warp + 1; w2 < kSelWarps; ++w2) higher += warp_sum[w2];
+    if (higher < remaining && remaining <= higher + mine) {  // exactly one thread: the k-th key is in its pair
+      if (higher + tot[1] >= remaining) { sel_digit = 2 * tid + 1; sel_above = higher; }
+      else { sel_digit = 2 * tid; sel_above = higher + tot[1]; }
     }
     __syncthreads();
-    if (warp == 0) {
-      // lane L owns digits 8L .. 8L+7; find the digit where the count from the top reaches `remaining`
-      uint32_t mine = 0;
-      for (int t = 0; t < 8; ++t) mine += total[lane * 8 + t];
-      uint32_t above = mine;                                // inclusive suffix sum over lanes
-      for (int off = 1; off < 32; off <<= 1) {
-        const uint32_t v = __shfl_down_sync(0xffffffffu, above, off);
-        if (lane + off < 32) above += v;
-      }
-      const uint32_t higher = above - mine;                 // keys in digits owned by higher lanes
-      if (higher < remaining && remaining <= above) {
-        uint32_t acc = higher;
-        for (int t = 7; t >= 0; --t) {
-          const uint32_t c = total[lane * 8 + t];
-          if (acc + c >= remaining) { sel_digit = lane * 8 + t; sel_above = acc; break; }
-          acc += c;
-        }
-      }
-    }
+    const uint32_t dsel = sel_digit;
+    // lower-rank keys in digits above the selected one are all kept: they precede this CTA's output
+    uint32_t la = (2u * tid > dsel ? low[0] : 0u) + (2u * tid + 1u > dsel ? low[1] : 0u);
+    for (int off = 16; off > 0; off >>= 1) la += __shfl_down_sync(0xffffffffu, la, off);
+    if (lane == 0 && la) atomicAdd(&lower_above, la);
     __syncthreads();
-    prefix |= sel_digit << shift;
-    mask |= 255u << shift;
+    gt_before_cta += lower_above;
+    if (pass == 2) eq_before_cta = lower[dsel];
+    prefix |= dsel << shift;
+    mask |= dmask << shift;
     remaining -= sel_above;
+    __syncthreads();                                        // sel_* and lower_above are rewritten next pass
   }
   const uint32_t T = prefix;                                // the k-th largest key
   const uint32_t need_eq = remaining;                       // ties at T to take, from the left
 
-  // ---- count keys above / at the threshold: warp w owns a contiguous run of the slice
+  // ---- keys above / at the threshold inside this CTA: warp w owns a contiguous run of the slice
   const int run = ((slice / kSelWarps) + 31) & ~31;
   const int wlo = min(hi, lo + warp * run), whi = min(hi, wlo + run);
   uint32_t ngt = 0, neq = 0;
@@ -157,28 +172,12 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
   }
   if (lane == 0) { warp_gt[warp] = ngt; warp_eq[warp] = neq; }
   __syncthreads();
-  if (warp == 0) {
-    uint32_t g = warp_gt[lane], e = warp_eq[lane];
-    const uint32_t g0 = g, e0 = e;
-    for (int off = 1; off < 32; off <<= 1) {
-      const uint32_t vg = __shfl_up_sync(0xffffffffu, g, off), ve = __shfl_up_sync(0xffffffffu, e, off);
-      if (lane >= off) { g += vg; e += ve; }
-    }
-    warp_gt[lane] = g - g0;                                 // exclusive prefix inside the CTA
-    warp_eq[lane] = e - e0;
-    if (lane == 31) { cta_cnt[0] = g; cta_cnt[1] = e; }
+  uint32_t gt_before = gt_before_cta, eq_before = eq_before_cta;
+  for (int w2 = 0; w2 < warp; ++w2) { gt_before += warp_gt[w2]; eq_before += warp_eq[w2]; }
+  if (rank == C - 1 && tid == kSelThreads - 1) {            // the last thread can see the grand total
+    if (gt_before + ngt + min(eq_before + neq, need_eq) != static_cast<uint32_t>(k))
+      atomicOr(p.status, kStatusSelectMismatch);
   }
-  cluster.sync();                                           // counts of every CTA visible
-  uint32_t gt_before = warp_gt[warp], eq_before = warp_eq[warp];
-  uint32_t all_gt = 0;
-  for (int c = 0; c < C; ++c) {
-    const uint32_t* rc = cluster.map_shared_rank(cta_cnt, c);
-    const uint32_t g = rc[0], e = rc[1];
-    if (c < rank) { gt_before += g; eq_before += e; }
-    all_gt += g;
-  }
-  if (rank == 0 && tid == 0 && all_gt + need_eq != static_cast<uint32_t>(k))
-    atomicOr(p.status, kStatusSelectMismatch);
 
   // ---- emit in ascending position: rank of i among the kept = (#greater before i) + min(#equal before i, need_eq)
   for (int base = wlo; base < whi; base += 32) {
