@@ -157,7 +157,7 @@ int launch_scores_generic(ScoreParams& sp, int batch, cudaStream_t st) {
   sp.slots_per_chunk = 1;
   rowstats_generic_kernel<T, D><<<dim3(stat_tiles, sp.num_kv_heads), kGenRowBlock, 0, st>>>(sp);
   mark(st, "rowstats_generic");
-  combine_stats_kernel<<<dim3((sp.rows + 31) / 32, sp.num_kv_heads, batch), 256, 0, st>>>(sp, std::log2(static_cast<float>(sp.group)));
+  combine_stats_kernel<<<dim3((sp.rows + 31) / 32, sp.num_kv_heads, batch), kCombineThreads, 0, st>>>(sp, std::log2(static_cast<float>(sp.group)));
   mark(st, "combine_stats");
   scores_generic_kernel<T, D><<<dim3(score_tiles, sp.num_kv_heads), kGenScoreKeys, 0, st>>>(sp);
   mark(st, "scores_generic");
@@ -281,7 +281,7 @@ int launch_scores_tc(const pkv_config* c, const pkv_tensor& q, const pkv_tensor&
   const int grid_b = static_cast<int>(std::min<long long>(sms, static_cast<long long>(score_items) * sp.num_kv_heads));
   score_tc_kernel<D, 0><<<grid_a, kTcThreads, TcSmem<D>::kTotal, st>>>(q_map, k_map, tp);
   mark(st, "rowstats_tc");
-  combine_stats_kernel<<<dim3((sp.rows + 31) / 32, sp.num_kv_heads, batch), 256, 0, st>>>(sp, std::log2(static_cast<float>(sp.group)));
+  combine_stats_kernel<<<dim3((sp.rows + 31) / 32, sp.num_kv_heads, batch), kCombineThreads, 0, st>>>(sp, std::log2(static_cast<float>(sp.group)));
   mark(st, "combine_stats");
   score_tc_kernel<D, 1><<<grid_b, kTcThreads, TcSmem<D>::kTotal, st>>>(q_map, k_map, tp);
   mark(st, "scores_tc");
@@ -330,14 +330,14 @@ int run_select(const pkv_config* c, const float* scores, int64_t ld, const SeqTa
   int cluster = 1;
   while (cluster < kSelMaxCluster && (max_p + cluster - 1) / cluster > 8192) cluster *= 2;
   const int slice = ((max_p + cluster - 1) / cluster + 31) & ~31;
-  sp.slice_cap = slice <= kSelSliceCap ? slice : 0;
-  const size_t smem = static_cast<size_t>(sp.slice_cap) * sizeof(uint32_t);
+  sp.cached = slice <= kSelSliceCap ? 1 : 0;
+  const size_t smem = sp.cached ? static_cast<size_t>(slice) * 6 : 0;
   static bool attr_done[64] = {};  // the attribute is per device; setting it twice is harmless
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return PKV_ERR_CUDA;
   if (dev >= 64 || !attr_done[dev]) {
-    if (cudaFuncSetAttribute(pool_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             kSelSliceCap * static_cast<int>(sizeof(uint32_t))) != cudaSuccess)
+    if (cudaFuncSetAttribute(pool_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSelSliceCap * 6) !=
+        cudaSuccess)
       return PKV_ERR_CUDA;
     if (dev < 64) attr_done[dev] = true;
   }

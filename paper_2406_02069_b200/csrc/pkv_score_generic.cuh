@@ -98,26 +98,34 @@ __global__ void __launch_bounds__(kGenRowBlock) rowstats_generic_kernel(const Sc
   }
 }
 
-// grid (ceil(rows / 32), H_kv, batch), block 256: merge the chunk partials of each window row.
-// Thread (rl, sg) = (tid % 32, tid / 32) takes row r0 + rl and every 8th partial slot starting at sg, so
-// a warp reads 32 consecutive rows of one slot (256 contiguous bytes); the 8 slot groups of a row are
-// merged through shared memory.  extra_log2 = log2(G) folds the mean over the group's query heads
-// into the normaliser.
-__global__ void __launch_bounds__(256) combine_stats_kernel(const ScoreParams p, float extra_log2) {
-  __shared__ float sm[8][32], sz[8][32];
+// grid (ceil(rows / 32), H_kv, batch), block 1024: merge the chunk partials of each window row.
+// Thread (rl, sg) = (tid % 32, tid / 32) takes row r0 + rl and every 32nd partial slot starting at sg, so
+// a warp reads 32 consecutive rows of one slot (256 contiguous bytes); loads are issued four at a time
+// before they are used.  The 32 slot groups of a row are merged through shared memory.
+// extra_log2 = log2(G) folds the mean over the group's query heads into the normaliser.
+constexpr int kCombineThreads = 1024;
+__global__ void __launch_bounds__(kCombineThreads) combine_stats_kernel(const ScoreParams p, float extra_log2) {
+  __shared__ float sm[32][33], sz[32][33];
   const int h = blockIdx.y, b = blockIdx.z;
   const int rl = threadIdx.x & 31, sg = threadIdx.x >> 5;
   const int r = blockIdx.x * 32 + rl;
   const int t0 = p.seq.stat_off[b] * p.slots_per_chunk, t1 = p.seq.stat_off[b + 1] * p.slots_per_chunk;
+  const int64_t slot_stride = static_cast<int64_t>(p.num_kv_heads) * p.rows;
   float m = -INFINITY, z = 0.f;
   if (r < p.rows) {
-    for (int t = t0 + sg; t < t1; t += 8) {
-      const float2 pz = p.partial[(static_cast<int64_t>(t) * p.num_kv_heads + h) * p.rows + r];
-      if (pz.x > -INFINITY) {                      // (-inf, 0) marks a slot that saw no key of this row
-        const float mn = fmaxf(m, pz.x);
-        z = z * exp2f(m - mn) + pz.y * exp2f(pz.x - mn);
-        m = mn;
-      }
+    const float2* base = p.partial + static_cast<int64_t>(h) * p.rows + r;
+    for (int t = t0 + sg; t < t1; t += 4 * 32) {
+      float2 pz[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        pz[u] = t + 32 * u < t1 ? base[(t + 32 * u) * slot_stride] : make_float2(-INFINITY, 0.f);
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (pz[u].x > -INFINITY) {                 // (-inf, 0) marks a slot that saw no key of this row
+          const float mn = fmaxf(m, pz[u].x);
+          z = z * exp2f(m - mn) + pz[u].y * exp2f(pz[u].x - mn);
+          m = mn;
+        }
     }
   }
   sm[sg][rl] = m;
@@ -125,9 +133,9 @@ __global__ void __launch_bounds__(256) combine_stats_kernel(const ScoreParams p,
   __syncthreads();
   if (sg == 0 && r < p.rows) {
     float mm = -INFINITY;
-    for (int g = 0; g < 8; ++g) mm = fmaxf(mm, sm[g][rl]);
+    for (int g = 0; g < 32; ++g) mm = fmaxf(mm, sm[g][rl]);
     float zz = 0.f;
-    for (int g = 0; g < 8; ++g)
+    for (int g = 0; g < 32; ++g)
       if (sm[g][rl] > -INFINITY) zz += sz[g][rl] * exp2f(sm[g][rl] - mm);
     p.lse2[(static_cast<int64_t>(b) * p.num_kv_heads + h) * p.rows + r] = mm + log2f(zz) + extra_log2;
   }

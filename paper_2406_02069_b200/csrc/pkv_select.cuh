@@ -1,21 +1,30 @@
 // Fused max-pool + per-head top-k + window retention (Section 4.2.2).
 //
 // One thread-block cluster per (sequence, KV head).  The prefix positions are
-// split into contiguous slices, one per CTA of the cluster; each CTA pools its
-// slice (reading a halo of (w-1)/2 scores on both sides) and keeps the pooled
-// values in shared memory as order-preserving 32-bit keys.  The k-th largest key
-// is found by a most-significant-digit radix search in three passes (11, 11 and
-// 10 bits): every CTA histograms its slice, the histograms are summed across the
-// cluster through distributed shared memory, and every CTA walks the summed
-// histogram to the same digit.  While summing, a CTA also accumulates the
-// histograms of the CTAs that own earlier positions, which gives it, with no
-// further exchange, how many kept keys precede its slice.  Ties at the threshold
-// go to the smaller position and kept positions are written in ascending order,
-// so the result is one canonical list:
-//   kept = { i : key_i > T }  plus the leftmost (k - |{key > T}|) positions with key_i == T.
-// The alpha window positions are appended after them.
+// split into contiguous slices, one per CTA of the cluster, and inside a CTA into
+// contiguous runs, one per warp, so that position order is (CTA rank, warp, order
+// inside the warp's run).
 //
-// Only cluster barriers are used for synchronisation (no flag spinning).
+//  1. The CTA stages its slice of raw scores in shared memory (coalesced), pools
+//     them (halo of (w-1)/2 scores on both sides, clipped to the prefix) and keeps
+//     the pooled values as order-preserving 32-bit keys.
+//  2. Candidate filter.  Every thread remembers the largest key it produced.  The
+//     k-th largest of those per-thread maxima is a lower bound L of the k-th largest
+//     key (k distinct keys >= it exist), found with one CTA-local 11-bit histogram.
+//     Each warp compacts the positions of its run whose key >= L into a candidate
+//     list, in order.  Typically only a few times k keys survive; in the worst case
+//     (all keys equal, or k larger than the thread count) L = 0 and all do.
+//  3. The k-th largest key T is found by a most-significant-digit radix search over
+//     the candidates in three passes (11, 11, 10 bits).  Per pass every CTA
+//     histograms its candidates, the histograms are summed across the cluster
+//     through distributed shared memory, and every CTA walks the sum to the same
+//     digit.  While summing, a CTA also accumulates the histograms of the CTAs that
+//     own earlier positions, which tells it how many kept keys precede its slice.
+//  4. kept = { i : key_i > T } plus the leftmost (k - |{key > T}|) positions with
+//     key_i == T, written in ascending position; the alpha window positions follow.
+//
+// Ties therefore go to the smaller position and the list is canonical.  Only
+// block and cluster barriers are used for synchronisation (no flag spinning).
 #pragma once
 
 #include <cooperative_groups.h>
@@ -29,7 +38,10 @@ namespace cg = cooperative_groups;
 constexpr int kSelThreads = 1024;
 constexpr int kSelWarps = kSelThreads / 32;
 constexpr int kSelMaxCluster = 8;
-constexpr int kSelSliceCap = 48 * 1024;   // keys a CTA can hold in shared memory (192 KB)
+constexpr int kSelBins = 2048;
+constexpr int kSelSliceCap = 16384;        // positions a CTA can hold in shared memory (6 bytes each)
+constexpr int kSelRunMax = kSelSliceCap / kSelWarps;   // positions per warp in that case
+constexpr int kSelPerLane = kSelRunMax / 32;           // ... and per lane
 
 struct SelectParams {
   const float* scores;      // [batch][H_kv][ld]
@@ -38,7 +50,7 @@ struct SelectParams {
   SeqTable seq;
   int32_t num_kv_heads;
   int32_t pool_radius;      // (w - 1) / 2
-  int32_t slice_cap;        // keys of shared memory each CTA has (0: keys are recomputed from global)
+  int32_t cached;           // 1: every CTA's slice fits kSelSliceCap and lives in shared memory
   uint32_t* status;
 };
 
@@ -55,23 +67,22 @@ __device__ __forceinline__ uint32_t pooled_key(const float* s, int i, int P, int
   return ordered_key(best);
 }
 
-constexpr int kSelBins = 2048;
-
 // grid (cluster * H_kv, batch), cluster (cluster, 1, 1), block kSelThreads,
-// dynamic shared memory slice_cap * 4 bytes.
+// dynamic shared memory 6 bytes per slice position when cached, else none.
 __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectParams p) {
-  extern __shared__ __align__(16) uint32_t keys[];          // this CTA's pooled keys (if cached)
+  extern __shared__ __align__(16) uint32_t keys[];          // [slice] raw scores, then pooled keys
   __shared__ uint32_t hist[2][kSelBins];                    // per-pass digit histogram (double buffered)
-  __shared__ uint32_t lower[kSelBins];                      // ... summed over the CTAs of lower rank only
+  __shared__ uint32_t lower[kSelBins];                      // histogram summed over the CTAs of lower rank
   __shared__ uint32_t warp_sum[kSelWarps];
   __shared__ uint32_t warp_gt[kSelWarps], warp_eq[kSelWarps];
-  __shared__ uint32_t sel_digit, sel_above, lower_above;
+  __shared__ uint32_t sel_digit, sel_above, lower_above, bound_digit;
 
   cg::cluster_group cluster = cg::this_cluster();
   const int C = cluster.dim_blocks().x;
   const int rank = cluster.block_rank();
   const int h = blockIdx.x / C, b = blockIdx.y;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t lt = (1u << lane) - 1u;
 
   const int n = p.seq.n[b], alpha = p.seq.alpha, P = n - alpha;
   const int count = p.seq.count[b];
@@ -90,28 +101,94 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
   const float* s = p.scores + (static_cast<int64_t>(b) * p.num_kv_heads + h) * p.ld_scores;
   const int slice = ((P + C - 1) / C + 31) & ~31;           // multiple of 32 positions per CTA
   const int lo = min(P, rank * slice), hi = min(P, lo + slice);
-  const bool cached = p.slice_cap >= slice;
+  const int run = ((slice / kSelWarps) + 31) & ~31;         // positions per warp, multiple of 32
+  const int wlo = min(hi, lo + warp * run), whi = min(hi, wlo + run);
+  const bool cached = p.cached != 0;                        // then run <= kSelRunMax
+  uint16_t* cand = reinterpret_cast<uint16_t*>(keys + slice) + warp * run;   // this warp's candidate list
+  const int radius = p.pool_radius;
 
-  if (cached)
-    for (int i = lo + tid; i < hi; i += kSelThreads) keys[i - lo] = pooled_key(s, i, P, p.pool_radius);
-  auto key_at = [&](int i) -> uint32_t {
-    return cached ? keys[i - lo] : pooled_key(s, i, P, p.pool_radius);
-  };
   for (int i = tid; i < 2 * kSelBins; i += kSelThreads) (&hist[0][0])[i] = 0;
+  int n_items = whi - wlo;                                  // items this warp walks in the passes below
+  if (cached) {
+    // ---- 1. stage raw scores, pool, keep keys
+    float* raw = reinterpret_cast<float*>(keys);
+    for (int i = lo + tid; i < hi; i += kSelThreads) raw[i - lo] = s[i];
+    __syncthreads();
+    uint32_t pk[kSelPerLane];
+    uint32_t tmax = 0;
+#pragma unroll
+    for (int it = 0; it < kSelPerLane; ++it) {
+      const int i = wlo + it * 32 + lane;
+      pk[it] = 0;
+      if (i < whi) {
+        const int a = max(0, i - radius), z = min(P - 1, i + radius);
+        float best = -INFINITY;
+        for (int t = a; t <= z; ++t) best = fmaxf(best, (t >= lo && t < hi) ? raw[t - lo] : s[t]);
+        pk[it] = ordered_key(best);
+        tmax = max(tmax, pk[it]);
+      }
+    }
+    __syncthreads();                                        // all raw scores read
+#pragma unroll
+    for (int it = 0; it < kSelPerLane; ++it) {
+      const int i = wlo + it * 32 + lane;
+      if (i < whi) keys[i - lo] = pk[it];
+    }
+    // ---- 2. lower bound of the k-th largest key from the per-thread maxima, then compaction
+    {
+      const uint32_t digit = tmax >> 21;
+      const uint32_t peers = __match_any_sync(0xffffffffu, digit);
+      if (lane == __ffs(peers) - 1) atomicAdd(&hist[1][digit], __popc(peers));
+    }
+    __syncthreads();
+    {
+      const uint2 v = reinterpret_cast<const uint2*>(hist[1])[tid];
+      const uint32_t mine = v.x + v.y;
+      uint32_t incl = mine;
+      for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t u = __shfl_down_sync(0xffffffffu, incl, off);
+        if (lane + off < 32) incl += u;
+      }
+      if (lane == 0) warp_sum[warp] = incl;
+      if (tid == 0) bound_digit = 0;                        // fewer than k maxima: no filtering
+      __syncthreads();
+      uint32_t higher = incl - mine;
+      for (int w2 = warp + 1; w2 < kSelWarps; ++w2) higher += warp_sum[w2];
+      const uint32_t kk = static_cast<uint32_t>(k);
+      if (higher < kk && kk <= higher + mine) bound_digit = (higher + v.y >= kk) ? 2 * tid + 1 : 2 * tid;
+      __syncthreads();
+      reinterpret_cast<uint2*>(hist[1])[tid] = make_uint2(0, 0);
+    }
+    const uint32_t bound = bound_digit << 21;
+    int ncand = 0;
+#pragma unroll
+    for (int it = 0; it < kSelPerLane; ++it) {
+      const int i = wlo + it * 32 + lane;
+      const bool c = i < whi && pk[it] >= bound;
+      const uint32_t bal = __ballot_sync(0xffffffffu, c);
+      if (c) cand[ncand + __popc(bal & lt)] = static_cast<uint16_t>(i - lo);
+      ncand += __popc(bal);
+    }
+    n_items = ncand;
+    __syncwarp();
+  }
   __syncthreads();
+  // item j of this warp -> (position, key)
+  auto item_pos = [&](int j) -> int { return cached ? lo + cand[j] : wlo + j; };
+  auto item_key = [&](int pos) -> uint32_t { return cached ? keys[pos - lo] : pooled_key(s, pos, P, radius); };
 
-  // ---- radix search for the k-th largest key
+  // ---- 3. radix search for the k-th largest key
   uint32_t prefix = 0, mask = 0, remaining = k;
   uint32_t gt_before_cta = 0, eq_before_cta = 0;            // kept-candidate keys owned by lower-rank CTAs
   for (int pass = 0; pass < 3; ++pass) {
     const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
     const uint32_t dmask = pass == 2 ? 1023u : 2047u;
     uint32_t* hcur = hist[pass & 1];
-    for (int base = lo + warp * 32; base < hi; base += kSelThreads) {
-      const int i = base + lane;
+    for (int j0 = 0; j0 < n_items; j0 += 32) {
+      const int j = j0 + lane;
       uint32_t digit = kSelBins;                            // kSelBins = does not take part
-      if (i < hi) {
-        const uint32_t key = key_at(i);
+      if (j < n_items) {
+        const uint32_t key = item_key(item_pos(j));
         if ((key & mask) == prefix) digit = (key >> shift) & dmask;
       }
       const uint32_t peers = __match_any_sync(0xffffffffu, digit);
@@ -120,11 +197,13 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
     cluster.sync();                                         // all histograms of this pass complete
     // every thread owns two adjacent digits
     uint32_t tot[2] = {0, 0}, low[2] = {0, 0};
-    for (int c = 0; c < C; ++c) {
-      const uint2 v = reinterpret_cast<const uint2*>(cluster.map_shared_rank(hcur, c))[tid];
-      tot[0] += v.x; tot[1] += v.y;
-      if (c < rank) { low[0] += v.x; low[1] += v.y; }
-    }
+#pragma unroll
+    for (int c = 0; c < kSelMaxCluster; ++c)
+      if (c < C) {
+        const uint2 v = reinterpret_cast<const uint2*>(cluster.map_shared_rank(hcur, c))[tid];
+        tot[0] += v.x; tot[1] += v.y;
+        if (c < rank) { low[0] += v.x; low[1] += v.y; }
+      }
     lower[2 * tid] = low[0]; lower[2 * tid + 1] = low[1];
     reinterpret_cast<uint2*>(hist[(pass + 1) & 1])[tid] = make_uint2(0, 0);   // next pass's buffer
     // keys in digits above this thread's pair: suffix sums inside the warp, then over warps
@@ -160,15 +239,13 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
   const uint32_t T = prefix;                                // the k-th largest key
   const uint32_t need_eq = remaining;                       // ties at T to take, from the left
 
-  // ---- keys above / at the threshold inside this CTA: warp w owns a contiguous run of the slice
-  const int run = ((slice / kSelWarps) + 31) & ~31;
-  const int wlo = min(hi, lo + warp * run), whi = min(hi, wlo + run);
+  // ---- 4. keys above / at the threshold inside this CTA, warp by warp, then emit in position order
   uint32_t ngt = 0, neq = 0;
-  for (int base = wlo; base < whi; base += 32) {
-    const int i = base + lane;
-    const uint32_t key = i < whi ? key_at(i) : 0u;
-    ngt += __popc(__ballot_sync(0xffffffffu, i < whi && key > T));
-    neq += __popc(__ballot_sync(0xffffffffu, i < whi && key == T));
+  for (int j0 = 0; j0 < n_items; j0 += 32) {
+    const int j = j0 + lane;
+    const uint32_t key = j < n_items ? item_key(item_pos(j)) : 0u;
+    ngt += __popc(__ballot_sync(0xffffffffu, j < n_items && key > T));
+    neq += __popc(__ballot_sync(0xffffffffu, j < n_items && key == T));
   }
   if (lane == 0) { warp_gt[warp] = ngt; warp_eq[warp] = neq; }
   __syncthreads();
@@ -178,16 +255,15 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
     if (gt_before + ngt + min(eq_before + neq, need_eq) != static_cast<uint32_t>(k))
       atomicOr(p.status, kStatusSelectMismatch);
   }
-
-  // ---- emit in ascending position: rank of i among the kept = (#greater before i) + min(#equal before i, need_eq)
-  for (int base = wlo; base < whi; base += 32) {
-    const int i = base + lane;
-    const uint32_t key = i < whi ? key_at(i) : 0u;
-    const bool is_gt = i < whi && key > T, is_eq = i < whi && key == T;
+  // rank of a kept position = (#greater before it) + min(#equal before it, need_eq)
+  for (int j0 = 0; j0 < n_items; j0 += 32) {
+    const int j = j0 + lane;
+    const int pos = j < n_items ? item_pos(j) : 0;
+    const uint32_t key = j < n_items ? item_key(pos) : 0u;
+    const bool is_gt = j < n_items && key > T, is_eq = j < n_items && key == T;
     const uint32_t bg = __ballot_sync(0xffffffffu, is_gt), be = __ballot_sync(0xffffffffu, is_eq);
-    const uint32_t lt = (1u << lane) - 1u;
     const uint32_t g = gt_before + __popc(bg & lt), e = eq_before + __popc(be & lt);
-    if (is_gt || (is_eq && e < need_eq)) out[g + min(e, need_eq)] = i;
+    if (is_gt || (is_eq && e < need_eq)) out[g + min(e, need_eq)] = pos;
     gt_before += __popc(bg);
     eq_before += __popc(be);
   }
