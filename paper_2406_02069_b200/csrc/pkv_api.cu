@@ -330,13 +330,14 @@ int run_select(const pkv_config* c, const float* scores, int64_t ld, const SeqTa
   int cluster = 1;
   while (cluster < kSelMaxCluster && (max_p + cluster - 1) / cluster > 8192) cluster *= 2;
   const int slice = ((max_p + cluster - 1) / cluster + 31) & ~31;
-  sp.cached = slice <= kSelSliceCap ? 1 : 0;
-  const size_t smem = sp.cached ? static_cast<size_t>(slice) * 6 : 0;
+  sp.cached = (slice <= kSelSliceCap && sp.pool_radius <= kSelHalo) ? 1 : 0;
+  const size_t smem = sp.cached ? static_cast<size_t>(slice) * 6 + 8 * kSelHalo : 0;
   static bool attr_done[64] = {};  // the attribute is per device; setting it twice is harmless
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return PKV_ERR_CUDA;
   if (dev >= 64 || !attr_done[dev]) {
-    if (cudaFuncSetAttribute(pool_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSelSliceCap * 6) !=
+    if (cudaFuncSetAttribute(pool_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             kSelSliceCap * 6 + 8 * kSelHalo) !=
         cudaSuccess)
       return PKV_ERR_CUDA;
     if (dev < 64) attr_done[dev] = true;

@@ -34,7 +34,7 @@ constexpr int kTcEpiThreads = 256;
 constexpr int kTcTileKeys = 128;        // keys per MMA tile
 constexpr int kTcKStages = 4;           // shared-memory stages of K tiles
 constexpr int kTcMaxRows = 256;         // window rows (G * alpha) the tensor-core path takes
-constexpr uint32_t kTcSpinCap = 1u << 22;
+constexpr long long kTcWaitCycles = 1ll << 31;   // bound of any one wait, in SM clocks
 
 struct TcParams {
   SeqTable seq;                 // stat_off / score_off count CHUNKS of chunk_tiles tiles
@@ -63,6 +63,7 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+// Non-blocking test of a barrier phase.
 __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
@@ -74,16 +75,29 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait: polls without blocking, backs off after the first polls, and gives up after
-// kTcSpinCap polls (of the order of a second).  Returns false if it gave up, or if another
-// thread did (abort flag).
+// Hardware-suspended wait for a barrier phase; returns false when the hardware's own time limit ran out.
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  The thread is suspended by the hardware between checks (no sleeping in software, which
+// would add its wake-up latency to every hand-off of the pipeline).  Gives up after kTcWaitCycles SM
+// clocks (of the order of a second) or when another thread gave up (abort flag); returns false then.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t it = 0; it < kTcSpinCap; ++it) {
-    if (mbar_test(bar, parity)) return true;
-    if (it >= 64u) {
-      __nanosleep(100);
-      if ((it & 255u) == 255u && *abort_flag) return false;
-    }
+  if (mbar_try(bar, parity)) return true;
+  const long long start = clock64();
+  for (;;) {
+    for (int i = 0; i < 32; ++i)
+      if (mbar_try(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (clock64() - start > kTcWaitCycles) break;
   }
   *abort_flag = 1;
   return false;
@@ -128,6 +142,76 @@ __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+
+// The special-function unit evaluates 16 exponentials per clock per SM, which is what bounds both
+// sweeps.  Every kTcPolyEvery-th exponential is therefore evaluated on the FMA pipe instead:
+// 2^x = 2^n * 2^f with n = round(x), f = x - n in [-0.5, 0.5]; 2^f by a cubic minimax polynomial
+// (largest relative error 7.5e-5, far inside the 2e-3 the scores are held to); 2^n by adding n to the
+// exponent field.  x is clamped to [-126, 127.5] so the exponent arithmetic cannot wrap.
+#ifndef PKV_POLY_EVERY
+#define PKV_POLY_EVERY 0
+#endif
+constexpr int kTcPolyEvery = PKV_POLY_EVERY;    // 0 = never
+
+template <bool kClampHigh>
+__device__ __forceinline__ float ex2_poly(float x) {
+  x = fmaxf(x, -126.0f);
+  if (kClampHigh) x = fminf(x, 127.5f);
+  const float t = x + 12582912.0f;              // 1.5 * 2^23: the low mantissa bits now hold round(x)
+  const float nf = t - 12582912.0f;
+  const float f = x - nf;
+  float q = fmaf(f, 0.0551716685295105f, 0.2426111251115799f);
+  q = fmaf(q, f, 0.6932609677314758f);
+  q = fmaf(q, f, 0.9999280571937561f);
+  // q * 2^n: add n to the exponent field.  The multiply-add form keeps this on the FMA pipe.
+  int bits;
+  asm("mad.lo.s32 %0, %1, 8388608, %2;" : "=r"(bits) : "r"(__float_as_int(t)), "r"(__float_as_int(q)));
+  return __int_as_float(bits);
+}
+template <bool kClampHigh>
+__device__ __forceinline__ float ex2_mixed(float x, int j) {
+  return (kTcPolyEvery > 0 && (j % (kTcPolyEvery > 0 ? kTcPolyEvery : 1)) == kTcPolyEvery - 1) ? ex2_poly<kClampHigh>(x)
+                                                                                              : ex2(x);
+}
+
+// Sweep A, 32 logits of one window row: z += sum_j 2^(v_j * c2 - m).  m is a reference exponent, not
+// necessarily the running maximum: it is only moved when a group's sum is not a moderate finite
+// number (the row's first group, where m = -inf, or a logit ~60 binades above the reference).
+__device__ __forceinline__ void rowstats_group(const uint32_t (&v)[32], float c2, float& m, float& z) {
+  float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+  for (int j = 0; j < 32; j += 4) {
+    a0 += ex2_mixed<true>(fmaf(__uint_as_float(v[j]), c2, -m), j);
+    a1 += ex2_mixed<true>(fmaf(__uint_as_float(v[j + 1]), c2, -m), j + 1);
+    a2 += ex2_mixed<true>(fmaf(__uint_as_float(v[j + 2]), c2, -m), j + 2);
+    a3 += ex2_mixed<true>(fmaf(__uint_as_float(v[j + 3]), c2, -m), j + 3);
+  }
+  float g = (a0 + a1) + (a2 + a3);
+  if (!(g < 1.0e18f)) {
+    float gm = __uint_as_float(v[0]);
+#pragma unroll
+    for (int j = 1; j < 32; ++j) gm = fmaxf(gm, __uint_as_float(v[j]));
+    const float mn = fmaxf(m, gm * c2);
+    z *= ex2(m - mn);
+    m = mn;
+    g = 0.f;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) g += ex2(fmaf(__uint_as_float(v[j]), c2, -m));
+  }
+  z += g;
+}
+
+// Sweep B, 32 window rows of one key: a += 2^(v_j * c2 - lse_j), lse from shared memory.
+__device__ __forceinline__ void score_group(const uint32_t (&v)[32], float c2, const float* lse, float (&a)[4]) {
+#pragma unroll
+  for (int j = 0; j < 32; j += 4) {
+    const float4 l4 = *reinterpret_cast<const float4*>(lse + j);
+    a[0] += ex2_mixed<false>(fmaf(__uint_as_float(v[j]), c2, -l4.x), j);
+    a[1] += ex2_mixed<false>(fmaf(__uint_as_float(v[j + 1]), c2, -l4.y), j + 1);
+    a[2] += ex2_mixed<false>(fmaf(__uint_as_float(v[j + 2]), c2, -l4.z), j + 2);
+    a[3] += ex2_mixed<false>(fmaf(__uint_as_float(v[j + 3]), c2, -l4.w), j + 3);
+  }
 }
 
 // Shared-memory matrix descriptor of a K-major bf16 operand whose rows are 128 bytes wide and
@@ -364,27 +448,24 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
                                  (two ? half * 128 : 0);
           const int key_base = t * kTcTileKeys;
           const bool masked = key_base + kTcTileKeys - 1 > P; // tile reaches into the window: per-element mask
-          for (int cg = 0; cg < kTcTileKeys; cg += 32) {
-            uint32_t v[32];
-            tc_ld32(taddr + cg, v);
-            tc_wait_ld();
-            if (!masked) {
-              float gm = __uint_as_float(v[0]);
+          if (!masked) {
+            // the load of the next 32 columns is in flight while the current 32 are processed
+            uint32_t va[32], vb[32];
+            tc_ld32(taddr, va);
 #pragma unroll
-              for (int j = 1; j < 32; ++j) gm = fmaxf(gm, __uint_as_float(v[j]));
-              const float mn = fmaxf(m, gm * c2);
-              z *= ex2(m - mn);
-              m = mn;
-              float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-#pragma unroll
-              for (int j = 0; j < 32; j += 4) {
-                a0 += ex2(fmaf(__uint_as_float(v[j]), c2, -m));
-                a1 += ex2(fmaf(__uint_as_float(v[j + 1]), c2, -m));
-                a2 += ex2(fmaf(__uint_as_float(v[j + 2]), c2, -m));
-                a3 += ex2(fmaf(__uint_as_float(v[j + 3]), c2, -m));
-              }
-              z += (a0 + a1) + (a2 + a3);
-            } else {
+            for (int cg = 0; cg < kTcTileKeys; cg += 64) {
+              tc_wait_ld();
+              tc_ld32(taddr + cg + 32, vb);
+              rowstats_group(va, c2, m, z);
+              tc_wait_ld();
+              if (cg + 64 < kTcTileKeys) tc_ld32(taddr + cg + 64, va);
+              rowstats_group(vb, c2, m, z);
+            }
+          } else {
+            for (int cg = 0; cg < kTcTileKeys; cg += 32) {
+              uint32_t v[32];
+              tc_ld32(taddr + cg, v);
+              tc_wait_ld();
               float gm = -INFINITY;
 #pragma unroll
               for (int j = 0; j < 32; ++j) {
@@ -439,25 +520,27 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
           if (!ok) break;
           tc_fence_after();
           const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + ts * stage_cols;
-          float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-          for (int cg = 0; cg < p.rows_pad; cg += 32) {
-            uint32_t v[32];
-            tc_ld32(taddr + cg, v);
-            tc_wait_ld();
-#pragma unroll
-            for (int j = 0; j < 32; j += 4) {
-              const float4 l4 = *reinterpret_cast<const float4*>(&lse_s[cg + j]);
-              a0 += ex2(fmaf(__uint_as_float(v[j]), c2, -l4.x));
-              a1 += ex2(fmaf(__uint_as_float(v[j + 1]), c2, -l4.y));
-              a2 += ex2(fmaf(__uint_as_float(v[j + 2]), c2, -l4.z));
-              a3 += ex2(fmaf(__uint_as_float(v[j + 3]), c2, -l4.w));
+          float acc[4] = {0.f, 0.f, 0.f, 0.f};
+          {
+            uint32_t va[32], vb[32];
+            tc_ld32(taddr, va);
+            for (int cg = 0; cg < p.rows_pad; cg += 64) {
+              const bool second = cg + 32 < p.rows_pad;
+              tc_wait_ld();
+              if (second) tc_ld32(taddr + cg + 32, vb);
+              score_group(va, c2, lse_s + cg, acc);
+              if (second) {
+                tc_wait_ld();
+                if (cg + 64 < p.rows_pad) tc_ld32(taddr + cg + 64, va);
+                score_group(vb, c2, lse_s + cg + 32, acc);
+              }
             }
           }
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(t_empty(ts));
           const int i = t * kTcTileKeys + lane_row;
-          if (i < P) srow[i] = (a0 + a1) + (a2 + a3);
+          if (i < P) srow[i] = (acc[0] + acc[1]) + (acc[2] + acc[3]);
         }
         if (!ok) break;
       }

@@ -42,6 +42,7 @@ constexpr int kSelBins = 2048;
 constexpr int kSelSliceCap = 16384;        // positions a CTA can hold in shared memory (6 bytes each)
 constexpr int kSelRunMax = kSelSliceCap / kSelWarps;   // positions per warp in that case
 constexpr int kSelPerLane = kSelRunMax / 32;           // ... and per lane
+constexpr int kSelHalo = 16;               // largest pool radius the shared-memory path stages
 
 struct SelectParams {
   const float* scores;      // [batch][H_kv][ld]
@@ -68,9 +69,10 @@ __device__ __forceinline__ uint32_t pooled_key(const float* s, int i, int P, int
 }
 
 // grid (cluster * H_kv, batch), cluster (cluster, 1, 1), block kSelThreads,
-// dynamic shared memory 6 bytes per slice position when cached, else none.
+// dynamic shared memory (6 bytes per slice position + 8 * kSelHalo) when cached, else none.
 __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectParams p) {
-  extern __shared__ __align__(16) uint32_t keys[];          // [slice] raw scores, then pooled keys
+  extern __shared__ __align__(16) uint32_t sel_smem[];      // [halo | slice | halo] raw scores, then pooled keys
+  uint32_t* keys = sel_smem + kSelHalo;
   __shared__ uint32_t hist[2][kSelBins];                    // per-pass digit histogram (double buffered)
   __shared__ uint32_t lower[kSelBins];                      // histogram summed over the CTAs of lower rank
   __shared__ uint32_t warp_sum[kSelWarps];
@@ -104,15 +106,16 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
   const int run = ((slice / kSelWarps) + 31) & ~31;         // positions per warp, multiple of 32
   const int wlo = min(hi, lo + warp * run), whi = min(hi, wlo + run);
   const bool cached = p.cached != 0;                        // then run <= kSelRunMax
-  uint16_t* cand = reinterpret_cast<uint16_t*>(keys + slice) + warp * run;   // this warp's candidate list
+  uint16_t* cand = reinterpret_cast<uint16_t*>(keys + slice + kSelHalo) + warp * run;   // this warp's candidates
   const int radius = p.pool_radius;
 
   for (int i = tid; i < 2 * kSelBins; i += kSelThreads) (&hist[0][0])[i] = 0;
   int n_items = whi - wlo;                                  // items this warp walks in the passes below
   if (cached) {
-    // ---- 1. stage raw scores, pool, keep keys
+    // ---- 1. stage raw scores with a halo (-inf outside the prefix), pool, keep keys
     float* raw = reinterpret_cast<float*>(keys);
-    for (int i = lo + tid; i < hi; i += kSelThreads) raw[i - lo] = s[i];
+    for (int i = lo - kSelHalo + tid; i < hi + kSelHalo; i += kSelThreads)
+      raw[i - lo] = (i >= 0 && i < P) ? s[i] : -INFINITY;
     __syncthreads();
     uint32_t pk[kSelPerLane];
     uint32_t tmax = 0;
@@ -121,9 +124,8 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
       const int i = wlo + it * 32 + lane;
       pk[it] = 0;
       if (i < whi) {
-        const int a = max(0, i - radius), z = min(P - 1, i + radius);
-        float best = -INFINITY;
-        for (int t = a; t <= z; ++t) best = fmaxf(best, (t >= lo && t < hi) ? raw[t - lo] : s[t]);
+        float best = raw[i - lo];
+        for (int t = 1; t <= radius; ++t) best = fmaxf(best, fmaxf(raw[i - lo - t], raw[i - lo + t]));
         pk[it] = ordered_key(best);
         tmax = max(tmax, pk[it]);
       }
@@ -134,14 +136,16 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
       const int i = wlo + it * 32 + lane;
       if (i < whi) keys[i - lo] = pk[it];
     }
-    // ---- 2. lower bound of the k-th largest key from the per-thread maxima, then compaction
-    {
-      const uint32_t digit = tmax >> 21;
+    // ---- 2. lower bound of the k-th largest key: the k-th largest per-thread maximum, resolved to its
+    //         top 22 bits by two CTA-local histogram passes; then compaction of the keys >= bound
+    uint32_t bprefix = 0, bmask = 0, brem = static_cast<uint32_t>(k);
+    for (int bp = 0; bp < 2; ++bp) {
+      const int shift = bp == 0 ? 21 : 10;
+      // threads whose maximum left the searched prefix do not take part in the second pass
+      const uint32_t digit = ((tmax & bmask) == bprefix) ? ((tmax >> shift) & 2047u) : kSelBins;
       const uint32_t peers = __match_any_sync(0xffffffffu, digit);
-      if (lane == __ffs(peers) - 1) atomicAdd(&hist[1][digit], __popc(peers));
-    }
-    __syncthreads();
-    {
+      if (digit < kSelBins && lane == __ffs(peers) - 1) atomicAdd(&hist[1][digit], __popc(peers));
+      __syncthreads();
       const uint2 v = reinterpret_cast<const uint2*>(hist[1])[tid];
       const uint32_t mine = v.x + v.y;
       uint32_t incl = mine;
@@ -150,16 +154,29 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
         if (lane + off < 32) incl += u;
       }
       if (lane == 0) warp_sum[warp] = incl;
-      if (tid == 0) bound_digit = 0;                        // fewer than k maxima: no filtering
+      if (tid == 0) { bound_digit = kSelBins; sel_above = 0; }   // kSelBins: fewer than brem maxima in play
       __syncthreads();
       uint32_t higher = incl - mine;
       for (int w2 = warp + 1; w2 < kSelWarps; ++w2) higher += warp_sum[w2];
-      const uint32_t kk = static_cast<uint32_t>(k);
-      if (higher < kk && kk <= higher + mine) bound_digit = (higher + v.y >= kk) ? 2 * tid + 1 : 2 * tid;
+      if (higher < brem && brem <= higher + mine) {
+        const bool upper = higher + v.y >= brem;
+        bound_digit = upper ? 2 * tid + 1 : 2 * tid;
+        sel_above = upper ? higher : higher + v.y;
+      }
       __syncthreads();
       reinterpret_cast<uint2*>(hist[1])[tid] = make_uint2(0, 0);
+      const uint32_t bd = bound_digit;
+      if (bd == kSelBins) {                                 // cannot bound (k exceeds the thread count): keep all
+        if (bp == 0) { bprefix = 0; bmask = 0; }
+        __syncthreads();
+        break;
+      }
+      bprefix |= bd << shift;
+      bmask |= 2047u << shift;
+      brem -= sel_above;
+      __syncthreads();                                      // histogram zeroed, bound_digit consumed
     }
-    const uint32_t bound = bound_digit << 21;
+    const uint32_t bound = bprefix;                         // lower edge of the resolved digits
     int ncand = 0;
 #pragma unroll
     for (int it = 0; it < kSelPerLane; ++it) {
