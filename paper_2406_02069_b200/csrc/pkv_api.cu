@@ -230,9 +230,10 @@ int launch_scores_tc(const pkv_config* c, const pkv_tensor& q, const pkv_tensor&
       return PKV_ERR_CUDA;
     attr_done[dev] = true;
   }
-  alignas(64) CUtensorMap q_map, k_map;
+  alignas(64) CUtensorMap q_map, k_map_a, k_map_b;
   if (!make_map(&q_map, q, D, c->window, c->num_q_heads, batch, c->window, sp.group) ||
-      !make_map(&k_map, k, D, max_n, c->num_kv_heads, batch, kTcTileKeys, 1))
+      !make_map(&k_map_a, k, D, max_n, c->num_kv_heads, batch, kTcTileKeysA, 1) ||
+      !make_map(&k_map_b, k, D, max_n, c->num_kv_heads, batch, kTcTileKeysB, 1))
     return PKV_ERR_CUDA;
 
   TcParams tp{};
@@ -249,41 +250,47 @@ int launch_scores_tc(const pkv_config* c, const pkv_tensor& q, const pkv_tensor&
   tp.ld_scores = sp.ld_scores;
   tp.status = status;
   // Key tiles per work item: the largest power of two that still spreads the items evenly over the SMs.
-  auto items_for = [&](int ct, bool prefix) {
+  auto items_for = [&](int ct, int tile_keys, bool prefix) {
     long long items = 0;
     for (int b = 0; b < batch; ++b) {
       const int keys = prefix ? sp.seq.n[b] - sp.seq.alpha : sp.seq.n[b];
-      const int tiles = (keys + kTcTileKeys - 1) / kTcTileKeys;
+      const int tiles = (keys + tile_keys - 1) / tile_keys;
       items += (tiles + ct - 1) / ct;
     }
     return items * sp.num_kv_heads;
   };
-  int ct = 16;
-  for (; ct > 1; ct /= 2) {
-    const long long items = items_for(ct, false);
-    const long long waves = (items + sms - 1) / sms;
-    if (items >= sms && static_cast<double>(items) / static_cast<double>(waves * sms) >= 0.93) break;
-  }
-  tp.chunk_tiles = ct;
+  auto pick = [&](int tile_keys, bool prefix) {
+    int ct = 16;
+    for (; ct > 1; ct /= 2) {
+      const long long items = items_for(ct, tile_keys, prefix);
+      const long long waves = (items + sms - 1) / sms;
+      if (items >= sms && static_cast<double>(items) / static_cast<double>(waves * sms) >= 0.93) break;
+    }
+    return ct;
+  };
+  tp.chunk_tiles_a = pick(kTcTileKeysA, false);
+  tp.chunk_tiles_b = pick(kTcTileKeysB, true);
   int stat_items = 0, score_items = 0;
   for (int b = 0; b < batch; ++b) {
     tp.seq.stat_off[b] = stat_items;
     tp.seq.score_off[b] = score_items;
-    stat_items += ((sp.seq.n[b] + kTcTileKeys - 1) / kTcTileKeys + ct - 1) / ct;
-    score_items += ((sp.seq.n[b] - sp.seq.alpha + kTcTileKeys - 1) / kTcTileKeys + ct - 1) / ct;
+    stat_items += ((sp.seq.n[b] + kTcTileKeysA - 1) / kTcTileKeysA + tp.chunk_tiles_a - 1) / tp.chunk_tiles_a;
+    score_items += ((sp.seq.n[b] - sp.seq.alpha + kTcTileKeysB - 1) / kTcTileKeysB + tp.chunk_tiles_b - 1) /
+                   tp.chunk_tiles_b;
   }
   tp.seq.stat_off[batch] = stat_items;
   tp.seq.score_off[batch] = score_items;
   sp.seq = tp.seq;
-  sp.slots_per_chunk = 2;
+  sp.slots_per_chunk = tp.row_blocks == 2 ? 2 : 4;    // partial slots each sweep-A work item writes
 
   const int grid_a = static_cast<int>(std::min<long long>(sms, static_cast<long long>(stat_items) * sp.num_kv_heads));
   const int grid_b = static_cast<int>(std::min<long long>(sms, static_cast<long long>(score_items) * sp.num_kv_heads));
-  score_tc_kernel<D, 0><<<grid_a, kTcThreads, TcSmem<D>::kTotal, st>>>(q_map, k_map, tp);
+  score_tc_kernel<D, 0><<<grid_a, kTcThreads, TcSmem<D>::kTotal, st>>>(q_map, k_map_a, tp);
   mark(st, "rowstats_tc");
-  combine_stats_kernel<<<dim3((sp.rows + 31) / 32, sp.num_kv_heads, batch), kCombineThreads, 0, st>>>(sp, std::log2(static_cast<float>(sp.group)));
+  combine_stats_kernel<<<dim3((sp.rows + 31) / 32, sp.num_kv_heads, batch), kCombineThreads, 0, st>>>(
+      sp, std::log2(static_cast<float>(sp.group)));
   mark(st, "combine_stats");
-  score_tc_kernel<D, 1><<<grid_b, kTcThreads, TcSmem<D>::kTotal, st>>>(q_map, k_map, tp);
+  score_tc_kernel<D, 1><<<grid_b, kTcThreads, TcSmem<D>::kTotal, st>>>(q_map, k_map_b, tp);
   mark(st, "scores_tc");
   return check_launch();
 }

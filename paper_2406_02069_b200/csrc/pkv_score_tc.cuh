@@ -3,18 +3,24 @@
 // Two sweeps over K, because the score of a key sums softmax rows that each have
 // their own normaliser (known only after a whole row has been seen):
 //
-//   sweep A  D[row r][key i] = Q K^T   (A operand = window queries, B operand = key tile)
+//   sweep A  D[row r][key i] = Q K^T   (A operand = 128 window rows, B operand = 256-key tile)
 //            TMEM lane = window row, so each epilogue thread owns one row and keeps its
-//            running max and sum of 2^x privately: no cross-thread reduction at all.
-//   sweep B  D[key i][row r] = K Q^T   (operands swapped)
+//            reference exponent and sum of 2^x privately: no cross-thread reduction at all.
+//   sweep B  D[key i][row r] = K Q^T   (A operand = 128-key tile, B operand = all window rows)
 //            TMEM lane = key, so each epilogue thread owns one key and sums
 //            2^(x_ri - lse2_r) over the rows r, reading lse2 from shared memory.
 //
 // x = (q . k) * log2(e) / sqrt(d).  Operands arrive by TMA (no multicast) into
-// 128-byte-swizzled shared memory; tcgen05.mma accumulates in TMEM; epilogue warps
-// read TMEM with tcgen05.ld.  Warp roles: warp 0 = TMA producer, warp 1 = MMA
-// issuer and TMEM owner, warps 4..11 = epilogue.  CTAs are persistent: each takes
-// a contiguous range of (sequence, KV head, key chunk) work items.
+// 128-byte-swizzled shared memory; tcgen05.mma accumulates in TMEM (two to four
+// accumulator stages of up to 256 columns); epilogue warps read TMEM with tcgen05.ld.
+// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner, warps 4..19 =
+// epilogue.  The exponentials bound both sweeps (16 per clock per SM); four epilogue
+// warps per scheduler are what it takes to keep that unit busy.  The 16 epilogue
+// warps form four groups (TMEM lane quarter = warp % 4, group = (warp - 4) / 4).
+// Accumulator stage u % 2 is read by the two groups g with g % 2 == u % 2, each taking
+// half of its columns, so while one pair of groups works on a stage the MMAs of the
+// next stage run.  CTAs are persistent: each takes a contiguous range of (sequence,
+// KV head, key chunk) work items.
 //
 // Every wait on an mbarrier is bounded.  A wait that runs out sets an abort flag in
 // shared memory and a status bit in the workspace; all roles then leave their loops,
@@ -28,11 +34,12 @@
 
 namespace pkv {
 
-constexpr int kTcThreads = 384;
+constexpr int kTcThreads = 640;         // 20 warps: producer, MMA issuer, 2 idle, 16 epilogue
 constexpr int kTcEpiWarp0 = 4;          // first epilogue warp
-constexpr int kTcEpiThreads = 256;
-constexpr int kTcTileKeys = 128;        // keys per MMA tile
-constexpr int kTcKStages = 4;           // shared-memory stages of K tiles
+constexpr int kTcEpiWarps = 16;         // four per scheduler, which is what keeps the exp unit fed
+constexpr int kTcTileKeysA = 256;       // keys per K tile in sweep A (the N of its MMAs)
+constexpr int kTcTileKeysB = 128;       // keys per K tile in sweep B (the M of its MMAs)
+constexpr int kTcKBytes = 128 * 1024;   // shared memory given to K stages (2 x 64 KB or 4 x 32 KB at d = 128)
 constexpr int kTcMaxRows = 256;         // window rows (G * alpha) the tensor-core path takes
 constexpr long long kTcWaitCycles = 1ll << 31;   // bound of any one wait, in SM clocks
 
@@ -41,10 +48,11 @@ struct TcParams {
   int32_t num_kv_heads, group, rows;      // rows = group * alpha (R)
   int32_t rows_pad;             // R rounded up to 32
   int32_t row_blocks;           // ceil(R / 128): M-blocks of sweep A
-  int32_t chunk_tiles;          // key tiles per work item
+  int32_t chunk_tiles_a;        // 256-key tiles per work item of sweep A
+  int32_t chunk_tiles_b;        // 128-key tiles per work item of sweep B
   float scale_log2;             // log2(e) / sqrt(d)
-  float2* partial;              // sweep A out: [chunk][2][H_kv][R] (max, sum) in the log2 domain; the two
-                                // epilogue warp groups each write their own slot of a chunk
+  float2* partial;              // sweep A out: [chunk][slots][H_kv][R] (reference exponent, sum); slots = 2 with
+                                // two row blocks, 4 with one: every epilogue warp group writes its own slot
   const float* lse2;            // sweep B in:  [batch][H_kv][R]
   float* scores;                // sweep B out: [batch][H_kv][ld]
   int64_t ld_scores;
@@ -247,11 +255,10 @@ template <int D>
 struct TcSmem {
   static constexpr int kHalves = D / 64;                       // 64-element (128-byte) column blocks
   static constexpr int kQBytes = kTcMaxRows * D * 2;
-  static constexpr int kKStageBytes = kTcTileKeys * D * 2;
   static constexpr int kQOff = 0;
   static constexpr int kKOff = kQBytes;
-  static constexpr int kMiscOff = kKOff + kTcKStages * kKStageBytes;
-  static constexpr int kMiscBytes = 12288;                     // barriers, per-warp copies of lse2
+  static constexpr int kMiscOff = kKOff + kTcKBytes;
+  static constexpr int kMiscBytes = 20 * 1024;                 // barriers, exchange buffers, per-warp lse2 copies
   static constexpr int kTotal = kMiscOff + kMiscBytes + 1024;  // + slack for manual 1024-byte alignment
 };
 
@@ -261,16 +268,21 @@ __global__ void __launch_bounds__(kTcThreads, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
                 const TcParams p) {
   using L = TcSmem<D>;
+  constexpr int kTileKeys = SWEEP == 0 ? kTcTileKeysA : kTcTileKeysB;
+  constexpr int kStageBytes = kTileKeys * D * 2;               // one K tile in shared memory
+  constexpr int kKStages = kTcKBytes / kStageBytes >= 4 ? 4 : kTcKBytes / kStageBytes;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* q_s = smem + L::kQOff;
   uint8_t* k_s = smem + L::kKOff;
   uint8_t* misc = smem + L::kMiscOff;
   uint64_t* bars = reinterpret_cast<uint64_t*>(misc);          // [0..3] k_full, [4..7] k_empty, [8..11] t_full,
-                                                               // [12..15] t_empty, [16] q_full, [17] q_empty
+                                                               // [12..15] t_empty, [16] q_full, [17] q_empty,
+                                                               // [18..19] x_full, [20..21] x_empty
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 256);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 260);
-  float* lse_all = reinterpret_cast<float*>(misc + 1024);      // sweep B: [8 warps][256] lse2 of the current head
+  float* xch = reinterpret_cast<float*>(misc + 1024);          // sweep B: [2][128] partial sums handed between groups
+  float* lse_all = reinterpret_cast<float*>(misc + 4096);      // sweep B: [16 warps][256] lse2 of the current head
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t bar0 = smem_u32(bars);
@@ -279,20 +291,28 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   auto t_full = [&](int s) { return bar0 + 8u * (8 + s); };
   auto t_empty = [&](int s) { return bar0 + 8u * (12 + s); };
   const uint32_t q_full = bar0 + 8u * 16, q_empty = bar0 + 8u * 17;
+  auto x_full = [&](int s) { return bar0 + 8u * (18 + s); };
+  auto x_empty = [&](int s) { return bar0 + 8u * (20 + s); };
 
-  // TMEM stages: sweep A holds row_blocks x 128 key columns per stage, sweep B rows_pad columns.
-  int stage_cols = SWEEP == 0 ? p.row_blocks * 128 : p.rows_pad;
-  if (stage_cols <= 32) stage_cols = 32; else if (stage_cols <= 64) stage_cols = 64;
-  else if (stage_cols <= 128) stage_cols = 128; else stage_cols = 256;
-  const int t_stages = min(4, 512 / stage_cols);
+  // Accumulator stages.  Sweep A: 256 key columns per unit (one row block x one K tile): two stages.
+  // Sweep B: rows_pad columns per unit (one K tile), rounded up to a power of two: two to four stages.
+  int stage_cols = 256;
+  if (SWEEP == 1) {
+    stage_cols = p.rows_pad <= 32 ? 32 : (p.rows_pad <= 64 ? 64 : (p.rows_pad <= 128 ? 128 : 256));
+  }
+  const int t_stages = SWEEP == 0 ? 2 : min(4, 512 / stage_cols);
+  const bool two_blocks = p.row_blocks == 2;                   // sweep A: units per K tile
+  const int split_b = ((p.rows_pad / 2) + 31) & ~31;           // sweep B: columns [0, split) and [split, rows_pad)
+  const bool second_half = SWEEP == 0 || split_b < p.rows_pad; // do the groups 2, 3 have columns to read?
 
   // ---- set-up
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kTcKStages; ++s) { mbar_init(k_full(s), 1); mbar_init(k_empty(s), 1); }
-    const uint32_t consumers = (SWEEP == 0 && p.row_blocks == 2) ? 8 : 4;   // epilogue warps that read one tile
+    for (int s = 0; s < 4; ++s) { mbar_init(k_full(s), 1); mbar_init(k_empty(s), 1); }
+    const uint32_t consumers = second_half ? 8 : 4;            // epilogue warps that read one accumulator stage
     for (int s = 0; s < 4; ++s) { mbar_init(t_full(s), 1); mbar_init(t_empty(s), consumers); }
     mbar_init(q_full, 1);
     mbar_init(q_empty, 1);
+    for (int s = 0; s < 2; ++s) { mbar_init(x_full(s), 4); mbar_init(x_empty(s), 4); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -311,6 +331,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
 
   // ---- this CTA's contiguous range of work items
   const int32_t* off = SWEEP == 0 ? p.seq.stat_off : p.seq.score_off;
+  const int chunk_tiles = SWEEP == 0 ? p.chunk_tiles_a : p.chunk_tiles_b;
   const int total = p.num_kv_heads * off[p.seq.batch];
   const int per = total / gridDim.x, rem = total % gridDim.x;
   const int item0 = blockIdx.x * per + min(static_cast<int>(blockIdx.x), rem);
@@ -321,7 +342,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   if (warp == 0) {
     // =========================================================== TMA producer
     if (lane == 0) {
-      uint32_t it = 0, heads_loaded = 0;
+      uint32_t it = 0, heads_loaded = 0;                       // it counts K tiles
       int cur_b = -1, cur_h = -1;
       bool ok = true;
       for (int id = item0; id < item1 && ok; ++id) {
@@ -336,23 +357,23 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
           cur_b = w.b; cur_h = w.h;
         }
         const int keys = span_keys(w.b);
-        const int tile0 = w.c * p.chunk_tiles;
-        const int tile1 = min(tile0 + p.chunk_tiles, (keys + kTcTileKeys - 1) / kTcTileKeys);
+        const int tile0 = w.c * chunk_tiles;
+        const int tile1 = min(tile0 + chunk_tiles, (keys + kTileKeys - 1) / kTileKeys);
         for (int t = tile0; t < tile1 && ok; ++t, ++it) {
-          const int s = it % kTcKStages;
-          ok = mbar_wait(k_empty(s), ((it / kTcKStages) & 1) ^ 1, abort_flag);
+          const int s = it % kKStages;
+          ok = mbar_wait(k_empty(s), ((it / kKStages) & 1) ^ 1, abort_flag);
           if (!ok) break;
-          mbar_expect_tx(k_full(s), L::kKStageBytes);
+          mbar_expect_tx(k_full(s), kStageBytes);
           for (int half = 0; half < L::kHalves; ++half)
-            tma_load_4d(smem_u32(k_s) + s * L::kKStageBytes + half * kTcTileKeys * 128, &k_map, k_full(s), half * 64,
-                        t * kTcTileKeys, w.h, w.b);
+            tma_load_4d(smem_u32(k_s) + s * kStageBytes + half * kTileKeys * 128, &k_map, k_full(s), half * 64,
+                        t * kTileKeys, w.h, w.b);
         }
       }
       if (!ok) {
         // drain: wait (bounded) for the copies still in flight before shared memory is given up
-        const uint32_t first = it > kTcKStages ? it - kTcKStages : 0;
+        const uint32_t first = it > kKStages ? it - kKStages : 0;
         for (uint32_t j = first; j < it; ++j)
-          for (uint32_t spin = 0; spin < (1u << 16) && !mbar_test(k_full(j % kTcKStages), (j / kTcKStages) & 1); ++spin)
+          for (uint32_t spin = 0; spin < (1u << 16) && !mbar_test(k_full(j % kKStages), (j / kKStages) & 1); ++spin)
             __nanosleep(64);
         if (heads_loaded > 0)
           for (uint32_t spin = 0; spin < (1u << 16) && !mbar_test(q_full, (heads_loaded - 1) & 1); ++spin) __nanosleep(64);
@@ -361,10 +382,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   } else if (warp == 1) {
     // =========================================================== MMA issuer
     if (lane == 0) {
-      uint32_t it = 0, heads_seen = 0;
+      uint32_t it = 0, u = 0, heads_seen = 0;                  // it counts K tiles, u accumulator units
       int cur_b = -1, cur_h = -1;
       bool ok = true;
-      const uint32_t idesc = SWEEP == 0 ? instr_desc_bf16(128, kTcTileKeys) : instr_desc_bf16(kTcTileKeys, p.rows_pad);
+      const uint32_t idesc = SWEEP == 0 ? instr_desc_bf16(128, kTcTileKeysA) : instr_desc_bf16(kTcTileKeysB, p.rows_pad);
       for (int id = item0; id < item1 && ok; ++id) {
         const TcItem w = tc_item(off, p.seq.batch, p.num_kv_heads, id);
         if (w.b != cur_b || w.h != cur_h) {
@@ -380,35 +401,31 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
           last_of_head = nx.b != w.b || nx.h != w.h;
         }
         const int keys = span_keys(w.b);
-        const int tile0 = w.c * p.chunk_tiles;
-        const int tile1 = min(tile0 + p.chunk_tiles, (keys + kTcTileKeys - 1) / kTcTileKeys);
+        const int tile0 = w.c * chunk_tiles;
+        const int tile1 = min(tile0 + chunk_tiles, (keys + kTileKeys - 1) / kTileKeys);
         for (int t = tile0; t < tile1 && ok; ++t, ++it) {
-          const int s = it % kTcKStages, ts = it % t_stages;
-          ok = mbar_wait(k_full(s), (it / kTcKStages) & 1, abort_flag) &&
-               mbar_wait(t_empty(ts), ((it / t_stages) & 1) ^ 1, abort_flag);
+          const int s = it % kKStages;
+          ok = mbar_wait(k_full(s), (it / kKStages) & 1, abort_flag);
           if (!ok) break;
-          tc_fence_after();
-          const uint32_t k_addr = smem_u32(k_s) + s * L::kKStageBytes;
+          const uint32_t k_addr = smem_u32(k_s) + s * kStageBytes;
           const uint32_t q_addr = smem_u32(q_s);
-          const uint32_t d_addr = tmem_base + ts * stage_cols;
-          if (SWEEP == 0) {
-            for (int mb = 0; mb < p.row_blocks; ++mb)
-#pragma unroll
-              for (int kk = 0; kk < D / 16; ++kk) {
-                const uint32_t qa = q_addr + (kk / 4) * kTcMaxRows * 128 + mb * 128 * 128 + (kk % 4) * 32;
-                const uint32_t ka = k_addr + (kk / 4) * kTcTileKeys * 128 + (kk % 4) * 32;
-                tc_mma_bf16(d_addr + mb * 128, smem_desc_sw128(qa), smem_desc_sw128(ka), idesc, kk > 0);
-              }
-          } else {
+          const int units = SWEEP == 0 ? p.row_blocks : 1;
+          for (int rb = 0; rb < units && ok; ++rb, ++u) {
+            const int ts = u % t_stages;
+            ok = mbar_wait(t_empty(ts), ((u / t_stages) & 1) ^ 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t d_addr = tmem_base + ts * stage_cols;
 #pragma unroll
             for (int kk = 0; kk < D / 16; ++kk) {
-              const uint32_t qa = q_addr + (kk / 4) * kTcMaxRows * 128 + (kk % 4) * 32;
-              const uint32_t ka = k_addr + (kk / 4) * kTcTileKeys * 128 + (kk % 4) * 32;
-              tc_mma_bf16(d_addr, smem_desc_sw128(ka), smem_desc_sw128(qa), idesc, kk > 0);
+              const uint32_t qa = q_addr + (kk / 4) * kTcMaxRows * 128 + rb * 128 * 128 + (kk % 4) * 32;
+              const uint32_t ka = k_addr + (kk / 4) * kTileKeys * 128 + (kk % 4) * 32;
+              if (SWEEP == 0) tc_mma_bf16(d_addr, smem_desc_sw128(qa), smem_desc_sw128(ka), idesc, kk > 0);
+              else tc_mma_bf16(d_addr, smem_desc_sw128(ka), smem_desc_sw128(qa), idesc, kk > 0);
             }
+            tc_commit(t_full(ts));
           }
-          tc_commit(k_empty(s));
-          tc_commit(t_full(ts));
+          if (ok) tc_commit(k_empty(s));
         }
         if (ok && last_of_head) tc_commit(q_empty);
       }
@@ -417,92 +434,84 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     // =========================================================== epilogue
     const int e = warp - kTcEpiWarp0;
     const int quarter = warp & 3;               // TMEM lanes 32*quarter .. +31 are this warp's
-    const int half = e >> 2;                    // which half of the work of a lane this warp takes
+    const int grp = e >> 2;                     // 0..3
+    const int par = grp & 1;                    // this group reads the units u with u % 2 == par
+    const int ch = grp >> 1;                    // ... and this half of their columns
     const int lane_row = quarter * 32 + lane;   // TMEM lane of this thread
     const float c2 = p.scale_log2;
-    uint32_t it = 0;
+    uint32_t u = 0, mine = 0;                   // units seen by the CTA / units this group's pair has read
     int cur_b = -1, cur_h = -1;
     bool ok = true;
     for (int id = item0; id < item1 && ok; ++id) {
       const TcItem w = tc_item(off, p.seq.batch, p.num_kv_heads, id);
       const int n = p.seq.n[w.b], alpha = p.seq.alpha, P = n - alpha;
       const int keys = span_keys(w.b);
-      const int tile0 = w.c * p.chunk_tiles;
-      const int tile1 = min(tile0 + p.chunk_tiles, (keys + kTcTileKeys - 1) / kTcTileKeys);
+      const int tile0 = w.c * chunk_tiles;
+      const int tile1 = min(tile0 + chunk_tiles, (keys + kTileKeys - 1) / kTileKeys);
       if (SWEEP == 0) {
-        // thread -> window row.  Two row blocks: each warp group owns one block and sees every tile.
-        // One row block: the groups take alternate tiles of the same 128 rows.  Either way each group
-        // writes its own partial slot, so no exchange between warps is needed.
-        const bool two = p.row_blocks == 2;
-        const int r = (two ? half * 128 : 0) + lane_row;
+        // thread -> window row.  With two row blocks the unit parity is the row block, so a group always
+        // works on the same block; with one, the pairs of groups take alternate K tiles.  Either way a
+        // thread keeps one (reference, sum) per work item and every group writes its own partial slot.
+        const int r = (two_blocks ? par * 128 : 0) + lane_row;
         const int last_visible = P + (r % alpha);             // row (g, j) sees keys 0 .. P + j
+        const int units = p.row_blocks;
         float m = -INFINITY, z = 0.f;
-        for (int t = tile0; t < tile1 && ok; ++t, ++it) {
-          if (!two && static_cast<int>(it & 1u) != half) continue;   // the other group's tile
-          const int ts = it % t_stages;
-          ok = mbar_wait(t_full(ts), (it / t_stages) & 1, abort_flag);
-          ok = __all_sync(0xffffffffu, ok);                   // whole warp proceeds together or not at all
-          if (!ok) break;
-          tc_fence_after();
-          const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + ts * stage_cols +
-                                 (two ? half * 128 : 0);
-          const int key_base = t * kTcTileKeys;
-          const bool masked = key_base + kTcTileKeys - 1 > P; // tile reaches into the window: per-element mask
-          if (!masked) {
-            // the load of the next 32 columns is in flight while the current 32 are processed
-            uint32_t va[32], vb[32];
-            tc_ld32(taddr, va);
-#pragma unroll
-            for (int cg = 0; cg < kTcTileKeys; cg += 64) {
-              tc_wait_ld();
-              tc_ld32(taddr + cg + 32, vb);
-              rowstats_group(va, c2, m, z);
-              tc_wait_ld();
-              if (cg + 64 < kTcTileKeys) tc_ld32(taddr + cg + 64, va);
-              rowstats_group(vb, c2, m, z);
-            }
-          } else {
-            for (int cg = 0; cg < kTcTileKeys; cg += 32) {
-              uint32_t v[32];
-              tc_ld32(taddr + cg, v);
-              tc_wait_ld();
-              float gm = -INFINITY;
-#pragma unroll
-              for (int j = 0; j < 32; ++j) {
-                const bool vis = key_base + cg + j <= last_visible;
-                const float x = vis ? __uint_as_float(v[j]) * c2 : -INFINITY;
-                v[j] = __float_as_uint(x);
-                gm = fmaxf(gm, x);
+        for (int t = tile0; t < tile1 && ok; ++t) {
+          for (int rb = 0; rb < units && ok; ++rb, ++u) {
+            if (static_cast<int>(u & 1u) != par) continue;    // the other pair's unit
+            const int ts = u & 1;
+            ok = mbar_wait(t_full(ts), (u >> 1) & 1, abort_flag);
+            ok = __all_sync(0xffffffffu, ok);                 // whole warp proceeds together or not at all
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + ts * stage_cols + ch * 128;
+            const int key_base = t * kTcTileKeysA + ch * 128;
+            if (key_base + 127 <= P) {                        // every key visible to every row: no mask
+              for (int cg = 0; cg < 128; cg += 32) {
+                uint32_t v[32];
+                tc_ld32(taddr + cg, v);
+                tc_wait_ld();
+                rowstats_group(v, c2, m, z);
               }
-              if (gm > -INFINITY) {
-                const float mn = fmaxf(m, gm);
-                z *= ex2(m - mn);
-                m = mn;
-                float a0 = 0.f;
+            } else {
+              for (int cg = 0; cg < 128; cg += 32) {
+                uint32_t v[32];
+                tc_ld32(taddr + cg, v);
+                tc_wait_ld();
+                float gm = -INFINITY;
 #pragma unroll
-                for (int j = 0; j < 32; ++j) a0 += ex2(__uint_as_float(v[j]) - m);
-                z += a0;
+                for (int j = 0; j < 32; ++j) {
+                  const bool vis = key_base + cg + j <= last_visible;
+                  const float x = vis ? __uint_as_float(v[j]) * c2 : -INFINITY;
+                  v[j] = __float_as_uint(x);
+                  gm = fmaxf(gm, x);
+                }
+                if (gm > -INFINITY) {
+                  const float mn = fmaxf(m, gm);
+                  z *= ex2(m - mn);
+                  m = mn;
+                  float a0 = 0.f;
+#pragma unroll
+                  for (int j = 0; j < 32; ++j) a0 += ex2(__uint_as_float(v[j]) - m);
+                  z += a0;
+                }
               }
             }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(t_empty(ts));
           }
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(t_empty(ts));
         }
         if (!ok) break;
         if (r < p.rows) {
+          const int slots = two_blocks ? 2 : 4;
+          const int slot = two_blocks ? ch : grp;
           const int64_t chunk = off[w.b] + w.c;
-          float2* slot0 = p.partial + ((chunk * 2 + 0) * p.num_kv_heads + w.h) * p.rows;
-          float2* slot1 = p.partial + ((chunk * 2 + 1) * p.num_kv_heads + w.h) * p.rows;
-          if (two) {                                          // this group alone saw row r
-            slot0[r] = make_float2(m, z);
-            slot1[r] = make_float2(-INFINITY, 0.f);
-          } else {
-            (half == 0 ? slot0 : slot1)[r] = make_float2(m, z);
-          }
+          p.partial[((chunk * slots + slot) * p.num_kv_heads + w.h) * p.rows + r] = make_float2(m, z);
         }
       } else {
-        // thread -> key; the two warp groups take alternate tiles, each thread sums all rows of its key
+        // thread -> key.  The pairs of groups take alternate K tiles; inside a pair the groups split the
+        // window rows (columns) of a key and group ch = 1 hands its partial sum to group ch = 0.
         float* lse_s = lse_all + e * 256;                     // this warp's private copy of lse2
         if (w.b != cur_b || w.h != cur_h) {
           __syncwarp();
@@ -512,35 +521,47 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
           cur_b = w.b; cur_h = w.h;
         }
         float* srow = p.scores + (static_cast<int64_t>(w.b) * p.num_kv_heads + w.h) * p.ld_scores;
-        for (int t = tile0; t < tile1 && ok; ++t, ++it) {
-          if (static_cast<int>(it & 1u) != half) continue;    // the other group's tile
-          const int ts = it % t_stages;
-          ok = mbar_wait(t_full(ts), (it / t_stages) & 1, abort_flag);
-          ok = __all_sync(0xffffffffu, ok);                   // whole warp proceeds together or not at all
+        const int col0 = ch == 0 ? 0 : split_b, col1 = ch == 0 ? split_b : p.rows_pad;
+        for (int t = tile0; t < tile1 && ok; ++t, ++u) {
+          if (static_cast<int>(u & 1u) != par) continue;      // the other pair's tile
+          if (ch == 1 && !second_half) continue;              // nothing for this group to read
+          const int ts = u % t_stages;
+          ok = mbar_wait(t_full(ts), (u / t_stages) & 1, abort_flag);
+          ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           tc_fence_after();
           const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + ts * stage_cols;
           float acc[4] = {0.f, 0.f, 0.f, 0.f};
-          {
-            uint32_t va[32], vb[32];
-            tc_ld32(taddr, va);
-            for (int cg = 0; cg < p.rows_pad; cg += 64) {
-              const bool second = cg + 32 < p.rows_pad;
-              tc_wait_ld();
-              if (second) tc_ld32(taddr + cg + 32, vb);
-              score_group(va, c2, lse_s + cg, acc);
-              if (second) {
-                tc_wait_ld();
-                if (cg + 64 < p.rows_pad) tc_ld32(taddr + cg + 64, va);
-                score_group(vb, c2, lse_s + cg + 32, acc);
-              }
-            }
+          for (int cg = col0; cg < col1; cg += 32) {
+            uint32_t v[32];
+            tc_ld32(taddr + cg, v);
+            tc_wait_ld();
+            score_group(v, c2, lse_s + cg, acc);
           }
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(t_empty(ts));
-          const int i = t * kTcTileKeys + lane_row;
-          if (i < P) srow[i] = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+          float sum = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+          if (second_half) {
+            if (ch == 1) {
+              ok = mbar_wait(x_empty(par), (mine & 1) ^ 1, abort_flag);
+              ok = __all_sync(0xffffffffu, ok);
+              if (!ok) break;
+              xch[par * 128 + lane_row] = sum;
+              __syncwarp();
+              if (lane == 0) mbar_arrive(x_full(par));
+            } else {
+              ok = mbar_wait(x_full(par), mine & 1, abort_flag);
+              ok = __all_sync(0xffffffffu, ok);
+              if (!ok) break;
+              sum += xch[par * 128 + lane_row];
+              __syncwarp();
+              if (lane == 0) mbar_arrive(x_empty(par));
+            }
+          }
+          ++mine;
+          const int i = t * kTcTileKeysB + lane_row;
+          if (ch == 0 && i < P) srow[i] = sum;
         }
         if (!ok) break;
       }
