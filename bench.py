@@ -35,7 +35,9 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from ncu captures, keyed by
 # kernel name, valid only for the kernel sources whose digest is given: any change to csrc/ voids them.
 NCU_TRAFFIC = {
-    # "kernel": {"csrc_digest": "...", "bytes_per_key_row": ...}
+    # profiles/score_tc_llama3_70b_128k.md: (read + written) bytes / (n * H_kv) key rows
+    "rowstats_tc": {"csrc_digest": "3e998e5764c412fd", "bytes_per_key_row": 262.3},
+    "scores_tc": {"csrc_digest": "3e998e5764c412fd", "bytes_per_key_row": 262.8},
 }
 
 
@@ -70,7 +72,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
@@ -84,23 +86,28 @@ class ClockSampler:
         except subprocess.TimeoutExpired:
             self.proc.kill()
             out, _ = self.proc.communicate()
-        sm, mx, reasons = [], 0.0, set()
+        rows, mx, reasons = [], 0.0, set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in out.splitlines():
             parts = [x.strip() for x in line.split(",")]
             if len(parts) < 7:
                 continue
             try:
-                sm.append(float(parts[0]))
+                rows.append((float(parts[0]), float(parts[2])))
                 mx = max(mx, float(parts[1]))
             except ValueError:
                 continue
             for name, val in zip(names, parts[3:7]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
-        sm.sort()
-        med = sm[len(sm) // 2] if sm else None
-        return {"sm_mhz": med, "sm_max_mhz": mx or None, "reasons": sorted(reasons), "samples": len(sm)}
+        # samples under load: the sampler also runs a little before and after the timed region
+        peak_w = max((w for _, w in rows), default=0.0)
+        loaded = [r for r in rows if r[1] >= 0.5 * peak_w] or rows
+        sm = sorted(c for c, _ in loaded)
+        watts = sorted(w for _, w in loaded)
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": mx or None, "reasons": sorted(reasons),
+                "samples": len(rows), "samples_under_load": len(loaded),
+                "power_w": watts[len(watts) // 2] if watts else None}
 
 
 def graded_bytes_per_layer(w, lens, count_rows, esz):
@@ -195,7 +202,7 @@ class HostOut:
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama3_70b_128k")
