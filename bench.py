@@ -202,7 +202,8 @@ class HostOut:
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=None,
+                    help="timed steps; default: as many as fill about one second (at least 5)")
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama3_70b_128k")
@@ -215,6 +216,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    auto_steps = args.steps is None
+    if auto_steps:
+        args.steps = 5
 
     from paper_2406_02069_b200 import workloads
     w = workloads.WORKLOADS[args.workload]
@@ -261,6 +265,17 @@ def main():
     for _ in range(args.warmup):
         streaming.compress_model(cfg, layers, lens, out, ws)
     pkv.check_status(ws)
+    if auto_steps:                                                  # size the timed region to about a second
+        c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        c0.record()
+        streaming.compress_model(cfg, layers, lens, out, ws)
+        c1.record()
+        torch.cuda.synchronize()
+        args.steps = int(min(5000, max(5, round(1000.0 / max(c0.elapsed_time(c1), 1e-3)))))
+        if dist is not None:
+            t = torch.tensor([args.steps], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            args.steps = int(t.item())
     sampler = ClockSampler(local)
     sampler.start()
     time.sleep(0.3)

@@ -245,7 +245,6 @@ int launch_scores_tc(const pkv_config* c, const pkv_tensor& q, const pkv_tensor&
   tp.row_blocks = (sp.rows + 127) / 128;
   tp.scale_log2 = sp.scale_log2;
   tp.partial = sp.partial;
-  tp.lse2 = sp.lse2;
   tp.scores = sp.scores;
   tp.ld_scores = sp.ld_scores;
   tp.status = status;
@@ -282,14 +281,13 @@ int launch_scores_tc(const pkv_config* c, const pkv_tensor& q, const pkv_tensor&
   tp.seq.score_off[batch] = score_items;
   sp.seq = tp.seq;
   sp.slots_per_chunk = tp.row_blocks == 2 ? 2 : 4;    // partial slots each sweep-A work item writes
+  tp.slots_per_chunk = sp.slots_per_chunk;
+  tp.group_log2 = std::log2(static_cast<float>(sp.group));
 
   const int grid_a = static_cast<int>(std::min<long long>(sms, static_cast<long long>(stat_items) * sp.num_kv_heads));
   const int grid_b = static_cast<int>(std::min<long long>(sms, static_cast<long long>(score_items) * sp.num_kv_heads));
   score_tc_kernel<D, 0><<<grid_a, kTcThreads, TcSmem<D>::kTotal, st>>>(q_map, k_map_a, tp);
   mark(st, "rowstats_tc");
-  combine_stats_kernel<<<dim3((sp.rows + 31) / 32, sp.num_kv_heads, batch), kCombineThreads, 0, st>>>(
-      sp, std::log2(static_cast<float>(sp.group)));
-  mark(st, "combine_stats");
   score_tc_kernel<D, 1><<<grid_b, kTcThreads, TcSmem<D>::kTotal, st>>>(q_map, k_map_b, tp);
   mark(st, "scores_tc");
   return check_launch();
@@ -323,8 +321,10 @@ int run_scores(const pkv_config* c, const pkv_tensor& q, const pkv_tensor& k, co
 }
 
 // ---------------------------------------------------------------- select
+// With k/v/k_out given the kernel also copies the kept rows (fused eviction); otherwise it writes indices only.
 int run_select(const pkv_config* c, const float* scores, int64_t ld, const SeqTable& table, int batch, int max_n,
-               int32_t* indices, const Workspace& w, cudaStream_t st) {
+               int32_t* indices, const Workspace& w, cudaStream_t st, const pkv_tensor* k = nullptr,
+               const pkv_tensor* v = nullptr, void* k_out = nullptr, void* v_out = nullptr) {
   SelectParams sp{};
   sp.scores = scores;
   sp.ld_scores = ld;
@@ -333,6 +333,14 @@ int run_select(const pkv_config* c, const float* scores, int64_t ld, const SeqTa
   sp.num_kv_heads = c->num_kv_heads;
   sp.pool_radius = (c->pool_kernel - 1) / 2;
   sp.status = w.status;
+  if (k_out) {
+    sp.k = view(*k);
+    sp.v = view(*v);
+    sp.k_out = k_out;
+    sp.v_out = v_out;
+    sp.elem_bytes = c->dtype == PKV_DTYPE_FP32 ? 4 : 2;
+    sp.pieces = c->head_dim * sp.elem_bytes / 16;
+  }
   const int max_p = max_n - c->window;
   int cluster = 1;
   while (cluster < kSelMaxCluster && (max_p + cluster - 1) / cluster > 8192) cluster *= 2;
@@ -362,7 +370,7 @@ int run_select(const pkv_config* c, const float* scores, int64_t ld, const SeqTa
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   if (cudaLaunchKernelEx(&cfg, pool_select_kernel, sp) != cudaSuccess) return PKV_ERR_CUDA;
-  mark(st, "pool_select");
+  mark(st, k_out ? "pool_select_gather" : "pool_select");
   return check_launch();
 }
 
@@ -516,8 +524,7 @@ int pyramidkv_compress_layer(const pkv_config* cfg, int32_t layer, pkv_tensor q_
   for (int b = 0; b < batch; ++b) any_compress |= table.count[b] < table.n[b];
   if (any_compress || scores_or_null)
     if (int rc = run_scores(cfg, q_win, k, table, batch, scores, ld, w, st)) return rc;
-  if (int rc = run_select(cfg, scores, ld, table, batch, max_n, indices, w, st)) return rc;
-  return run_gather(cfg, k, v, indices, table, rows, k_out, v_out, st);
+  return run_select(cfg, scores, ld, table, batch, max_n, indices, w, st, &k, &v, k_out, v_out);
 }
 
 int pyramidkv_profile_layer(const pkv_config* cfg, int32_t layer, pkv_tensor q_win, pkv_tensor k, pkv_tensor v,

@@ -53,6 +53,13 @@ struct SelectParams {
   int32_t pool_radius;      // (w - 1) / 2
   int32_t cached;           // 1: every CTA's slice fits kSelSliceCap and lives in shared memory
   uint32_t* status;
+  // Optional fused eviction by gather (k_out == nullptr: indices only).  Once a head's list is complete
+  // the cluster that produced it copies the listed rows of K and V into the packed cache.
+  TensorView k, v;
+  void* k_out;
+  void* v_out;
+  int32_t elem_bytes;       // 4 or 2
+  int32_t pieces;           // 16-byte pieces per row = d * elem_bytes / 16
 };
 
 // Monotone map float -> uint32 (larger float, larger key).  -0 is folded into +0 first.
@@ -96,9 +103,8 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
     for (int j = tid; j < alpha; j += kSelThreads) out[k + j] = P + j;
   if (k >= P) {                                             // nothing to evict: identity list
     for (int i = rank * kSelThreads + tid; i < P; i += C * kSelThreads) out[i] = i;
-    return;                                                 // uniform over the cluster
   }
-  if (k == 0) return;
+  if (k > 0 && k < P) {                                     // (uniform over the cluster)
 
   const float* s = p.scores + (static_cast<int64_t>(b) * p.num_kv_heads + h) * p.ld_scores;
   const int slice = ((P + C - 1) / C + 31) & ~31;           // multiple of 32 positions per CTA
@@ -284,7 +290,27 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
     gt_before += __popc(bg);
     eq_before += __popc(be);
   }
-  cluster.sync();                                           // nobody leaves while its shared memory may be read
+  }
+  cluster.sync();              // the list is complete; nobody leaves while its shared memory may be read
+
+  // ---- 5. eviction by gather (appendix on torch.gather), spread over the cluster: 16 bytes of K and of V
+  //         per thread and step
+  if (p.k_out != nullptr) {
+    const int64_t row0 = p.seq.row_off[b] + static_cast<int64_t>(h) * count;
+    const int total = count * p.pieces;
+    const char* kb = static_cast<const char*>(p.k.ptr) + (b * p.k.sb + h * p.k.sh) * p.elem_bytes;
+    const char* vb = static_cast<const char*>(p.v.ptr) + (b * p.v.sb + h * p.v.sh) * p.elem_bytes;
+    for (int g = rank * kSelThreads + tid; g < total; g += C * kSelThreads) {
+      const int row = g / p.pieces, piece = g - row * p.pieces;
+      const int pos = __ldcg(out + row);                    // written by other CTAs of the cluster: skip L1
+      const int64_t dst = (row0 + row) * p.pieces + piece;
+      static_cast<uint4*>(p.k_out)[dst] =
+          reinterpret_cast<const uint4*>(kb + static_cast<int64_t>(pos) * p.k.st * p.elem_bytes)[piece];
+      if (p.v_out)
+        static_cast<uint4*>(p.v_out)[dst] =
+            reinterpret_cast<const uint4*>(vb + static_cast<int64_t>(pos) * p.v.st * p.elem_bytes)[piece];
+    }
+  }
 }
 
 }  // namespace pkv
