@@ -6,6 +6,7 @@
 #include <algorithm>
 #include <cstring>
 #include <mutex>
+#include <utility>
 
 #include "pkv_common.cuh"
 #include "pkv_gather.cuh"
@@ -128,6 +129,23 @@ TensorView view(const pkv_tensor& t) { return TensorView{t.ptr, t.stride_batch, 
 
 int check_launch() { return cudaPeekAtLastError() == cudaSuccess ? PKV_OK : PKV_ERR_CUDA; }
 
+// Launch with programmatic stream serialisation: the kernel may be scheduled while its predecessor in
+// the stream drains; the kernels order themselves with pdl_wait() (pkv_common.cuh).
+template <typename... KArgs, typename... Args>
+void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+
 // Optional per-kernel timing (pyramidkv_profile_layer): when armed, an event is recorded after every launch.
 struct StageTimer {
   cudaEvent_t ev[PKV_MAX_STAGES + 1];
@@ -155,11 +173,12 @@ int launch_scores_generic(ScoreParams& sp, int batch, cudaStream_t st) {
   sp.seq.stat_off[batch] = stat_tiles;
   sp.seq.score_off[batch] = score_tiles;
   sp.slots_per_chunk = 1;
-  rowstats_generic_kernel<T, D><<<dim3(stat_tiles, sp.num_kv_heads), kGenRowBlock, 0, st>>>(sp);
+  launch_pdl(rowstats_generic_kernel<T, D>, dim3(stat_tiles, sp.num_kv_heads), kGenRowBlock, 0, st, sp);
   mark(st, "rowstats_generic");
-  combine_stats_kernel<<<dim3((sp.rows + 31) / 32, sp.num_kv_heads, batch), kCombineThreads, 0, st>>>(sp, std::log2(static_cast<float>(sp.group)));
+  launch_pdl(combine_stats_kernel, dim3((sp.rows + 31) / 32, sp.num_kv_heads, batch), kCombineThreads, 0, st, sp,
+             std::log2(static_cast<float>(sp.group)));
   mark(st, "combine_stats");
-  scores_generic_kernel<T, D><<<dim3(score_tiles, sp.num_kv_heads), kGenScoreKeys, 0, st>>>(sp);
+  launch_pdl(scores_generic_kernel<T, D>, dim3(score_tiles, sp.num_kv_heads), kGenScoreKeys, 0, st, sp);
   mark(st, "scores_generic");
   return check_launch();
 }
@@ -245,6 +264,7 @@ int launch_scores_tc(const pkv_config* c, const pkv_tensor& q, const pkv_tensor&
   tp.row_blocks = (sp.rows + 127) / 128;
   tp.scale_log2 = sp.scale_log2;
   tp.partial = sp.partial;
+  tp.lse2 = sp.lse2;
   tp.scores = sp.scores;
   tp.ld_scores = sp.ld_scores;
   tp.status = status;
@@ -281,14 +301,15 @@ int launch_scores_tc(const pkv_config* c, const pkv_tensor& q, const pkv_tensor&
   tp.seq.score_off[batch] = score_items;
   sp.seq = tp.seq;
   sp.slots_per_chunk = tp.row_blocks == 2 ? 2 : 4;    // partial slots each sweep-A work item writes
-  tp.slots_per_chunk = sp.slots_per_chunk;
-  tp.group_log2 = std::log2(static_cast<float>(sp.group));
 
   const int grid_a = static_cast<int>(std::min<long long>(sms, static_cast<long long>(stat_items) * sp.num_kv_heads));
   const int grid_b = static_cast<int>(std::min<long long>(sms, static_cast<long long>(score_items) * sp.num_kv_heads));
-  score_tc_kernel<D, 0><<<grid_a, kTcThreads, TcSmem<D>::kTotal, st>>>(q_map, k_map_a, tp);
+  launch_pdl(score_tc_kernel<D, 0>, grid_a, kTcThreads, TcSmem<D>::kTotal, st, q_map, k_map_a, tp);
   mark(st, "rowstats_tc");
-  score_tc_kernel<D, 1><<<grid_b, kTcThreads, TcSmem<D>::kTotal, st>>>(q_map, k_map_b, tp);
+  launch_pdl(combine_stats_kernel, dim3((sp.rows + 31) / 32, sp.num_kv_heads, batch), kCombineThreads, 0, st, sp,
+             std::log2(static_cast<float>(sp.group)));
+  mark(st, "combine_stats");
+  launch_pdl(score_tc_kernel<D, 1>, grid_b, kTcThreads, TcSmem<D>::kTotal, st, q_map, k_map_b, tp);
   mark(st, "scores_tc");
   return check_launch();
 }
@@ -362,13 +383,15 @@ int run_select(const pkv_config* c, const float* scores, int64_t ld, const SeqTa
   cfg.blockDim = dim3(kSelThreads);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = cluster;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   if (cudaLaunchKernelEx(&cfg, pool_select_kernel, sp) != cudaSuccess) return PKV_ERR_CUDA;
   mark(st, k_out ? "pool_select_gather" : "pool_select");
   return check_launch();
@@ -391,7 +414,7 @@ int run_gather(const pkv_config* c, const pkv_tensor& k, const pkv_tensor& v, co
   const int64_t threads = total_rows * gp.pieces;
   if (threads == 0) return PKV_OK;
   const unsigned blocks = static_cast<unsigned>((threads + kGatherThreads - 1) / kGatherThreads);
-  gather_rows_kernel<<<blocks, kGatherThreads, 0, st>>>(gp);
+  launch_pdl(gather_rows_kernel, blocks, kGatherThreads, 0, st, gp);
   mark(st, "gather_rows");
   return check_launch();
 }

@@ -32,6 +32,14 @@ enum : uint32_t {
   kStatusWaitExpired = 1u << 1,      // a bounded wait ran out
 };
 
+// Programmatic dependent launch: every kernel of the library is launched so that it may start while
+// the kernel before it in the stream is still draining.  A kernel first lets its own successor be
+// scheduled (pdl_trigger), does whatever set-up touches no global memory, and then waits for the
+// preceding kernel to have completed and flushed its writes (pdl_wait) before it reads or writes
+// global memory.  Without a preceding kernel both are no-ops.
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ float to_float(float x) { return x; }
 __device__ __forceinline__ float to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
 

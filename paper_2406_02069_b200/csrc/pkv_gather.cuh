@@ -24,6 +24,8 @@ struct GatherParams {
 };
 
 __global__ void __launch_bounds__(kGatherThreads) gather_rows_kernel(const GatherParams p) {
+  pdl_trigger();
+  pdl_wait();
   const int64_t gid = static_cast<int64_t>(blockIdx.x) * kGatherThreads + threadIdx.x;
   const int64_t row = gid / p.pieces;
   const int piece = static_cast<int>(gid % p.pieces);

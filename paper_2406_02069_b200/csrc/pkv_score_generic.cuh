@@ -40,6 +40,8 @@ struct ScoreParams {
 template <typename T, int D>
 __global__ void __launch_bounds__(kGenRowBlock) rowstats_generic_kernel(const ScoreParams p) {
   __shared__ __align__(16) float ktile[kGenKeyTile][D];
+  pdl_trigger();
+  pdl_wait();
   const int tile = blockIdx.x, h = blockIdx.y;
   const int b = find_sequence(p.seq.stat_off, p.seq.batch, tile);
   const int n = p.seq.n[b], alpha = p.seq.alpha, P = n - alpha;
@@ -106,6 +108,8 @@ __global__ void __launch_bounds__(kGenRowBlock) rowstats_generic_kernel(const Sc
 constexpr int kCombineThreads = 1024;
 __global__ void __launch_bounds__(kCombineThreads) combine_stats_kernel(const ScoreParams p, float extra_log2) {
   __shared__ float sm[32][33], sz[32][33];
+  pdl_trigger();
+  pdl_wait();
   const int h = blockIdx.y, b = blockIdx.z;
   const int rl = threadIdx.x & 31, sg = threadIdx.x >> 5;
   const int r = blockIdx.x * 32 + rl;
@@ -146,6 +150,8 @@ template <typename T, int D>
 __global__ void __launch_bounds__(kGenScoreKeys) scores_generic_kernel(const ScoreParams p) {
   __shared__ __align__(16) float qs[kGenQRows][D];
   __shared__ float lse_s[kGenQRows];
+  pdl_trigger();
+  pdl_wait();
   const int tile = blockIdx.x, h = blockIdx.y;
   const int b = find_sequence(p.seq.score_off, p.seq.batch, tile);
   const int alpha = p.seq.alpha, P = p.seq.n[b] - alpha;

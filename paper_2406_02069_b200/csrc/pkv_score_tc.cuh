@@ -53,8 +53,7 @@ struct TcParams {
   float scale_log2;             // log2(e) / sqrt(d)
   float2* partial;              // sweep A out: [chunk][slots][H_kv][R] (reference exponent, sum); slots = 2 with
                                 // two row blocks, 4 with one: every epilogue warp group writes its own slot
-  int32_t slots_per_chunk;      // partial slots per sweep-A work item (2 or 4)
-  float group_log2;             // log2(G): folds the mean over the group's query heads into the normaliser
+  const float* lse2;            // sweep B in:  [batch][H_kv][R]
   float* scores;                // sweep B out: [batch][H_kv][ld]
   int64_t ld_scores;
   uint32_t* status;
@@ -279,12 +278,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   uint8_t* misc = smem + L::kMiscOff;
   uint64_t* bars = reinterpret_cast<uint64_t*>(misc);          // [0..3] k_full, [4..7] k_empty, [8..11] t_full,
                                                                // [12..15] t_empty, [16] q_full, [17] q_empty,
-                                                               // [18..19] x_full, [20..21] x_empty,
-                                                               // [22] lse_ready, [23] lse_copied
+                                                               // [18..19] x_full, [20..21] x_empty
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 256);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 260);
   float* xch = reinterpret_cast<float*>(misc + 1024);          // sweep B: [2][128] partial sums handed between groups
-  float* lse_sh = reinterpret_cast<float*>(misc + 2048);       // sweep B: [256] lse2 of the head being set up
   float* lse_all = reinterpret_cast<float*>(misc + 4096);      // sweep B: [16 warps][256] lse2 of the current head
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -296,7 +293,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   const uint32_t q_full = bar0 + 8u * 16, q_empty = bar0 + 8u * 17;
   auto x_full = [&](int s) { return bar0 + 8u * (18 + s); };
   auto x_empty = [&](int s) { return bar0 + 8u * (20 + s); };
-  const uint32_t lse_ready = bar0 + 8u * 22, lse_copied = bar0 + 8u * 23;
 
   // Accumulator stages.  Sweep A: 256 key columns per unit (one row block x one K tile): two stages.
   // Sweep B: rows_pad columns per unit (one K tile), rounded up to a power of two: two to four stages.
@@ -309,7 +305,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   const int split_b = ((p.rows_pad / 2) + 31) & ~31;           // sweep B: columns [0, split) and [split, rows_pad)
   const bool second_half = SWEEP == 0 || split_b < p.rows_pad; // do the groups 2, 3 have columns to read?
 
-  // ---- set-up
+  // ---- set-up (shared memory and TMEM only: it may overlap the tail of the preceding kernel)
+  pdl_trigger();
   if (threadIdx.x == 0) {
     for (int s = 0; s < 4; ++s) { mbar_init(k_full(s), 1); mbar_init(k_empty(s), 1); }
     const uint32_t consumers = second_half ? 8 : 4;            // epilogue warps that read one accumulator stage
@@ -317,8 +314,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     mbar_init(q_full, 1);
     mbar_init(q_empty, 1);
     for (int s = 0; s < 2; ++s) { mbar_init(x_full(s), 4); mbar_init(x_empty(s), 4); }
-    mbar_init(lse_ready, kTcEpiWarps);
-    mbar_init(lse_copied, kTcEpiWarps);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -334,6 +329,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();                                                  // from here on global memory is read and written
 
   // ---- this CTA's contiguous range of work items
   const int32_t* off = SWEEP == 0 ? p.seq.stat_off : p.seq.score_off;
@@ -445,7 +441,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     const int ch = grp >> 1;                    // ... and this half of their columns
     const int lane_row = quarter * 32 + lane;   // TMEM lane of this thread
     const float c2 = p.scale_log2;
-    uint32_t u = 0, mine = 0, heads_set = 0;    // units seen by the CTA / read by this group's pair / heads set up
+    uint32_t u = 0, mine = 0;                   // units seen by the CTA / units this group's pair has read
     int cur_b = -1, cur_h = -1;
     bool ok = true;
     for (int id = item0; id < item1 && ok; ++id) {
@@ -520,47 +516,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         // window rows (columns) of a key and group ch = 1 hands its partial sum to group ch = 0.
         float* lse_s = lse_all + e * 256;                     // this warp's private copy of lse2
         if (w.b != cur_b || w.h != cur_h) {
-          // New head: merge sweep A's partial (reference, sum) pairs into lse2_r = log2 sum_i 2^(x_ri) + log2 G.
-          // The 16 warps take 16 rows each, lanes stride over the partial slots; the result goes through
-          // one shared array into every warp's private copy.  This runs while the first K tiles of the
-          // head are already being loaded and multiplied.
-          if (heads_set > 0) {                                // everyone has copied the previous head's values
-            ok = mbar_wait(lse_copied, (heads_set - 1) & 1, abort_flag);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-          }
-          const int slot0 = p.seq.stat_off[w.b] * p.slots_per_chunk;
-          const int slot1 = p.seq.stat_off[w.b + 1] * p.slots_per_chunk;
-          const int64_t slot_stride = static_cast<int64_t>(p.num_kv_heads) * p.rows;
-          for (int rr = 0; rr < 256 / kTcEpiWarps; ++rr) {
-            const int r = e * (256 / kTcEpiWarps) + rr;
-            float m = -INFINITY, z = 0.f;
-            if (r < p.rows) {
-              const float2* src = p.partial + static_cast<int64_t>(w.h) * p.rows + r;
-              for (int t = slot0 + lane; t < slot1; t += 32) {
-                const float2 pz = src[t * slot_stride];
-                if (pz.x > -INFINITY) {                       // (-inf, 0): that slot saw no key of this row
-                  const float mn = fmaxf(m, pz.x);
-                  z = z * exp2f(m - mn) + pz.y * exp2f(pz.x - mn);
-                  m = mn;
-                }
-              }
-            }
-            float mm = m;
-            for (int o = 16; o > 0; o >>= 1) mm = fmaxf(mm, __shfl_xor_sync(0xffffffffu, mm, o));
-            float zz = m > -INFINITY ? z * exp2f(m - mm) : 0.f;
-            for (int o = 16; o > 0; o >>= 1) zz += __shfl_xor_sync(0xffffffffu, zz, o);
-            if (lane == 0) lse_sh[r] = r < p.rows ? mm + log2f(zz) + p.group_log2 : INFINITY;
-          }
           __syncwarp();
-          if (lane == 0) mbar_arrive(lse_ready);
-          ok = mbar_wait(lse_ready, heads_set & 1, abort_flag);
-          ok = __all_sync(0xffffffffu, ok);
-          if (!ok) break;
-          for (int i = lane; i < 256; i += 32) lse_s[i] = lse_sh[i];
+          const float* src = p.lse2 + (static_cast<int64_t>(w.b) * p.num_kv_heads + w.h) * p.rows;
+          for (int i = lane; i < 256; i += 32) lse_s[i] = i < p.rows ? src[i] : INFINITY;
           __syncwarp();
-          if (lane == 0) mbar_arrive(lse_copied);
-          ++heads_set;
           cur_b = w.b; cur_h = w.h;
         }
         float* srow = p.scores + (static_cast<int64_t>(w.b) * p.num_kv_heads + w.h) * p.ld_scores;

@@ -86,6 +86,8 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
   __shared__ uint32_t warp_gt[kSelWarps], warp_eq[kSelWarps];
   __shared__ uint32_t sel_digit, sel_above, lower_above, bound_digit;
 
+  pdl_trigger();
+  pdl_wait();
   cg::cluster_group cluster = cg::this_cluster();
   const int C = cluster.dim_blocks().x;
   const int rank = cluster.block_rank();
