@@ -73,6 +73,10 @@ struct Workspace {
   float2* partial;
   float* scores;
   int64_t ld_scores;
+  uint2* sel_cand;           // selection: candidate (key, position) pairs, [heads][sel_cand_stride]
+  int64_t sel_cand_stride;
+  uint32_t* sel_cnt;         // selection: pairs per cluster rank, [heads][kSelMaxCluster]
+  size_t score_scratch_bytes;   // bytes of the leading regions that the score kernels alone need
   size_t bytes;
 };
 
@@ -88,8 +92,12 @@ Workspace carve(const pkv_config* c, int batch, int max_n, void* base) {
   w.status = reinterpret_cast<uint32_t*>(take(kAlign));
   w.lse2 = reinterpret_cast<float*>(take(heads * rows * sizeof(float)));
   w.partial = reinterpret_cast<float2*>(take(heads * chunks * 2 * rows * sizeof(float2)));   // 2 slots per chunk
+  w.score_scratch_bytes = off;
   w.ld_scores = static_cast<int64_t>((static_cast<size_t>(max_n) + 63) / 64 * 64);
   w.scores = reinterpret_cast<float*>(take(heads * w.ld_scores * sizeof(float)));
+  w.sel_cand_stride = static_cast<int64_t>(max_n) + 32 * kSelMaxCluster;   // cluster * slice never exceeds this
+  w.sel_cand = reinterpret_cast<uint2*>(take(heads * w.sel_cand_stride * sizeof(uint2)));
+  w.sel_cnt = reinterpret_cast<uint32_t*>(take(heads * kSelMaxCluster * sizeof(uint32_t)));
   w.bytes = off;
   return w;
 }
@@ -354,6 +362,9 @@ int run_select(const pkv_config* c, const float* scores, int64_t ld, const SeqTa
   sp.num_kv_heads = c->num_kv_heads;
   sp.pool_radius = (c->pool_kernel - 1) / 2;
   sp.status = w.status;
+  sp.cand = w.sel_cand;
+  sp.cand_stride = w.sel_cand_stride;
+  sp.cand_cnt = w.sel_cnt;
   if (k_out) {
     sp.k = view(*k);
     sp.v = view(*v);
@@ -368,6 +379,7 @@ int run_select(const pkv_config* c, const float* scores, int64_t ld, const SeqTa
   const int slice = ((max_p + cluster - 1) / cluster + 31) & ~31;
   sp.cached = (slice <= kSelSliceCap && sp.pool_radius <= kSelHalo) ? 1 : 0;
   const size_t smem = sp.cached ? static_cast<size_t>(slice) * 6 + 8 * kSelHalo : 0;
+  sp.smem_pairs = static_cast<int32_t>(smem / sizeof(uint2));
   static bool attr_done[64] = {};  // the attribute is per device; setting it twice is harmless
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return PKV_ERR_CUDA;
@@ -636,12 +648,10 @@ extern "C" int pyramidkv_score_window_static(const pkv_config* cfg, pkv_tensor q
   int64_t rows;
   if (int rc = build_table(cfg, seq_lens, batch, 0, &table, &max_n, &rows)) return rc;
   if (ld_scores < max_n - cfg->window) return PKV_ERR_INVALID_ARG;
-  // Scratch the score kernels need: everything the usual workspace holds ahead of its score buffer.
-  // (the score buffer is the workspace's last region and is supplied by the caller here)
+  // Scratch the score kernels need: the workspace's leading regions (status word, normalisers, chunk
+  // statistics); the score buffer is supplied by the caller and the selection scratch is not used here.
   const Workspace sizing = carve(cfg, batch, max_n, nullptr);
-  const size_t score_region =
-      align_up(static_cast<size_t>(batch) * cfg->num_kv_heads * sizing.ld_scores * sizeof(float));
-  const size_t need = sizing.bytes - score_region;
+  const size_t need = sizing.score_scratch_bytes;
   if (need > PKV_STATIC_SCRATCH_BYTES) return PKV_ERR_STATIC_SCRATCH;
   void* base = static_scratch_address();
   if (!base) return PKV_ERR_CUDA;

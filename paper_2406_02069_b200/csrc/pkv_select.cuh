@@ -1,27 +1,28 @@
-// Fused max-pool + per-head top-k + window retention (Section 4.2.2).
+// Fused max-pool + per-head top-k + window retention (+ optional eviction by gather), Section 4.2.2.
 //
 // One thread-block cluster per (sequence, KV head).  The prefix positions are
 // split into contiguous slices, one per CTA of the cluster, and inside a CTA into
 // contiguous runs, one per warp, so that position order is (CTA rank, warp, order
 // inside the warp's run).
 //
-//  1. The CTA stages its slice of raw scores in shared memory (coalesced), pools
-//     them (halo of (w-1)/2 scores on both sides, clipped to the prefix) and keeps
-//     the pooled values as order-preserving 32-bit keys.
+//  1. Every CTA stages its slice of raw scores in shared memory (coalesced), pools
+//     them (halo of (w-1)/2 scores on both sides, clipped to the prefix) into
+//     order-preserving 32-bit keys held in registers.
 //  2. Candidate filter.  Every thread remembers the largest key it produced.  The
-//     k-th largest of those per-thread maxima is a lower bound L of the k-th largest
-//     key (k distinct keys >= it exist), found with one CTA-local 11-bit histogram.
-//     Each warp compacts the positions of its run whose key >= L into a candidate
-//     list, in order.  Typically only a few times k keys survive; in the worst case
-//     (all keys equal, or k larger than the thread count) L = 0 and all do.
-//  3. The k-th largest key T is found by a most-significant-digit radix search over
-//     the candidates in three passes (11, 11, 10 bits).  Per pass every CTA
-//     histograms its candidates, the histograms are summed across the cluster
-//     through distributed shared memory, and every CTA walks the sum to the same
-//     digit.  While summing, a CTA also accumulates the histograms of the CTAs that
-//     own earlier positions, which tells it how many kept keys precede its slice.
-//  4. kept = { i : key_i > T } plus the leftmost (k - |{key > T}|) positions with
-//     key_i == T, written in ascending position; the alpha window positions follow.
+//     k-th largest of those per-thread maxima is a lower bound of the k-th largest
+//     key (k distinct keys >= it exist); its top 22 bits are found with two CTA-local
+//     11-bit histogram passes.  The CTA writes the (key, position) pairs of its slice
+//     that reach the bound, in position order, to its region of a scratch buffer in
+//     global memory.  Typically a few times k pairs survive in the whole cluster; in
+//     the worst case (all keys equal, or k larger than the thread count) all do.
+//  3. After one cluster barrier CTA 0 alone finishes: it concatenates the regions
+//     (they are already in position order), finds the k-th largest key T by a
+//     most-significant-digit radix search in three passes (11, 11, 10 bits) over the
+//     candidates, and emits
+//       kept = { i : key_i > T } plus the leftmost (k - |{key > T}|) positions with key_i == T
+//     in ascending position; the alpha window positions follow.
+//  4. After a second cluster barrier all CTAs of the cluster copy the kept rows of K
+//     and V (when asked to).
 //
 // Ties therefore go to the smaller position and the list is canonical.  Only
 // block and cluster barriers are used for synchronisation (no flag spinning).
@@ -51,7 +52,11 @@ struct SelectParams {
   SeqTable seq;
   int32_t num_kv_heads;
   int32_t pool_radius;      // (w - 1) / 2
-  int32_t cached;           // 1: every CTA's slice fits kSelSliceCap and lives in shared memory
+  int32_t cached;           // 1: every CTA's slice fits kSelSliceCap and is staged in shared memory
+  int32_t smem_pairs;       // (key, position) pairs CTA 0 can hold in its dynamic shared memory
+  uint2* cand;              // scratch: [batch * H_kv][cand_stride] candidate pairs, one region per CTA rank
+  int64_t cand_stride;      // >= cluster * slice
+  uint32_t* cand_cnt;       // scratch: [batch * H_kv][kSelMaxCluster] pairs written per region
   uint32_t* status;
   // Optional fused eviction by gather (k_out == nullptr: indices only).  Once a head's list is complete
   // the cluster that produced it copies the listed rows of K and V into the packed cache.
@@ -78,13 +83,11 @@ __device__ __forceinline__ uint32_t pooled_key(const float* s, int i, int P, int
 // grid (cluster * H_kv, batch), cluster (cluster, 1, 1), block kSelThreads,
 // dynamic shared memory (6 bytes per slice position + 8 * kSelHalo) when cached, else none.
 __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectParams p) {
-  extern __shared__ __align__(16) uint32_t sel_smem[];      // [halo | slice | halo] raw scores, then pooled keys
-  uint32_t* keys = sel_smem + kSelHalo;
+  extern __shared__ __align__(16) uint32_t sel_smem[];      // [halo | slice | halo] raw scores; later CTA 0's pairs
   __shared__ uint32_t hist[2][kSelBins];                    // per-pass digit histogram (double buffered)
-  __shared__ uint32_t lower[kSelBins];                      // histogram summed over the CTAs of lower rank
   __shared__ uint32_t warp_sum[kSelWarps];
   __shared__ uint32_t warp_gt[kSelWarps], warp_eq[kSelWarps];
-  __shared__ uint32_t sel_digit, sel_above, lower_above, bound_digit;
+  __shared__ uint32_t sel_digit, sel_above, bound_digit;
 
   pdl_trigger();
   pdl_wait();
@@ -99,6 +102,7 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
   const int count = p.seq.count[b];
   const int k = count - alpha;                              // prefix rows to keep, 0 <= k <= P
   int32_t* out = p.indices + p.seq.row_off[b] + static_cast<int64_t>(h) * count;
+  const bool selecting = k > 0 && k < P;                    // uniform over the cluster
 
   // The window positions close the list (Section 4.2.1: always retained).
   if (rank == 0)
@@ -106,194 +110,199 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
   if (k >= P) {                                             // nothing to evict: identity list
     for (int i = rank * kSelThreads + tid; i < P; i += C * kSelThreads) out[i] = i;
   }
-  if (k > 0 && k < P) {                                     // (uniform over the cluster)
 
-  const float* s = p.scores + (static_cast<int64_t>(b) * p.num_kv_heads + h) * p.ld_scores;
+  const int64_t head = static_cast<int64_t>(b) * p.num_kv_heads + h;
   const int slice = ((P + C - 1) / C + 31) & ~31;           // multiple of 32 positions per CTA
-  const int lo = min(P, rank * slice), hi = min(P, lo + slice);
-  const int run = ((slice / kSelWarps) + 31) & ~31;         // positions per warp, multiple of 32
-  const int wlo = min(hi, lo + warp * run), whi = min(hi, wlo + run);
-  const bool cached = p.cached != 0;                        // then run <= kSelRunMax
-  uint16_t* cand = reinterpret_cast<uint16_t*>(keys + slice + kSelHalo) + warp * run;   // this warp's candidates
-  const int radius = p.pool_radius;
-
+  uint2* regions = p.cand + head * p.cand_stride;           // region of CTA c starts at c * slice
+  uint32_t* counts = p.cand_cnt + head * kSelMaxCluster;
   for (int i = tid; i < 2 * kSelBins; i += kSelThreads) (&hist[0][0])[i] = 0;
-  int n_items = whi - wlo;                                  // items this warp walks in the passes below
-  if (cached) {
-    // ---- 1. stage raw scores with a halo (-inf outside the prefix), pool, keep keys
-    float* raw = reinterpret_cast<float*>(keys);
-    for (int i = lo - kSelHalo + tid; i < hi + kSelHalo; i += kSelThreads)
-      raw[i - lo] = (i >= 0 && i < P) ? s[i] : -INFINITY;
-    __syncthreads();
-    uint32_t pk[kSelPerLane];
-    uint32_t tmax = 0;
-#pragma unroll
-    for (int it = 0; it < kSelPerLane; ++it) {
-      const int i = wlo + it * 32 + lane;
-      pk[it] = 0;
-      if (i < whi) {
-        float best = raw[i - lo];
-        for (int t = 1; t <= radius; ++t) best = fmaxf(best, fmaxf(raw[i - lo - t], raw[i - lo + t]));
-        pk[it] = ordered_key(best);
-        tmax = max(tmax, pk[it]);
-      }
-    }
-    __syncthreads();                                        // all raw scores read
-#pragma unroll
-    for (int it = 0; it < kSelPerLane; ++it) {
-      const int i = wlo + it * 32 + lane;
-      if (i < whi) keys[i - lo] = pk[it];
-    }
-    // ---- 2. lower bound of the k-th largest key: the k-th largest per-thread maximum, resolved to its
-    //         top 22 bits by two CTA-local histogram passes; then compaction of the keys >= bound
-    uint32_t bprefix = 0, bmask = 0, brem = static_cast<uint32_t>(k);
-    for (int bp = 0; bp < 2; ++bp) {
-      const int shift = bp == 0 ? 21 : 10;
-      // threads whose maximum left the searched prefix do not take part in the second pass
-      const uint32_t digit = ((tmax & bmask) == bprefix) ? ((tmax >> shift) & 2047u) : kSelBins;
-      const uint32_t peers = __match_any_sync(0xffffffffu, digit);
-      if (digit < kSelBins && lane == __ffs(peers) - 1) atomicAdd(&hist[1][digit], __popc(peers));
+
+  if (selecting) {
+    const float* s = p.scores + head * p.ld_scores;
+    const int lo = min(P, rank * slice), hi = min(P, lo + slice);
+    const int run = ((slice / kSelWarps) + 31) & ~31;       // positions per warp, multiple of 32
+    const int wlo = min(hi, lo + warp * run), whi = min(hi, wlo + run);
+    const int radius = p.pool_radius;
+    uint2* region = regions + static_cast<int64_t>(rank) * slice;
+    if (p.cached) {                                         // then run <= kSelRunMax
+      // ---- 1. stage raw scores with a halo (-inf outside the prefix) and pool
+      float* raw = reinterpret_cast<float*>(sel_smem + kSelHalo);
+      for (int i = lo - kSelHalo + tid; i < hi + kSelHalo; i += kSelThreads)
+        raw[i - lo] = (i >= 0 && i < P) ? s[i] : -INFINITY;
       __syncthreads();
-      const uint2 v = reinterpret_cast<const uint2*>(hist[1])[tid];
+      uint32_t pk[kSelPerLane];
+      uint32_t tmax = 0;
+#pragma unroll
+      for (int it = 0; it < kSelPerLane; ++it) {
+        const int i = wlo + it * 32 + lane;
+        pk[it] = 0;
+        if (i < whi) {
+          float best = raw[i - lo];
+          for (int t = 1; t <= radius; ++t) best = fmaxf(best, fmaxf(raw[i - lo - t], raw[i - lo + t]));
+          pk[it] = ordered_key(best);
+          tmax = max(tmax, pk[it]);
+        }
+      }
+      // ---- 2. lower bound of the k-th largest key: the k-th largest per-thread maximum, resolved to its
+      //         top 22 bits by two CTA-local histogram passes
+      uint32_t bprefix = 0, bmask = 0, brem = static_cast<uint32_t>(k);
+      for (int bp = 0; bp < 2; ++bp) {
+        const int shift = bp == 0 ? 21 : 10;
+        // threads whose maximum left the searched prefix do not take part in the second pass
+        const uint32_t digit = ((tmax & bmask) == bprefix) ? ((tmax >> shift) & 2047u) : kSelBins;
+        const uint32_t peers = __match_any_sync(0xffffffffu, digit);
+        if (digit < kSelBins && lane == __ffs(peers) - 1) atomicAdd(&hist[1][digit], __popc(peers));
+        __syncthreads();
+        const uint2 v = reinterpret_cast<const uint2*>(hist[1])[tid];
+        const uint32_t mine = v.x + v.y;
+        uint32_t incl = mine;
+        for (int off = 1; off < 32; off <<= 1) {
+          const uint32_t u = __shfl_down_sync(0xffffffffu, incl, off);
+          if (lane + off < 32) incl += u;
+        }
+        if (lane == 0) warp_sum[warp] = incl;
+        if (tid == 0) { bound_digit = kSelBins; sel_above = 0; }   // kSelBins: fewer than brem maxima in play
+        __syncthreads();
+        uint32_t higher = incl - mine;
+        for (int w2 = warp + 1; w2 < kSelWarps; ++w2) higher += warp_sum[w2];
+        if (higher < brem && brem <= higher + mine) {
+          const bool upper = higher + v.y >= brem;
+          bound_digit = upper ? 2 * tid + 1 : 2 * tid;
+          sel_above = upper ? higher : higher + v.y;
+        }
+        __syncthreads();
+        reinterpret_cast<uint2*>(hist[1])[tid] = make_uint2(0, 0);
+        const uint32_t bd = bound_digit;
+        if (bd == kSelBins) {                               // cannot bound (k exceeds the thread count): keep all
+          if (bp == 0) { bprefix = 0; bmask = 0; }
+          __syncthreads();
+          break;
+        }
+        bprefix |= bd << shift;
+        bmask |= 2047u << shift;
+        brem -= sel_above;
+        __syncthreads();                                    // histogram zeroed, bound_digit consumed
+      }
+      const uint32_t bound = bprefix;                       // lower edge of the resolved digits
+      // candidates of this warp's run, then their place among the CTA's
+      uint32_t wc = 0;
+#pragma unroll
+      for (int it = 0; it < kSelPerLane; ++it) {
+        const int i = wlo + it * 32 + lane;
+        wc += __popc(__ballot_sync(0xffffffffu, i < whi && pk[it] >= bound));
+      }
+      if (lane == 0) warp_gt[warp] = wc;
+      __syncthreads();
+      uint32_t base = 0;
+      for (int w2 = 0; w2 < warp; ++w2) base += warp_gt[w2];
+      if (tid == kSelThreads - 1) counts[rank] = base + wc;
+#pragma unroll
+      for (int it = 0; it < kSelPerLane; ++it) {
+        const int i = wlo + it * 32 + lane;
+        const bool c = i < whi && pk[it] >= bound;
+        const uint32_t bal = __ballot_sync(0xffffffffu, c);
+        if (c) region[base + __popc(bal & lt)] = make_uint2(pk[it], static_cast<uint32_t>(i));
+        base += __popc(bal);
+      }
+    } else {
+      // slices too long for shared memory, or a very wide pool: every position is a candidate
+      for (int i = lo + tid; i < hi; i += kSelThreads) region[i - lo] = make_uint2(pooled_key(s, i, P, radius), i);
+      if (tid == 0) counts[rank] = hi - lo;
+    }
+  }
+  cluster.sync();                                           // every region and its count are written
+
+  if (selecting && rank == 0) {
+    // ---- 3. CTA 0: concatenate the regions, radix search, emit
+    uint32_t pre[kSelMaxCluster + 1];
+    pre[0] = 0;
+#pragma unroll
+    for (int c = 0; c < kSelMaxCluster; ++c) pre[c + 1] = pre[c] + (c < C ? __ldcg(counts + c) : 0u);
+    const int N = static_cast<int>(pre[kSelMaxCluster]);
+    auto fetch = [&](int j) -> uint2 {                      // pair j of the concatenation, from global memory
+      int c = 0;
+#pragma unroll
+      for (int q = 1; q < kSelMaxCluster; ++q) c += static_cast<uint32_t>(j) >= pre[q] ? 1 : 0;
+      return __ldcg(regions + static_cast<int64_t>(c) * slice + (j - static_cast<int>(pre[c])));
+    };
+    uint2* flat = reinterpret_cast<uint2*>(sel_smem);
+    const int held = min(N, p.smem_pairs);
+    for (int j = tid; j < held; j += kSelThreads) flat[j] = fetch(j);
+    __syncthreads();
+    auto item = [&](int j) -> uint2 { return j < held ? flat[j] : fetch(j); };
+
+    uint32_t prefix = 0, mask = 0, remaining = k;
+    for (int pass = 0; pass < 3; ++pass) {
+      const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
+      const uint32_t dmask = pass == 2 ? 1023u : 2047u;
+      uint32_t* hcur = hist[pass & 1];
+      for (int j0 = warp * 32; j0 < N; j0 += kSelThreads) {
+        const int j = j0 + lane;
+        uint32_t digit = kSelBins;                          // kSelBins = does not take part
+        if (j < N) {
+          const uint32_t key = item(j).x;
+          if ((key & mask) == prefix) digit = (key >> shift) & dmask;
+        }
+        const uint32_t peers = __match_any_sync(0xffffffffu, digit);
+        if (digit < kSelBins && lane == __ffs(peers) - 1) atomicAdd(&hcur[digit], __popc(peers));
+      }
+      __syncthreads();
+      const uint2 v = reinterpret_cast<const uint2*>(hcur)[tid];           // every thread owns two adjacent digits
+      reinterpret_cast<uint2*>(hist[(pass + 1) & 1])[tid] = make_uint2(0, 0);   // next pass's buffer
       const uint32_t mine = v.x + v.y;
-      uint32_t incl = mine;
+      uint32_t incl = mine;                                 // keys in this and the higher pairs of the warp
       for (int off = 1; off < 32; off <<= 1) {
         const uint32_t u = __shfl_down_sync(0xffffffffu, incl, off);
         if (lane + off < 32) incl += u;
       }
       if (lane == 0) warp_sum[warp] = incl;
-      if (tid == 0) { bound_digit = kSelBins; sel_above = 0; }   // kSelBins: fewer than brem maxima in play
       __syncthreads();
       uint32_t higher = incl - mine;
       for (int w2 = warp + 1; w2 < kSelWarps; ++w2) higher += warp_sum[w2];
-      if (higher < brem && brem <= higher + mine) {
-        const bool upper = higher + v.y >= brem;
-        bound_digit = upper ? 2 * tid + 1 : 2 * tid;
-        sel_above = upper ? higher : higher + v.y;
+      if (higher < remaining && remaining <= higher + mine) {  // exactly one thread: the k-th key is in its pair
+        if (higher + v.y >= remaining) { sel_digit = 2 * tid + 1; sel_above = higher; }
+        else { sel_digit = 2 * tid; sel_above = higher + v.y; }
       }
       __syncthreads();
-      reinterpret_cast<uint2*>(hist[1])[tid] = make_uint2(0, 0);
-      const uint32_t bd = bound_digit;
-      if (bd == kSelBins) {                                 // cannot bound (k exceeds the thread count): keep all
-        if (bp == 0) { bprefix = 0; bmask = 0; }
-        __syncthreads();
-        break;
-      }
-      bprefix |= bd << shift;
-      bmask |= 2047u << shift;
-      brem -= sel_above;
-      __syncthreads();                                      // histogram zeroed, bound_digit consumed
+      prefix |= sel_digit << shift;
+      mask |= dmask << shift;
+      remaining -= sel_above;
+      __syncthreads();                                      // sel_* are rewritten next pass
     }
-    const uint32_t bound = bprefix;                         // lower edge of the resolved digits
-    int ncand = 0;
-#pragma unroll
-    for (int it = 0; it < kSelPerLane; ++it) {
-      const int i = wlo + it * 32 + lane;
-      const bool c = i < whi && pk[it] >= bound;
-      const uint32_t bal = __ballot_sync(0xffffffffu, c);
-      if (c) cand[ncand + __popc(bal & lt)] = static_cast<uint16_t>(i - lo);
-      ncand += __popc(bal);
-    }
-    n_items = ncand;
-    __syncwarp();
-  }
-  __syncthreads();
-  // item j of this warp -> (position, key)
-  auto item_pos = [&](int j) -> int { return cached ? lo + cand[j] : wlo + j; };
-  auto item_key = [&](int pos) -> uint32_t { return cached ? keys[pos - lo] : pooled_key(s, pos, P, radius); };
+    const uint32_t T = prefix;                              // the k-th largest key
+    const uint32_t need_eq = remaining;                     // ties at T to take, from the left
 
-  // ---- 3. radix search for the k-th largest key
-  uint32_t prefix = 0, mask = 0, remaining = k;
-  uint32_t gt_before_cta = 0, eq_before_cta = 0;            // kept-candidate keys owned by lower-rank CTAs
-  for (int pass = 0; pass < 3; ++pass) {
-    const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
-    const uint32_t dmask = pass == 2 ? 1023u : 2047u;
-    uint32_t* hcur = hist[pass & 1];
-    for (int j0 = 0; j0 < n_items; j0 += 32) {
+    // keys above / at the threshold, warp by warp over contiguous chunks of the concatenation
+    const int chunk = (((N + kSelWarps - 1) / kSelWarps) + 31) & ~31;
+    const int j_lo = min(N, warp * chunk), j_hi = min(N, j_lo + chunk);
+    uint32_t ngt = 0, neq = 0;
+    for (int j0 = j_lo; j0 < j_hi; j0 += 32) {
       const int j = j0 + lane;
-      uint32_t digit = kSelBins;                            // kSelBins = does not take part
-      if (j < n_items) {
-        const uint32_t key = item_key(item_pos(j));
-        if ((key & mask) == prefix) digit = (key >> shift) & dmask;
-      }
-      const uint32_t peers = __match_any_sync(0xffffffffu, digit);
-      if (digit < kSelBins && lane == __ffs(peers) - 1) atomicAdd(&hcur[digit], __popc(peers));
+      const uint32_t key = j < j_hi ? item(j).x : 0u;
+      ngt += __popc(__ballot_sync(0xffffffffu, j < j_hi && key > T));
+      neq += __popc(__ballot_sync(0xffffffffu, j < j_hi && key == T));
     }
-    cluster.sync();                                         // all histograms of this pass complete
-    // every thread owns two adjacent digits
-    uint32_t tot[2] = {0, 0}, low[2] = {0, 0};
-#pragma unroll
-    for (int c = 0; c < kSelMaxCluster; ++c)
-      if (c < C) {
-        const uint2 v = reinterpret_cast<const uint2*>(cluster.map_shared_rank(hcur, c))[tid];
-        tot[0] += v.x; tot[1] += v.y;
-        if (c < rank) { low[0] += v.x; low[1] += v.y; }
-      }
-    lower[2 * tid] = low[0]; lower[2 * tid + 1] = low[1];
-    reinterpret_cast<uint2*>(hist[(pass + 1) & 1])[tid] = make_uint2(0, 0);   // next pass's buffer
-    // keys in digits above this thread's pair: suffix sums inside the warp, then over warps
-    const uint32_t mine = tot[0] + tot[1];
-    uint32_t incl = mine;
-    for (int off = 1; off < 32; off <<= 1) {
-      const uint32_t v = __shfl_down_sync(0xffffffffu, incl, off);
-      if (lane + off < 32) incl += v;
+    if (lane == 0) { warp_gt[warp] = ngt; warp_eq[warp] = neq; }
+    __syncthreads();
+    uint32_t gt_before = 0, eq_before = 0;
+    for (int w2 = 0; w2 < warp; ++w2) { gt_before += warp_gt[w2]; eq_before += warp_eq[w2]; }
+    if (tid == kSelThreads - 1) {                           // the last thread can see the grand total
+      if (gt_before + ngt + min(eq_before + neq, need_eq) != static_cast<uint32_t>(k))
+        atomicOr(p.status, kStatusSelectMismatch);
     }
-    if (lane == 0) warp_sum[warp] = incl;
-    if (tid == 0) lower_above = 0;
-    __syncthreads();
-    uint32_t higher = incl - mine;
-    for (int w2 = warp + 1; w2 < kSelWarps; ++w2) higher += warp_sum[w2];
-    if (higher < remaining && remaining <= higher + mine) {  // exactly one thread: the k-th key is in its pair
-      if (higher + tot[1] >= remaining) { sel_digit = 2 * tid + 1; sel_above = higher; }
-      else { sel_digit = 2 * tid; sel_above = higher + tot[1]; }
+    // rank of a kept position = (#greater before it) + min(#equal before it, need_eq)
+    for (int j0 = j_lo; j0 < j_hi; j0 += 32) {
+      const int j = j0 + lane;
+      const uint2 kv = j < j_hi ? item(j) : make_uint2(0u, 0u);
+      const bool is_gt = j < j_hi && kv.x > T, is_eq = j < j_hi && kv.x == T;
+      const uint32_t bg = __ballot_sync(0xffffffffu, is_gt), be = __ballot_sync(0xffffffffu, is_eq);
+      const uint32_t g = gt_before + __popc(bg & lt), e = eq_before + __popc(be & lt);
+      if (is_gt || (is_eq && e < need_eq)) out[g + min(e, need_eq)] = static_cast<int32_t>(kv.y);
+      gt_before += __popc(bg);
+      eq_before += __popc(be);
     }
-    __syncthreads();
-    const uint32_t dsel = sel_digit;
-    // lower-rank keys in digits above the selected one are all kept: they precede this CTA's output
-    uint32_t la = (2u * tid > dsel ? low[0] : 0u) + (2u * tid + 1u > dsel ? low[1] : 0u);
-    for (int off = 16; off > 0; off >>= 1) la += __shfl_down_sync(0xffffffffu, la, off);
-    if (lane == 0 && la) atomicAdd(&lower_above, la);
-    __syncthreads();
-    gt_before_cta += lower_above;
-    if (pass == 2) eq_before_cta = lower[dsel];
-    prefix |= dsel << shift;
-    mask |= dmask << shift;
-    remaining -= sel_above;
-    __syncthreads();                                        // sel_* and lower_above are rewritten next pass
   }
-  const uint32_t T = prefix;                                // the k-th largest key
-  const uint32_t need_eq = remaining;                       // ties at T to take, from the left
-
-  // ---- 4. keys above / at the threshold inside this CTA, warp by warp, then emit in position order
-  uint32_t ngt = 0, neq = 0;
-  for (int j0 = 0; j0 < n_items; j0 += 32) {
-    const int j = j0 + lane;
-    const uint32_t key = j < n_items ? item_key(item_pos(j)) : 0u;
-    ngt += __popc(__ballot_sync(0xffffffffu, j < n_items && key > T));
-    neq += __popc(__ballot_sync(0xffffffffu, j < n_items && key == T));
-  }
-  if (lane == 0) { warp_gt[warp] = ngt; warp_eq[warp] = neq; }
-  __syncthreads();
-  uint32_t gt_before = gt_before_cta, eq_before = eq_before_cta;
-  for (int w2 = 0; w2 < warp; ++w2) { gt_before += warp_gt[w2]; eq_before += warp_eq[w2]; }
-  if (rank == C - 1 && tid == kSelThreads - 1) {            // the last thread can see the grand total
-    if (gt_before + ngt + min(eq_before + neq, need_eq) != static_cast<uint32_t>(k))
-      atomicOr(p.status, kStatusSelectMismatch);
-  }
-  // rank of a kept position = (#greater before it) + min(#equal before it, need_eq)
-  for (int j0 = 0; j0 < n_items; j0 += 32) {
-    const int j = j0 + lane;
-    const int pos = j < n_items ? item_pos(j) : 0;
-    const uint32_t key = j < n_items ? item_key(pos) : 0u;
-    const bool is_gt = j < n_items && key > T, is_eq = j < n_items && key == T;
-    const uint32_t bg = __ballot_sync(0xffffffffu, is_gt), be = __ballot_sync(0xffffffffu, is_eq);
-    const uint32_t g = gt_before + __popc(bg & lt), e = eq_before + __popc(be & lt);
-    if (is_gt || (is_eq && e < need_eq)) out[g + min(e, need_eq)] = pos;
-    gt_before += __popc(bg);
-    eq_before += __popc(be);
-  }
-  }
-  cluster.sync();              // the list is complete; nobody leaves while its shared memory may be read
+  cluster.sync();                                           // the list is complete
 
   // ---- 5. eviction by gather (appendix on torch.gather), spread over the cluster: 16 bytes of K and of V
   //         per thread and step
