@@ -224,6 +224,29 @@ int pyramidkv_compress_layer(const pkv_config* cfg, int32_t layer,
                              void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Hand-off from the prefill attention (Section 4.1: the scores come from the very attention rows the
+ * prefill has just computed, Eq. 2).  A prefill attention kernel that ran over the window rows
+ * already holds each row's log-sum-exp; given it, the first of the two K sweeps (the one that only
+ * finds the row normalisers) is skipped and the scores need a single pass over K.
+ *   window_lse  device, [batch][H_q][alpha] floats, contiguous: for query head g and window row j of
+ *               sequence b the natural logarithm of  sum over keys i <= P_b + j of exp(q . k_i / sqrt(d)),
+ *               i.e. the causal softmax denominator of that row in log form.
+ * Everything else as pyramidkv_score_window / pyramidkv_compress_layer; results agree with them to
+ * rounding when window_lse is exact.  A wrong window_lse gives wrongly scaled scores: it is not
+ * checked.  Errors: as the base calls, plus INVALID_ARG for a null window_lse.
+ */
+int pyramidkv_score_window_lse(const pkv_config* cfg, pkv_tensor q_win, pkv_tensor k, const float* window_lse,
+                               const int32_t* seq_lens, int32_t batch,
+                               float* scores, int64_t ld_scores,
+                               void* workspace, size_t workspace_bytes, void* stream);
+int pyramidkv_compress_layer_lse(const pkv_config* cfg, int32_t layer,
+                                 pkv_tensor q_win, pkv_tensor k, pkv_tensor v, const float* window_lse,
+                                 const int32_t* seq_lens, int32_t batch,
+                                 void* k_out, void* v_out, int32_t* indices,
+                                 float* scores_or_null, int64_t ld_scores,
+                                 void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Measuring aid; the paper has no counterpart.  Same arguments and results as
  * pyramidkv_compress_layer, but a CUDA event is recorded after every kernel the
  * call launches, the stream is synchronised, and the device time of each kernel
@@ -239,6 +262,15 @@ int pyramidkv_profile_layer(const pkv_config* cfg, int32_t layer,
                             float* scores_or_null, int64_t ld_scores,
                             void* workspace, size_t workspace_bytes, void* stream,
                             float* stage_ms, char (*stage_names)[32], int32_t* num_stages);
+
+/* The same measuring aid for pyramidkv_compress_layer_lse. */
+int pyramidkv_profile_layer_lse(const pkv_config* cfg, int32_t layer,
+                                pkv_tensor q_win, pkv_tensor k, pkv_tensor v, const float* window_lse,
+                                const int32_t* seq_lens, int32_t batch,
+                                void* k_out, void* v_out, int32_t* indices,
+                                float* scores_or_null, int64_t ld_scores,
+                                void* workspace, size_t workspace_bytes, void* stream,
+                                float* stage_ms, char (*stage_names)[32], int32_t* num_stages);
 
 /*
  * Synchronises `stream` and reads the workspace status word.  For tests and

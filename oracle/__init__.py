@@ -49,6 +49,9 @@ def _load() -> ctypes.CDLL:
         lib.orc_window_scores.argtypes = [ctypes.c_void_p, ctypes.c_void_p] + [ctypes.c_int] * 6 + \
                                          [ctypes.c_void_p, ctypes.c_void_p]
         lib.orc_window_scores.restype = None
+        lib.orc_window_scores_lse.argtypes = [ctypes.c_void_p, ctypes.c_void_p] + [ctypes.c_int] * 6 + \
+                                             [ctypes.c_void_p] * 3
+        lib.orc_window_scores_lse.restype = None
         lib.orc_pool_max.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_void_p]
         lib.orc_pool_max.restype = ctypes.c_int
         lib.orc_select_topk.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_void_p]
@@ -107,6 +110,18 @@ def window_scores(q_win: torch.Tensor, k: torch.Tensor):
     _load().orc_window_scores(q_win.data_ptr(), k.data_ptr(), _dtype_code(k), hq, hkv, d, alpha, n,
                               scores.ctypes.data, mass.ctypes.data)
     return scores, mass
+
+
+def window_lse(q_win: torch.Tensor, k: torch.Tensor) -> np.ndarray:
+    """Natural-log softmax denominators of the window rows, float64 [H_q][alpha] (Eq. 2, causal rows)."""
+    q_win, k = _host(q_win), _host(k)
+    hq, alpha, d = q_win.shape
+    hkv, n, _ = k.shape
+    scores = np.zeros((hkv, n - alpha), dtype=np.float32)
+    lse = np.zeros((hq, alpha), dtype=np.float64)
+    _load().orc_window_scores_lse(q_win.data_ptr(), k.data_ptr(), _dtype_code(k), hq, hkv, d, alpha, n,
+                                  scores.ctypes.data, None, lse.ctypes.data)
+    return lse
 
 
 def pool_max(x: np.ndarray, w: int) -> np.ndarray:

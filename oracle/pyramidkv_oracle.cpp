@@ -112,8 +112,10 @@ int orc_kept_count(int avg_budget, int alpha, int k_layer, int n) {
 //   window_mass [H_kv]      double, may be null: the same sum taken over the
 //                           window columns i >= P, so that for every head
 //                           sum_i scores + window_mass = alpha.
-void orc_window_scores(const void* q, const void* k, int dtype, int num_q_heads, int num_kv_heads,
-                       int d, int alpha, int n, float* scores, double* window_mass) {
+//   row_lse     [H_q][alpha] double, may be null: log of each row's softmax denominator,
+//                           log sum_{i <= P+j} exp(logit[i]) (what a prefill attention kernel keeps).
+void orc_window_scores_lse(const void* q, const void* k, int dtype, int num_q_heads, int num_kv_heads,
+                           int d, int alpha, int n, float* scores, double* window_mass, double* row_lse) {
   const int group = num_q_heads / num_kv_heads;
   const int P = n - alpha;
   const double scale = 1.0 / std::sqrt(static_cast<double>(d));
@@ -148,6 +150,7 @@ void orc_window_scores(const void* q, const void* k, int dtype, int num_q_heads,
         for (int i = 0; i < visible; ++i) logit[i] = std::exp(logit[i] - mx);
         double z = 0.0;
         for (int i = 0; i < visible; ++i) z += logit[i];
+        if (row_lse) row_lse[static_cast<int64_t>(hq) * alpha + j] = mx + std::log(z);
         // Eq. 3: add this row's attention to every key it sees.
 #pragma omp parallel for schedule(static)
         for (int i = 0; i < visible; ++i) acc[i] += logit[i] / z;
@@ -162,6 +165,11 @@ void orc_window_scores(const void* q, const void* k, int dtype, int num_q_heads,
       window_mass[h] = wm * inv_group;
     }
   }
+}
+
+void orc_window_scores(const void* q, const void* k, int dtype, int num_q_heads, int num_kv_heads,
+                       int d, int alpha, int n, float* scores, double* window_mass) {
+  orc_window_scores_lse(q, k, dtype, num_q_heads, num_kv_heads, d, alpha, n, scores, window_mass, nullptr);
 }
 
 // ---------------------------------------------------------------------------

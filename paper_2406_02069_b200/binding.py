@@ -27,7 +27,8 @@ PKV_STATIC_SCRATCH_BYTES = 8 << 20
 EXPORTS = ("pyramidkv_strerror", "pyramidkv_layer_budgets", "pyramidkv_kept_count",
            "pyramidkv_workspace_bytes", "pyramidkv_score_window", "pyramidkv_select_topk",
            "pyramidkv_gather_compact", "pyramidkv_compress_layer", "pyramidkv_profile_layer",
-           "pyramidkv_check_status", "pyramidkv_score_window_static")
+           "pyramidkv_check_status", "pyramidkv_score_window_static", "pyramidkv_score_window_lse",
+           "pyramidkv_compress_layer_lse", "pyramidkv_profile_layer_lse")
 PKV_MAX_STAGES = 8
 
 
@@ -71,6 +72,10 @@ def _load() -> ctypes.CDLL:
     lib.pyramidkv_compress_layer.argtypes = [CFG, I32, PkvTensor, PkvTensor, PkvTensor, P, I32, P, P, P, P, I64,
                                              P, SZ, P]
     lib.pyramidkv_profile_layer.argtypes = lib.pyramidkv_compress_layer.argtypes + [P, P, P]
+    lib.pyramidkv_score_window_lse.argtypes = [CFG, PkvTensor, PkvTensor, P, P, I32, P, I64, P, SZ, P]
+    lib.pyramidkv_compress_layer_lse.argtypes = [CFG, I32, PkvTensor, PkvTensor, PkvTensor, P, P, I32, P, P, P, P,
+                                                 I64, P, SZ, P]
+    lib.pyramidkv_profile_layer_lse.argtypes = lib.pyramidkv_compress_layer_lse.argtypes + [P, P, P]
     lib.pyramidkv_check_status.argtypes = [P, P, P]
     for name in EXPORTS:
         if name not in ("pyramidkv_strerror", "pyramidkv_workspace_bytes"):
@@ -157,9 +162,23 @@ def total_rows(cfg: PkvConfig, k_layer: int, seq_lens: Sequence[int]) -> int:
     return sum(cfg.num_kv_heads * kept_count(cfg, k_layer, n) for n in seq_lens)
 
 
+def _lse_ptr(window_lse: torch.Tensor) -> int:
+    if window_lse.dtype != torch.float32 or not window_lse.is_contiguous():
+        raise ValueError("window_lse must be a contiguous float32 [batch][H_q][alpha] tensor")
+    return window_lse.data_ptr()
+
+
 def score_window(cfg: PkvConfig, q_win: torch.Tensor, k: torch.Tensor, seq_lens: Sequence[int],
-                 scores: torch.Tensor, workspace: torch.Tensor, stream=None) -> None:
+                 scores: torch.Tensor, workspace: torch.Tensor, stream=None,
+                 window_lse: Optional[torch.Tensor] = None) -> None:
+    """window_lse given: the prefill's natural-log row normalisers are used and one K sweep is skipped."""
     lens, batch = _lens(seq_lens)
+    if window_lse is not None:
+        _check(_lib.pyramidkv_score_window_lse(ctypes.byref(cfg), _tensor(q_win), _tensor(k), _lse_ptr(window_lse),
+                                               lens, batch, scores.data_ptr(), scores.stride(1),
+                                               workspace.data_ptr(), workspace.numel(), _stream(stream)),
+               "pyramidkv_score_window_lse")
+        return
     _check(_lib.pyramidkv_score_window(ctypes.byref(cfg), _tensor(q_win), _tensor(k), lens, batch,
                                        scores.data_ptr(), scores.stride(1), workspace.data_ptr(),
                                        workspace.numel(), _stream(stream)), "pyramidkv_score_window")
@@ -199,8 +218,16 @@ def gather_compact(cfg: PkvConfig, k: torch.Tensor, v: Optional[torch.Tensor], i
 
 def compress_layer(cfg: PkvConfig, layer: int, q_win: torch.Tensor, k: torch.Tensor, v: torch.Tensor,
                    seq_lens: Sequence[int], k_out: torch.Tensor, v_out: torch.Tensor, indices: torch.Tensor,
-                   workspace: torch.Tensor, scores: Optional[torch.Tensor] = None, stream=None) -> None:
+                   workspace: torch.Tensor, scores: Optional[torch.Tensor] = None, stream=None,
+                   window_lse: Optional[torch.Tensor] = None) -> None:
     lens, batch = _lens(seq_lens)
+    if window_lse is not None:
+        _check(_lib.pyramidkv_compress_layer_lse(
+            ctypes.byref(cfg), int(layer), _tensor(q_win), _tensor(k), _tensor(v), _lse_ptr(window_lse), lens, batch,
+            k_out.data_ptr(), v_out.data_ptr(), indices.data_ptr(),
+            scores.data_ptr() if scores is not None else None, scores.stride(1) if scores is not None else 0,
+            workspace.data_ptr(), workspace.numel(), _stream(stream)), "pyramidkv_compress_layer_lse")
+        return
     _check(_lib.pyramidkv_compress_layer(ctypes.byref(cfg), int(layer), _tensor(q_win), _tensor(k), _tensor(v), lens,
                                          batch, k_out.data_ptr(), v_out.data_ptr(), indices.data_ptr(),
                                          scores.data_ptr() if scores is not None else None,
@@ -211,12 +238,18 @@ def compress_layer(cfg: PkvConfig, layer: int, q_win: torch.Tensor, k: torch.Ten
 
 def profile_layer(cfg: PkvConfig, layer: int, q_win: torch.Tensor, k: torch.Tensor, v: torch.Tensor,
                   seq_lens: Sequence[int], k_out: torch.Tensor, v_out: torch.Tensor, indices: torch.Tensor,
-                  workspace: torch.Tensor, stream=None):
+                  workspace: torch.Tensor, stream=None, window_lse: Optional[torch.Tensor] = None):
     """compress_layer with per-kernel device times: returns [(kernel name, milliseconds), ...]."""
     lens, batch = _lens(seq_lens)
     ms = (ctypes.c_float * PKV_MAX_STAGES)()
     names = ((ctypes.c_char * 32) * PKV_MAX_STAGES)()
     n = ctypes.c_int32(0)
+    if window_lse is not None:
+        _check(_lib.pyramidkv_profile_layer_lse(
+            ctypes.byref(cfg), int(layer), _tensor(q_win), _tensor(k), _tensor(v), _lse_ptr(window_lse), lens, batch,
+            k_out.data_ptr(), v_out.data_ptr(), indices.data_ptr(), None, 0, workspace.data_ptr(), workspace.numel(),
+            _stream(stream), ms, names, ctypes.byref(n)), "pyramidkv_profile_layer_lse")
+        return [(names[i].value.decode(), float(ms[i])) for i in range(n.value)]
     _check(_lib.pyramidkv_profile_layer(ctypes.byref(cfg), int(layer), _tensor(q_win), _tensor(k), _tensor(v), lens,
                                         batch, k_out.data_ptr(), v_out.data_ptr(), indices.data_ptr(), None, 0,
                                         workspace.data_ptr(), workspace.numel(), _stream(stream), ms, names,

@@ -181,11 +181,13 @@ int launch_scores_generic(ScoreParams& sp, int batch, cudaStream_t st) {
   sp.seq.stat_off[batch] = stat_tiles;
   sp.seq.score_off[batch] = score_tiles;
   sp.slots_per_chunk = 1;
-  launch_pdl(rowstats_generic_kernel<T, D>, dim3(stat_tiles, sp.num_kv_heads), kGenRowBlock, 0, st, sp);
-  mark(st, "rowstats_generic");
-  launch_pdl(combine_stats_kernel, dim3((sp.rows + 31) / 32, sp.num_kv_heads, batch), kCombineThreads, 0, st, sp,
-             std::log2(static_cast<float>(sp.group)));
-  mark(st, "combine_stats");
+  if (sp.lse_in == sp.lse2) {                    // normalisers not supplied: sweep A and its merge
+    launch_pdl(rowstats_generic_kernel<T, D>, dim3(stat_tiles, sp.num_kv_heads), kGenRowBlock, 0, st, sp);
+    mark(st, "rowstats_generic");
+    launch_pdl(combine_stats_kernel, dim3((sp.rows + 31) / 32, sp.num_kv_heads, batch), kCombineThreads, 0, st, sp,
+               std::log2(static_cast<float>(sp.group)));
+    mark(st, "combine_stats");
+  }
   launch_pdl(scores_generic_kernel<T, D>, dim3(score_tiles, sp.num_kv_heads), kGenScoreKeys, 0, st, sp);
   mark(st, "scores_generic");
   return check_launch();
@@ -272,7 +274,9 @@ int launch_scores_tc(const pkv_config* c, const pkv_tensor& q, const pkv_tensor&
   tp.row_blocks = (sp.rows + 127) / 128;
   tp.scale_log2 = sp.scale_log2;
   tp.partial = sp.partial;
-  tp.lse2 = sp.lse2;
+  tp.lse2 = sp.lse_in;
+  tp.lse_scale = sp.lse_scale;
+  tp.lse_add = sp.lse_add;
   tp.scores = sp.scores;
   tp.ld_scores = sp.ld_scores;
   tp.status = status;
@@ -312,18 +316,21 @@ int launch_scores_tc(const pkv_config* c, const pkv_tensor& q, const pkv_tensor&
 
   const int grid_a = static_cast<int>(std::min<long long>(sms, static_cast<long long>(stat_items) * sp.num_kv_heads));
   const int grid_b = static_cast<int>(std::min<long long>(sms, static_cast<long long>(score_items) * sp.num_kv_heads));
-  launch_pdl(score_tc_kernel<D, 0>, grid_a, kTcThreads, TcSmem<D>::kTotal, st, q_map, k_map_a, tp);
-  mark(st, "rowstats_tc");
-  launch_pdl(combine_stats_kernel, dim3((sp.rows + 31) / 32, sp.num_kv_heads, batch), kCombineThreads, 0, st, sp,
-             std::log2(static_cast<float>(sp.group)));
-  mark(st, "combine_stats");
+  if (sp.lse_in == sp.lse2) {                    // normalisers not supplied: sweep A and its merge
+    launch_pdl(score_tc_kernel<D, 0>, grid_a, kTcThreads, TcSmem<D>::kTotal, st, q_map, k_map_a, tp);
+    mark(st, "rowstats_tc");
+    launch_pdl(combine_stats_kernel, dim3((sp.rows + 31) / 32, sp.num_kv_heads, batch), kCombineThreads, 0, st, sp,
+               std::log2(static_cast<float>(sp.group)));
+    mark(st, "combine_stats");
+  }
   launch_pdl(score_tc_kernel<D, 1>, grid_b, kTcThreads, TcSmem<D>::kTotal, st, q_map, k_map_b, tp);
   mark(st, "scores_tc");
   return check_launch();
 }
 
+// window_lse: null, or the caller's natural-log row normalisers [batch][H_q][alpha] (then sweep A is skipped).
 int run_scores(const pkv_config* c, const pkv_tensor& q, const pkv_tensor& k, const SeqTable& table, int batch,
-               float* scores, int64_t ld, const Workspace& w, cudaStream_t st) {
+               float* scores, int64_t ld, const Workspace& w, cudaStream_t st, const float* window_lse = nullptr) {
   ScoreParams sp{};
   sp.q = view(q);
   sp.k = view(k);
@@ -334,6 +341,9 @@ int run_scores(const pkv_config* c, const pkv_tensor& q, const pkv_tensor& k, co
   sp.scale_log2 = static_cast<float>(1.4426950408889634 / std::sqrt(static_cast<double>(c->head_dim)));
   sp.partial = w.partial;
   sp.lse2 = w.lse2;
+  sp.lse_in = window_lse ? window_lse : w.lse2;
+  sp.lse_scale = window_lse ? 1.4426950408889634f : 1.0f;
+  sp.lse_add = window_lse ? std::log2(static_cast<float>(sp.group)) : 0.0f;
   sp.scores = scores;
   sp.ld_scores = ld;
   if (tc_eligible(c)) {
@@ -473,9 +483,9 @@ size_t pyramidkv_workspace_bytes(const pkv_config* cfg, int32_t batch, int32_t m
   return carve(cfg, batch, max_seq_len, nullptr).bytes;
 }
 
-int pyramidkv_score_window(const pkv_config* cfg, pkv_tensor q_win, pkv_tensor k, const int32_t* seq_lens,
-                           int32_t batch, float* scores, int64_t ld_scores, void* workspace,
-                           size_t workspace_bytes, void* stream) {
+static int score_window_impl(const pkv_config* cfg, pkv_tensor q_win, pkv_tensor k, const float* window_lse,
+                             const int32_t* seq_lens, int32_t batch, float* scores, int64_t ld_scores,
+                             void* workspace, size_t workspace_bytes, void* stream) {
   if (!config_ok(cfg)) return PKV_ERR_INVALID_ARG;
   if (int rc = config_supported(cfg)) return rc;
   const int eb = cfg->dtype == PKV_DTYPE_FP32 ? 4 : 2;
@@ -487,7 +497,22 @@ int pyramidkv_score_window(const pkv_config* cfg, pkv_tensor q_win, pkv_tensor k
   if (ld_scores < max_n - cfg->window) return PKV_ERR_INVALID_ARG;
   Workspace w;
   if (int rc = workspace_check(cfg, batch, max_n, workspace, workspace_bytes, &w)) return rc;
-  return run_scores(cfg, q_win, k, table, batch, scores, ld_scores, w, static_cast<cudaStream_t>(stream));
+  return run_scores(cfg, q_win, k, table, batch, scores, ld_scores, w, static_cast<cudaStream_t>(stream), window_lse);
+}
+
+int pyramidkv_score_window(const pkv_config* cfg, pkv_tensor q_win, pkv_tensor k, const int32_t* seq_lens,
+                           int32_t batch, float* scores, int64_t ld_scores, void* workspace,
+                           size_t workspace_bytes, void* stream) {
+  return score_window_impl(cfg, q_win, k, nullptr, seq_lens, batch, scores, ld_scores, workspace, workspace_bytes,
+                           stream);
+}
+
+int pyramidkv_score_window_lse(const pkv_config* cfg, pkv_tensor q_win, pkv_tensor k, const float* window_lse,
+                               const int32_t* seq_lens, int32_t batch, float* scores, int64_t ld_scores,
+                               void* workspace, size_t workspace_bytes, void* stream) {
+  if (!window_lse) return PKV_ERR_INVALID_ARG;
+  return score_window_impl(cfg, q_win, k, window_lse, seq_lens, batch, scores, ld_scores, workspace,
+                           workspace_bytes, stream);
 }
 
 int pyramidkv_select_topk(const pkv_config* cfg, const float* scores, int64_t ld_scores, const int32_t* seq_lens,
@@ -523,10 +548,10 @@ int pyramidkv_gather_compact(const pkv_config* cfg, pkv_tensor k, pkv_tensor v, 
   return run_gather(cfg, k, v, indices, table, rows, k_out, v_out, static_cast<cudaStream_t>(stream));
 }
 
-int pyramidkv_compress_layer(const pkv_config* cfg, int32_t layer, pkv_tensor q_win, pkv_tensor k, pkv_tensor v,
-                             const int32_t* seq_lens, int32_t batch, void* k_out, void* v_out, int32_t* indices,
-                             float* scores_or_null, int64_t ld_scores, void* workspace, size_t workspace_bytes,
-                             void* stream) {
+static int compress_layer_impl(const pkv_config* cfg, int32_t layer, pkv_tensor q_win, pkv_tensor k, pkv_tensor v,
+                               const float* window_lse, const int32_t* seq_lens, int32_t batch, void* k_out,
+                               void* v_out, int32_t* indices, float* scores_or_null, int64_t ld_scores,
+                               void* workspace, size_t workspace_bytes, void* stream) {
   if (!config_ok(cfg)) return PKV_ERR_INVALID_ARG;
   if (int rc = config_supported(cfg)) return rc;
   if (layer < 0 || layer >= cfg->num_layers) return PKV_ERR_INVALID_ARG;
@@ -558,14 +583,32 @@ int pyramidkv_compress_layer(const pkv_config* cfg, int32_t layer, pkv_tensor q_
   bool any_compress = false;
   for (int b = 0; b < batch; ++b) any_compress |= table.count[b] < table.n[b];
   if (any_compress || scores_or_null)
-    if (int rc = run_scores(cfg, q_win, k, table, batch, scores, ld, w, st)) return rc;
+    if (int rc = run_scores(cfg, q_win, k, table, batch, scores, ld, w, st, window_lse)) return rc;
   return run_select(cfg, scores, ld, table, batch, max_n, indices, w, st, &k, &v, k_out, v_out);
 }
 
-int pyramidkv_profile_layer(const pkv_config* cfg, int32_t layer, pkv_tensor q_win, pkv_tensor k, pkv_tensor v,
-                            const int32_t* seq_lens, int32_t batch, void* k_out, void* v_out, int32_t* indices,
-                            float* scores_or_null, int64_t ld_scores, void* workspace, size_t workspace_bytes,
-                            void* stream, float* stage_ms, char (*stage_names)[32], int32_t* num_stages) {
+int pyramidkv_compress_layer(const pkv_config* cfg, int32_t layer, pkv_tensor q_win, pkv_tensor k, pkv_tensor v,
+                             const int32_t* seq_lens, int32_t batch, void* k_out, void* v_out, int32_t* indices,
+                             float* scores_or_null, int64_t ld_scores, void* workspace, size_t workspace_bytes,
+                             void* stream) {
+  return compress_layer_impl(cfg, layer, q_win, k, v, nullptr, seq_lens, batch, k_out, v_out, indices,
+                             scores_or_null, ld_scores, workspace, workspace_bytes, stream);
+}
+
+int pyramidkv_compress_layer_lse(const pkv_config* cfg, int32_t layer, pkv_tensor q_win, pkv_tensor k, pkv_tensor v,
+                                 const float* window_lse, const int32_t* seq_lens, int32_t batch, void* k_out,
+                                 void* v_out, int32_t* indices, float* scores_or_null, int64_t ld_scores,
+                                 void* workspace, size_t workspace_bytes, void* stream) {
+  if (!window_lse) return PKV_ERR_INVALID_ARG;
+  return compress_layer_impl(cfg, layer, q_win, k, v, window_lse, seq_lens, batch, k_out, v_out, indices,
+                             scores_or_null, ld_scores, workspace, workspace_bytes, stream);
+}
+
+static int profile_layer_impl(const pkv_config* cfg, int32_t layer, pkv_tensor q_win, pkv_tensor k, pkv_tensor v,
+                              const float* window_lse, const int32_t* seq_lens, int32_t batch, void* k_out,
+                              void* v_out, int32_t* indices, float* scores_or_null, int64_t ld_scores,
+                              void* workspace, size_t workspace_bytes, void* stream, float* stage_ms,
+                              char (*stage_names)[32], int32_t* num_stages) {
   if (!stage_ms || !stage_names || !num_stages) return PKV_ERR_INVALID_ARG;
   StageTimer timer;
   for (auto& e : timer.ev)
@@ -573,8 +616,8 @@ int pyramidkv_profile_layer(const pkv_config* cfg, int32_t layer, pkv_tensor q_w
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   cudaEventRecord(timer.ev[0], st);
   g_timer = &timer;
-  int rc = pyramidkv_compress_layer(cfg, layer, q_win, k, v, seq_lens, batch, k_out, v_out, indices, scores_or_null,
-                                    ld_scores, workspace, workspace_bytes, stream);
+  int rc = compress_layer_impl(cfg, layer, q_win, k, v, window_lse, seq_lens, batch, k_out, v_out, indices,
+                               scores_or_null, ld_scores, workspace, workspace_bytes, stream);
   g_timer = nullptr;
   if (rc == PKV_OK && cudaStreamSynchronize(st) != cudaSuccess) rc = PKV_ERR_CUDA;
   *num_stages = 0;
@@ -587,6 +630,25 @@ int pyramidkv_profile_layer(const pkv_config* cfg, int32_t layer, pkv_tensor q_w
   }
   for (auto& e : timer.ev) cudaEventDestroy(e);
   return rc;
+}
+
+int pyramidkv_profile_layer(const pkv_config* cfg, int32_t layer, pkv_tensor q_win, pkv_tensor k, pkv_tensor v,
+                            const int32_t* seq_lens, int32_t batch, void* k_out, void* v_out, int32_t* indices,
+                            float* scores_or_null, int64_t ld_scores, void* workspace, size_t workspace_bytes,
+                            void* stream, float* stage_ms, char (*stage_names)[32], int32_t* num_stages) {
+  return profile_layer_impl(cfg, layer, q_win, k, v, nullptr, seq_lens, batch, k_out, v_out, indices, scores_or_null,
+                            ld_scores, workspace, workspace_bytes, stream, stage_ms, stage_names, num_stages);
+}
+
+int pyramidkv_profile_layer_lse(const pkv_config* cfg, int32_t layer, pkv_tensor q_win, pkv_tensor k, pkv_tensor v,
+                                const float* window_lse, const int32_t* seq_lens, int32_t batch, void* k_out,
+                                void* v_out, int32_t* indices, float* scores_or_null, int64_t ld_scores,
+                                void* workspace, size_t workspace_bytes, void* stream, float* stage_ms,
+                                char (*stage_names)[32], int32_t* num_stages) {
+  if (!window_lse) return PKV_ERR_INVALID_ARG;
+  return profile_layer_impl(cfg, layer, q_win, k, v, window_lse, seq_lens, batch, k_out, v_out, indices,
+                            scores_or_null, ld_scores, workspace, workspace_bytes, stream, stage_ms, stage_names,
+                            num_stages);
 }
 
 int pyramidkv_check_status(const void* workspace, void* stream, uint32_t* detail_or_null) {

@@ -32,6 +32,8 @@ struct ScoreParams {
   float2* partial;                       // [sum_b chunks_b][slots_per_chunk][H_kv][rows] (max, sum)
   int32_t slots_per_chunk;               // partial slots each chunk writes (1 here, 2 for the tensor-core sweep)
   float* lse2;                           // [batch][H_kv][rows]
+  const float* lse_in;                   // normalisers the score sweep reads: lse2, or the caller's
+  float lse_scale, lse_add;              // applied on load: (1, 0), or (log2 e, log2 G) for natural-log input
   float* scores;                         // [batch][H_kv][ld]
   int64_t ld_scores;
 };
@@ -179,7 +181,9 @@ __global__ void __launch_bounds__(kGenScoreKeys) scores_generic_kernel(const Sco
     }
     if (threadIdx.x < kGenQRows) {
       const int r = r0 + threadIdx.x;
-      lse_s[threadIdx.x] = r < p.rows ? p.lse2[(static_cast<int64_t>(b) * p.num_kv_heads + h) * p.rows + r] : INFINITY;
+      lse_s[threadIdx.x] =
+          r < p.rows ? fmaf(p.lse_in[(static_cast<int64_t>(b) * p.num_kv_heads + h) * p.rows + r], p.lse_scale, p.lse_add)
+                     : INFINITY;
     }
     __syncthreads();
     const int rn = min(kGenQRows, p.rows - r0);

@@ -53,7 +53,9 @@ struct TcParams {
   float scale_log2;             // log2(e) / sqrt(d)
   float2* partial;              // sweep A out: [chunk][slots][H_kv][R] (reference exponent, sum); slots = 2 with
                                 // two row blocks, 4 with one: every epilogue warp group writes its own slot
-  const float* lse2;            // sweep B in:  [batch][H_kv][R]
+  const float* lse2;            // sweep B in:  [batch][H_kv][R] row normalisers (log of the row's sum of exps)
+  float lse_scale, lse_add;     // lse2_r = lse2[r] * lse_scale + lse_add: (1, 0) for the library's own sweep A,
+                                // (log2 e, log2 G) for natural-log normalisers handed in by the caller
   float* scores;                // sweep B out: [batch][H_kv][ld]
   int64_t ld_scores;
   uint32_t* status;
@@ -518,7 +520,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         if (w.b != cur_b || w.h != cur_h) {
           __syncwarp();
           const float* src = p.lse2 + (static_cast<int64_t>(w.b) * p.num_kv_heads + w.h) * p.rows;
-          for (int i = lane; i < 256; i += 32) lse_s[i] = i < p.rows ? src[i] : INFINITY;
+          for (int i = lane; i < 256; i += 32) lse_s[i] = i < p.rows ? fmaf(src[i], p.lse_scale, p.lse_add) : INFINITY;
           __syncwarp();
           cur_b = w.b; cur_h = w.h;
         }

@@ -85,6 +85,44 @@ def test_scores_bf16_shapes(hq, hkv, alpha, d, lens):
         assert (got[b, :, n - alpha:] == -1.0).all()
 
 
+@pytest.mark.parametrize("w", [SCALED[0], SCALED[2], SCALED[3], SCALED[4]], ids=lambda w: w.name)
+def test_single_sweep_with_prefill_lse_matches_oracle(w):
+    """Hand-off mode: the window rows' log-sum-exp comes from outside (here: from the oracle)."""
+    cfg = pkv.config_of(w)
+    lens = small_lens(w)
+    budgets = pkv.layer_budgets(cfg)
+    layer = w.num_layers - 1
+    x = workloads.make_layer(w, layer, device=DEV, seq_lens=lens)
+    qc, kc = x.q_win.cpu(), x.k.cpu()
+    lse = np.stack([oracle.window_lse(qc[b], kc[b, :, :n]) for b, n in enumerate(lens)]).astype(np.float32)
+    lse_dev = torch.from_numpy(lse).to(DEV)
+    ws = pkv.new_workspace(cfg, len(lens), max(lens), DEV)
+    scores = torch.full((len(lens), w.num_kv_heads, max(lens)), -1.0, dtype=torch.float32, device=DEV)
+    pkv.score_window(cfg, x.q_win, x.k, lens, scores, ws, window_lse=lse_dev)
+    pkv.check_status(ws)
+    got = scores.cpu().numpy()
+    for b, n in enumerate(lens):
+        want, _ = oracle.window_scores(qc[b], kc[b, :, :n])
+        assert_scores_close(got[b, :, : n - w.window], want, "%s seq %d" % (w.name, b))
+    # the whole layer through the same mode equals the self-contained call
+    kl = budgets[layer]
+    rows = pkv.total_rows(cfg, kl, lens)
+    outs = []
+    for use_lse in (False, True):
+        k_out = torch.empty(rows, w.head_dim, dtype=x.k.dtype, device=DEV)
+        v_out = torch.empty_like(k_out)
+        idx = torch.empty(rows, dtype=torch.int32, device=DEV)
+        pkv.compress_layer(cfg, layer, x.q_win, x.k, x.v, lens, k_out, v_out, idx, ws,
+                           window_lse=lse_dev if use_lse else None)
+        pkv.check_status(ws)
+        outs.append((idx.cpu().numpy(), k_out.cpu(), v_out.cpu()))
+    counts = [pkv.kept_count(cfg, kl, n) for n in lens]
+    heads = [np.array_equal(outs[0][0][sl], outs[1][0][sl]) for _, _, sl in packed_rows(counts, w.num_kv_heads)]
+    assert np.mean(heads) >= 0.9, "only %d of %d heads keep the same list in both modes" % (sum(heads), len(heads))
+    if all(heads):
+        assert torch.equal(outs[0][1], outs[1][1]) and torch.equal(outs[0][2], outs[1][2])
+
+
 @pytest.mark.parametrize("P,k,w", [(1, 1, 1), (5, 2, 7), (33, 32, 3), (100, 0, 5), (100, 100, 5), (100, 250, 5),
                                    (1000, 37, 7), (4064, 188, 7), (8193, 500, 7), (20000, 4, 7), (40000, 937, 7),
                                    (131040, 188, 7), (70001, 2016, 1)])

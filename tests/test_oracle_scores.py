@@ -146,3 +146,20 @@ def test_bf16_inputs_are_widened_exactly():
     a, _ = oracle.window_scores(q, k)
     b, _ = oracle.window_scores(q.float(), k.float())
     np.testing.assert_array_equal(a, b)
+
+
+def test_row_lse_matches_library_logsumexp():
+    """The log-denominators handed to the single-sweep mode are torch.logsumexp of the masked logits."""
+    hq, hkv, alpha, n, d = 6, 2, 5, 70, 16
+    q, k = draw(hq, hkv, alpha, n, d, seed=31)
+    got = oracle.window_lse(q, k)
+    group = hq // hkv
+    logits = torch.einsum("gjd,gnd->gjn", q.double(), k.double().repeat_interleave(group, dim=0)) / math.sqrt(d)
+    mask = torch.arange(n).view(1, 1, n) > torch.arange(n - alpha, n).view(1, alpha, 1)
+    want = torch.logsumexp(logits.masked_fill(mask, float("-inf")), dim=-1).numpy()
+    np.testing.assert_allclose(got, want, rtol=1e-12, atol=1e-12)
+    # and scores are exactly exp(logit - lse) summed over rows, averaged over the group
+    s, _ = oracle.window_scores(q, k)
+    att = torch.exp(logits.masked_fill(mask, float("-inf")) - torch.from_numpy(got).unsqueeze(-1))
+    want_s = att.sum(dim=1).view(hkv, group, n).mean(dim=1)[:, : n - alpha].numpy()
+    np.testing.assert_allclose(s, want_s, rtol=3e-7)
