@@ -29,10 +29,11 @@ class LayerOutputs:
 
 def compress_model(cfg: pkv.PkvConfig, layers, seq_lens: Sequence[int], out: LayerOutputs,
                    workspace: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
-    """layers: sequence of objects with .q_win, .k, .v device tensors, one per layer."""
+    """layers: sequence of objects with .q_win, .k, .v device tensors, one per layer; a layer that also
+    has .window_lse (the prefill's log-sum-exp of the window rows) is scored in a single K sweep."""
     for l, x in enumerate(layers):
         pkv.compress_layer(cfg, l, x.q_win, x.k, x.v, seq_lens, out.k[l], out.v[l], out.idx[l], workspace,
-                           stream=stream)
+                           stream=stream, window_lse=getattr(x, "window_lse", None))
 
 
 class HostPipeline:
@@ -49,7 +50,8 @@ class HostPipeline:
                          v=torch.empty(kv_shape, dtype=dtype, device=device),
                          ko=torch.empty(max_rows, cfg.head_dim, dtype=dtype, device=device),
                          vo=torch.empty(max_rows, cfg.head_dim, dtype=dtype, device=device),
-                         io=torch.empty(max_rows, dtype=torch.int32, device=device)) for _ in range(2)]
+                         io=torch.empty(max_rows, dtype=torch.int32, device=device),
+                         lse=torch.empty(q_shape[:3], dtype=torch.float32, device=device)) for _ in range(2)]
         self.workspace = pkv.new_workspace(cfg, len(self.seq_lens), max(self.seq_lens), device)
         self.copy_in = torch.cuda.Stream(device=device)
         self.compute = torch.cuda.Stream(device=device)
@@ -72,14 +74,19 @@ class HostPipeline:
                 buf["q"].copy_(src.q_win, non_blocking=True)
                 buf["k"].copy_(src.k, non_blocking=True)
                 buf["v"].copy_(src.v, non_blocking=True)
+                lse = getattr(src, "window_lse", None)
+                if lse is not None:
+                    buf["lse"].copy_(lse, non_blocking=True)
                 loaded[l].record(self.copy_in)
-            self.h2d_bytes += sum(t.numel() * t.element_size() for t in (src.q_win, src.k, src.v))
+            moved = [src.q_win, src.k, src.v] + ([lse] if lse is not None else [])
+            self.h2d_bytes += sum(t.numel() * t.element_size() for t in moved)
             with torch.cuda.stream(self.compute):
                 self.compute.wait_event(loaded[l])
                 if l >= 2:
                     self.compute.wait_event(drained[l - 2])       # outputs of this buffer were copied out
                 pkv.compress_layer(self.cfg, l, buf["q"], buf["k"], buf["v"], self.seq_lens, buf["ko"], buf["vo"],
-                                   buf["io"], self.workspace, stream=self.compute)
+                                   buf["io"], self.workspace, stream=self.compute,
+                                   window_lse=buf["lse"] if lse is not None else None)
                 computed[l].record(self.compute)
             with torch.cuda.stream(self.copy_out):
                 self.copy_out.wait_event(computed[l])
