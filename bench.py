@@ -253,7 +253,7 @@ def main():
         return
 
     import paper_2406_02069_b200 as pkv
-    from paper_2406_02069_b200 import streaming
+    from paper_2406_02069_b200 import parallel, streaming
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -311,14 +311,10 @@ def main():
     ev1.record()
     barrier()
     clocks = sampler.stop()
-    ms = ev0.elapsed_time(ev1)
-    if dist is not None:
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    # whole-job rate: tokens of all ranks over the slowest rank's device time
+    value, ms, _ = parallel.job_throughput(tokens * args.steps, ev0.elapsed_time(ev1), device="cuda")
     pkv.check_status(ws)
     ms_per_step = ms / args.steps
-    value = world * tokens / (ms_per_step * 1e-3)
 
     # ---- per-kernel device times (events between the launches of each layer's call), same inputs and launch shapes
     stages = {}
@@ -380,13 +376,9 @@ def main():
             pipe.run(hl, ho)
         e1.record()
         barrier()
-        e_ms = e0.elapsed_time(e1)
-        if dist is not None:
-            t = torch.tensor([e_ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e_ms = float(t.item())
+        e_value, e_ms, _ = parallel.job_throughput(tokens * args.e2e_steps, e0.elapsed_time(e1), device="cuda")
         pkv.check_status(pipe.workspace)
-        line["e2e"] = {"value": world * tokens / (e_ms / args.e2e_steps * 1e-3), "unit": UNIT,
+        line["e2e"] = {"value": e_value, "unit": UNIT,
                        "h2d_bytes_per_step": pipe.h2d_bytes, "d2h_bytes_per_step": pipe.d2h_bytes,
                        "steps": args.e2e_steps, "ms_per_step": e_ms / args.e2e_steps,
                        "note": "host side cycles %d distinct pinned layers; every layer is copied in every step" % ring}
