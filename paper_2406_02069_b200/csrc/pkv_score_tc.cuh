@@ -185,18 +185,44 @@ __device__ __forceinline__ float ex2_mixed(float x, int j) {
                                                                                               : ex2(x);
 }
 
+// Packed pairs of fp32 (one instruction for two multiply-adds or two adds): the scale-and-shift in front
+// of each exponential and the accumulation behind it go through these, which halves their issue slots.
+__device__ __forceinline__ unsigned long long pack2(float lo, float hi) {
+  unsigned long long r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(unsigned long long r, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(r));
+}
+__device__ __forceinline__ unsigned long long fma2(unsigned long long a, unsigned long long b, unsigned long long c) {
+  unsigned long long d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ unsigned long long add2(unsigned long long a, unsigned long long b) {
+  unsigned long long d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+
 // Sweep A, 32 logits of one window row: z += sum_j 2^(v_j * c2 - m).  m is a reference exponent, not
 // necessarily the running maximum: it is only moved when a group's sum is not a moderate finite
 // number (the row's first group, where m = -inf, or a logit ~60 binades above the reference).
 __device__ __forceinline__ void rowstats_group(const uint32_t (&v)[32], float c2, float& m, float& z) {
-  float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+  const unsigned long long cc = pack2(c2, c2), mm = pack2(-m, -m);
+  unsigned long long acc01 = pack2(0.f, 0.f), acc23 = acc01;
 #pragma unroll
   for (int j = 0; j < 32; j += 4) {
-    a0 += ex2_mixed<true>(fmaf(__uint_as_float(v[j]), c2, -m), j);
-    a1 += ex2_mixed<true>(fmaf(__uint_as_float(v[j + 1]), c2, -m), j + 1);
-    a2 += ex2_mixed<true>(fmaf(__uint_as_float(v[j + 2]), c2, -m), j + 2);
-    a3 += ex2_mixed<true>(fmaf(__uint_as_float(v[j + 3]), c2, -m), j + 3);
+    float x0, x1, x2, x3;
+    unpack2(fma2(pack2(__uint_as_float(v[j]), __uint_as_float(v[j + 1])), cc, mm), x0, x1);
+    unpack2(fma2(pack2(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3])), cc, mm), x2, x3);
+    acc01 = add2(acc01, pack2(ex2_mixed<true>(x0, j), ex2_mixed<true>(x1, j + 1)));
+    acc23 = add2(acc23, pack2(ex2_mixed<true>(x2, j + 2), ex2_mixed<true>(x3, j + 3)));
   }
+  float a0, a1, a2, a3;
+  unpack2(acc01, a0, a1);
+  unpack2(acc23, a2, a3);
   float g = (a0 + a1) + (a2 + a3);
   if (!(g < 1.0e18f)) {
     float gm = __uint_as_float(v[0]);
@@ -212,15 +238,19 @@ __device__ __forceinline__ void rowstats_group(const uint32_t (&v)[32], float c2
   z += g;
 }
 
-// Sweep B, 32 window rows of one key: a += 2^(v_j * c2 - lse_j), lse from shared memory.
-__device__ __forceinline__ void score_group(const uint32_t (&v)[32], float c2, const float* lse, float (&a)[4]) {
+// Sweep B, 32 window rows of one key: acc += 2^(v_j * c2 + nlse_j); nlse = -lse2 sits in shared memory
+// (negated when it was loaded), acc holds two packed pairs of partial sums.
+__device__ __forceinline__ void score_group(const uint32_t (&v)[32], float c2, const float* nlse,
+                                            unsigned long long (&acc)[2]) {
+  const unsigned long long cc = pack2(c2, c2);
 #pragma unroll
   for (int j = 0; j < 32; j += 4) {
-    const float4 l4 = *reinterpret_cast<const float4*>(lse + j);
-    a[0] += ex2_mixed<false>(fmaf(__uint_as_float(v[j]), c2, -l4.x), j);
-    a[1] += ex2_mixed<false>(fmaf(__uint_as_float(v[j + 1]), c2, -l4.y), j + 1);
-    a[2] += ex2_mixed<false>(fmaf(__uint_as_float(v[j + 2]), c2, -l4.z), j + 2);
-    a[3] += ex2_mixed<false>(fmaf(__uint_as_float(v[j + 3]), c2, -l4.w), j + 3);
+    const ulonglong2 l4 = *reinterpret_cast<const ulonglong2*>(nlse + j);     // four floats as two packed pairs
+    float x0, x1, x2, x3;
+    unpack2(fma2(pack2(__uint_as_float(v[j]), __uint_as_float(v[j + 1])), cc, l4.x), x0, x1);
+    unpack2(fma2(pack2(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3])), cc, l4.y), x2, x3);
+    acc[0] = add2(acc[0], pack2(ex2_mixed<false>(x0, j), ex2_mixed<false>(x1, j + 1)));
+    acc[1] = add2(acc[1], pack2(ex2_mixed<false>(x2, j + 2), ex2_mixed<false>(x3, j + 3)));
   }
 }
 
@@ -459,6 +489,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         const int r = (two_blocks ? par * 128 : 0) + lane_row;
         const int last_visible = P + (r % alpha);             // row (g, j) sees keys 0 .. P + j
         const int units = p.row_blocks;
+        // a warp whose 32 TMEM lanes are all padding rows (R < 128) has nothing to evaluate
+        const bool warp_has_rows = (two_blocks ? par * 128 : 0) + quarter * 32 < p.rows;
         float m = -INFINITY, z = 0.f;
         for (int t = tile0; t < tile1 && ok; ++t) {
           for (int rb = 0; rb < units && ok; ++rb, ++u) {
@@ -470,7 +502,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
             tc_fence_after();
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + ts * stage_cols + ch * 128;
             const int key_base = t * kTcTileKeysA + ch * 128;
-            if (key_base + 127 <= P) {                        // every key visible to every row: no mask
+            if (!warp_has_rows) {
+              // only the hand-shake below
+            } else if (key_base + 127 <= P) {                 // every key visible to every row: no mask
               for (int cg = 0; cg < 128; cg += 32) {
                 uint32_t v[32];
                 tc_ld32(taddr + cg, v);
@@ -520,7 +554,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         if (w.b != cur_b || w.h != cur_h) {
           __syncwarp();
           const float* src = p.lse2 + (static_cast<int64_t>(w.b) * p.num_kv_heads + w.h) * p.rows;
-          for (int i = lane; i < 256; i += 32) lse_s[i] = i < p.rows ? fmaf(src[i], p.lse_scale, p.lse_add) : INFINITY;
+          for (int i = lane; i < 256; i += 32)       // stored negated: the epilogue adds it
+            lse_s[i] = i < p.rows ? -fmaf(src[i], p.lse_scale, p.lse_add) : -INFINITY;
           __syncwarp();
           cur_b = w.b; cur_h = w.h;
         }
@@ -535,7 +570,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
           if (!ok) break;
           tc_fence_after();
           const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + ts * stage_cols;
-          float acc[4] = {0.f, 0.f, 0.f, 0.f};
+          unsigned long long acc[2] = {pack2(0.f, 0.f), pack2(0.f, 0.f)};
           for (int cg = col0; cg < col1; cg += 32) {
             uint32_t v[32];
             tc_ld32(taddr + cg, v);
@@ -545,7 +580,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(t_empty(ts));
-          float sum = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+          float s0, s1, s2, s3;
+          unpack2(acc[0], s0, s1);
+          unpack2(acc[1], s2, s3);
+          float sum = (s0 + s1) + (s2 + s3);
           if (second_half) {
             if (ch == 1) {
               ok = mbar_wait(x_empty(par), (mine & 1) ^ 1, abort_flag);
