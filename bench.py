@@ -36,8 +36,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
 # kernel name, valid only for the kernel sources whose digest is given: any change to csrc/ voids them.
 NCU_TRAFFIC = {
     # profiles/score_tc_llama3_70b_128k.md: (read + written) bytes / (n * H_kv) key rows
-    "rowstats_tc": {"csrc_digest": "3e998e5764c412fd", "bytes_per_key_row": 262.3},
-    "scores_tc": {"csrc_digest": "3e998e5764c412fd", "bytes_per_key_row": 262.8},
+    "rowstats_tc": {"csrc_digest": "8b40a59e6ec5b93c", "bytes_per_key_row": 262.7},
+    "scores_tc": {"csrc_digest": "8b40a59e6ec5b93c", "bytes_per_key_row": 263.4},
 }
 
 
