@@ -119,30 +119,37 @@ def graded_bytes_per_layer(w, lens, count_rows, esz):
     return k_read + q_read + 2 * moved + 4 * count_rows
 
 
-def cpu_baseline_sample(w, layer_inputs, lens, budgets, budget_s=20.0):
-    """Times the oracle, as it stands, on (sequence 0, a few KV heads) of layer 0 and scales to all layers."""
+def cpu_baseline_sample(w, layer_inputs, lens, budgets, budget_s=20.0, min_s=10.0):
+    """Times the oracle, as it stands, on (sequence 0, one KV head at a time) of the first layers until
+    min_s..budget_s seconds of CPU work are spent, and scales to all layers.  layer_inputs: one layer
+    or a list of layers (layer l at index l)."""
     import oracle
+    many = layer_inputs if isinstance(layer_inputs, (list, tuple)) else [layer_inputs]
     n = lens[0]
-    q = layer_inputs.q_win[0].cpu()
-    k = layer_inputs.k[0, :, :n].cpu()
-    v = layer_inputs.v[0, :, :n].cpu()
     g = w.group
-    heads_done, t_total = 0, 0.0
-    while heads_done < w.num_kv_heads:
-        h = heads_done
-        t0 = time.perf_counter()
-        oracle.compress_layer(q[h * g:(h + 1) * g], k[h:h + 1], v[h:h + 1], pool_kernel=w.pool_kernel,
-                              avg_budget=w.avg_budget, k_layer=budgets[0], want_scores=False)
-        t_total += time.perf_counter() - t0
-        heads_done += 1
-        if t_total * (heads_done + 1) / heads_done > budget_s:
+    units, t_total, used_layers = 0, 0.0, 0
+    for l, x in enumerate(many):
+        q = x.q_win[0].cpu()
+        k = x.k[0, :, :n].cpu()
+        v = x.v[0, :, :n].cpu()
+        used_layers += 1
+        for h in range(w.num_kv_heads):
+            t0 = time.perf_counter()
+            oracle.compress_layer(q[h * g:(h + 1) * g], k[h:h + 1], v[h:h + 1], pool_kernel=w.pool_kernel,
+                                  avg_budget=w.avg_budget, k_layer=budgets[l], want_scores=False)
+            t_total += time.perf_counter() - t0
+            units += 1
+            if t_total * (units + 1) / units > budget_s:
+                break
+        if t_total >= min_s or t_total * (units + 1) / units > budget_s:
             break
-    # one (sequence, head) unit costs t_total / heads_done; all layers, all heads, all sequences (by length)
-    per_token_head = t_total / heads_done / n
-    full = per_token_head * sum(lens) * w.num_kv_heads * w.num_layers
+    # one (sequence, head, layer) unit costs t_total / units; all layers, heads and sequences (by length)
+    per_token_unit = t_total / units / n
+    full = per_token_unit * sum(lens) * w.num_kv_heads * w.num_layers
     return {"value": sum(lens) / full, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-            "sample": "layer 0, sequence 0 (n=%d), %d of %d KV heads with their %d query heads each; "
-                      "%.1f s of CPU work scaled by heads x layers x tokens" % (n, heads_done, w.num_kv_heads, g, t_total)}
+            "sample": "sequence 0 (n=%d), %d (layer, KV head) units from the first %d layer(s), each head with its %d "
+                      "query heads; %.1f s of CPU work scaled by heads x layers x tokens"
+                      % (n, units, used_layers, g, t_total)}
 
 
 def run_reference(args, w):
@@ -384,7 +391,7 @@ def main():
                        "note": "host side cycles %d distinct pinned layers; every layer is copied in every step" % ring}
 
     if rank == 0 and not args.no_cpu_baseline and world == 1:
-        line["cpu_baseline"] = cpu_baseline_sample(w, layers[0], lens, out.budgets)
+        line["cpu_baseline"] = cpu_baseline_sample(w, layers[:16], lens, out.budgets)
     if rank == 0:
         print(json.dumps(line))
     if dist is not None:

@@ -224,6 +224,43 @@ def test_compress_layer_matches_oracle(w):
         assert identical >= 0.9 * total, "only %d of %d index lists identical" % (identical, total)
 
 
+@pytest.mark.parametrize("w,layers", [
+    (workloads.LLAMA2_7B, (0, 31)), (workloads.LLAMA3_8B, (0, 31)), (workloads.LLAMA3_70B, (0, 79)),
+    (workloads.MISTRAL_RAGGED, (0,)), (workloads.with_budget(workloads.MISTRAL_RAGGED, 2048), (31,)),
+], ids=lambda x: getattr(x, "name", str(x)))
+def test_full_size_layers_match_oracle(w, layers):
+    """The configurations at their full sizes, in the launch shapes bench.py times: every score of the
+    layer, every kept list and the gathered rows against the oracle (about a second of CPU per head)."""
+    cfg = pkv.config_of(w)
+    lens = w.seq_lens()
+    budgets = pkv.layer_budgets(cfg)
+    ws = pkv.new_workspace(cfg, len(lens), max(lens), DEV)
+    for layer in layers:
+        kl = budgets[layer]
+        x = workloads.make_layer(w, layer, device=DEV)
+        rows = pkv.total_rows(cfg, kl, lens)
+        k_out = torch.empty(rows, w.head_dim, dtype=x.k.dtype, device=DEV)
+        v_out = torch.empty_like(k_out)
+        idx = torch.empty(rows, dtype=torch.int32, device=DEV)
+        scores = torch.full((len(lens), w.num_kv_heads, max(lens)), -1.0, dtype=torch.float32, device=DEV)
+        pkv.compress_layer(cfg, layer, x.q_win, x.k, x.v, lens, k_out, v_out, idx, ws, scores=scores)
+        pkv.check_status(ws)
+        ref = oracle.compress_batch(x.q_win.cpu(), x.k.cpu(), x.v.cpu(), lens, pool_kernel=w.pool_kernel,
+                                    avg_budget=w.avg_budget, k_layer=kl)
+        got_scores, got_idx = scores.cpu().numpy(), idx.cpu().numpy()
+        for b, n in enumerate(lens):
+            assert_scores_close(got_scores[b, :, : n - w.window], ref["scores"][b], "%s layer %d seq %d" % (w.name, layer, b))
+        identical = 0
+        for b, h, sl in packed_rows(ref["counts"], w.num_kv_heads):
+            identical += bool(assert_indices_match(got_idx[sl], ref["indices"][sl], ref["scores"][b][h], w.pool_kernel,
+                                                   w.window, "%s layer %d b %d h %d" % (w.name, layer, b, h)))
+            sel = idx[sl].long()
+            assert torch.equal(k_out[sl], x.k[b, h, sel]) and torch.equal(v_out[sl], x.v[b, h, sel])
+        assert identical >= 0.9 * len(ref["counts"]) * w.num_kv_heads
+        del x, k_out, v_out, scores
+        torch.cuda.empty_cache()
+
+
 def test_three_calls_equal_the_fused_call():
     w = workloads.scaled(workloads.LLAMA3_8B, num_layers=2, seq_len=3000, name="l3_3k")
     cfg = pkv.config_of(w)
