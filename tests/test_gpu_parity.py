@@ -261,6 +261,41 @@ def test_full_size_layers_match_oracle(w, layers):
         torch.cuda.empty_cache()
 
 
+def test_layer_calls_can_be_captured_in_a_cuda_graph():
+    """Nothing in the per-layer call synchronises or allocates, so a step can be captured once and replayed."""
+    w = workloads.scaled(workloads.LLAMA3_8B, num_layers=3, seq_len=3000, name="l3_graph")
+    cfg = pkv.config_of(w)
+    lens = w.seq_lens()
+    budgets = pkv.layer_budgets(cfg)
+    layers = [workloads.make_layer(w, l, device=DEV) for l in range(w.num_layers)]
+    ws = pkv.new_workspace(cfg, 1, max(lens), DEV)
+    rows = [pkv.total_rows(cfg, kl, lens) for kl in budgets]
+    outs = [(torch.zeros(r, w.head_dim, dtype=torch.bfloat16, device=DEV), torch.zeros(r, w.head_dim, dtype=torch.bfloat16, device=DEV),
+             torch.zeros(r, dtype=torch.int32, device=DEV)) for r in rows]
+
+    def step():
+        for l, x in enumerate(layers):
+            pkv.compress_layer(cfg, l, x.q_win, x.k, x.v, lens, outs[l][0], outs[l][1], outs[l][2], ws)
+
+    step()                                                          # eager: also runs every first-use set-up
+    torch.cuda.synchronize()
+    want = [tuple(t.clone() for t in o) for o in outs]
+    graph, side = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            step()
+    for o in outs:
+        for t in o:
+            t.zero_()
+    for _ in range(2):
+        graph.replay()
+    torch.cuda.synchronize()
+    pkv.check_status(ws)
+    for o, wnt in zip(outs, want):
+        for a_, b_ in zip(o, wnt):
+            assert torch.equal(a_, b_)
+
+
 def test_three_calls_equal_the_fused_call():
     w = workloads.scaled(workloads.LLAMA3_8B, num_layers=2, seq_len=3000, name="l3_3k")
     cfg = pkv.config_of(w)
