@@ -247,6 +247,33 @@ int pyramidkv_compress_layer_lse(const pkv_config* cfg, int32_t layer,
                                  void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Decode attention over the compact cache of one layer (Section 4.1: after compression only K_s, V_s
+ * are used for inference; Section 4.2.2: evicted entries take part in no later computation).  For one
+ * new token per sequence, query head g attends to every kept row of its KV head:
+ *     out[b][g] = softmax(q[b][g] . K_s^T / sqrt(d)) V_s      (no mask: every kept token precedes it).
+ *   q          device, [batch][H_q][d] of the config dtype, contiguous, 16-byte aligned
+ *   k_cache, v_cache  device, packed rows as written by pyramidkv_compress_layer for budget k_layer
+ *   out        device, [batch][H_q][d] floats
+ * Positions are not needed here: K rows carry their rotary embedding as computed at prefill.
+ * Errors: INVALID_ARG, UNSUPPORTED, CUDA.
+ */
+int pyramidkv_decode_attention(const pkv_config* cfg, const void* q, const void* k_cache, const void* v_cache,
+                               const int32_t* seq_lens, int32_t batch, int32_t k_layer, float* out, void* stream);
+
+/*
+ * Attention recall of a layer's selection (appendix "Attention Recall Rate Experiment": the share of
+ * the attention computed with the kept keys relative to all keys), per sequence and KV head, averaged
+ * over the alpha window rows and the group's query heads.  With the scores of Eq. 3 this is
+ *     recall[b][h] = 1 - (sum of scores[b][h][i] over evicted prefix positions i) / alpha,
+ * since each window row's attention sums to one and the window keys are always kept.
+ *   scores, indices  device, as produced for this layer; recall  device, [batch][H_kv] floats
+ * Errors: INVALID_ARG, CUDA.
+ */
+int pyramidkv_attention_recall(const pkv_config* cfg, const float* scores, int64_t ld_scores,
+                               const int32_t* indices, const int32_t* seq_lens, int32_t batch,
+                               int32_t k_layer, float* recall, void* stream);
+
+/*
  * Measuring aid; the paper has no counterpart.  Same arguments and results as
  * pyramidkv_compress_layer, but a CUDA event is recorded after every kernel the
  * call launches, the stream is synchronised, and the device time of each kernel

@@ -62,6 +62,10 @@ def _load() -> ctypes.CDLL:
         lib.orc_window_attention.argtypes = [ctypes.c_void_p] * 4 + [ctypes.c_int] * 5 + \
                                             [ctypes.c_void_p]
         lib.orc_window_attention.restype = None
+        lib.orc_decode_attention.argtypes = [ctypes.c_void_p] * 3 + [ctypes.c_int] * 3 + [ctypes.c_void_p]
+        lib.orc_decode_attention.restype = None
+        lib.orc_attention_recall.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_void_p, ctypes.c_int]
+        lib.orc_attention_recall.restype = ctypes.c_double
         lib.orc_num_threads.argtypes = []
         lib.orc_num_threads.restype = ctypes.c_int
         _lib = lib
@@ -194,3 +198,20 @@ def window_attention(q_head: torch.Tensor, k_rows: torch.Tensor, v_rows: torch.T
     _load().orc_window_attention(q_head.data_ptr(), k_rows.data_ptr(), v_rows.data_ptr(),
                                  pos.ctypes.data, _dtype_code(k_rows), d, alpha, n, c, out.ctypes.data)
     return out
+
+
+def decode_attention(q_row: torch.Tensor, k_rows: torch.Tensor, v_rows: torch.Tensor) -> np.ndarray:
+    """softmax(q K_s^T / sqrt(d)) V_s for one query vector over cached rows.  float64 [d]."""
+    q_row, k_rows, v_rows = _host(q_row), _host(k_rows), _host(v_rows)
+    c, d = k_rows.shape
+    out = np.zeros(d, dtype=np.float64)
+    _load().orc_decode_attention(q_row.data_ptr(), k_rows.data_ptr(), v_rows.data_ptr(), _dtype_code(k_rows), d, c,
+                                 out.ctypes.data)
+    return out
+
+
+def attention_recall(scores_row: np.ndarray, alpha: int, kept: np.ndarray) -> float:
+    """Share of the window's attention on kept keys for one KV head (scores_row: its Eq. 3 scores)."""
+    s = np.ascontiguousarray(scores_row, dtype=np.float32)
+    kp = np.ascontiguousarray(kept, dtype=np.int32)
+    return float(_load().orc_attention_recall(s.ctypes.data, s.shape[0], int(alpha), kp.ctypes.data, kp.shape[0]))

@@ -276,6 +276,41 @@ void orc_window_attention(const void* q, const void* kc, const void* vc, const i
   }
 }
 
+// ---------------------------------------------------------------------------
+// Section 4.1: inference after compression uses only the kept rows.  One new token's query attends to
+// every cached row of its KV head (no mask: all of them precede it).
+//   q [d]; kc, vc [c][d]; out [d] double.
+void orc_decode_attention(const void* q, const void* kc, const void* vc, int dtype, int d, int c, double* out) {
+  const double scale = 1.0 / std::sqrt(static_cast<double>(d));
+  std::vector<double> w(c);
+  double mx = -std::numeric_limits<double>::infinity();
+  for (int r = 0; r < c; ++r) {
+    double dot = 0.0;
+    for (int t = 0; t < d; ++t) dot += elem(q, dtype, t) * elem(kc, dtype, static_cast<int64_t>(r) * d + t);
+    w[r] = dot * scale;
+    mx = std::max(mx, w[r]);
+  }
+  double z = 0.0;
+  for (int r = 0; r < c; ++r) { w[r] = std::exp(w[r] - mx); z += w[r]; }
+  for (int t = 0; t < d; ++t) {
+    double o = 0.0;
+    for (int r = 0; r < c; ++r) o += (w[r] / z) * elem(vc, dtype, static_cast<int64_t>(r) * d + t);
+    out[t] = o;
+  }
+}
+
+// Appendix on the attention recall rate: share of the window rows' attention that lands on kept keys,
+// averaged over the alpha rows and the group's query heads.  scores [P] are the Eq. 3 scores of one KV
+// head (they already hold the group mean of the row sums), kept [c] its kept positions (window included).
+double orc_attention_recall(const float* scores, int P, int alpha, const int32_t* kept, int c) {
+  double all = 0.0, on_kept = 0.0;
+  for (int i = 0; i < P; ++i) all += scores[i];
+  for (int r = 0; r < c; ++r)
+    if (kept[r] < P) on_kept += scores[kept[r]];
+  const double window_mass = alpha - all;                 // every row's attention sums to one
+  return (on_kept + window_mass) / alpha;
+}
+
 int orc_num_threads() {
 #ifdef _OPENMP
   return omp_get_max_threads();

@@ -28,7 +28,8 @@ EXPORTS = ("pyramidkv_strerror", "pyramidkv_layer_budgets", "pyramidkv_kept_coun
            "pyramidkv_workspace_bytes", "pyramidkv_score_window", "pyramidkv_select_topk",
            "pyramidkv_gather_compact", "pyramidkv_compress_layer", "pyramidkv_profile_layer",
            "pyramidkv_check_status", "pyramidkv_score_window_static", "pyramidkv_score_window_lse",
-           "pyramidkv_compress_layer_lse", "pyramidkv_profile_layer_lse")
+           "pyramidkv_compress_layer_lse", "pyramidkv_profile_layer_lse", "pyramidkv_decode_attention",
+           "pyramidkv_attention_recall")
 PKV_MAX_STAGES = 8
 
 
@@ -76,6 +77,8 @@ def _load() -> ctypes.CDLL:
     lib.pyramidkv_compress_layer_lse.argtypes = [CFG, I32, PkvTensor, PkvTensor, PkvTensor, P, P, I32, P, P, P, P,
                                                  I64, P, SZ, P]
     lib.pyramidkv_profile_layer_lse.argtypes = lib.pyramidkv_compress_layer_lse.argtypes + [P, P, P]
+    lib.pyramidkv_decode_attention.argtypes = [CFG, P, P, P, P, I32, I32, P, P]
+    lib.pyramidkv_attention_recall.argtypes = [CFG, P, I64, P, P, I32, I32, P, P]
     lib.pyramidkv_check_status.argtypes = [P, P, P]
     for name in EXPORTS:
         if name not in ("pyramidkv_strerror", "pyramidkv_workspace_bytes"):
@@ -255,6 +258,26 @@ def profile_layer(cfg: PkvConfig, layer: int, q_win: torch.Tensor, k: torch.Tens
                                         workspace.data_ptr(), workspace.numel(), _stream(stream), ms, names,
                                         ctypes.byref(n)), "pyramidkv_profile_layer")
     return [(names[i].value.decode(), float(ms[i])) for i in range(n.value)]
+
+
+def decode_attention(cfg: PkvConfig, q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor,
+                     seq_lens: Sequence[int], k_layer: int, out: torch.Tensor, stream=None) -> None:
+    """One new token per sequence attends to the compact cache of a layer: q [batch][H_q][d] -> out fp32."""
+    lens, batch = _lens(seq_lens)
+    if not (q.is_contiguous() and k_cache.is_contiguous() and v_cache.is_contiguous() and out.is_contiguous()):
+        raise ValueError("decode_attention takes contiguous tensors")
+    _check(_lib.pyramidkv_decode_attention(ctypes.byref(cfg), q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(),
+                                           lens, batch, int(k_layer), out.data_ptr(), _stream(stream)),
+           "pyramidkv_decode_attention")
+
+
+def attention_recall(cfg: PkvConfig, scores: torch.Tensor, indices: torch.Tensor, seq_lens: Sequence[int],
+                     k_layer: int, recall: torch.Tensor, stream=None) -> None:
+    """Share of the window's attention that falls on kept keys, per (sequence, KV head)."""
+    lens, batch = _lens(seq_lens)
+    _check(_lib.pyramidkv_attention_recall(ctypes.byref(cfg), scores.data_ptr(), scores.stride(1),
+                                           indices.data_ptr(), lens, batch, int(k_layer), recall.data_ptr(),
+                                           _stream(stream)), "pyramidkv_attention_recall")
 
 
 def check_status(workspace: torch.Tensor, stream=None) -> int:

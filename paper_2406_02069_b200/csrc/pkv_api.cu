@@ -9,6 +9,7 @@
 #include <utility>
 
 #include "pkv_common.cuh"
+#include "pkv_extras.cuh"
 #include "pkv_gather.cuh"
 #include "pkv_score_generic.cuh"
 #include "pkv_score_tc.cuh"
@@ -649,6 +650,60 @@ int pyramidkv_profile_layer_lse(const pkv_config* cfg, int32_t layer, pkv_tensor
   return profile_layer_impl(cfg, layer, q_win, k, v, window_lse, seq_lens, batch, k_out, v_out, indices,
                             scores_or_null, ld_scores, workspace, workspace_bytes, stream, stage_ms, stage_names,
                             num_stages);
+}
+
+int pyramidkv_decode_attention(const pkv_config* cfg, const void* q, const void* k_cache, const void* v_cache,
+                               const int32_t* seq_lens, int32_t batch, int32_t k_layer, float* out, void* stream) {
+  if (!config_ok(cfg)) return PKV_ERR_INVALID_ARG;
+  if (int rc = config_supported(cfg)) return rc;
+  if (!q || !k_cache || !v_cache || !out) return PKV_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(q) % 16 || reinterpret_cast<uintptr_t>(k_cache) % 16 ||
+      reinterpret_cast<uintptr_t>(v_cache) % 16)
+    return PKV_ERR_INVALID_ARG;
+  SeqTable table;
+  int max_n;
+  int64_t rows;
+  if (int rc = build_table(cfg, seq_lens, batch, k_layer, &table, &max_n, &rows)) return rc;
+  DecodeParams dp{};
+  dp.q = q;
+  dp.k_cache = k_cache;
+  dp.v_cache = v_cache;
+  dp.out = out;
+  dp.seq = table;
+  dp.num_kv_heads = cfg->num_kv_heads;
+  dp.group = cfg->num_q_heads / cfg->num_kv_heads;
+  dp.scale_log2 = static_cast<float>(1.4426950408889634 / std::sqrt(static_cast<double>(cfg->head_dim)));
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const dim3 grid(cfg->num_q_heads, batch);
+  if (cfg->dtype == PKV_DTYPE_FP32) {
+    if (cfg->head_dim == 64) launch_pdl(decode_attention_kernel<float, 64>, grid, kDecThreads, 0, st, dp);
+    else launch_pdl(decode_attention_kernel<float, 128>, grid, kDecThreads, 0, st, dp);
+  } else {
+    if (cfg->head_dim == 64) launch_pdl(decode_attention_kernel<__nv_bfloat16, 64>, grid, kDecThreads, 0, st, dp);
+    else launch_pdl(decode_attention_kernel<__nv_bfloat16, 128>, grid, kDecThreads, 0, st, dp);
+  }
+  return check_launch();
+}
+
+int pyramidkv_attention_recall(const pkv_config* cfg, const float* scores, int64_t ld_scores, const int32_t* indices,
+                               const int32_t* seq_lens, int32_t batch, int32_t k_layer, float* recall,
+                               void* stream) {
+  if (!config_ok(cfg)) return PKV_ERR_INVALID_ARG;
+  if (!scores || !indices || !recall) return PKV_ERR_INVALID_ARG;
+  SeqTable table;
+  int max_n;
+  int64_t rows;
+  if (int rc = build_table(cfg, seq_lens, batch, k_layer, &table, &max_n, &rows)) return rc;
+  if (ld_scores < max_n - cfg->window) return PKV_ERR_INVALID_ARG;
+  RecallParams rp{};
+  rp.scores = scores;
+  rp.ld_scores = ld_scores;
+  rp.indices = indices;
+  rp.recall = recall;
+  rp.seq = table;
+  rp.num_kv_heads = cfg->num_kv_heads;
+  launch_pdl(attention_recall_kernel, dim3(cfg->num_kv_heads, batch), 256, 0, static_cast<cudaStream_t>(stream), rp);
+  return check_launch();
 }
 
 int pyramidkv_check_status(const void* workspace, void* stream, uint32_t* detail_or_null) {

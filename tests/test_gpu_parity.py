@@ -296,6 +296,41 @@ def test_layer_calls_can_be_captured_in_a_cuda_graph():
             assert torch.equal(a_, b_)
 
 
+@pytest.mark.parametrize("w", [SCALED[0], SCALED[2], SCALED[4]], ids=lambda w: w.name)
+def test_decode_attention_and_recall_over_the_compact_cache(w):
+    """After compression a new token attends to the kept rows only; recall says how much attention they hold."""
+    cfg = pkv.config_of(w)
+    lens = small_lens(w)
+    layer = 0
+    kl = pkv.layer_budgets(cfg)[layer]
+    x = workloads.make_layer(w, layer, device=DEV, seq_lens=lens)
+    ws = pkv.new_workspace(cfg, len(lens), max(lens), DEV)
+    rows = pkv.total_rows(cfg, kl, lens)
+    k_out = torch.empty(rows, w.head_dim, dtype=x.k.dtype, device=DEV)
+    v_out = torch.empty_like(k_out)
+    idx = torch.empty(rows, dtype=torch.int32, device=DEV)
+    scores = torch.zeros(len(lens), w.num_kv_heads, max(lens), dtype=torch.float32, device=DEV)
+    pkv.compress_layer(cfg, layer, x.q_win, x.k, x.v, lens, k_out, v_out, idx, ws, scores=scores)
+    g = torch.Generator(device="cpu").manual_seed(77)
+    q_new = torch.randn(len(lens), w.num_q_heads, w.head_dim, generator=g).to(x.k.dtype)
+    out = torch.zeros(len(lens), w.num_q_heads, w.head_dim, dtype=torch.float32, device=DEV)
+    pkv.decode_attention(cfg, q_new.to(DEV), k_out, v_out, lens, kl, out)
+    recall = torch.zeros(len(lens), w.num_kv_heads, dtype=torch.float32, device=DEV)
+    pkv.attention_recall(cfg, scores, idx, lens, kl, recall)
+    pkv.check_status(ws)
+    out_h, rec_h = out.cpu().numpy(), recall.cpu().numpy()
+    kc, vc, ic, sc = k_out.cpu(), v_out.cpu(), idx.cpu().numpy(), scores.cpu().numpy()
+    counts = [pkv.kept_count(cfg, kl, n) for n in lens]
+    for b, h, sl in packed_rows(counts, w.num_kv_heads):
+        for gq in range(w.group):
+            hq = h * w.group + gq
+            want = oracle.decode_attention(q_new[b, hq], kc[sl], vc[sl])
+            np.testing.assert_allclose(out_h[b, hq], want, rtol=2e-3, atol=2e-4)
+        want_r = oracle.attention_recall(sc[b, h, : lens[b] - w.window], w.window, ic[sl])
+        assert abs(rec_h[b, h] - want_r) < 1e-4
+        assert 0.0 < rec_h[b, h] <= 1.0 + 1e-5
+
+
 def test_three_calls_equal_the_fused_call():
     w = workloads.scaled(workloads.LLAMA3_8B, num_layers=2, seq_len=3000, name="l3_3k")
     cfg = pkv.config_of(w)

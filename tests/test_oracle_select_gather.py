@@ -200,3 +200,44 @@ def test_kept_positions_follow_the_papers_position_example():
         k[0, p] += 20.0 * u                                 # make exactly the printed prefix positions stand out
     r = oracle.compress_layer(q, k, v, pool_kernel=1, avg_budget=len(printed), k_layer=len(printed) - 1)
     assert list(r["kept"][0]) == printed
+
+
+# ----------------------------------------------------------------------------- consumers of the compact cache
+def test_decode_attention_is_library_softmax_attention():
+    g = torch.Generator().manual_seed(9)
+    d, c = 32, 57
+    q = torch.randn(d, generator=g)
+    k = torch.randn(c, d, generator=g)
+    v = torch.randn(c, d, generator=g)
+    got = oracle.decode_attention(q, k, v)
+    want = torch.softmax((k.double() @ q.double()) / np.sqrt(d), dim=0) @ v.double()
+    np.testing.assert_allclose(got, want.numpy(), rtol=1e-12, atol=1e-13)
+    # a single cached row returns that row's value; permuting the cache changes nothing
+    np.testing.assert_allclose(oracle.decode_attention(q, k[:1], v[:1]), v[0].double().numpy(), rtol=1e-12)
+    perm = torch.randperm(c, generator=g)
+    np.testing.assert_allclose(oracle.decode_attention(q, k[perm], v[perm]), got, rtol=1e-10, atol=1e-12)
+
+
+def test_attention_recall_definition_and_monotonicity():
+    """Recall = kept share of the window rows' attention, from the full attention matrix (library softmax)."""
+    hq, hkv, alpha, n, d = 4, 2, 4, 90, 16
+    q, k, v = draw(hq, hkv, alpha, n, d, seed=17)
+    P = n - alpha
+    group = hq // hkv
+    logits = torch.einsum("gjd,gnd->gjn", q.double(), k.double().repeat_interleave(group, dim=0)) / np.sqrt(d)
+    mask = torch.arange(n).view(1, 1, n) > torch.arange(P, n).view(1, alpha, 1)
+    att = torch.softmax(logits.masked_fill(mask, float("-inf")), dim=-1)            # [H_q][alpha][n]
+    prev = None
+    for kl in (5, 20, 60, P):
+        r = oracle.compress_layer(q, k, v, pool_kernel=1, avg_budget=alpha + kl, k_layer=kl)
+        vals = []
+        for h in range(hkv):
+            kept = torch.from_numpy(r["kept"][h]).long()
+            want = att[h * group:(h + 1) * group][:, :, kept].sum(dim=-1).mean().item()   # mean over heads and rows
+            got = oracle.attention_recall(r["scores"][h], alpha, r["kept"][h])
+            assert abs(got - want) < 1e-6
+            vals.append(got)
+        if prev is not None:
+            assert all(a >= b - 1e-9 for a, b in zip(vals, prev))                     # more budget, more recall
+        prev = vals
+    assert all(abs(x - 1.0) < 1e-6 for x in prev)                                     # nothing evicted
