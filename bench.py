@@ -33,18 +33,19 @@ UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from ncu captures, keyed by
-# kernel name, valid only for the kernel sources whose digest is given: any change to csrc/ voids them.
+# kernel name, valid only while the kernel's source files have the digest given: a change voids them.
+TC_SOURCES = ("pkv_score_tc.cuh", "pkv_common.cuh")
 NCU_TRAFFIC = {
     # profiles/score_tc_llama3_70b_128k.md: (read + written) bytes / (n * H_kv) key rows
-    "rowstats_tc": {"csrc_digest": "8b40a59e6ec5b93c", "bytes_per_key_row": 262.7},
-    "scores_tc": {"csrc_digest": "8b40a59e6ec5b93c", "bytes_per_key_row": 263.4},
+    "rowstats_tc": {"sources": TC_SOURCES, "digest": "83d46454d1fc6417", "bytes_per_key_row": 262.7},
+    "scores_tc": {"sources": TC_SOURCES, "digest": "83d46454d1fc6417", "bytes_per_key_row": 263.4},
 }
 
 
-def csrc_digest() -> str:
+def csrc_digest(names) -> str:
     h = hashlib.sha256()
     d = os.path.join(ROOT, "paper_2406_02069_b200", "csrc")
-    for name in sorted(os.listdir(d)):
+    for name in sorted(names):
         with open(os.path.join(d, name), "rb") as f:
             h.update(name.encode() + b"\0" + f.read())
     return h.hexdigest()[:16]
@@ -355,7 +356,7 @@ def main():
     achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
     traffic = None
     tr = NCU_TRAFFIC.get(dominant)
-    if tr and tr.get("csrc_digest") == csrc_digest():
+    if tr and tr["digest"] == csrc_digest(tr["sources"]):
         traffic = tr["bytes_per_key_row"] * sum(lens) * w.num_kv_heads
     graded = sum(graded_bytes_per_layer(w, lens, r, esz) for r in out.rows)
     path_gbs = graded / (ms_per_step * 1e-3) / 1e9
