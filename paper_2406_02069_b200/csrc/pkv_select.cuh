@@ -116,6 +116,9 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
   uint2* regions = p.cand + head * p.cand_stride;           // region of CTA c starts at c * slice
   uint32_t* counts = p.cand_cnt + head * kSelMaxCluster;
   for (int i = tid; i < 2 * kSelBins; i += kSelThreads) (&hist[0][0])[i] = 0;
+  // A cluster of one keeps its candidates in shared memory when they fit: no trip through global memory.
+  bool local_pairs = false;
+  int local_count = 0;
 
   if (selecting) {
     const float* s = p.scores + head * p.ld_scores;
@@ -193,15 +196,21 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
       }
       if (lane == 0) warp_gt[warp] = wc;
       __syncthreads();
-      uint32_t base = 0;
-      for (int w2 = 0; w2 < warp; ++w2) base += warp_gt[w2];
-      if (tid == kSelThreads - 1) counts[rank] = base + wc;
+      uint32_t base = 0, all_cand = 0;
+      for (int w2 = 0; w2 < kSelWarps; ++w2) {
+        if (w2 < warp) base += warp_gt[w2];
+        all_cand += warp_gt[w2];
+      }
+      if (tid == kSelThreads - 1) counts[rank] = all_cand;
+      local_pairs = C == 1 && static_cast<int>(all_cand) <= p.smem_pairs;
+      local_count = static_cast<int>(all_cand);
+      uint2* dst = local_pairs ? reinterpret_cast<uint2*>(sel_smem) : region;   // the raw scores are dead by now
 #pragma unroll
       for (int it = 0; it < kSelPerLane; ++it) {
         const int i = wlo + it * 32 + lane;
         const bool c = i < whi && pk[it] >= bound;
         const uint32_t bal = __ballot_sync(0xffffffffu, c);
-        if (c) region[base + __popc(bal & lt)] = make_uint2(pk[it], static_cast<uint32_t>(i));
+        if (c) dst[base + __popc(bal & lt)] = make_uint2(pk[it], static_cast<uint32_t>(i));
         base += __popc(bal);
       }
     } else {
@@ -210,7 +219,7 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
       if (tid == 0) counts[rank] = hi - lo;
     }
   }
-  cluster.sync();                                           // every region and its count are written
+  if (C == 1) __syncthreads(); else cluster.sync();         // every region and its count are written
 
   if (selecting && rank == 0) {
     // ---- 3. CTA 0: concatenate the regions, radix search, emit
@@ -218,7 +227,7 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
     pre[0] = 0;
 #pragma unroll
     for (int c = 0; c < kSelMaxCluster; ++c) pre[c + 1] = pre[c] + (c < C ? __ldcg(counts + c) : 0u);
-    const int N = static_cast<int>(pre[kSelMaxCluster]);
+    const int N = local_pairs ? local_count : static_cast<int>(pre[kSelMaxCluster]);
     auto fetch = [&](int j) -> uint2 {                      // pair j of the concatenation, from global memory
       int c = 0;
 #pragma unroll
@@ -227,8 +236,10 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
     };
     uint2* flat = reinterpret_cast<uint2*>(sel_smem);
     const int held = min(N, p.smem_pairs);
-    for (int j = tid; j < held; j += kSelThreads) flat[j] = fetch(j);
-    __syncthreads();
+    if (!local_pairs) {
+      for (int j = tid; j < held; j += kSelThreads) flat[j] = fetch(j);
+      __syncthreads();
+    }
     auto item = [&](int j) -> uint2 { return j < held ? flat[j] : fetch(j); };
 
     uint32_t prefix = 0, mask = 0, remaining = k;
@@ -302,7 +313,7 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
       eq_before += __popc(be);
     }
   }
-  cluster.sync();                                           // the list is complete
+  if (C == 1) __syncthreads(); else cluster.sync();         // the list is complete
 
   // ---- 5. eviction by gather (appendix on torch.gather), spread over the cluster: 16 bytes of K and of V
   //         per thread and step
