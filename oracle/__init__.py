@@ -6,7 +6,7 @@ restatement in ``pyramidkv_oracle.cpp`` (built with g++ into
 package and the CUDA package imports nothing from here.  Only the tests, the
 smoke check and the benchmark's CPU-baseline leg may call it.
 
-All tensors are CPU torch tensors (float32 or bfloat16); shapes are per sequence:
+All tensors are CPU torch tensors (float32, bfloat16 or float16); shapes are per sequence:
 ``q_win [H_q][alpha][d]``, ``k, v [H_kv][n][d]``.
 """
 from __future__ import annotations
@@ -54,9 +54,11 @@ def _load() -> ctypes.CDLL:
         lib.orc_window_scores_lse.restype = None
         lib.orc_pool_max.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_void_p]
         lib.orc_pool_max.restype = ctypes.c_int
+        lib.orc_pool_avg.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_void_p]
+        lib.orc_pool_avg.restype = ctypes.c_int
         lib.orc_select_topk.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_void_p]
         lib.orc_select_topk.restype = ctypes.c_int
-        lib.orc_compress_layer.argtypes = [ctypes.c_void_p] * 3 + [ctypes.c_int] * 9 + \
+        lib.orc_compress_layer.argtypes = [ctypes.c_void_p] * 3 + [ctypes.c_int] * 10 + \
                                           [ctypes.c_void_p] * 4
         lib.orc_compress_layer.restype = ctypes.c_int
         lib.orc_window_attention.argtypes = [ctypes.c_void_p] * 4 + [ctypes.c_int] * 5 + \
@@ -77,7 +79,9 @@ def _dtype_code(t: torch.Tensor) -> int:
         return 0
     if t.dtype == torch.bfloat16:
         return 1
-    raise TypeError("oracle takes float32 or bfloat16 tensors, got %s" % t.dtype)
+    if t.dtype == torch.float16:
+        return 2
+    raise TypeError("oracle takes float32, bfloat16 or float16 tensors, got %s" % t.dtype)
 
 
 def _host(t: torch.Tensor) -> torch.Tensor:
@@ -137,6 +141,16 @@ def pool_max(x: np.ndarray, w: int) -> np.ndarray:
     return out
 
 
+def pool_avg(x: np.ndarray, w: int) -> np.ndarray:
+    """Mean-pool variant: zeros outside the prefix, always divided by w, float arithmetic left to right."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    assert x.ndim == 1
+    out = np.empty_like(x)
+    if _load().orc_pool_avg(x.ctypes.data, x.shape[0], w, out.ctypes.data) != 0:
+        raise ValueError("pool width must be odd and >= 1")
+    return out
+
+
 def select_topk(pooled: np.ndarray, k: int) -> np.ndarray:
     pooled = np.ascontiguousarray(pooled, dtype=np.float32)
     assert pooled.ndim == 1
@@ -147,7 +161,8 @@ def select_topk(pooled: np.ndarray, k: int) -> np.ndarray:
 
 
 def compress_layer(q_win: torch.Tensor, k: torch.Tensor, v: torch.Tensor, *, pool_kernel: int,
-                   avg_budget: int, k_layer: int, want_scores: bool = True) -> Dict[str, object]:
+                   avg_budget: int, k_layer: int, want_scores: bool = True,
+                   pool_kind: str = "max") -> Dict[str, object]:
     """One layer, one sequence.  Returns kept [H_kv][c] int32, k_out/v_out [H_kv][c][d], scores."""
     q_win, k, v = _host(q_win), _host(k), _host(v)
     hq, alpha, d = q_win.shape
@@ -159,7 +174,8 @@ def compress_layer(q_win: torch.Tensor, k: torch.Tensor, v: torch.Tensor, *, poo
     v_out = torch.empty((hkv, c, d), dtype=v.dtype)
     scores = np.zeros((hkv, n - alpha), dtype=np.float32) if want_scores else None
     got = _load().orc_compress_layer(q_win.data_ptr(), k.data_ptr(), v.data_ptr(), _dtype_code(k),
-                                     hq, hkv, d, alpha, pool_kernel, avg_budget, k_layer, n,
+                                     hq, hkv, d, alpha, pool_kernel, {"max": 0, "avg": 1}[pool_kind], avg_budget,
+                                     k_layer, n,
                                      kept.ctypes.data, k_out.data_ptr(), v_out.data_ptr(),
                                      scores.ctypes.data if want_scores else None)
     assert got == c
@@ -167,7 +183,7 @@ def compress_layer(q_win: torch.Tensor, k: torch.Tensor, v: torch.Tensor, *, poo
 
 
 def compress_batch(q_win: torch.Tensor, k: torch.Tensor, v: torch.Tensor, seq_lens: Sequence[int], *,
-                   pool_kernel: int, avg_budget: int, k_layer: int) -> Dict[str, object]:
+                   pool_kernel: int, avg_budget: int, k_layer: int, pool_kind: str = "max") -> Dict[str, object]:
     """One layer of a ragged batch (tensors padded to the longest sequence).
 
     Packed output: sequences in batch order; inside a sequence head after head,
@@ -176,7 +192,7 @@ def compress_batch(q_win: torch.Tensor, k: torch.Tensor, v: torch.Tensor, seq_le
     rows_k, rows_v, rows_i, scores, counts = [], [], [], [], []
     for b, n in enumerate(seq_lens):
         r = compress_layer(q_win[b], k[b, :, :n], v[b, :, :n], pool_kernel=pool_kernel,
-                           avg_budget=avg_budget, k_layer=k_layer)
+                           avg_budget=avg_budget, k_layer=k_layer, pool_kind=pool_kind)
         d = k.shape[-1]
         rows_k.append(r["k_out"].reshape(-1, d))
         rows_v.append(r["v_out"].reshape(-1, d))

@@ -20,14 +20,17 @@
 // causal among themselves; GQA scores are the mean over the query heads of a
 // group; pooling is a centred max clipped at both ends; ties are broken by
 // (value descending, position ascending); kept positions are emitted ascending.
+// Variants reachable through arguments: a mean pool (zeros outside the prefix,
+// divided by the full width, in float) and binary16 inputs.
 //
 // Arithmetic: every floating-point accumulation is in double; scores are
 // rounded once to float at the end of the score step, and the pool and the
 // selection work on those floats.
 //
 // Pins (tests/test_oracle_*.py): budget closed forms and sums; softmax mass
-// invariant; Q = 0 closed form; library softmax / max_pool1d / sort on small
-// inputs; brute-force subset search; identity when the context fits the budget.
+// invariant; Q = 0 closed form; library softmax / max_pool1d / avg_pool1d / sort
+// on small inputs; brute-force subset search; identity when the context fits the
+// budget; every finite 16-bit pattern against the library's widening.
 // Absolute score values on random data have no value printed in the paper.
 
 #include <algorithm>
@@ -50,9 +53,21 @@ inline double widen_bf16(uint16_t bits) {
   return static_cast<double>(f);
 }
 
-// Element (row, c) of a [rows][d] matrix stored as float (dtype 0) or bfloat16 bits (dtype 1).
+// IEEE 754 binary16: 1 sign bit, 5 exponent bits (bias 15), 10 fraction bits.  Every value is exact in double.
+inline double widen_fp16(uint16_t bits) {
+  const int sign = bits >> 15, e = (bits >> 10) & 31, frac = bits & 1023;
+  double mag;
+  if (e == 0) mag = std::ldexp(static_cast<double>(frac), -24);                 // zero and subnormals
+  else if (e == 31) mag = frac ? std::nan("") : HUGE_VAL;
+  else mag = std::ldexp(1.0 + static_cast<double>(frac) / 1024.0, e - 15);
+  return sign ? -mag : mag;
+}
+
+// Element (row, c) of a [rows][d] matrix stored as float (dtype 0), bfloat16 bits (dtype 1) or binary16 bits
+// (dtype 2).
 inline double elem(const void* base, int dtype, int64_t index) {
   if (dtype == 0) return static_cast<double>(static_cast<const float*>(base)[index]);
+  if (dtype == 2) return widen_fp16(static_cast<const uint16_t*>(base)[index]);
   return widen_bf16(static_cast<const uint16_t*>(base)[index]);
 }
 
@@ -103,7 +118,7 @@ int orc_kept_count(int avg_budget, int alpha, int k_layer, int n) {
 // Section 4.2.2, Eq. 2 and Eq. 3, one sequence.
 //   q   [H_q][alpha][d]   window queries (the last alpha positions), contiguous
 //   k   [H_kv][n][d]      keys, contiguous
-//   dtype 0 = float, 1 = bfloat16 bit patterns
+//   dtype 0 = float, 1 = bfloat16 bit patterns, 2 = binary16 bit patterns
 // Window row j sits at absolute position P + j (P = n - alpha) and, the model
 // being autoregressive, sees keys 0 .. P + j.  Each row is a softmax over what
 // it sees.  The score of prefix key i < P is the sum over the alpha rows of
@@ -189,6 +204,24 @@ int orc_pool_max(const float* in, int P, int w, float* out) {
   return 0;
 }
 
+// The same layer as a mean (the variant the section's "pooling layer" also admits): centred window of odd
+// width w, stride 1, positions outside [0, P) count as zeros, the sum is always divided by w.  The result
+// decides a top-k, so its precision is part of the definition: float additions from the left-most
+// window position to the right-most, then one float division by w.
+int orc_pool_avg(const float* in, int P, int w, float* out) {
+  if (w < 1 || (w % 2) == 0) return -1;
+  const int r = (w - 1) / 2;
+  for (int i = 0; i < P; ++i) {
+    float sum = 0.0f;
+    for (int t = -r; t <= r; ++t) {
+      const int x = i + t;
+      if (x >= 0 && x < P) sum = sum + in[x];
+    }
+    out[i] = sum / static_cast<float>(w);
+  }
+  return 0;
+}
+
 // ---------------------------------------------------------------------------
 // Section 4.2.2: keep the k highest-scored prefix positions.  Order all P
 // positions by (value descending, position ascending), keep the first
@@ -214,7 +247,7 @@ int orc_select_topk(const float* pooled, int P, int k, int32_t* idx_out) {
 //   scores_out  out [H_kv][P] float, may be null
 // Returns c.
 int orc_compress_layer(const void* q, const void* k, const void* v, int dtype, int num_q_heads,
-                       int num_kv_heads, int d, int alpha, int pool_w, int avg_budget, int k_layer,
+                       int num_kv_heads, int d, int alpha, int pool_w, int pool_kind, int avg_budget, int k_layer,
                        int n, int32_t* kept, void* k_out, void* v_out, float* scores_out) {
   const int P = n - alpha;
   const int c = orc_kept_count(avg_budget, alpha, k_layer, n);
@@ -231,7 +264,8 @@ int orc_compress_layer(const void* q, const void* k, const void* v, int dtype, i
     if (keep_all) {
       for (int i = 0; i < P; ++i) row[cnt++] = i;
     } else {
-      orc_pool_max(scores.data() + static_cast<int64_t>(h) * P, P, pool_w, pooled.data());
+      if (pool_kind == 1) orc_pool_avg(scores.data() + static_cast<int64_t>(h) * P, P, pool_w, pooled.data());
+      else orc_pool_max(scores.data() + static_cast<int64_t>(h) * P, P, pool_w, pooled.data());
       cnt = orc_select_topk(pooled.data(), P, k_layer, row);
     }
     for (int i = P; i < n; ++i) row[cnt++] = i;             // instruction tokens, always kept

@@ -39,6 +39,68 @@ def test_pool_spreads_one_spike_over_w_positions():
     np.testing.assert_array_equal(oracle.pool_max(x, 7), x)
 
 
+# ----------------------------------------------------------------------------- mean pool (variant)
+@pytest.mark.parametrize("P,w", [(1, 1), (1, 5), (2, 7), (3, 3), (17, 5), (100, 7), (64, 1), (9, 9), (5, 11)])
+def test_avg_pool_equals_library_avg_pool(P, w):
+    rng = np.random.default_rng(P * 37 + w)
+    x = rng.random(P).astype(np.float32)
+    got = oracle.pool_avg(x, w)
+    want = torch.nn.functional.avg_pool1d(torch.from_numpy(x).double().view(1, 1, P), kernel_size=w, stride=1,
+                                          padding=(w - 1) // 2).view(-1).numpy()     # zeros outside, divided by w
+    np.testing.assert_allclose(got, want, rtol=(w + 1) * 2.0 ** -24, atol=0)
+    if w == 1:
+        np.testing.assert_array_equal(got, x)
+
+
+@pytest.mark.parametrize("w", [3, 5, 7, 11])
+def test_avg_pool_is_exact_on_small_integers(w):
+    # Integer inputs make every partial sum exact, so only the final division rounds: the result must be the
+    # float nearest to the rational sum / w.
+    rng = np.random.default_rng(w)
+    P = 50
+    x = rng.integers(0, 9, P).astype(np.float32)
+    got = oracle.pool_avg(x, w)
+    r = (w - 1) // 2
+    for i in range(P):
+        total = int(sum(x[max(0, i - r): min(P, i + r + 1)]))
+        assert got[i] == np.float32(total / w), (i, total)
+
+
+def test_avg_pool_divides_by_full_width_at_the_edges():
+    x = np.zeros(30, dtype=np.float32)
+    x[0] = 7.0                                              # at the left edge: 4 windows of width 7 contain it
+    got = oracle.pool_avg(x, 7)
+    np.testing.assert_array_equal(got[:4], np.ones(4, dtype=np.float32))
+    assert not got[4:].any()
+    x[:] = 0
+    x[15] = 7.0                                             # interior spike: spread over 7 positions, mass kept
+    got = oracle.pool_avg(x, 7)
+    assert list(np.nonzero(got)[0]) == list(range(12, 19)) and got.sum() == 7.0
+
+
+def test_avg_and_max_pool_choose_differently():
+    s = np.zeros(60, dtype=np.float32)
+    s[10] = 1.0                                             # a lone spike
+    s[30:37] = 0.5                                          # a plateau as wide as the pool
+    assert list(oracle.select_topk(oracle.pool_max(s, 7), 1)) == [7]       # spike wins, left-most of its ties
+    assert list(oracle.select_topk(oracle.pool_avg(s, 7), 1)) == [33]      # plateau centre wins (0.5 > 1/7)
+
+
+def test_layer_with_avg_pool_is_pool_then_select():
+    g = torch.Generator().manual_seed(21)
+    q = torch.randn(4, 8, 64, generator=g)
+    k = torch.randn(2, 300, 64, generator=g)
+    v = torch.randn(2, 300, 64, generator=g)
+    r = oracle.compress_layer(q, k, v, pool_kernel=5, avg_budget=64, k_layer=40, pool_kind="avg")
+    for h in range(2):
+        want = oracle.select_topk(oracle.pool_avg(r["scores"][h], 5), 40)
+        assert list(r["kept"][h][:40]) == list(want)
+        assert list(r["kept"][h][40:]) == list(range(292, 300))
+        assert torch.equal(r["k_out"][h], k[h][torch.from_numpy(r["kept"][h]).long()])
+    m = oracle.compress_layer(q, k, v, pool_kernel=5, avg_budget=64, k_layer=40)
+    assert not np.array_equal(m["kept"], r["kept"])          # the two pools do select different rows here
+
+
 # ----------------------------------------------------------------------------- selection
 def brute_force_select(p, k):
     order = sorted(range(len(p)), key=lambda i: (-float(p[i]), i))
