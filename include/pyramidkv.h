@@ -63,8 +63,11 @@ extern "C" {
 
 #define PKV_DTYPE_FP32 0
 #define PKV_DTYPE_BF16 1
+#define PKV_DTYPE_FP16 2          /* IEEE binary16 */
 
-#define PKV_POOL_MAX 0
+#define PKV_POOL_MAX 0            /* centred max, window clipped to the prefix (the graded reading of Section 4.2.2) */
+#define PKV_POOL_AVG 1            /* centred mean: zeros outside the prefix, always divided by the width; float
+                                     additions left to right, then one float division (it decides the top-k) */
 
 #define PKV_MAX_BATCH 64          /* sequences per call */
 #define PKV_MAX_STAGES 8          /* kernels one pyramidkv_compress_layer call may launch */
@@ -77,7 +80,7 @@ typedef struct pkv_config {
   int32_t head_dim;      /* d: 64 or 128 */
   int32_t window;        /* alpha >= 1: instruction tokens, always kept (Section 4.2.1) */
   int32_t pool_kernel;   /* odd width of the score pooling, 1 = none (Section 4.2.2) */
-  int32_t pool_kind;     /* PKV_POOL_MAX */
+  int32_t pool_kind;     /* PKV_POOL_MAX or PKV_POOL_AVG */
   int32_t dtype;         /* PKV_DTYPE_*: element type shared by K, V and Q_win */
   int32_t avg_budget;    /* B: mean rows kept per layer and KV head, window rows included; >= alpha */
   int32_t reserved;      /* must be 0 */

@@ -99,7 +99,7 @@ def strerror(status: int) -> str:
 
 def make_config(*, num_layers: int, num_q_heads: int, num_kv_heads: int, head_dim: int, window: int,
                 pool_kernel: int, dtype: str, avg_budget: int, beta: float = 20.0, pool_kind: int = 0) -> PkvConfig:
-    code = {"fp32": 0, "bf16": 1, torch.float32: 0, torch.bfloat16: 1}[dtype]
+    code = {"fp32": 0, "bf16": 1, "fp16": 2, torch.float32: 0, torch.bfloat16: 1, torch.float16: 2}[dtype]
     return PkvConfig(num_layers, num_q_heads, num_kv_heads, head_dim, window, pool_kernel, pool_kind, code,
                      avg_budget, 0, float(beta))
 
@@ -108,7 +108,7 @@ def config_of(w) -> PkvConfig:
     """Config of a workloads.Workload."""
     return make_config(num_layers=w.num_layers, num_q_heads=w.num_q_heads, num_kv_heads=w.num_kv_heads,
                        head_dim=w.head_dim, window=w.window, pool_kernel=w.pool_kernel, dtype=w.dtype,
-                       avg_budget=w.avg_budget, beta=w.beta)
+                       avg_budget=w.avg_budget, beta=w.beta, pool_kind={"max": 0, "avg": 1}[w.pool_kind])
 
 
 def _tensor(t: Optional[torch.Tensor]) -> PkvTensor:

@@ -35,9 +35,10 @@ bool config_ok(const pkv_config* c) {
 }
 
 int config_supported(const pkv_config* c) {
-  if (c->dtype != PKV_DTYPE_FP32 && c->dtype != PKV_DTYPE_BF16) return PKV_ERR_UNSUPPORTED;
+  if (c->dtype != PKV_DTYPE_FP32 && c->dtype != PKV_DTYPE_BF16 && c->dtype != PKV_DTYPE_FP16)
+    return PKV_ERR_UNSUPPORTED;
   if (c->head_dim != 64 && c->head_dim != 128) return PKV_ERR_UNSUPPORTED;
-  if (c->pool_kind != PKV_POOL_MAX) return PKV_ERR_UNSUPPORTED;
+  if (c->pool_kind != PKV_POOL_MAX && c->pool_kind != PKV_POOL_AVG) return PKV_ERR_UNSUPPORTED;
   return PKV_OK;
 }
 
@@ -211,10 +212,10 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-// Tensor map of a bf16 [batch][head][token][d] view: dims (d, token, head, batch), box (64, box_tok, box_head, 1),
+// Tensor map of a 16-bit [batch][head][token][d] view: dims (d, token, head, batch), box (64, box_tok, box_head, 1),
 // 128-byte swizzle, zero fill outside the tensor.
-bool make_map(CUtensorMap* map, const pkv_tensor& t, int d, uint64_t tokens, uint64_t heads, uint64_t batch,
-              uint32_t box_tok, uint32_t box_head) {
+bool make_map(CUtensorMap* map, const pkv_tensor& t, bool fp16, int d, uint64_t tokens, uint64_t heads,
+              uint64_t batch, uint32_t box_tok, uint32_t box_head) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (!fn) return false;
   const cuuint64_t dims[4] = {static_cast<cuuint64_t>(d), tokens, heads, batch};
@@ -222,14 +223,14 @@ bool make_map(CUtensorMap* map, const pkv_tensor& t, int d, uint64_t tokens, uin
   const cuuint64_t strides[3] = {bytes(t.stride_token), bytes(t.stride_head), bytes(t.stride_batch)};
   const cuuint32_t box[4] = {64, box_tok, box_head, 1};
   const cuuint32_t estr[4] = {1, 1, 1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(t.ptr), dims, strides, box, estr,
+  return fn(map, fp16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(t.ptr), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 bool tc_eligible(const pkv_config* c) {
   const int g = c->num_q_heads / c->num_kv_heads;
-  return c->dtype == PKV_DTYPE_BF16 && g * c->window <= kTcMaxRows && c->window <= 256 && g <= 256;
+  return (c->dtype == PKV_DTYPE_BF16 || c->dtype == PKV_DTYPE_FP16) && g * c->window <= kTcMaxRows && c->window <= 256 && g <= 256;
 }
 
 int device_sm_count() {
@@ -261,9 +262,10 @@ int launch_scores_tc(const pkv_config* c, const pkv_tensor& q, const pkv_tensor&
     attr_done[dev] = true;
   }
   alignas(64) CUtensorMap q_map, k_map_a, k_map_b;
-  if (!make_map(&q_map, q, D, c->window, c->num_q_heads, batch, c->window, sp.group) ||
-      !make_map(&k_map_a, k, D, max_n, c->num_kv_heads, batch, kTcTileKeysA, 1) ||
-      !make_map(&k_map_b, k, D, max_n, c->num_kv_heads, batch, kTcTileKeysB, 1))
+  const bool fp16 = c->dtype == PKV_DTYPE_FP16;
+  if (!make_map(&q_map, q, fp16, D, c->window, c->num_q_heads, batch, c->window, sp.group) ||
+      !make_map(&k_map_a, k, fp16, D, max_n, c->num_kv_heads, batch, kTcTileKeysA, 1) ||
+      !make_map(&k_map_b, k, fp16, D, max_n, c->num_kv_heads, batch, kTcTileKeysB, 1))
     return PKV_ERR_CUDA;
 
   TcParams tp{};
@@ -272,6 +274,7 @@ int launch_scores_tc(const pkv_config* c, const pkv_tensor& q, const pkv_tensor&
   tp.group = sp.group;
   tp.rows = sp.rows;
   tp.rows_pad = (sp.rows + 31) / 32 * 32;
+  tp.fp16 = fp16 ? 1 : 0;
   tp.row_blocks = (sp.rows + 127) / 128;
   tp.scale_log2 = sp.scale_log2;
   tp.partial = sp.partial;
@@ -356,6 +359,9 @@ int run_scores(const pkv_config* c, const pkv_tensor& q, const pkv_tensor& k, co
   if (c->dtype == PKV_DTYPE_FP32)
     return c->head_dim == 64 ? launch_scores_generic<float, 64>(sp, batch, st)
                              : launch_scores_generic<float, 128>(sp, batch, st);
+  if (c->dtype == PKV_DTYPE_FP16)
+    return c->head_dim == 64 ? launch_scores_generic<__half, 64>(sp, batch, st)
+                             : launch_scores_generic<__half, 128>(sp, batch, st);
   return c->head_dim == 64 ? launch_scores_generic<__nv_bfloat16, 64>(sp, batch, st)
                            : launch_scores_generic<__nv_bfloat16, 128>(sp, batch, st);
 }
@@ -372,6 +378,7 @@ int run_select(const pkv_config* c, const float* scores, int64_t ld, const SeqTa
   sp.seq = table;
   sp.num_kv_heads = c->num_kv_heads;
   sp.pool_radius = (c->pool_kernel - 1) / 2;
+  sp.pool_avg = c->pool_kind == PKV_POOL_AVG ? 1 : 0;
   sp.status = w.status;
   sp.cand = w.sel_cand;
   sp.cand_stride = w.sel_cand_stride;
@@ -678,6 +685,9 @@ int pyramidkv_decode_attention(const pkv_config* cfg, const void* q, const void*
   if (cfg->dtype == PKV_DTYPE_FP32) {
     if (cfg->head_dim == 64) launch_pdl(decode_attention_kernel<float, 64>, grid, kDecThreads, 0, st, dp);
     else launch_pdl(decode_attention_kernel<float, 128>, grid, kDecThreads, 0, st, dp);
+  } else if (cfg->dtype == PKV_DTYPE_FP16) {
+    if (cfg->head_dim == 64) launch_pdl(decode_attention_kernel<__half, 64>, grid, kDecThreads, 0, st, dp);
+    else launch_pdl(decode_attention_kernel<__half, 128>, grid, kDecThreads, 0, st, dp);
   } else {
     if (cfg->head_dim == 64) launch_pdl(decode_attention_kernel<__nv_bfloat16, 64>, grid, kDecThreads, 0, st, dp);
     else launch_pdl(decode_attention_kernel<__nv_bfloat16, 128>, grid, kDecThreads, 0, st, dp);

@@ -1,4 +1,4 @@
-// Window-score kernels on the sm_100a tensor cores (Section 4.2.2, Eq. 2 and Eq. 3), bf16 inputs.
+// Window-score kernels on the sm_100a tensor cores (Section 4.2.2, Eq. 2 and Eq. 3), bf16 or fp16 inputs.
 //
 // Two sweeps over K, because the score of a key sums softmax rows that each have
 // their own normaliser (known only after a whole row has been seen):
@@ -47,6 +47,7 @@ struct TcParams {
   SeqTable seq;                 // stat_off / score_off count CHUNKS of chunk_tiles tiles
   int32_t num_kv_heads, group, rows;      // rows = group * alpha (R)
   int32_t rows_pad;             // R rounded up to 32
+  int32_t fp16;                 // 1: Q and K hold binary16, 0: bfloat16 (both operands always share the type)
   int32_t row_blocks;           // ceil(R / 128): M-blocks of sweep A
   int32_t chunk_tiles_a;        // 256-key tiles per work item of sweep A
   int32_t chunk_tiles_b;        // 128-key tiles per work item of sweep B
@@ -126,7 +127,7 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+__device__ __forceinline__ void tc_mma_f16kind(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                             uint32_t accumulate) {
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
@@ -266,9 +267,11 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
   d |= static_cast<uint64_t>(2) << 61;                         // 128-byte swizzle
   return d;
 }
-// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M x N tile.
-__device__ __forceinline__ uint32_t instr_desc_bf16(int M, int N) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(N >> 3) << 17) |
+// Instruction descriptor: 16-bit x 16-bit -> fp32, both operands K-major and of one type (format code 1 =
+// bf16, 0 = fp16, for A at bit 7 and B at bit 10), M x N tile.
+__device__ __forceinline__ uint32_t instr_desc_16bit(int M, int N, int fp16) {
+  const uint32_t fmt = fp16 ? 0u : 1u;
+  return (1u << 4) | (fmt << 7) | (fmt << 10) | (static_cast<uint32_t>(N >> 3) << 17) |
          (static_cast<uint32_t>(M >> 4) << 24);
 }
 
@@ -419,7 +422,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       uint32_t it = 0, u = 0, heads_seen = 0;                  // it counts K tiles, u accumulator units
       int cur_b = -1, cur_h = -1;
       bool ok = true;
-      const uint32_t idesc = SWEEP == 0 ? instr_desc_bf16(128, kTcTileKeysA) : instr_desc_bf16(kTcTileKeysB, p.rows_pad);
+      const uint32_t idesc = SWEEP == 0 ? instr_desc_16bit(128, kTcTileKeysA, p.fp16)
+                                        : instr_desc_16bit(kTcTileKeysB, p.rows_pad, p.fp16);
       for (int id = item0; id < item1 && ok; ++id) {
         const TcItem w = tc_item(off, p.seq.batch, p.num_kv_heads, id);
         if (w.b != cur_b || w.h != cur_h) {
@@ -454,8 +458,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
             for (int kk = 0; kk < D / 16; ++kk) {
               const uint32_t qa = q_addr + (kk / 4) * kTcMaxRows * 128 + rb * 128 * 128 + (kk % 4) * 32;
               const uint32_t ka = k_addr + (kk / 4) * kTileKeys * 128 + (kk % 4) * 32;
-              if (SWEEP == 0) tc_mma_bf16(d_addr, smem_desc_sw128(qa), smem_desc_sw128(ka), idesc, kk > 0);
-              else tc_mma_bf16(d_addr, smem_desc_sw128(ka), smem_desc_sw128(qa), idesc, kk > 0);
+              if (SWEEP == 0) tc_mma_f16kind(d_addr, smem_desc_sw128(qa), smem_desc_sw128(ka), idesc, kk > 0);
+              else tc_mma_f16kind(d_addr, smem_desc_sw128(ka), smem_desc_sw128(qa), idesc, kk > 0);
             }
             tc_commit(t_full(ts));
           }

@@ -52,6 +52,7 @@ struct SelectParams {
   SeqTable seq;
   int32_t num_kv_heads;
   int32_t pool_radius;      // (w - 1) / 2
+  int32_t pool_avg;         // 0: centred max clipped to the prefix; 1: centred mean, zeros outside, divided by w
   int32_t cached;           // 1: every CTA's slice fits kSelSliceCap and is staged in shared memory
   int32_t smem_pairs;       // (key, position) pairs CTA 0 can hold in its dynamic shared memory
   uint2* cand;              // scratch: [batch * H_kv][cand_stride] candidate pairs, one region per CTA rank
@@ -73,10 +74,17 @@ __device__ __forceinline__ uint32_t ordered_key(float x) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-__device__ __forceinline__ uint32_t pooled_key(const float* s, int i, int P, int radius) {
+// The mean pool decides a top-k, so its rounding is fixed: float additions from the left-most position of the
+// window to the right-most, then one float division by the width.
+__device__ __forceinline__ uint32_t pooled_key(const float* s, int i, int P, int radius, int avg) {
   const int lo = max(0, i - radius), hi = min(P - 1, i + radius);
   float best = s[lo];
-  for (int t = lo + 1; t <= hi; ++t) best = fmaxf(best, s[t]);
+  if (avg) {
+    for (int t = lo + 1; t <= hi; ++t) best = __fadd_rn(best, s[t]);
+    best = __fdiv_rn(best, static_cast<float>(2 * radius + 1));
+  } else {
+    for (int t = lo + 1; t <= hi; ++t) best = fmaxf(best, s[t]);
+  }
   return ordered_key(best);
 }
 
@@ -128,10 +136,12 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
     const int radius = p.pool_radius;
     uint2* region = regions + static_cast<int64_t>(rank) * slice;
     if (p.cached) {                                         // then run <= kSelRunMax
-      // ---- 1. stage raw scores with a halo (-inf outside the prefix) and pool
+      // ---- 1. stage raw scores with a halo (outside the prefix: -inf for the max, 0 for the mean) and pool
       float* raw = reinterpret_cast<float*>(sel_smem + kSelHalo);
+      const float outside = p.pool_avg ? 0.0f : -INFINITY;
+      const float width = static_cast<float>(2 * radius + 1);
       for (int i = lo - kSelHalo + tid; i < hi + kSelHalo; i += kSelThreads)
-        raw[i - lo] = (i >= 0 && i < P) ? s[i] : -INFINITY;
+        raw[i - lo] = (i >= 0 && i < P) ? s[i] : outside;
       __syncthreads();
       uint32_t pk[kSelPerLane];
       uint32_t tmax = 0;
@@ -140,8 +150,15 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
         const int i = wlo + it * 32 + lane;
         pk[it] = 0;
         if (i < whi) {
-          float best = raw[i - lo];
-          for (int t = 1; t <= radius; ++t) best = fmaxf(best, fmaxf(raw[i - lo - t], raw[i - lo + t]));
+          float best;
+          if (p.pool_avg) {                                 // left to right; adding the zeros outside changes nothing
+            best = raw[i - lo - radius];
+            for (int t = 1 - radius; t <= radius; ++t) best = __fadd_rn(best, raw[i - lo + t]);
+            best = __fdiv_rn(best, width);
+          } else {
+            best = raw[i - lo];
+            for (int t = 1; t <= radius; ++t) best = fmaxf(best, fmaxf(raw[i - lo - t], raw[i - lo + t]));
+          }
           pk[it] = ordered_key(best);
           tmax = max(tmax, pk[it]);
         }
@@ -215,7 +232,7 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
       }
     } else {
       // slices too long for shared memory, or a very wide pool: every position is a candidate
-      for (int i = lo + tid; i < hi; i += kSelThreads) region[i - lo] = make_uint2(pooled_key(s, i, P, radius), i);
+      for (int i = lo + tid; i < hi; i += kSelThreads) region[i - lo] = make_uint2(pooled_key(s, i, P, radius, p.pool_avg), i);
       if (tid == 0) counts[rank] = hi - lo;
     }
   }

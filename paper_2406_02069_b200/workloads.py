@@ -40,7 +40,7 @@ class Workload:
     batch: int
     seq_len_lo: int          # per-sequence length is uniform in [lo, hi]
     seq_len_hi: int
-    dtype: str               # "fp32" | "bf16"
+    dtype: str               # "fp32" | "bf16" | "fp16"
     window: int              # alpha
     pool_kernel: int         # w
     avg_budget: int          # B, window rows included
@@ -53,13 +53,14 @@ class Workload:
     sink_gain: float = 2.0
     needle_gain: float = 1.5
     seed: int = 0
+    pool_kind: str = "max"   # "max" | "avg" (the mean-pool variant)
 
     @property
     def group(self) -> int:
         return self.num_q_heads // self.num_kv_heads
 
     def torch_dtype(self) -> torch.dtype:
-        return {"fp32": torch.float32, "bf16": torch.bfloat16}[self.dtype]
+        return {"fp32": torch.float32, "bf16": torch.bfloat16, "fp16": torch.float16}[self.dtype]
 
     def seq_lens(self) -> List[int]:
         """Per-sequence context lengths, drawn once from the workload seed."""
@@ -97,9 +98,10 @@ def with_budget(w: Workload, avg_budget: int) -> Workload:
 
 
 def scaled(w: Workload, *, num_layers: Optional[int] = None, seq_len: Optional[int] = None,
-           batch: Optional[int] = None, name: Optional[str] = None) -> Workload:
-    """A smaller case of the same shape family (for tests the oracle finishes in seconds)."""
-    kw = {}
+           batch: Optional[int] = None, name: Optional[str] = None, **fields) -> Workload:
+    """A smaller case of the same shape family (for tests the oracle finishes in seconds); further keyword
+    arguments replace fields by name (dtype, pool_kind, window, beta ...)."""
+    kw = dict(fields)
     if num_layers is not None:
         kw["num_layers"] = num_layers
     if seq_len is not None:

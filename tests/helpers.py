@@ -18,7 +18,7 @@ def assert_scores_close(got: np.ndarray, want: np.ndarray, what=""):
 
 
 def assert_indices_match(got_row: np.ndarray, want_row: np.ndarray, oracle_scores_row: np.ndarray, w: int,
-                         alpha: int, what=""):
+                         alpha: int, what="", pool_kind="max"):
     """Kept lists of one (sequence, head): identical, or differing only where the oracle's pooled
     score is within tolerance of the oracle's k-th pooled value (the threshold)."""
     assert len(got_row) == len(want_row), what
@@ -28,7 +28,8 @@ def assert_indices_match(got_row: np.ndarray, want_row: np.ndarray, oracle_score
     if np.array_equal(got_row, want_row):
         return True
     P = oracle_scores_row.shape[0]
-    pooled = oracle.pool_max(oracle_scores_row, w).astype(np.float64)
+    pool = oracle.pool_avg if pool_kind == "avg" else oracle.pool_max
+    pooled = pool(oracle_scores_row, w).astype(np.float64)
     k = len(want_row) - alpha
     kth = np.sort(pooled)[::-1][k - 1]
     diff = np.setxor1d(got_row[:k], want_row[:k])

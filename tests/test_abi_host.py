@@ -96,6 +96,12 @@ def test_validation_happens_before_any_device_work():
                           dtype="bf16", avg_budget=64)
     st = lib.pyramidkv_score_window(ctypes.byref(bad), fake, fake, lens, 1, 4096, 128, 4096, 1 << 30, None)
     assert st == binding.PKV_ERR_UNSUPPORTED
+    for field, value in (("dtype", 3), ("pool_kind", 2)):           # codes past fp16 / the mean pool are not built
+        odd_cfg = pkv.make_config(num_layers=4, num_q_heads=8, num_kv_heads=2, head_dim=128, window=8, pool_kernel=7,
+                                  dtype="fp16", avg_budget=64, pool_kind=1)
+        setattr(odd_cfg, field, value)
+        st = lib.pyramidkv_score_window(ctypes.byref(odd_cfg), fake, fake, lens, 1, 4096, 128, 4096, 1 << 30, None)
+        assert st == binding.PKV_ERR_UNSUPPORTED
     assert pkv.strerror(binding.PKV_ERR_WORKSPACE).startswith("workspace")
 
 
