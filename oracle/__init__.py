@@ -68,6 +68,13 @@ def _load() -> ctypes.CDLL:
         lib.orc_decode_attention.restype = None
         lib.orc_attention_recall.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_void_p, ctypes.c_int]
         lib.orc_attention_recall.restype = ctypes.c_double
+        lib.orc_pages_needed.argtypes = [ctypes.c_int] * 5
+        lib.orc_pages_needed.restype = ctypes.c_int
+        lib.orc_scatter_paged.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_void_p,
+                                          ctypes.c_int, ctypes.c_void_p]
+        lib.orc_scatter_paged.restype = ctypes.c_int
+        lib.orc_read_paged.argtypes = lib.orc_scatter_paged.argtypes
+        lib.orc_read_paged.restype = ctypes.c_int
         lib.orc_num_threads.argtypes = []
         lib.orc_num_threads.restype = ctypes.c_int
         _lib = lib
@@ -231,3 +238,34 @@ def attention_recall(scores_row: np.ndarray, alpha: int, kept: np.ndarray) -> fl
     s = np.ascontiguousarray(scores_row, dtype=np.float32)
     kp = np.ascontiguousarray(kept, dtype=np.int32)
     return float(_load().orc_attention_recall(s.ctypes.data, s.shape[0], int(alpha), kp.ctypes.data, kp.shape[0]))
+
+
+def pages_needed(avg_budget: int, alpha: int, k_layer: int, n: int, page_size: int) -> int:
+    """Pages one KV head of an n-token sequence needs in a layer with budget k_layer."""
+    got = int(_load().orc_pages_needed(avg_budget, alpha, k_layer, n, page_size))
+    if got < 0:
+        raise ValueError("page_size must be >= 1")
+    return got
+
+
+def scatter_paged(rows: torch.Tensor, table: np.ndarray, page_size: int, pool: torch.Tensor) -> None:
+    """Place rows [c][d] of one head into pool [num_pages][page_size][d] through its block table (in place)."""
+    rows = _host(rows)
+    assert pool.is_contiguous() and pool.dtype == rows.dtype and pool.shape[1:] == (page_size, rows.shape[1])
+    tab = np.ascontiguousarray(table, dtype=np.int32)
+    c, d = rows.shape
+    assert tab.shape[0] >= (c + page_size - 1) // page_size
+    if _load().orc_scatter_paged(rows.data_ptr(), c, d * rows.element_size(), page_size, tab.ctypes.data,
+                                 pool.shape[0], pool.data_ptr()) != 0:
+        raise ValueError("block table names a page outside the pool")
+
+
+def read_paged(pool: torch.Tensor, table: np.ndarray, count: int, page_size: int) -> torch.Tensor:
+    """The `count` rows of one head, in list order, read back through its block table."""
+    assert pool.is_contiguous() and pool.shape[1] == page_size
+    tab = np.ascontiguousarray(table, dtype=np.int32)
+    rows = torch.empty((count, pool.shape[2]), dtype=pool.dtype)
+    if _load().orc_read_paged(pool.data_ptr(), count, pool.shape[2] * pool.element_size(), page_size,
+                              tab.ctypes.data, pool.shape[0], rows.data_ptr()) != 0:
+        raise ValueError("block table names a page outside the pool")
+    return rows

@@ -13,6 +13,7 @@
 //   pool      Section 4.2.2          a pooling layer applied to the scores (max, odd width)
 //   select    Section 4.2.2          top k^l per head, plus the last alpha tokens always
 //   gather    Appendix (eviction by gather): copy the kept rows into a new tensor
+//   paged     Appendix (paged attention): the same rows placed in pages through a per-layer block table
 //
 // Where the paper is silent the readings are: the budget B counts the alpha
 // window rows, the pyramid is laid over B - alpha; real budgets are floored and
@@ -343,6 +344,46 @@ double orc_attention_recall(const float* scores, int P, int alpha, const int32_t
     if (kept[r] < P) on_kept += scores[kept[r]];
   const double window_mass = alpha - all;                 // every row's attention sums to one
   return (on_kept + window_mass) / alpha;
+}
+
+// ---------------------------------------------------------------------------
+// Appendix on paged attention: a per-layer block table per sequence, so that each layer's cache lives in
+// pages of its own and can be found "without the use of fixed memory offsets".  Layout used here: a pool
+// of pages, each holding page_size rows of one KV head; row r of a head's kept list sits in the page
+// table[r / page_size] at slot r % page_size.
+int orc_pages_needed(int avg_budget, int alpha, int k_layer, int n, int page_size) {
+  if (page_size < 1) return -1;
+  const int c = orc_kept_count(avg_budget, alpha, k_layer, n);
+  return (c + page_size - 1) / page_size;
+}
+
+// rows [c][row_bytes] of one head -> pool [num_pages][page_size][row_bytes] through table [ceil(c/page_size)].
+// Returns 0, or -1 when a table entry names a page outside the pool (nothing is written then).
+int orc_scatter_paged(const void* rows, int c, int row_bytes, int page_size, const int32_t* table, int num_pages,
+                      void* pool) {
+  const int pages = (c + page_size - 1) / page_size;
+  for (int j = 0; j < pages; ++j)
+    if (table[j] < 0 || table[j] >= num_pages) return -1;
+  for (int r = 0; r < c; ++r) {
+    const size_t dst = (static_cast<size_t>(table[r / page_size]) * page_size + (r % page_size)) * row_bytes;
+    std::memcpy(static_cast<char*>(pool) + dst, static_cast<const char*>(rows) + static_cast<size_t>(r) * row_bytes,
+                row_bytes);
+  }
+  return 0;
+}
+
+// The inverse walk: the c rows of one head, in list order, read back through its table.
+int orc_read_paged(const void* pool, int c, int row_bytes, int page_size, const int32_t* table, int num_pages,
+                   void* rows) {
+  const int pages = (c + page_size - 1) / page_size;
+  for (int j = 0; j < pages; ++j)
+    if (table[j] < 0 || table[j] >= num_pages) return -1;
+  for (int r = 0; r < c; ++r) {
+    const size_t src = (static_cast<size_t>(table[r / page_size]) * page_size + (r % page_size)) * row_bytes;
+    std::memcpy(static_cast<char*>(rows) + static_cast<size_t>(r) * row_bytes, static_cast<const char*>(pool) + src,
+                row_bytes);
+  }
+  return 0;
 }
 
 int orc_num_threads() {
