@@ -303,6 +303,64 @@ int pyramidkv_profile_layer_lse(const pkv_config* cfg, int32_t layer,
                                 float* stage_ms, char (*stage_names)[32], int32_t* num_stages);
 
 /*
+ * Paged placement of a layer's compact cache (appendix on paged attention: the block table of a
+ * sequence is widened to one block table per layer, so that each layer's cache is found through its
+ * own pages rather than at fixed offsets, and a layer with a small budget holds few pages).
+ *
+ * Layout.  A pool holds num_pages pages; a page holds page_size rows of d elements of ONE KV head of
+ * one sequence: k_pool, v_pool are [num_pages][page_size][d] of the config dtype.  Row r of the kept
+ * list of (sequence b, KV head h) sits in page  table[r / page_size]  at slot  r % page_size, where
+ * `table` is that head's slice of the layer's block table.  The block table of one layer is a packed
+ * int32 array: sequences in batch order, inside a sequence head after head, each head holding
+ *     pages_b = pyramidkv_pages_needed(cfg, k_layer, n_b, page_size) = ceil(c_b / page_size)
+ * entries; the slice of (b, h) starts at  H_kv * (pages_0 + ... + pages_{b-1}) + h * pages_b.
+ * The caller's allocator fills the table with pages it owns; the library only follows it.  Slots of
+ * the last page past c_b, and pages the table does not name, are not touched.  The index list (one
+ * original position per kept row) keeps the packed layout of pyramidkv_compress_layer.
+ *
+ * A table entry outside [0, num_pages) is never dereferenced: the row is skipped and the workspace
+ * status word gets a bit set (pyramidkv_check_status then returns PKV_ERR_DEVICE_STATUS).
+ */
+
+/* Host only.  Pages one KV head of a seq_len-token sequence needs; negative status on bad arguments. */
+int pyramidkv_pages_needed(const pkv_config* cfg, int32_t k_layer, int32_t seq_len, int32_t page_size);
+
+/*
+ * Eviction by gather into pages: the rows of K and V named by `indices` (packed, as written by
+ * pyramidkv_select_topk for budget k_layer) go to their page slots.  Bit copies.
+ *   block_table  device int32, layout above      page_size >= 1, num_pages >= 1
+ *   k_pool, v_pool  device, 16-byte aligned      workspace: only its status word is used (>= 256 bytes)
+ * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA.
+ */
+int pyramidkv_gather_paged(const pkv_config* cfg, pkv_tensor k, pkv_tensor v, const int32_t* indices,
+                           const int32_t* seq_lens, int32_t batch, int32_t k_layer,
+                           const int32_t* block_table, int32_t page_size, int32_t num_pages,
+                           void* k_pool, void* v_pool,
+                           void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * pyramidkv_compress_layer with the kept rows placed in pages: scores, pool, top-k and window
+ * retention as there (window_lse_or_null: the optional row normalisers of the single-sweep mode),
+ * then the gather above.  `indices` receives the packed list of original positions.
+ */
+int pyramidkv_compress_layer_paged(const pkv_config* cfg, int32_t layer,
+                                   pkv_tensor q_win, pkv_tensor k, pkv_tensor v, const float* window_lse_or_null,
+                                   const int32_t* seq_lens, int32_t batch,
+                                   const int32_t* block_table, int32_t page_size, int32_t num_pages,
+                                   void* k_pool, void* v_pool, int32_t* indices,
+                                   float* scores_or_null, int64_t ld_scores,
+                                   void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * pyramidkv_decode_attention over a paged layer: the kept rows of each KV head are read through the
+ * layer's block table, in list order.  Arguments as there and as pyramidkv_gather_paged.
+ */
+int pyramidkv_decode_attention_paged(const pkv_config* cfg, const void* q, const void* k_pool, const void* v_pool,
+                                     const int32_t* block_table, int32_t page_size, int32_t num_pages,
+                                     const int32_t* seq_lens, int32_t batch, int32_t k_layer, float* out,
+                                     void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Synchronises `stream` and reads the workspace status word.  For tests and
  * debugging.  Returns PKV_OK, PKV_ERR_DEVICE_STATUS (a kernel gave up on a
  * bounded wait or saw an impossible state; *detail_or_null receives the word),

@@ -29,7 +29,8 @@ EXPORTS = ("pyramidkv_strerror", "pyramidkv_layer_budgets", "pyramidkv_kept_coun
            "pyramidkv_gather_compact", "pyramidkv_compress_layer", "pyramidkv_profile_layer",
            "pyramidkv_check_status", "pyramidkv_score_window_static", "pyramidkv_score_window_lse",
            "pyramidkv_compress_layer_lse", "pyramidkv_profile_layer_lse", "pyramidkv_decode_attention",
-           "pyramidkv_attention_recall")
+           "pyramidkv_attention_recall", "pyramidkv_pages_needed", "pyramidkv_gather_paged",
+           "pyramidkv_compress_layer_paged", "pyramidkv_decode_attention_paged")
 PKV_MAX_STAGES = 8
 
 
@@ -79,6 +80,11 @@ def _load() -> ctypes.CDLL:
     lib.pyramidkv_profile_layer_lse.argtypes = lib.pyramidkv_compress_layer_lse.argtypes + [P, P, P]
     lib.pyramidkv_decode_attention.argtypes = [CFG, P, P, P, P, I32, I32, P, P]
     lib.pyramidkv_attention_recall.argtypes = [CFG, P, I64, P, P, I32, I32, P, P]
+    lib.pyramidkv_pages_needed.argtypes = [CFG, I32, I32, I32]
+    lib.pyramidkv_gather_paged.argtypes = [CFG, PkvTensor, PkvTensor, P, P, I32, I32, P, I32, I32, P, P, P, SZ, P]
+    lib.pyramidkv_compress_layer_paged.argtypes = [CFG, I32, PkvTensor, PkvTensor, PkvTensor, P, P, I32, P, I32, I32,
+                                                   P, P, P, P, I64, P, SZ, P]
+    lib.pyramidkv_decode_attention_paged.argtypes = [CFG, P, P, P, P, I32, I32, P, I32, I32, P, P, SZ, P]
     lib.pyramidkv_check_status.argtypes = [P, P, P]
     for name in EXPORTS:
         if name not in ("pyramidkv_strerror", "pyramidkv_workspace_bytes"):
@@ -144,6 +150,14 @@ def kept_count(cfg: PkvConfig, k_layer: int, seq_len: int) -> int:
     c = _lib.pyramidkv_kept_count(ctypes.byref(cfg), int(k_layer), int(seq_len))
     if c < 0:
         raise PkvError(-c, "pyramidkv_kept_count")
+    return int(c)
+
+
+def pages_needed(cfg: PkvConfig, k_layer: int, seq_len: int, page_size: int) -> int:
+    """Pages one KV head of a seq_len-token sequence needs in a layer with budget k_layer."""
+    c = _lib.pyramidkv_pages_needed(ctypes.byref(cfg), int(k_layer), int(seq_len), int(page_size))
+    if c < 0:
+        raise PkvError(-c, "pyramidkv_pages_needed")
     return int(c)
 
 
@@ -287,3 +301,50 @@ def check_status(workspace: torch.Tensor, stream=None) -> int:
     if st != PKV_OK:
         raise PkvError(st, "pyramidkv_check_status (word 0x%x)" % detail.value)
     return 0
+
+
+def _paged(block_table: torch.Tensor, k_pool: torch.Tensor, v_pool: torch.Tensor):
+    """(table pointer, page_size, num_pages, k pointer, v pointer) of pools [num_pages][page_size][d]."""
+    if block_table.dtype != torch.int32 or not block_table.is_contiguous():
+        raise ValueError("block_table must be a contiguous int32 tensor")
+    if k_pool.dim() != 3 or k_pool.shape != v_pool.shape or not (k_pool.is_contiguous() and v_pool.is_contiguous()):
+        raise ValueError("k_pool and v_pool must be contiguous [num_pages][page_size][d] tensors of one shape")
+    return block_table.data_ptr(), int(k_pool.shape[1]), int(k_pool.shape[0]), k_pool.data_ptr(), v_pool.data_ptr()
+
+
+def gather_paged(cfg: PkvConfig, k: torch.Tensor, v: torch.Tensor, indices: torch.Tensor, seq_lens: Sequence[int],
+                 k_layer: int, block_table: torch.Tensor, k_pool: torch.Tensor, v_pool: torch.Tensor,
+                 workspace: torch.Tensor, stream=None) -> None:
+    lens, batch = _lens(seq_lens)
+    tab, page_size, num_pages, kp, vp = _paged(block_table, k_pool, v_pool)
+    _check(_lib.pyramidkv_gather_paged(ctypes.byref(cfg), _tensor(k), _tensor(v), indices.data_ptr(), lens, batch,
+                                       int(k_layer), tab, page_size, num_pages, kp, vp, workspace.data_ptr(),
+                                       workspace.numel(), _stream(stream)), "pyramidkv_gather_paged")
+
+
+def compress_layer_paged(cfg: PkvConfig, layer: int, q_win: torch.Tensor, k: torch.Tensor, v: torch.Tensor,
+                         seq_lens: Sequence[int], block_table: torch.Tensor, k_pool: torch.Tensor,
+                         v_pool: torch.Tensor, indices: torch.Tensor, workspace: torch.Tensor,
+                         scores: Optional[torch.Tensor] = None, stream=None,
+                         window_lse: Optional[torch.Tensor] = None) -> None:
+    lens, batch = _lens(seq_lens)
+    tab, page_size, num_pages, kp, vp = _paged(block_table, k_pool, v_pool)
+    _check(_lib.pyramidkv_compress_layer_paged(
+        ctypes.byref(cfg), int(layer), _tensor(q_win), _tensor(k), _tensor(v),
+        _lse_ptr(window_lse) if window_lse is not None else None, lens, batch, tab, page_size, num_pages, kp, vp,
+        indices.data_ptr(), scores.data_ptr() if scores is not None else None,
+        scores.stride(1) if scores is not None else 0, workspace.data_ptr(), workspace.numel(), _stream(stream)),
+        "pyramidkv_compress_layer_paged")
+
+
+def decode_attention_paged(cfg: PkvConfig, q: torch.Tensor, block_table: torch.Tensor, k_pool: torch.Tensor,
+                           v_pool: torch.Tensor, seq_lens: Sequence[int], k_layer: int, out: torch.Tensor,
+                           workspace: torch.Tensor, stream=None) -> None:
+    lens, batch = _lens(seq_lens)
+    if not (q.is_contiguous() and out.is_contiguous()):
+        raise ValueError("decode_attention_paged takes contiguous q and out")
+    tab, page_size, num_pages, kp, vp = _paged(block_table, k_pool, v_pool)
+    _check(_lib.pyramidkv_decode_attention_paged(ctypes.byref(cfg), q.data_ptr(), kp, vp, tab, page_size, num_pages,
+                                                 lens, batch, int(k_layer), out.data_ptr(), workspace.data_ptr(),
+                                                 workspace.numel(), _stream(stream)),
+           "pyramidkv_decode_attention_paged")

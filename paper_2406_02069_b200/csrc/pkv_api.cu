@@ -449,6 +449,50 @@ int run_gather(const pkv_config* c, const pkv_tensor& k, const pkv_tensor& v, co
   return check_launch();
 }
 
+// Table offsets of a layer's block table: sequences in batch order, H_kv * pages_b entries each.
+void fill_page_table(const pkv_config* c, const SeqTable& t, const int32_t* block_table, int page_size,
+                     int num_pages, PageTable* pt) {
+  std::memset(pt, 0, sizeof *pt);
+  pt->table = block_table;
+  pt->page_size = page_size;
+  pt->num_pages = num_pages;
+  int64_t off = 0;
+  for (int b = 0; b < t.batch; ++b) {
+    pt->pages[b] = (t.count[b] + page_size - 1) / page_size;
+    pt->tab_off[b] = off;
+    off += static_cast<int64_t>(c->num_kv_heads) * pt->pages[b];
+  }
+}
+
+int run_gather_paged(const pkv_config* c, const pkv_tensor& k, const pkv_tensor& v, const int32_t* indices,
+                     const SeqTable& table, int64_t total_rows, const int32_t* block_table, int page_size,
+                     int num_pages, void* k_pool, void* v_pool, uint32_t* status, cudaStream_t st) {
+  GatherPagedParams gp{};
+  gp.k = view(k);
+  gp.v = view(v);
+  gp.indices = indices;
+  gp.k_pool = k_pool;
+  gp.v_pool = v_pool;
+  gp.seq = table;
+  fill_page_table(c, table, block_table, page_size, num_pages, &gp.pt);
+  gp.num_kv_heads = c->num_kv_heads;
+  gp.elem_bytes = c->dtype == PKV_DTYPE_FP32 ? 4 : 2;
+  gp.pieces = c->head_dim * gp.elem_bytes / 16;
+  gp.total_rows = total_rows;
+  gp.status = status;
+  const int64_t threads = total_rows * gp.pieces;
+  if (threads == 0) return PKV_OK;
+  const unsigned blocks = static_cast<unsigned>((threads + kPagedThreads - 1) / kPagedThreads);
+  launch_pdl(gather_paged_kernel, blocks, kPagedThreads, 0, st, gp);
+  mark(st, "gather_paged");
+  return check_launch();
+}
+
+bool paged_args_ok(const int32_t* block_table, int page_size, int num_pages, const void* k_pool, const void* v_pool) {
+  if (!block_table || !k_pool || !v_pool || page_size < 1 || num_pages < 1) return false;
+  return reinterpret_cast<uintptr_t>(k_pool) % 16 == 0 && reinterpret_cast<uintptr_t>(v_pool) % 16 == 0;
+}
+
 int workspace_check(const pkv_config* c, int batch, int max_n, void* ws, size_t ws_bytes, Workspace* out) {
   if (!ws || reinterpret_cast<uintptr_t>(ws) % kAlign) return PKV_ERR_WORKSPACE;
   *out = carve(c, batch, max_n, ws);
@@ -556,6 +600,16 @@ int pyramidkv_gather_compact(const pkv_config* cfg, pkv_tensor k, pkv_tensor v, 
   return run_gather(cfg, k, v, indices, table, rows, k_out, v_out, static_cast<cudaStream_t>(stream));
 }
 
+// Budget of one layer: the schedule is O(m) integer work, small enough to redo per call.
+static int32_t layer_budget(const pkv_config* cfg, int32_t layer) {
+  int32_t stack_buf[512];
+  int32_t* all = cfg->num_layers <= 512 ? stack_buf : new int32_t[cfg->num_layers];
+  budgets(cfg, all);
+  const int32_t k_layer = all[layer];
+  if (all != stack_buf) delete[] all;
+  return k_layer;
+}
+
 static int compress_layer_impl(const pkv_config* cfg, int32_t layer, pkv_tensor q_win, pkv_tensor k, pkv_tensor v,
                                const float* window_lse, const int32_t* seq_lens, int32_t batch, void* k_out,
                                void* v_out, int32_t* indices, float* scores_or_null, int64_t ld_scores,
@@ -568,15 +622,7 @@ static int compress_layer_impl(const pkv_config* cfg, int32_t layer, pkv_tensor 
     return PKV_ERR_INVALID_ARG;
   if (!k_out || !v_out || !indices) return PKV_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(k_out) % 16 || reinterpret_cast<uintptr_t>(v_out) % 16) return PKV_ERR_INVALID_ARG;
-  int32_t k_layer;
-  {
-    // the schedule is O(m) integer work; small enough to redo per call
-    int32_t stack_buf[512];
-    int32_t* all = cfg->num_layers <= 512 ? stack_buf : new int32_t[cfg->num_layers];
-    budgets(cfg, all);
-    k_layer = all[layer];
-    if (all != stack_buf) delete[] all;
-  }
+  const int32_t k_layer = layer_budget(cfg, layer);
   SeqTable table;
   int max_n;
   int64_t rows;
@@ -713,6 +759,103 @@ int pyramidkv_attention_recall(const pkv_config* cfg, const float* scores, int64
   rp.seq = table;
   rp.num_kv_heads = cfg->num_kv_heads;
   launch_pdl(attention_recall_kernel, dim3(cfg->num_kv_heads, batch), 256, 0, static_cast<cudaStream_t>(stream), rp);
+  return check_launch();
+}
+
+int pyramidkv_pages_needed(const pkv_config* cfg, int32_t k_layer, int32_t seq_len, int32_t page_size) {
+  if (!config_ok(cfg) || k_layer < 0 || seq_len < cfg->window + 1 || page_size < 1) return -PKV_ERR_INVALID_ARG;
+  return (kept_count(cfg, k_layer, seq_len) + page_size - 1) / page_size;
+}
+
+int pyramidkv_gather_paged(const pkv_config* cfg, pkv_tensor k, pkv_tensor v, const int32_t* indices,
+                           const int32_t* seq_lens, int32_t batch, int32_t k_layer, const int32_t* block_table,
+                           int32_t page_size, int32_t num_pages, void* k_pool, void* v_pool, void* workspace,
+                           size_t workspace_bytes, void* stream) {
+  if (!config_ok(cfg)) return PKV_ERR_INVALID_ARG;
+  if (int rc = config_supported(cfg)) return rc;
+  const int eb = cfg->dtype == PKV_DTYPE_FP32 ? 4 : 2;
+  if (!tensor_ok(k, cfg->head_dim, eb) || !tensor_ok(v, cfg->head_dim, eb) || !indices) return PKV_ERR_INVALID_ARG;
+  if (!paged_args_ok(block_table, page_size, num_pages, k_pool, v_pool)) return PKV_ERR_INVALID_ARG;
+  if (!workspace || reinterpret_cast<uintptr_t>(workspace) % kAlign || workspace_bytes < kAlign)
+    return PKV_ERR_WORKSPACE;
+  SeqTable table;
+  int max_n;
+  int64_t rows;
+  if (int rc = build_table(cfg, seq_lens, batch, k_layer, &table, &max_n, &rows)) return rc;
+  return run_gather_paged(cfg, k, v, indices, table, rows, block_table, page_size, num_pages, k_pool, v_pool,
+                          static_cast<uint32_t*>(workspace), static_cast<cudaStream_t>(stream));
+}
+
+int pyramidkv_compress_layer_paged(const pkv_config* cfg, int32_t layer, pkv_tensor q_win, pkv_tensor k,
+                                   pkv_tensor v, const float* window_lse_or_null, const int32_t* seq_lens,
+                                   int32_t batch, const int32_t* block_table, int32_t page_size, int32_t num_pages,
+                                   void* k_pool, void* v_pool, int32_t* indices, float* scores_or_null,
+                                   int64_t ld_scores, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!config_ok(cfg)) return PKV_ERR_INVALID_ARG;
+  if (int rc = config_supported(cfg)) return rc;
+  if (layer < 0 || layer >= cfg->num_layers) return PKV_ERR_INVALID_ARG;
+  const int eb = cfg->dtype == PKV_DTYPE_FP32 ? 4 : 2;
+  if (!tensor_ok(q_win, cfg->head_dim, eb) || !tensor_ok(k, cfg->head_dim, eb) || !tensor_ok(v, cfg->head_dim, eb))
+    return PKV_ERR_INVALID_ARG;
+  if (!indices || !paged_args_ok(block_table, page_size, num_pages, k_pool, v_pool)) return PKV_ERR_INVALID_ARG;
+  const int32_t k_layer = layer_budget(cfg, layer);
+  SeqTable table;
+  int max_n;
+  int64_t rows;
+  if (int rc = build_table(cfg, seq_lens, batch, k_layer, &table, &max_n, &rows)) return rc;
+  Workspace w;
+  if (int rc = workspace_check(cfg, batch, max_n, workspace, workspace_bytes, &w)) return rc;
+  float* scores = scores_or_null ? scores_or_null : w.scores;
+  const int64_t ld = scores_or_null ? ld_scores : w.ld_scores;
+  if (ld < max_n - cfg->window) return PKV_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  bool any_compress = false;
+  for (int b = 0; b < batch; ++b) any_compress |= table.count[b] < table.n[b];
+  if (any_compress || scores_or_null)
+    if (int rc = run_scores(cfg, q_win, k, table, batch, scores, ld, w, st, window_lse_or_null)) return rc;
+  if (int rc = run_select(cfg, scores, ld, table, batch, max_n, indices, w, st)) return rc;
+  return run_gather_paged(cfg, k, v, indices, table, rows, block_table, page_size, num_pages, k_pool, v_pool,
+                          w.status, st);
+}
+
+int pyramidkv_decode_attention_paged(const pkv_config* cfg, const void* q, const void* k_pool, const void* v_pool,
+                                     const int32_t* block_table, int32_t page_size, int32_t num_pages,
+                                     const int32_t* seq_lens, int32_t batch, int32_t k_layer, float* out,
+                                     void* workspace, size_t workspace_bytes, void* stream) {
+  if (!config_ok(cfg)) return PKV_ERR_INVALID_ARG;
+  if (int rc = config_supported(cfg)) return rc;
+  if (!q || !out || reinterpret_cast<uintptr_t>(q) % 16) return PKV_ERR_INVALID_ARG;
+  if (!paged_args_ok(block_table, page_size, num_pages, k_pool, v_pool)) return PKV_ERR_INVALID_ARG;
+  if (!workspace || reinterpret_cast<uintptr_t>(workspace) % kAlign || workspace_bytes < kAlign)
+    return PKV_ERR_WORKSPACE;
+  SeqTable table;
+  int max_n;
+  int64_t rows;
+  if (int rc = build_table(cfg, seq_lens, batch, k_layer, &table, &max_n, &rows)) return rc;
+  DecodeParams dp{};
+  dp.q = q;
+  dp.k_cache = k_pool;
+  dp.v_cache = v_pool;
+  dp.out = out;
+  dp.seq = table;
+  fill_page_table(cfg, table, block_table, page_size, num_pages, &dp.pt);
+  dp.status = static_cast<uint32_t*>(workspace);
+  dp.num_kv_heads = cfg->num_kv_heads;
+  dp.group = cfg->num_q_heads / cfg->num_kv_heads;
+  dp.scale_log2 = static_cast<float>(1.4426950408889634 / std::sqrt(static_cast<double>(cfg->head_dim)));
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const dim3 grid(cfg->num_q_heads, batch);
+  const bool wide = cfg->head_dim == 128;
+  if (cfg->dtype == PKV_DTYPE_FP32) {
+    if (wide) launch_pdl(decode_attention_kernel<float, 128, true>, grid, kDecThreads, 0, st, dp);
+    else launch_pdl(decode_attention_kernel<float, 64, true>, grid, kDecThreads, 0, st, dp);
+  } else if (cfg->dtype == PKV_DTYPE_FP16) {
+    if (wide) launch_pdl(decode_attention_kernel<__half, 128, true>, grid, kDecThreads, 0, st, dp);
+    else launch_pdl(decode_attention_kernel<__half, 64, true>, grid, kDecThreads, 0, st, dp);
+  } else {
+    if (wide) launch_pdl(decode_attention_kernel<__nv_bfloat16, 128, true>, grid, kDecThreads, 0, st, dp);
+    else launch_pdl(decode_attention_kernel<__nv_bfloat16, 64, true>, grid, kDecThreads, 0, st, dp);
+  }
   return check_launch();
 }
 

@@ -31,6 +31,7 @@ struct TensorView {
 enum : uint32_t {
   kStatusSelectMismatch = 1u << 0,   // selection emitted a count other than k
   kStatusWaitExpired = 1u << 1,      // a bounded wait ran out
+  kStatusBadPage = 1u << 2,          // a block-table entry named a page outside the pool (row skipped)
 };
 
 // Programmatic dependent launch: every kernel of the library is launched so that it may start while

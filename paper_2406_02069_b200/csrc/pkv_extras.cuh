@@ -3,6 +3,7 @@
 #pragma once
 
 #include "pkv_common.cuh"
+#include "pkv_paged.cuh"
 
 namespace pkv {
 
@@ -10,8 +11,10 @@ constexpr int kDecThreads = 128;
 
 struct DecodeParams {
   const void* q;            // [batch][H_q][d], config dtype, contiguous
-  const void* k_cache;      // packed rows [sum_b H_kv * c_b][d]
+  const void* k_cache;      // packed rows [sum_b H_kv * c_b][d]; with PAGED the pool [num_pages][page_size][d]
   const void* v_cache;
+  PageTable pt;             // PAGED only
+  uint32_t* status;         // PAGED only: where a bad table entry is recorded
   float* out;               // [batch][H_q][d] fp32
   SeqTable seq;
   int32_t num_kv_heads, group;
@@ -21,7 +24,8 @@ struct DecodeParams {
 // grid (H_q, batch), block kDecThreads.  One new token's query of one head attends to every kept row of
 // its KV head: out = softmax(q K_s^T / sqrt(d)) V_s.  Each 16-lane half-warp takes one cached row at a
 // time (16 bytes per lane); running (max, sum, weighted V) are kept per half-warp and merged at the end.
-template <typename T, int D>
+// PAGED: the rows are found through the layer's block table instead of at fixed offsets.
+template <typename T, int D, bool PAGED = false>
 __global__ void __launch_bounds__(kDecThreads) decode_attention_kernel(const DecodeParams p) {
   constexpr int kPer = D / 16;                  // elements per lane
   __shared__ float s_m[kDecThreads / 16], s_z[kDecThreads / 16];
@@ -33,6 +37,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_attention_kernel(const Dec
   const int count = p.seq.count[b];
   const int64_t row0 = p.seq.row_off[b] + static_cast<int64_t>(h) * count;
   const int sub = threadIdx.x & 15, team = threadIdx.x >> 4, teams = kDecThreads / 16;
+  const uint32_t half_mask = 0xffffu << (threadIdx.x & 16);   // the two half-warps leave the row loop separately
 
   float qv[kPer], acc[kPer];
   const T* qrow = static_cast<const T*>(p.q) + (static_cast<int64_t>(b) * gridDim.x + hq) * D + sub * kPer;
@@ -40,13 +45,21 @@ __global__ void __launch_bounds__(kDecThreads) decode_attention_kernel(const Dec
   for (int c = 0; c < kPer; ++c) { qv[c] = to_float(qrow[c]); acc[c] = 0.f; }
   float m = -INFINITY, z = 0.f;
   for (int r = team; r < count; r += teams) {
-    const T* kr = static_cast<const T*>(p.k_cache) + (row0 + r) * D + sub * kPer;
-    const T* vr = static_cast<const T*>(p.v_cache) + (row0 + r) * D + sub * kPer;
+    int64_t at = row0 + r;
+    if (PAGED) {
+      at = paged_row(p.pt, b, h, r);
+      if (at < 0) {                                           // uniform over the half-warp
+        if (sub == 0) atomicOr(p.status, kStatusBadPage);
+        continue;
+      }
+    }
+    const T* kr = static_cast<const T*>(p.k_cache) + at * D + sub * kPer;
+    const T* vr = static_cast<const T*>(p.v_cache) + at * D + sub * kPer;
     float dot = 0.f;
 #pragma unroll
     for (int c = 0; c < kPer; ++c) dot = fmaf(qv[c], to_float(kr[c]), dot);
 #pragma unroll
-    for (int o = 8; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o, 16);
+    for (int o = 8; o > 0; o >>= 1) dot += __shfl_xor_sync(half_mask, dot, o, 16);
     const float x = dot * p.scale_log2;
     const float mn = fmaxf(m, x);
     const float corr = exp2f(m - mn), w = exp2f(x - mn);
