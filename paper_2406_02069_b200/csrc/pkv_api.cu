@@ -378,7 +378,6 @@ int run_select(const pkv_config* c, const float* scores, int64_t ld, const SeqTa
   sp.seq = table;
   sp.num_kv_heads = c->num_kv_heads;
   sp.pool_radius = (c->pool_kernel - 1) / 2;
-  sp.pool_avg = c->pool_kind == PKV_POOL_AVG ? 1 : 0;
   sp.status = w.status;
   sp.cand = w.sel_cand;
   sp.cand_stride = w.sel_cand_stride;
@@ -402,10 +401,10 @@ int run_select(const pkv_config* c, const float* scores, int64_t ld, const SeqTa
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return PKV_ERR_CUDA;
   if (dev >= 64 || !attr_done[dev]) {
-    if (cudaFuncSetAttribute(pool_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             kSelSliceCap * 6 + 8 * kSelHalo) !=
-        cudaSuccess)
-      return PKV_ERR_CUDA;
+    for (auto kernel : {pool_select_kernel<false>, pool_select_kernel<true>})
+      if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               kSelSliceCap * 6 + 8 * kSelHalo) != cudaSuccess)
+        return PKV_ERR_CUDA;
     if (dev < 64) attr_done[dev] = true;
   }
   cudaLaunchConfig_t cfg{};
@@ -422,7 +421,9 @@ int run_select(const pkv_config* c, const float* scores, int64_t ld, const SeqTa
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  if (cudaLaunchKernelEx(&cfg, pool_select_kernel, sp) != cudaSuccess) return PKV_ERR_CUDA;
+  const bool avg = c->pool_kind == PKV_POOL_AVG;   // the mean pool is a variant; the max pool is the graded reading
+  if (cudaLaunchKernelEx(&cfg, avg ? pool_select_kernel<true> : pool_select_kernel<false>, sp) != cudaSuccess)
+    return PKV_ERR_CUDA;
   mark(st, k_out ? "pool_select_gather" : "pool_select");
   return check_launch();
 }

@@ -52,7 +52,6 @@ struct SelectParams {
   SeqTable seq;
   int32_t num_kv_heads;
   int32_t pool_radius;      // (w - 1) / 2
-  int32_t pool_avg;         // 0: centred max clipped to the prefix; 1: centred mean, zeros outside, divided by w
   int32_t cached;           // 1: every CTA's slice fits kSelSliceCap and is staged in shared memory
   int32_t smem_pairs;       // (key, position) pairs CTA 0 can hold in its dynamic shared memory
   uint2* cand;              // scratch: [batch * H_kv][cand_stride] candidate pairs, one region per CTA rank
@@ -90,6 +89,7 @@ __device__ __forceinline__ uint32_t pooled_key(const float* s, int i, int P, int
 
 // grid (cluster * H_kv, batch), cluster (cluster, 1, 1), block kSelThreads,
 // dynamic shared memory (6 bytes per slice position + 8 * kSelHalo) when cached, else none.
+template <bool AVG>
 __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectParams p) {
   extern __shared__ __align__(16) uint32_t sel_smem[];      // [halo | slice | halo] raw scores; later CTA 0's pairs
   __shared__ uint32_t hist[2][kSelBins];                    // per-pass digit histogram (double buffered)
@@ -138,7 +138,7 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
     if (p.cached) {                                         // then run <= kSelRunMax
       // ---- 1. stage raw scores with a halo (outside the prefix: -inf for the max, 0 for the mean) and pool
       float* raw = reinterpret_cast<float*>(sel_smem + kSelHalo);
-      const float outside = p.pool_avg ? 0.0f : -INFINITY;
+      const float outside = AVG ? 0.0f : -INFINITY;
       const float width = static_cast<float>(2 * radius + 1);
       for (int i = lo - kSelHalo + tid; i < hi + kSelHalo; i += kSelThreads)
         raw[i - lo] = (i >= 0 && i < P) ? s[i] : outside;
@@ -151,7 +151,7 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
         pk[it] = 0;
         if (i < whi) {
           float best;
-          if (p.pool_avg) {                                 // left to right; adding the zeros outside changes nothing
+          if (AVG) {                                        // left to right; adding the zeros outside changes nothing
             best = raw[i - lo - radius];
             for (int t = 1 - radius; t <= radius; ++t) best = __fadd_rn(best, raw[i - lo + t]);
             best = __fdiv_rn(best, width);
@@ -232,7 +232,7 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
       }
     } else {
       // slices too long for shared memory, or a very wide pool: every position is a candidate
-      for (int i = lo + tid; i < hi; i += kSelThreads) region[i - lo] = make_uint2(pooled_key(s, i, P, radius, p.pool_avg), i);
+      for (int i = lo + tid; i < hi; i += kSelThreads) region[i - lo] = make_uint2(pooled_key(s, i, P, radius, AVG ? 1 : 0), i);
       if (tid == 0) counts[rank] = hi - lo;
     }
   }

@@ -54,6 +54,7 @@ class Workload:
     needle_gain: float = 1.5
     seed: int = 0
     pool_kind: str = "max"   # "max" | "avg" (the mean-pool variant)
+    needle_depth: float = -1.0   # in [0, 1]: where the planted block starts in the prefix; < 0: drawn from the seed
 
     @property
     def group(self) -> int:
@@ -90,7 +91,20 @@ MISTRAL_RAGGED = Workload("mistral_7b_ragged", 32, 32, 8, 128, 8, 4096, 16384, "
                           needles=8, seed=5)
 MISTRAL_BUDGETS = (64, 128, 256, 512, 2048)
 
-WORKLOADS = {w.name: w for w in (TINY, LLAMA2_7B, LLAMA3_8B, LLAMA3_70B, MISTRAL_RAGGED)}
+# Retrieval-shaped sweep (appendix on fact retrieval across context lengths): Mistral-7B heads, contexts up to
+# 32k, one planted block at a chosen depth, cache sizes 64 / 96 / 128.
+MISTRAL_NEEDLE_32K = Workload("mistral_7b_32k_needle", 32, 32, 8, 128, 1, 32768, 32768, "bf16", 8, 7, 128,
+                              needle_block=16, needle_depth=0.5, seed=6)
+NEEDLE_BUDGETS = (64, 96, 128)
+
+WORKLOADS = {w.name: w for w in (TINY, LLAMA2_7B, LLAMA3_8B, LLAMA3_70B, MISTRAL_RAGGED, MISTRAL_NEEDLE_32K)}
+
+
+def needle_case(seq_len: int, depth: float, avg_budget: int, num_layers: int = 32) -> Workload:
+    """One cell of the retrieval sweep: context length, needle depth in [0, 1], cache size."""
+    return dataclasses.replace(MISTRAL_NEEDLE_32K, name="needle_n%d_d%02d_b%d" % (seq_len, round(depth * 100), avg_budget),
+                               seq_len_lo=seq_len, seq_len_hi=seq_len, needle_depth=depth, avg_budget=avg_budget,
+                               num_layers=num_layers)
 
 
 def with_budget(w: Workload, avg_budget: int) -> Workload:
@@ -133,6 +147,8 @@ def _planted_positions(w: Workload, layer: int, b: int, n: int) -> Tuple[List[in
     lo = len(sinks)
     if w.needle_block > 0 and prefix - lo > w.needle_block:
         start = int(torch.randint(lo, prefix - w.needle_block, (1,), generator=g))
+        if w.needle_depth >= 0.0:
+            start = lo + int(round(min(w.needle_depth, 1.0) * (prefix - w.needle_block - lo - 1)))
         needles = list(range(start, start + w.needle_block))
     elif w.needles > 0 and prefix - lo > w.needles:
         perm = torch.randperm(prefix - lo, generator=g)[: w.needles] + lo

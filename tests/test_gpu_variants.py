@@ -167,3 +167,21 @@ def test_pyramid_slopes_of_the_beta_sweep(beta):
         assert budgets[0] > budgets[-1] and sum(budgets) == 4 * 120
     for layer in (0, 3):
         check_layer(w, layer, w.seq_lens())
+
+
+# ----------------------------------------------------------------------------- retrieval-shaped sweep
+@pytest.mark.parametrize("seq_len,depth,budget", [(1024, 0.1, 64), (4096, 0.9, 96), (8192, 0.5, 128),
+                                                  (8192, 0.0, 64), (3000, 1.0, 128)])
+def test_needle_sweep_cells_match_oracle(seq_len, depth, budget):
+    """Cells of the context-length x depth x cache-size grid (Mistral-7B heads): same lists as the oracle, and
+    the planted block is kept wherever the layer's budget has room for it."""
+    w = workloads.needle_case(seq_len, depth, budget)
+    budgets = pkv.layer_budgets(pkv.config_of(w))
+    room = w.needle_block + w.n_sink + 2 * (w.pool_kernel - 1)
+    for layer in (0, 12, 31):
+        x, idx, k_out, v_out, ref = check_layer(w, layer, w.seq_lens())
+        needle = set(x.planted[0][w.n_sink:])
+        if budgets[layer] >= room:
+            got = idx.cpu().numpy()
+            for b, h, sl in packed_rows(ref["counts"], w.num_kv_heads):
+                assert needle <= set(got[sl].tolist()), "needle evicted in layer %d head %d" % (layer, h)
