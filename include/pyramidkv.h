@@ -361,6 +361,47 @@ int pyramidkv_decode_attention_paged(const pkv_config* cfg, const void* q, const
                                      void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Sequence-sharded compression, for contexts whose K does not fit one GPU.  The keys (and values) of a
+ * sequence are split into contiguous position ranges, one per GPU; every GPU holds the window queries.
+ * The window keys (the last alpha positions) all lie on the shard that ends the sequence, which must also
+ * hold at least one prefix key.  A layer then takes these steps (Section 4.2.2 on each shard, with the one
+ * exchange Eq. 2's softmax needs); the two exchanges are the caller's (any all-gather / all-reduce):
+ *   1. pyramidkv_shard_window_lse   every shard: partial normalisers of the window rows over its keys
+ *      -- all-gather the parts --
+ *   2. pyramidkv_merge_lse          the rows' full normalisers
+ *   3. pyramidkv_shard_scores       every shard: Eq. 3 scores of its own prefix keys (one K sweep)
+ *      -- all-gather the score ranges into the sequence's score row --
+ *   4. pyramidkv_select_topk        every shard runs the same selection on the full score row
+ *   5. pyramidkv_shard_gather       every shard copies the kept rows it owns into a zero-filled packed
+ *      buffer  -- all-reduce (integer sum, each row has one owner) if every GPU wants the whole cache --
+ * The result equals pyramidkv_compress_layer on the unsharded tensors (scores to rounding, rows bit for bit).
+ *
+ *   k_shard, v_shard  this GPU's keys/values: token t of the view is position shard_begin[b] + t
+ *   shard_keys   host [batch]: keys of sequence b in this shard (>= 1)
+ *   window_keys  host [batch]: alpha if this shard ends sequence b (then shard_keys[b] >= alpha + 1), else 0
+ *   lse_out, parts, window_lse  device floats [batch][H_q][alpha]: natural log of a sum of exponentials
+ * Errors: as pyramidkv_score_window; INVALID_ARG for a window_keys entry other than 0 or alpha.
+ */
+int pyramidkv_shard_window_lse(const pkv_config* cfg, pkv_tensor q_win, pkv_tensor k_shard,
+                               const int32_t* shard_keys, const int32_t* window_keys, int32_t batch,
+                               float* lse_out, void* workspace, size_t workspace_bytes, void* stream);
+/* parts: device [num_shards][count] floats; out: device [count];  out = log(sum over shards of exp(part)). */
+int pyramidkv_merge_lse(const float* parts, int32_t num_shards, int64_t count, float* out, void* stream);
+/* scores: device [batch][H_kv][ld_scores], the first shard_keys[b] - window_keys[b] of each row are written. */
+int pyramidkv_shard_scores(const pkv_config* cfg, pkv_tensor q_win, pkv_tensor k_shard, const float* window_lse,
+                           const int32_t* shard_keys, const int32_t* window_keys, int32_t batch,
+                           float* scores, int64_t ld_scores,
+                           void* workspace, size_t workspace_bytes, void* stream);
+/*
+ * indices, k_out, v_out: the packed layout of the WHOLE layer (seq_lens are the full lengths); only the
+ * rows whose position lies in [shard_begin[b], shard_begin[b] + shard_keys[b]) are written.
+ */
+int pyramidkv_shard_gather(const pkv_config* cfg, pkv_tensor k_shard, pkv_tensor v_shard, const int32_t* indices,
+                           const int32_t* seq_lens, int32_t batch, int32_t k_layer,
+                           const int32_t* shard_begin, const int32_t* shard_keys,
+                           void* k_out, void* v_out, void* stream);
+
+/*
  * Synchronises `stream` and reads the workspace status word.  For tests and
  * debugging.  Returns PKV_OK, PKV_ERR_DEVICE_STATUS (a kernel gave up on a
  * bounded wait or saw an impossible state; *detail_or_null receives the word),

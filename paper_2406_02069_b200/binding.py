@@ -30,7 +30,8 @@ EXPORTS = ("pyramidkv_strerror", "pyramidkv_layer_budgets", "pyramidkv_kept_coun
            "pyramidkv_check_status", "pyramidkv_score_window_static", "pyramidkv_score_window_lse",
            "pyramidkv_compress_layer_lse", "pyramidkv_profile_layer_lse", "pyramidkv_decode_attention",
            "pyramidkv_attention_recall", "pyramidkv_pages_needed", "pyramidkv_gather_paged",
-           "pyramidkv_compress_layer_paged", "pyramidkv_decode_attention_paged")
+           "pyramidkv_compress_layer_paged", "pyramidkv_decode_attention_paged", "pyramidkv_shard_window_lse",
+           "pyramidkv_merge_lse", "pyramidkv_shard_scores", "pyramidkv_shard_gather")
 PKV_MAX_STAGES = 8
 
 
@@ -85,6 +86,10 @@ def _load() -> ctypes.CDLL:
     lib.pyramidkv_compress_layer_paged.argtypes = [CFG, I32, PkvTensor, PkvTensor, PkvTensor, P, P, I32, P, I32, I32,
                                                    P, P, P, P, I64, P, SZ, P]
     lib.pyramidkv_decode_attention_paged.argtypes = [CFG, P, P, P, P, I32, I32, P, I32, I32, P, P, SZ, P]
+    lib.pyramidkv_shard_window_lse.argtypes = [CFG, PkvTensor, PkvTensor, P, P, I32, P, P, SZ, P]
+    lib.pyramidkv_merge_lse.argtypes = [P, I32, I64, P, P]
+    lib.pyramidkv_shard_scores.argtypes = [CFG, PkvTensor, PkvTensor, P, P, P, I32, P, I64, P, SZ, P]
+    lib.pyramidkv_shard_gather.argtypes = [CFG, PkvTensor, PkvTensor, P, P, I32, I32, P, P, P, P, P]
     lib.pyramidkv_check_status.argtypes = [P, P, P]
     for name in EXPORTS:
         if name not in ("pyramidkv_strerror", "pyramidkv_workspace_bytes"):
@@ -348,3 +353,45 @@ def decode_attention_paged(cfg: PkvConfig, q: torch.Tensor, block_table: torch.T
                                                  lens, batch, int(k_layer), out.data_ptr(), workspace.data_ptr(),
                                                  workspace.numel(), _stream(stream)),
            "pyramidkv_decode_attention_paged")
+
+
+# ----------------------------------------------------------------------------- sequence-sharded steps
+def shard_window_lse(cfg: PkvConfig, q_win: torch.Tensor, k_shard: torch.Tensor, shard_keys: Sequence[int],
+                     window_keys: Sequence[int], lse_out: torch.Tensor, workspace: torch.Tensor, stream=None) -> None:
+    """Partial normalisers (natural log) of the window rows over this shard's keys -> lse_out [batch][H_q][alpha]."""
+    keys, batch = _lens(shard_keys)
+    wkeys, _ = _lens(window_keys)
+    _check(_lib.pyramidkv_shard_window_lse(ctypes.byref(cfg), _tensor(q_win), _tensor(k_shard), keys, wkeys, batch,
+                                           _lse_ptr(lse_out), workspace.data_ptr(), workspace.numel(),
+                                           _stream(stream)), "pyramidkv_shard_window_lse")
+
+
+def merge_lse(parts: torch.Tensor, out: torch.Tensor, stream=None) -> None:
+    """parts [num_shards][...] float32 -> out [...] = log(sum over shards of exp(part))."""
+    if parts.dtype != torch.float32 or out.dtype != torch.float32 or not (parts.is_contiguous() and out.is_contiguous()):
+        raise ValueError("merge_lse takes contiguous float32 tensors")
+    if parts.numel() != parts.shape[0] * out.numel():
+        raise ValueError("parts must be [num_shards] + out.shape")
+    _check(_lib.pyramidkv_merge_lse(parts.data_ptr(), int(parts.shape[0]), out.numel(), out.data_ptr(),
+                                    _stream(stream)), "pyramidkv_merge_lse")
+
+
+def shard_scores(cfg: PkvConfig, q_win: torch.Tensor, k_shard: torch.Tensor, window_lse: torch.Tensor,
+                 shard_keys: Sequence[int], window_keys: Sequence[int], scores: torch.Tensor,
+                 workspace: torch.Tensor, stream=None) -> None:
+    keys, batch = _lens(shard_keys)
+    wkeys, _ = _lens(window_keys)
+    _check(_lib.pyramidkv_shard_scores(ctypes.byref(cfg), _tensor(q_win), _tensor(k_shard), _lse_ptr(window_lse), keys,
+                                       wkeys, batch, scores.data_ptr(), scores.stride(1), workspace.data_ptr(),
+                                       workspace.numel(), _stream(stream)), "pyramidkv_shard_scores")
+
+
+def shard_gather(cfg: PkvConfig, k_shard: torch.Tensor, v_shard: torch.Tensor, indices: torch.Tensor,
+                 seq_lens: Sequence[int], k_layer: int, shard_begin: Sequence[int], shard_keys: Sequence[int],
+                 k_out: torch.Tensor, v_out: torch.Tensor, stream=None) -> None:
+    lens, batch = _lens(seq_lens)
+    begin, _ = _lens(shard_begin)
+    keys, _ = _lens(shard_keys)
+    _check(_lib.pyramidkv_shard_gather(ctypes.byref(cfg), _tensor(k_shard), _tensor(v_shard), indices.data_ptr(), lens,
+                                       batch, int(k_layer), begin, keys, k_out.data_ptr(), v_out.data_ptr(),
+                                       _stream(stream)), "pyramidkv_shard_gather")

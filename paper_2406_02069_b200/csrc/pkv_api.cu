@@ -14,6 +14,7 @@
 #include "pkv_score_generic.cuh"
 #include "pkv_score_tc.cuh"
 #include "pkv_select.cuh"
+#include "pkv_shard.cuh"
 
 namespace pkv {
 namespace {
@@ -118,6 +119,7 @@ int build_table(const pkv_config* c, const int32_t* seq_lens, int batch, int k_l
     const int n = seq_lens[b];
     if (n < c->window + 1) return PKV_ERR_INVALID_ARG;
     t->n[b] = n;
+    t->prefix[b] = n - c->window;
     t->count[b] = kept_count(c, k_layer, n);
     t->row_off[b] = rows;
     rows += static_cast<int64_t>(c->num_kv_heads) * t->count[b];
@@ -178,7 +180,7 @@ int launch_scores_generic(ScoreParams& sp, int batch, cudaStream_t st) {
     sp.seq.stat_off[b] = stat_tiles;
     sp.seq.score_off[b] = score_tiles;
     stat_tiles += (sp.seq.n[b] + kGenChunk - 1) / kGenChunk;
-    score_tiles += (sp.seq.n[b] - sp.seq.alpha + kGenScoreKeys - 1) / kGenScoreKeys;
+    score_tiles += (sp.seq.prefix[b] + kGenScoreKeys - 1) / kGenScoreKeys;
   }
   sp.seq.stat_off[batch] = stat_tiles;
   sp.seq.score_off[batch] = score_tiles;
@@ -190,6 +192,7 @@ int launch_scores_generic(ScoreParams& sp, int batch, cudaStream_t st) {
                std::log2(static_cast<float>(sp.group)));
     mark(st, "combine_stats");
   }
+  if (sp.stats_only) return check_launch();
   launch_pdl(scores_generic_kernel<T, D>, dim3(score_tiles, sp.num_kv_heads), kGenScoreKeys, 0, st, sp);
   mark(st, "scores_generic");
   return check_launch();
@@ -288,7 +291,7 @@ int launch_scores_tc(const pkv_config* c, const pkv_tensor& q, const pkv_tensor&
   auto items_for = [&](int ct, int tile_keys, bool prefix) {
     long long items = 0;
     for (int b = 0; b < batch; ++b) {
-      const int keys = prefix ? sp.seq.n[b] - sp.seq.alpha : sp.seq.n[b];
+      const int keys = prefix ? sp.seq.prefix[b] : sp.seq.n[b];
       const int tiles = (keys + tile_keys - 1) / tile_keys;
       items += (tiles + ct - 1) / ct;
     }
@@ -310,7 +313,7 @@ int launch_scores_tc(const pkv_config* c, const pkv_tensor& q, const pkv_tensor&
     tp.seq.stat_off[b] = stat_items;
     tp.seq.score_off[b] = score_items;
     stat_items += ((sp.seq.n[b] + kTcTileKeysA - 1) / kTcTileKeysA + tp.chunk_tiles_a - 1) / tp.chunk_tiles_a;
-    score_items += ((sp.seq.n[b] - sp.seq.alpha + kTcTileKeysB - 1) / kTcTileKeysB + tp.chunk_tiles_b - 1) /
+    score_items += ((sp.seq.prefix[b] + kTcTileKeysB - 1) / kTcTileKeysB + tp.chunk_tiles_b - 1) /
                    tp.chunk_tiles_b;
   }
   tp.seq.stat_off[batch] = stat_items;
@@ -327,6 +330,7 @@ int launch_scores_tc(const pkv_config* c, const pkv_tensor& q, const pkv_tensor&
                std::log2(static_cast<float>(sp.group)));
     mark(st, "combine_stats");
   }
+  if (sp.stats_only) return check_launch();
   launch_pdl(score_tc_kernel<D, 1>, grid_b, kTcThreads, TcSmem<D>::kTotal, st, q_map, k_map_b, tp);
   mark(st, "scores_tc");
   return check_launch();
@@ -334,8 +338,10 @@ int launch_scores_tc(const pkv_config* c, const pkv_tensor& q, const pkv_tensor&
 
 // window_lse: null, or the caller's natural-log row normalisers [batch][H_q][alpha] (then sweep A is skipped).
 int run_scores(const pkv_config* c, const pkv_tensor& q, const pkv_tensor& k, const SeqTable& table, int batch,
-               float* scores, int64_t ld, const Workspace& w, cudaStream_t st, const float* window_lse = nullptr) {
+               float* scores, int64_t ld, const Workspace& w, cudaStream_t st, const float* window_lse = nullptr,
+               bool stats_only = false) {
   ScoreParams sp{};
+  sp.stats_only = stats_only ? 1 : 0;
   sp.q = view(q);
   sp.k = view(k);
   sp.seq = table;
@@ -492,6 +498,26 @@ int run_gather_paged(const pkv_config* c, const pkv_tensor& k, const pkv_tensor&
 bool paged_args_ok(const int32_t* block_table, int page_size, int num_pages, const void* k_pool, const void* v_pool) {
   if (!block_table || !k_pool || !v_pool || page_size < 1 || num_pages < 1) return false;
   return reinterpret_cast<uintptr_t>(k_pool) % 16 == 0 && reinterpret_cast<uintptr_t>(v_pool) % 16 == 0;
+}
+
+// Table of a call on one shard of each sequence: n = keys held here, prefix = those that are scored.
+int build_shard_table(const pkv_config* c, const int32_t* shard_keys, const int32_t* window_keys, int batch,
+                      SeqTable* t, int* max_n) {
+  if (!shard_keys || !window_keys || batch < 1) return PKV_ERR_INVALID_ARG;
+  if (batch > PKV_MAX_BATCH) return PKV_ERR_UNSUPPORTED;
+  std::memset(t, 0, sizeof *t);
+  t->batch = batch;
+  t->alpha = c->window;
+  int mx = 0;
+  for (int b = 0; b < batch; ++b) {
+    if (window_keys[b] != 0 && window_keys[b] != c->window) return PKV_ERR_INVALID_ARG;
+    if (shard_keys[b] < window_keys[b] + 1) return PKV_ERR_INVALID_ARG;
+    t->n[b] = shard_keys[b];
+    t->prefix[b] = shard_keys[b] - window_keys[b];
+    if (shard_keys[b] > mx) mx = shard_keys[b];
+  }
+  *max_n = mx;
+  return PKV_OK;
 }
 
 int workspace_check(const pkv_config* c, int batch, int max_n, void* ws, size_t ws_bytes, Workspace* out) {
@@ -857,6 +883,91 @@ int pyramidkv_decode_attention_paged(const pkv_config* cfg, const void* q, const
     if (wide) launch_pdl(decode_attention_kernel<__nv_bfloat16, 128, true>, grid, kDecThreads, 0, st, dp);
     else launch_pdl(decode_attention_kernel<__nv_bfloat16, 64, true>, grid, kDecThreads, 0, st, dp);
   }
+  return check_launch();
+}
+
+int pyramidkv_shard_window_lse(const pkv_config* cfg, pkv_tensor q_win, pkv_tensor k_shard,
+                               const int32_t* shard_keys, const int32_t* window_keys, int32_t batch, float* lse_out,
+                               void* workspace, size_t workspace_bytes, void* stream) {
+  if (!config_ok(cfg)) return PKV_ERR_INVALID_ARG;
+  if (int rc = config_supported(cfg)) return rc;
+  const int eb = cfg->dtype == PKV_DTYPE_FP32 ? 4 : 2;
+  if (!tensor_ok(q_win, cfg->head_dim, eb) || !tensor_ok(k_shard, cfg->head_dim, eb) || !lse_out)
+    return PKV_ERR_INVALID_ARG;
+  SeqTable table;
+  int max_n;
+  if (int rc = build_shard_table(cfg, shard_keys, window_keys, batch, &table, &max_n)) return rc;
+  Workspace w;
+  if (int rc = workspace_check(cfg, batch, max_n + cfg->window, workspace, workspace_bytes, &w)) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (int rc = run_scores(cfg, q_win, k_shard, table, batch, w.scores, w.ld_scores, w, st, nullptr, true)) return rc;
+  const int64_t count = static_cast<int64_t>(batch) * cfg->num_q_heads * cfg->window;
+  const float log2_group = std::log2(static_cast<float>(cfg->num_q_heads / cfg->num_kv_heads));
+  launch_pdl(export_lse_kernel, static_cast<unsigned>((count + kShardThreads - 1) / kShardThreads), kShardThreads, 0,
+             st, static_cast<const float*>(w.lse2), log2_group, lse_out, count);
+  return check_launch();
+}
+
+int pyramidkv_merge_lse(const float* parts, int32_t num_shards, int64_t count, float* out, void* stream) {
+  if (!parts || !out || num_shards < 1 || count < 1) return PKV_ERR_INVALID_ARG;
+  launch_pdl(merge_lse_kernel, static_cast<unsigned>((count + kShardThreads - 1) / kShardThreads), kShardThreads, 0,
+             static_cast<cudaStream_t>(stream), parts, static_cast<int>(num_shards), count, out);
+  return check_launch();
+}
+
+int pyramidkv_shard_scores(const pkv_config* cfg, pkv_tensor q_win, pkv_tensor k_shard, const float* window_lse,
+                           const int32_t* shard_keys, const int32_t* window_keys, int32_t batch, float* scores,
+                           int64_t ld_scores, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!config_ok(cfg)) return PKV_ERR_INVALID_ARG;
+  if (int rc = config_supported(cfg)) return rc;
+  const int eb = cfg->dtype == PKV_DTYPE_FP32 ? 4 : 2;
+  if (!tensor_ok(q_win, cfg->head_dim, eb) || !tensor_ok(k_shard, cfg->head_dim, eb) || !window_lse || !scores)
+    return PKV_ERR_INVALID_ARG;
+  SeqTable table;
+  int max_n;
+  if (int rc = build_shard_table(cfg, shard_keys, window_keys, batch, &table, &max_n)) return rc;
+  for (int b = 0; b < batch; ++b)
+    if (ld_scores < table.prefix[b]) return PKV_ERR_INVALID_ARG;
+  Workspace w;
+  if (int rc = workspace_check(cfg, batch, max_n + cfg->window, workspace, workspace_bytes, &w)) return rc;
+  return run_scores(cfg, q_win, k_shard, table, batch, scores, ld_scores, w, static_cast<cudaStream_t>(stream),
+                    window_lse);
+}
+
+int pyramidkv_shard_gather(const pkv_config* cfg, pkv_tensor k_shard, pkv_tensor v_shard, const int32_t* indices,
+                           const int32_t* seq_lens, int32_t batch, int32_t k_layer, const int32_t* shard_begin,
+                           const int32_t* shard_keys, void* k_out, void* v_out, void* stream) {
+  if (!config_ok(cfg)) return PKV_ERR_INVALID_ARG;
+  if (int rc = config_supported(cfg)) return rc;
+  const int eb = cfg->dtype == PKV_DTYPE_FP32 ? 4 : 2;
+  if (!tensor_ok(k_shard, cfg->head_dim, eb) || !tensor_ok(v_shard, cfg->head_dim, eb)) return PKV_ERR_INVALID_ARG;
+  if (!indices || !k_out || !v_out || !shard_begin || !shard_keys) return PKV_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(k_out) % 16 || reinterpret_cast<uintptr_t>(v_out) % 16) return PKV_ERR_INVALID_ARG;
+  SeqTable table;
+  int max_n;
+  int64_t rows;
+  if (int rc = build_table(cfg, seq_lens, batch, k_layer, &table, &max_n, &rows)) return rc;
+  GatherShardParams gp{};
+  gp.k = view(k_shard);
+  gp.v = view(v_shard);
+  gp.indices = indices;
+  gp.k_out = k_out;
+  gp.v_out = v_out;
+  gp.seq = table;
+  for (int b = 0; b < batch; ++b) {
+    if (shard_begin[b] < 0 || shard_keys[b] < 0 || shard_begin[b] + shard_keys[b] > seq_lens[b])
+      return PKV_ERR_INVALID_ARG;
+    gp.begin[b] = shard_begin[b];
+    gp.keys[b] = shard_keys[b];
+  }
+  gp.num_kv_heads = cfg->num_kv_heads;
+  gp.elem_bytes = eb;
+  gp.pieces = cfg->head_dim * eb / 16;
+  gp.total_rows = rows;
+  const int64_t threads = rows * gp.pieces;
+  if (threads == 0) return PKV_OK;
+  launch_pdl(gather_shard_kernel, static_cast<unsigned>((threads + kShardThreads - 1) / kShardThreads), kShardThreads,
+             0, static_cast<cudaStream_t>(stream), gp);
   return check_launch();
 }
 

@@ -14,7 +14,9 @@ namespace pkv {
 struct SeqTable {
   int32_t batch;
   int32_t alpha;
-  int32_t n[PKV_MAX_BATCH];              // tokens of sequence b
+  int32_t n[PKV_MAX_BATCH];              // keys of sequence b held by the K tensor of this call
+  int32_t prefix[PKV_MAX_BATCH];         // how many of them are scored prefix keys: n - alpha for a whole
+                                         // sequence; all of them on a shard that does not hold the window
   int32_t count[PKV_MAX_BATCH];          // rows each KV head of sequence b keeps in this layer
   int64_t row_off[PKV_MAX_BATCH];        // first packed output row of sequence b
   int32_t stat_off[PKV_MAX_BATCH + 1];   // running sum of key chunks per sequence (row statistics sweep)

@@ -36,6 +36,7 @@ struct ScoreParams {
   float lse_scale, lse_add;              // applied on load: (1, 0), or (log2 e, log2 G) for natural-log input
   float* scores;                         // [batch][H_kv][ld]
   int64_t ld_scores;
+  int32_t stats_only;                    // host side: stop after the row normalisers (no score sweep)
 };
 
 // grid (total chunks, H_kv), block kGenRowBlock.
@@ -46,7 +47,7 @@ __global__ void __launch_bounds__(kGenRowBlock) rowstats_generic_kernel(const Sc
   pdl_wait();
   const int tile = blockIdx.x, h = blockIdx.y;
   const int b = find_sequence(p.seq.stat_off, p.seq.batch, tile);
-  const int n = p.seq.n[b], alpha = p.seq.alpha, P = n - alpha;
+  const int n = p.seq.n[b], alpha = p.seq.alpha, P = p.seq.prefix[b];
   const int key0 = (tile - p.seq.stat_off[b]) * kGenChunk;
   const int key1 = min(n, key0 + kGenChunk);
   const T* kbase = static_cast<const T*>(p.k.ptr) + b * p.k.sb + h * p.k.sh;
@@ -156,7 +157,7 @@ __global__ void __launch_bounds__(kGenScoreKeys) scores_generic_kernel(const Sco
   pdl_wait();
   const int tile = blockIdx.x, h = blockIdx.y;
   const int b = find_sequence(p.seq.score_off, p.seq.batch, tile);
-  const int alpha = p.seq.alpha, P = p.seq.n[b] - alpha;
+  const int alpha = p.seq.alpha, P = p.seq.prefix[b];
   const int i = (tile - p.seq.score_off[b]) * kGenScoreKeys + threadIdx.x;
   const bool live = i < P;
   float kreg[D];

@@ -374,7 +374,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   const int item0 = blockIdx.x * per + min(static_cast<int>(blockIdx.x), rem);
   const int item1 = item0 + per + (static_cast<int>(blockIdx.x) < rem ? 1 : 0);
   // keys an item of sequence b spans: sweep A covers all n keys, sweep B the prefix only
-  auto span_keys = [&](int b) { return SWEEP == 0 ? p.seq.n[b] : p.seq.n[b] - p.seq.alpha; };
+  auto span_keys = [&](int b) { return SWEEP == 0 ? p.seq.n[b] : p.seq.prefix[b]; };
 
   if (warp == 0) {
     // =========================================================== TMA producer
@@ -482,7 +482,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     bool ok = true;
     for (int id = item0; id < item1 && ok; ++id) {
       const TcItem w = tc_item(off, p.seq.batch, p.num_kv_heads, id);
-      const int n = p.seq.n[w.b], alpha = p.seq.alpha, P = n - alpha;
+      const int n = p.seq.n[w.b], alpha = p.seq.alpha, P = p.seq.prefix[w.b];
       const int keys = span_keys(w.b);
       const int tile0 = w.c * chunk_tiles;
       const int tile1 = min(tile0 + chunk_tiles, (keys + kTileKeys - 1) / kTileKeys);
@@ -491,7 +491,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         // works on the same block; with one, the pairs of groups take alternate K tiles.  Either way a
         // thread keeps one (reference, sum) per work item and every group writes its own partial slot.
         const int r = (two_blocks ? par * 128 : 0) + lane_row;
-        const int last_visible = P + (r % alpha);             // row (g, j) sees keys 0 .. P + j
+        const int last_visible = min(P + (r % alpha), n - 1); // row (g, j) sees keys 0 .. P + j that exist here
         const int units = p.row_blocks;
         // a warp whose 32 TMEM lanes are all padding rows (R < 128) has nothing to evaluate
         const bool warp_has_rows = (two_blocks ? par * 128 : 0) + quarter * 32 < p.rows;
@@ -508,7 +508,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
             const int key_base = t * kTcTileKeysA + ch * 128;
             if (!warp_has_rows) {
               // only the hand-shake below
-            } else if (key_base + 127 <= P) {                 // every key visible to every row: no mask
+            } else if (key_base + 127 <= min(P, n - 1)) {     // every key visible to every row: no mask
               for (int cg = 0; cg < 128; cg += 32) {
                 uint32_t v[32];
                 tc_ld32(taddr + cg, v);
