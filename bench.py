@@ -37,8 +37,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
 TC_SOURCES = ("pkv_score_tc.cuh", "pkv_common.cuh")
 NCU_TRAFFIC = {
     # profiles/score_tc_llama3_70b_128k.md: (read + written) bytes / (n * H_kv) key rows
-    "rowstats_tc": {"sources": TC_SOURCES, "digest": "83d46454d1fc6417", "bytes_per_key_row": 262.7},
-    "scores_tc": {"sources": TC_SOURCES, "digest": "83d46454d1fc6417", "bytes_per_key_row": 263.4},
+    "rowstats_tc": {"sources": TC_SOURCES, "digest": "a10eb2af3bd01f01", "bytes_per_key_row": 262.3},
+    "scores_tc": {"sources": TC_SOURCES, "digest": "a10eb2af3bd01f01", "bytes_per_key_row": 260.0},
 }
 
 
