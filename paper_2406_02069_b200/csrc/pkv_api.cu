@@ -400,8 +400,8 @@ int run_select(const pkv_config* c, const float* scores, int64_t ld, const SeqTa
   int cluster = 1;
   while (cluster < kSelMaxCluster && (max_p + cluster - 1) / cluster > 8192) cluster *= 2;
   const int slice = ((max_p + cluster - 1) / cluster + 31) & ~31;
-  sp.cached = (slice <= kSelSliceCap && sp.pool_radius <= kSelHalo) ? 1 : 0;
-  const size_t smem = sp.cached ? static_cast<size_t>(slice) * 6 + 8 * kSelHalo : 0;
+  sp.cached = sp.pool_radius <= kSelHalo ? 1 : 0;
+  const size_t smem = sp.cached ? static_cast<size_t>(std::min(slice, kSelSliceCap)) * 6 + 8 * kSelHalo : 0;
   sp.smem_pairs = static_cast<int32_t>(smem / sizeof(uint2));
   static bool attr_done[64] = {};  // the attribute is per device; setting it twice is harmless
   int dev = 0;

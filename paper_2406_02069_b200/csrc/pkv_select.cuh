@@ -52,7 +52,7 @@ struct SelectParams {
   SeqTable seq;
   int32_t num_kv_heads;
   int32_t pool_radius;      // (w - 1) / 2
-  int32_t cached;           // 1: every CTA's slice fits kSelSliceCap and is staged in shared memory
+  int32_t cached;           // 1: the pool radius fits kSelHalo, slices are staged in shared memory round by round
   int32_t smem_pairs;       // (key, position) pairs CTA 0 can hold in its dynamic shared memory
   uint2* cand;              // scratch: [batch * H_kv][cand_stride] candidate pairs, one region per CTA rank
   int64_t cand_stride;      // >= cluster * slice
@@ -131,37 +131,53 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
   if (selecting) {
     const float* s = p.scores + head * p.ld_scores;
     const int lo = min(P, rank * slice), hi = min(P, lo + slice);
-    const int run = ((slice / kSelWarps) + 31) & ~31;       // positions per warp, multiple of 32
-    const int wlo = min(hi, lo + warp * run), whi = min(hi, wlo + run);
     const int radius = p.pool_radius;
     uint2* region = regions + static_cast<int64_t>(rank) * slice;
-    if (p.cached) {                                         // then run <= kSelRunMax
-      // ---- 1. stage raw scores with a halo (outside the prefix: -inf for the max, 0 for the mean) and pool
+    if (p.cached) {                                         // the pool's reach fits the staged halo
+      // The slice is taken in rounds of at most kSelSliceCap positions (one round up to 131072 keys per head
+      // with a cluster of 8).  Round: stage raw scores with a halo (outside the prefix: -inf for the max, 0
+      // for the mean), pool them into one key per lane and step.
       float* raw = reinterpret_cast<float*>(sel_smem + kSelHalo);
       const float outside = AVG ? 0.0f : -INFINITY;
       const float width = static_cast<float>(2 * radius + 1);
-      for (int i = lo - kSelHalo + tid; i < hi + kSelHalo; i += kSelThreads)
-        raw[i - lo] = (i >= 0 && i < P) ? s[i] : outside;
-      __syncthreads();
+      const int rounds = (hi - lo + kSelSliceCap - 1) / kSelSliceCap;
+      const int run = ((min(slice, kSelSliceCap) / kSelWarps) + 31) & ~31;   // positions per warp and round
       uint32_t pk[kSelPerLane];
+      int wlo = hi, whi = hi;
+      auto pool_round = [&](int r) {
+        const int rlo = lo + r * kSelSliceCap, rhi = min(hi, rlo + kSelSliceCap);
+        __syncthreads();                                    // the previous round's readers are done
+        for (int i = rlo - kSelHalo + tid; i < rhi + kSelHalo; i += kSelThreads)
+          raw[i - rlo] = (i >= 0 && i < P) ? s[i] : outside;
+        __syncthreads();
+        wlo = min(rhi, rlo + warp * run);
+        whi = min(rhi, wlo + run);
+#pragma unroll
+        for (int it = 0; it < kSelPerLane; ++it) {
+          const int i = wlo + it * 32 + lane;
+          pk[it] = 0;
+          if (i < whi) {
+            float best;
+            if (AVG) {                                      // left to right; adding the zeros outside changes nothing
+              best = raw[i - rlo - radius];
+              for (int t = 1 - radius; t <= radius; ++t) best = __fadd_rn(best, raw[i - rlo + t]);
+              best = __fdiv_rn(best, width);
+            } else {
+              best = raw[i - rlo];
+              for (int t = 1; t <= radius; ++t) best = fmaxf(best, fmaxf(raw[i - rlo - t], raw[i - rlo + t]));
+            }
+            pk[it] = ordered_key(best);
+          }
+        }
+      };
+      // ---- 1. every thread's largest pooled key over the whole slice
       uint32_t tmax = 0;
 #pragma unroll
-      for (int it = 0; it < kSelPerLane; ++it) {
-        const int i = wlo + it * 32 + lane;
-        pk[it] = 0;
-        if (i < whi) {
-          float best;
-          if (AVG) {                                        // left to right; adding the zeros outside changes nothing
-            best = raw[i - lo - radius];
-            for (int t = 1 - radius; t <= radius; ++t) best = __fadd_rn(best, raw[i - lo + t]);
-            best = __fdiv_rn(best, width);
-          } else {
-            best = raw[i - lo];
-            for (int t = 1; t <= radius; ++t) best = fmaxf(best, fmaxf(raw[i - lo - t], raw[i - lo + t]));
-          }
-          pk[it] = ordered_key(best);
-          tmax = max(tmax, pk[it]);
-        }
+      for (int it = 0; it < kSelPerLane; ++it) pk[it] = 0;
+      for (int r = 0; r < rounds; ++r) {
+        pool_round(r);
+#pragma unroll
+        for (int it = 0; it < kSelPerLane; ++it) tmax = max(tmax, pk[it]);
       }
       // ---- 2. lower bound of the k-th largest key: the k-th largest per-thread maximum, resolved to its
       //         top 22 bits by two CTA-local histogram passes
@@ -204,34 +220,39 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
         __syncthreads();                                    // histogram zeroed, bound_digit consumed
       }
       const uint32_t bound = bprefix;                       // lower edge of the resolved digits
-      // candidates of this warp's run, then their place among the CTA's
-      uint32_t wc = 0;
+      // ---- 2b. candidates (keys >= bound) of every round, in position order, to this CTA's region
+      uint32_t filled = 0;
+      for (int r = 0; r < rounds; ++r) {
+        if (rounds > 1) pool_round(r);                      // a single round still holds its keys in registers
+        uint32_t wc = 0;
 #pragma unroll
-      for (int it = 0; it < kSelPerLane; ++it) {
-        const int i = wlo + it * 32 + lane;
-        wc += __popc(__ballot_sync(0xffffffffu, i < whi && pk[it] >= bound));
-      }
-      if (lane == 0) warp_gt[warp] = wc;
-      __syncthreads();
-      uint32_t base = 0, all_cand = 0;
-      for (int w2 = 0; w2 < kSelWarps; ++w2) {
-        if (w2 < warp) base += warp_gt[w2];
-        all_cand += warp_gt[w2];
-      }
-      if (tid == kSelThreads - 1) counts[rank] = all_cand;
-      local_pairs = C == 1 && static_cast<int>(all_cand) <= p.smem_pairs;
-      local_count = static_cast<int>(all_cand);
-      uint2* dst = local_pairs ? reinterpret_cast<uint2*>(sel_smem) : region;   // the raw scores are dead by now
+        for (int it = 0; it < kSelPerLane; ++it) {
+          const int i = wlo + it * 32 + lane;
+          wc += __popc(__ballot_sync(0xffffffffu, i < whi && pk[it] >= bound));
+        }
+        if (lane == 0) warp_gt[warp] = wc;
+        __syncthreads();
+        uint32_t base = filled, all_cand = 0;
+        for (int w2 = 0; w2 < kSelWarps; ++w2) {
+          if (w2 < warp) base += warp_gt[w2];
+          all_cand += warp_gt[w2];
+        }
+        local_pairs = C == 1 && rounds == 1 && static_cast<int>(all_cand) <= p.smem_pairs;
+        uint2* dst = local_pairs ? reinterpret_cast<uint2*>(sel_smem) : region;   // the raw scores are dead by now
 #pragma unroll
-      for (int it = 0; it < kSelPerLane; ++it) {
-        const int i = wlo + it * 32 + lane;
-        const bool c = i < whi && pk[it] >= bound;
-        const uint32_t bal = __ballot_sync(0xffffffffu, c);
-        if (c) dst[base + __popc(bal & lt)] = make_uint2(pk[it], static_cast<uint32_t>(i));
-        base += __popc(bal);
+        for (int it = 0; it < kSelPerLane; ++it) {
+          const int i = wlo + it * 32 + lane;
+          const bool c = i < whi && pk[it] >= bound;
+          const uint32_t bal = __ballot_sync(0xffffffffu, c);
+          if (c) dst[base + __popc(bal & lt)] = make_uint2(pk[it], static_cast<uint32_t>(i));
+          base += __popc(bal);
+        }
+        filled += all_cand;
       }
+      local_count = static_cast<int>(filled);
+      if (tid == 0) counts[rank] = filled;
     } else {
-      // slices too long for shared memory, or a very wide pool: every position is a candidate
+      // a very wide pool: every position is a candidate
       for (int i = lo + tid; i < hi; i += kSelThreads) region[i - lo] = make_uint2(pooled_key(s, i, P, radius, AVG ? 1 : 0), i);
       if (tid == 0) counts[rank] = hi - lo;
     }
