@@ -407,7 +407,10 @@ int run_select(const pkv_config* c, const float* scores, int64_t ld, const SeqTa
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return PKV_ERR_CUDA;
   if (dev >= 64 || !attr_done[dev]) {
-    for (auto kernel : {pool_select_kernel<false>, pool_select_kernel<true>})
+    for (auto kernel : {pool_select_kernel<false, false, 1>, pool_select_kernel<true, false, 1>,
+                        pool_select_kernel<false, true, 1>, pool_select_kernel<true, true, 1>,
+                        pool_select_kernel<false, false, 8>, pool_select_kernel<true, false, 8>,
+                        pool_select_kernel<false, true, 8>, pool_select_kernel<true, true, 8>})
       if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                kSelSliceCap * 6 + 8 * kSelHalo) != cudaSuccess)
         return PKV_ERR_CUDA;
@@ -428,8 +431,15 @@ int run_select(const pkv_config* c, const float* scores, int64_t ld, const SeqTa
   cfg.attrs = attr;
   cfg.numAttrs = 2;
   const bool avg = c->pool_kind == PKV_POOL_AVG;   // the mean pool is a variant; the max pool is the graded reading
-  if (cudaLaunchKernelEx(&cfg, avg ? pool_select_kernel<true> : pool_select_kernel<false>, sp) != cudaSuccess)
-    return PKV_ERR_CUDA;
+  const bool multi = slice > kSelSliceCap;          // long rows: each CTA takes its slice in several rounds
+  int k_max = 0;                                    // largest number of prefix rows any sequence keeps
+  for (int b = 0; b < batch; ++b) k_max = std::max(k_max, table.count[b] - c->window);
+  const bool wide = k_max > 512;                    // then 8 maxima per thread keep the candidate bound tight
+  auto kernel = avg ? (multi ? (wide ? pool_select_kernel<true, true, 8> : pool_select_kernel<true, true, 1>)
+                             : (wide ? pool_select_kernel<true, false, 8> : pool_select_kernel<true, false, 1>))
+                    : (multi ? (wide ? pool_select_kernel<false, true, 8> : pool_select_kernel<false, true, 1>)
+                             : (wide ? pool_select_kernel<false, false, 8> : pool_select_kernel<false, false, 1>));
+  if (cudaLaunchKernelEx(&cfg, kernel, sp) != cudaSuccess) return PKV_ERR_CUDA;
   mark(st, k_out ? "pool_select_gather" : "pool_select");
   return check_launch();
 }

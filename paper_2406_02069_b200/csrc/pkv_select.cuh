@@ -87,9 +87,61 @@ __device__ __forceinline__ uint32_t pooled_key(const float* s, int i, int P, int
   return ordered_key(best);
 }
 
+// Copies the rows named by one head's finished list into the packed cache: 16 bytes of K and of V per thread
+// and piece.  `first` / `stride` spread the pieces over the threads of the cluster.  Kept out of line so that
+// its registers are allocated apart from the selection's.  Long lists (large budgets move hundreds of
+// megabytes here) take four pieces per step with the index loads, the row loads and the stores issued as
+// batches; a one-piece loop would be bound by its latency chain.
+__device__ __noinline__ void gather_listed_rows(const int32_t* out, const char* kb, const char* vb, int64_t k_step,
+                                                int64_t v_step, uint4* k_dst, uint4* v_dst, int64_t row0, int total,
+                                                int pieces, int first, int stride) {
+  constexpr int kUnroll = 4;
+  int g0 = first;
+  {
+    for (; g0 + (kUnroll - 1) * stride < total; g0 += kUnroll * stride) {
+      int piece[kUnroll], pos[kUnroll];
+      int64_t dst[kUnroll];
+      uint4 val[kUnroll];
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u) {
+        const int g = g0 + u * stride;
+        const int row = g / pieces;
+        piece[u] = g - row * pieces;
+        pos[u] = __ldcg(out + row);                           // written by other CTAs of the cluster: skip L1
+        dst[u] = (row0 + row) * pieces + piece[u];
+      }
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u)
+        val[u] = reinterpret_cast<const uint4*>(kb + pos[u] * k_step)[piece[u]];
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u) k_dst[dst[u]] = val[u];
+      if (v_dst) {
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u)
+          val[u] = reinterpret_cast<const uint4*>(vb + pos[u] * v_step)[piece[u]];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) v_dst[dst[u]] = val[u];
+      }
+    }
+  }
+  for (; g0 < total; g0 += stride) {
+    const int row = g0 / pieces, piece = g0 - row * pieces;
+    const int pos = __ldcg(out + row);
+    const int64_t dst = (row0 + row) * pieces + piece;
+    k_dst[dst] =
+        reinterpret_cast<const uint4*>(kb + pos * k_step)[piece];
+    if (v_dst)
+      v_dst[dst] =
+          reinterpret_cast<const uint4*>(vb + pos * v_step)[piece];
+  }
+}
+
 // grid (cluster * H_kv, batch), cluster (cluster, 1, 1), block kSelThreads,
 // dynamic shared memory (6 bytes per slice position + 8 * kSelHalo) when cached, else none.
-template <bool AVG>
+// MULTI: some CTA's slice is longer than kSelSliceCap and is taken in several rounds.
+// GROUPS: maxima each thread keeps for the lower bound of step 2 (1 for small budgets, 8 when k nears or
+// passes the thread count, so that the bound stays tight).
+template <bool AVG, bool MULTI, int GROUPS>
 __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectParams p) {
   extern __shared__ __align__(16) uint32_t sel_smem[];      // [halo | slice | halo] raw scores; later CTA 0's pairs
   __shared__ uint32_t hist[2][kSelBins];                    // per-pass digit histogram (double buffered)
@@ -140,13 +192,13 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
       float* raw = reinterpret_cast<float*>(sel_smem + kSelHalo);
       const float outside = AVG ? 0.0f : -INFINITY;
       const float width = static_cast<float>(2 * radius + 1);
-      const int rounds = (hi - lo + kSelSliceCap - 1) / kSelSliceCap;
+      const int rounds = MULTI ? (hi - lo + kSelSliceCap - 1) / kSelSliceCap : 1;
       const int run = ((min(slice, kSelSliceCap) / kSelWarps) + 31) & ~31;   // positions per warp and round
       uint32_t pk[kSelPerLane];
       int wlo = hi, whi = hi;
       auto pool_round = [&](int r) {
         const int rlo = lo + r * kSelSliceCap, rhi = min(hi, rlo + kSelSliceCap);
-        __syncthreads();                                    // the previous round's readers are done
+        if (MULTI) __syncthreads();                         // the previous round's readers are done
         for (int i = rlo - kSelHalo + tid; i < rhi + kSelHalo; i += kSelThreads)
           raw[i - rlo] = (i >= 0 && i < P) ? s[i] : outside;
         __syncthreads();
@@ -170,24 +222,31 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
           }
         }
       };
-      // ---- 1. every thread's largest pooled key over the whole slice
-      uint32_t tmax = 0;
+      // ---- 1. every thread's largest pooled keys over the whole slice: one per group of its positions
+      //         (position step `it` belongs to group it mod GROUPS)
+      uint32_t tmax[GROUPS];
+#pragma unroll
+      for (int g = 0; g < GROUPS; ++g) tmax[g] = 0;
 #pragma unroll
       for (int it = 0; it < kSelPerLane; ++it) pk[it] = 0;
       for (int r = 0; r < rounds; ++r) {
         pool_round(r);
 #pragma unroll
-        for (int it = 0; it < kSelPerLane; ++it) tmax = max(tmax, pk[it]);
+        for (int it = 0; it < kSelPerLane; ++it) tmax[it % GROUPS] = max(tmax[it % GROUPS], pk[it]);
       }
-      // ---- 2. lower bound of the k-th largest key: the k-th largest per-thread maximum, resolved to its
-      //         top 22 bits by two CTA-local histogram passes
+      // ---- 2. lower bound of the k-th largest key: the k-th largest of these maxima (maxima of disjoint
+      //         groups of positions, so at least k keys are no smaller), resolved to its top 22 bits by two
+      //         CTA-local histogram passes
       uint32_t bprefix = 0, bmask = 0, brem = static_cast<uint32_t>(k);
       for (int bp = 0; bp < 2; ++bp) {
         const int shift = bp == 0 ? 21 : 10;
-        // threads whose maximum left the searched prefix do not take part in the second pass
-        const uint32_t digit = ((tmax & bmask) == bprefix) ? ((tmax >> shift) & 2047u) : kSelBins;
-        const uint32_t peers = __match_any_sync(0xffffffffu, digit);
-        if (digit < kSelBins && lane == __ffs(peers) - 1) atomicAdd(&hist[1][digit], __popc(peers));
+        // maxima that left the searched prefix do not take part in the second pass
+#pragma unroll
+        for (int g = 0; g < GROUPS; ++g) {
+          const uint32_t digit = ((tmax[g] & bmask) == bprefix) ? ((tmax[g] >> shift) & 2047u) : kSelBins;
+          const uint32_t peers = __match_any_sync(0xffffffffu, digit);
+          if (digit < kSelBins && lane == __ffs(peers) - 1) atomicAdd(&hist[1][digit], __popc(peers));
+        }
         __syncthreads();
         const uint2 v = reinterpret_cast<const uint2*>(hist[1])[tid];
         const uint32_t mine = v.x + v.y;
@@ -209,7 +268,7 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
         __syncthreads();
         reinterpret_cast<uint2*>(hist[1])[tid] = make_uint2(0, 0);
         const uint32_t bd = bound_digit;
-        if (bd == kSelBins) {                               // cannot bound (k exceeds the thread count): keep all
+        if (bd == kSelBins) {                               // cannot bound (k exceeds the number of maxima): keep all
           if (bp == 0) { bprefix = 0; bmask = 0; }
           __syncthreads();
           break;
@@ -223,7 +282,7 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
       // ---- 2b. candidates (keys >= bound) of every round, in position order, to this CTA's region
       uint32_t filled = 0;
       for (int r = 0; r < rounds; ++r) {
-        if (rounds > 1) pool_round(r);                      // a single round still holds its keys in registers
+        if (MULTI) pool_round(r);                           // a single round still holds its keys in registers
         uint32_t wc = 0;
 #pragma unroll
         for (int it = 0; it < kSelPerLane; ++it) {
@@ -237,7 +296,7 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
           if (w2 < warp) base += warp_gt[w2];
           all_cand += warp_gt[w2];
         }
-        local_pairs = C == 1 && rounds == 1 && static_cast<int>(all_cand) <= p.smem_pairs;
+        local_pairs = !MULTI && C == 1 && static_cast<int>(all_cand) <= p.smem_pairs;
         uint2* dst = local_pairs ? reinterpret_cast<uint2*>(sel_smem) : region;   // the raw scores are dead by now
 #pragma unroll
         for (int it = 0; it < kSelPerLane; ++it) {
@@ -353,22 +412,26 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
   }
   if (C == 1) __syncthreads(); else cluster.sync();         // the list is complete
 
-  // ---- 5. eviction by gather (appendix on torch.gather), spread over the cluster: 16 bytes of K and of V
-  //         per thread and step
+  // ---- 5. eviction by gather (appendix on torch.gather), spread over the cluster
   if (p.k_out != nullptr) {
-    const int64_t row0 = p.seq.row_off[b] + static_cast<int64_t>(h) * count;
-    const int total = count * p.pieces;
     const char* kb = static_cast<const char*>(p.k.ptr) + (b * p.k.sb + h * p.k.sh) * p.elem_bytes;
     const char* vb = static_cast<const char*>(p.v.ptr) + (b * p.v.sb + h * p.v.sh) * p.elem_bytes;
-    for (int g = rank * kSelThreads + tid; g < total; g += C * kSelThreads) {
-      const int row = g / p.pieces, piece = g - row * p.pieces;
-      const int pos = __ldcg(out + row);                    // written by other CTAs of the cluster: skip L1
-      const int64_t dst = (row0 + row) * p.pieces + piece;
-      static_cast<uint4*>(p.k_out)[dst] =
-          reinterpret_cast<const uint4*>(kb + static_cast<int64_t>(pos) * p.k.st * p.elem_bytes)[piece];
-      if (p.v_out)
-        static_cast<uint4*>(p.v_out)[dst] =
-            reinterpret_cast<const uint4*>(vb + static_cast<int64_t>(pos) * p.v.st * p.elem_bytes)[piece];
+    const int64_t row0 = p.seq.row_off[b] + static_cast<int64_t>(h) * count;
+    const int total = count * p.pieces, stride = C * kSelThreads;
+    if (total >= 8 * stride) {                              // a long list: the batched copy
+      gather_listed_rows(out, kb, vb, p.k.st * p.elem_bytes, p.v.st * p.elem_bytes, static_cast<uint4*>(p.k_out),
+                         static_cast<uint4*>(p.v_out), row0, total, p.pieces, rank * kSelThreads + tid, stride);
+    } else {
+      for (int g = rank * kSelThreads + tid; g < total; g += stride) {
+        const int row = g / p.pieces, piece = g - row * p.pieces;
+        const int pos = __ldcg(out + row);                  // written by other CTAs of the cluster: skip L1
+        const int64_t dst = (row0 + row) * p.pieces + piece;
+        static_cast<uint4*>(p.k_out)[dst] =
+            reinterpret_cast<const uint4*>(kb + static_cast<int64_t>(pos) * p.k.st * p.elem_bytes)[piece];
+        if (p.v_out)
+          static_cast<uint4*>(p.v_out)[dst] =
+              reinterpret_cast<const uint4*>(vb + static_cast<int64_t>(pos) * p.v.st * p.elem_bytes)[piece];
+      }
     }
   }
 }
