@@ -94,7 +94,10 @@ Workspace carve(const pkv_config* c, int batch, int max_n, void* base) {
   const size_t chunks = (static_cast<size_t>(max_n) + kPartialChunk - 1) / kPartialChunk;
   w.status = reinterpret_cast<uint32_t*>(take(kAlign));
   w.lse2 = reinterpret_cast<float*>(take(heads * rows * sizeof(float)));
-  w.partial = reinterpret_cast<float2*>(take(heads * chunks * 2 * rows * sizeof(float2)));   // 2 slots per chunk
+  // fp32-pipe sweep: 2 slots per chunk and head; tensor-core sweep: up to 4 slots per segment, one segment per
+  // run of a CTA over a head (at most CTAs + heads of them)
+  const size_t partial_slots = std::max(heads * chunks * 2, (static_cast<size_t>(kTcMaxGrid) + heads) * 4);
+  w.partial = reinterpret_cast<float2*>(take(partial_slots * rows * sizeof(float2)));
   w.score_scratch_bytes = off;
   w.ld_scores = static_cast<int64_t>((static_cast<size_t>(max_n) + 63) / 64 * 64);
   w.scores = reinterpret_cast<float*>(take(heads * w.ld_scores * sizeof(float)));
@@ -321,7 +324,9 @@ int launch_scores_tc(const pkv_config* c, const pkv_tensor& q, const pkv_tensor&
   sp.seq = tp.seq;
   sp.slots_per_chunk = tp.row_blocks == 2 ? 2 : 4;    // partial slots each sweep-A work item writes
 
-  const int grid_a = static_cast<int>(std::min<long long>(sms, static_cast<long long>(stat_items) * sp.num_kv_heads));
+  const int grid_a = static_cast<int>(std::min<long long>(std::min(sms, kTcMaxGrid),
+                                                          static_cast<long long>(stat_items) * sp.num_kv_heads));
+  sp.stat_grid = grid_a;
   const int grid_b = static_cast<int>(std::min<long long>(sms, static_cast<long long>(score_items) * sp.num_kv_heads));
   if (sp.lse_in == sp.lse2) {                    // normalisers not supplied: sweep A and its merge
     launch_pdl(score_tc_kernel<D, 0>, grid_a, kTcThreads, TcSmem<D>::kTotal, st, q_map, k_map_a, tp);

@@ -37,6 +37,9 @@ struct ScoreParams {
   float* scores;                         // [batch][H_kv][ld]
   int64_t ld_scores;
   int32_t stats_only;                    // host side: stop after the row normalisers (no score sweep)
+  int32_t stat_grid;                     // 0: partial is [chunk][slot][H_kv][rows] (fp32-pipe sweep).  > 0: CTAs of
+                                         // the tensor-core sweep, which writes [segment][slot][rows] with segment =
+                                         // CTA + head for every run of a CTA over one head's chunks
 };
 
 // grid (total chunks, H_kv), block kGenRowBlock.
@@ -116,11 +119,28 @@ __global__ void __launch_bounds__(kCombineThreads) combine_stats_kernel(const Sc
   const int h = blockIdx.y, b = blockIdx.z;
   const int rl = threadIdx.x & 31, sg = threadIdx.x >> 5;
   const int r = blockIdx.x * 32 + rl;
-  const int t0 = p.seq.stat_off[b] * p.slots_per_chunk, t1 = p.seq.stat_off[b + 1] * p.slots_per_chunk;
-  const int64_t slot_stride = static_cast<int64_t>(p.num_kv_heads) * p.rows;
+  int t0 = p.seq.stat_off[b] * p.slots_per_chunk, t1 = p.seq.stat_off[b + 1] * p.slots_per_chunk;
+  int64_t slot_stride = static_cast<int64_t>(p.num_kv_heads) * p.rows;
+  int64_t first = static_cast<int64_t>(h) * p.rows;
+  if (p.stat_grid > 0) {
+    // The sweep's CTAs take contiguous item ranges (items ordered sequence, head, chunk): the first `rem`
+    // CTAs per + 1 items, the others per.  This head's items fall to CTAs c0..c1, one segment each.
+    const int nc = p.seq.stat_off[b + 1] - p.seq.stat_off[b];
+    const int total = p.num_kv_heads * p.seq.stat_off[p.seq.batch];
+    const int per = total / p.stat_grid, rem = total % p.stat_grid;
+    const int edge = rem * (per + 1);
+    const int i0 = p.num_kv_heads * p.seq.stat_off[b] + h * nc, i1 = i0 + nc - 1;
+    const int c0 = i0 < edge ? i0 / (per + 1) : rem + (i0 - edge) / per;
+    const int c1 = i1 < edge ? i1 / (per + 1) : rem + (i1 - edge) / per;
+    const int hg = b * p.num_kv_heads + h;
+    t0 = (c0 + hg) * p.slots_per_chunk;
+    t1 = (c1 + hg + 1) * p.slots_per_chunk;
+    slot_stride = p.rows;
+    first = 0;
+  }
   float m = -INFINITY, z = 0.f;
   if (r < p.rows) {
-    const float2* base = p.partial + static_cast<int64_t>(h) * p.rows + r;
+    const float2* base = p.partial + first + r;
     for (int t = t0 + sg; t < t1; t += 4 * 32) {
       float2 pz[4];
 #pragma unroll

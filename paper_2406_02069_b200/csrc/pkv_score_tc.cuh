@@ -40,6 +40,7 @@ constexpr int kTcEpiWarps = 16;         // four per scheduler, which is what kee
 constexpr int kTcTileKeysA = 256;       // keys per K tile in sweep A (the N of its MMAs)
 constexpr int kTcTileKeysB = 128;       // keys per K tile in sweep B (the M of its MMAs)
 constexpr int kTcKBytes = 128 * 1024;   // shared memory given to K stages (2 x 64 KB or 4 x 32 KB at d = 128)
+constexpr int kTcMaxGrid = 256;         // CTAs of a sweep at most (the workspace holds a partial segment per CTA)
 constexpr int kTcMaxRows = 256;         // window rows (G * alpha) the tensor-core path takes
 constexpr long long kTcWaitCycles = 1ll << 31;   // bound of any one wait, in SM clocks
 
@@ -52,8 +53,9 @@ struct TcParams {
   int32_t chunk_tiles_a;        // 256-key tiles per work item of sweep A
   int32_t chunk_tiles_b;        // 128-key tiles per work item of sweep B
   float scale_log2;             // log2(e) / sqrt(d)
-  float2* partial;              // sweep A out: [chunk][slots][H_kv][R] (reference exponent, sum); slots = 2 with
-                                // two row blocks, 4 with one: every epilogue warp group writes its own slot
+  float2* partial;              // sweep A out: [segment][slots][R] (reference exponent, sum); a segment is one
+                                // CTA's run over one (sequence, head); slots = 2 with two row blocks, 4 with
+                                // one: every epilogue warp group writes its own slot
   const float* lse2;            // sweep B in:  [batch][H_kv][R] row normalisers (log of the row's sum of exps)
   float lse_scale, lse_add;     // lse2_r = lse2[r] * lse_scale + lse_add: (1, 0) for the library's own sweep A,
                                 // (log2 e, log2 G) for natural-log normalisers handed in by the caller
@@ -480,6 +482,20 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     uint32_t u = 0, mine = 0;                   // units seen by the CTA / units this group's pair has read
     int cur_b = -1, cur_h = -1;
     bool ok = true;
+    // Sweep A: a thread's (reference, sum) runs on over consecutive work items of one (sequence, head) and is
+    // written once per run, to the segment numbered blockIdx.x + head: along the item order either the CTA
+    // or the head advances from one run to the next, so the numbers are distinct, and the merge kernel finds
+    // a head's segments from the CTAs its items fall to.
+    float m = -INFINITY, z = 0.f;
+    int run_b = -1, run_h = -1;
+    auto flush_run = [&]() {
+      const int r = (two_blocks ? par * 128 : 0) + lane_row;
+      if (run_b < 0 || r >= p.rows) return;
+      const int slots = two_blocks ? 2 : 4;
+      const int slot = two_blocks ? ch : grp;
+      const int64_t seg = static_cast<int64_t>(blockIdx.x) + run_b * p.num_kv_heads + run_h;
+      p.partial[(seg * slots + slot) * p.rows + r] = make_float2(m, z);
+    };
     for (int id = item0; id < item1 && ok; ++id) {
       const TcItem w = tc_item(off, p.seq.batch, p.num_kv_heads, id);
       const int n = p.seq.n[w.b], alpha = p.seq.alpha, P = p.seq.prefix[w.b];
@@ -489,13 +505,19 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       if (SWEEP == 0) {
         // thread -> window row.  With two row blocks the unit parity is the row block, so a group always
         // works on the same block; with one, the pairs of groups take alternate K tiles.  Either way a
-        // thread keeps one (reference, sum) per work item and every group writes its own partial slot.
+        // thread keeps one (reference, sum) per run of work items and every group writes its own partial slot.
         const int r = (two_blocks ? par * 128 : 0) + lane_row;
         const int last_visible = min(P + (r % alpha), n - 1); // row (g, j) sees keys 0 .. P + j that exist here
         const int units = p.row_blocks;
         // a warp whose 32 TMEM lanes are all padding rows (R < 128) has nothing to evaluate
         const bool warp_has_rows = (two_blocks ? par * 128 : 0) + quarter * 32 < p.rows;
-        float m = -INFINITY, z = 0.f;
+        if (w.b != run_b || w.h != run_h) {
+          flush_run();
+          m = -INFINITY;
+          z = 0.f;
+          run_b = w.b;
+          run_h = w.h;
+        }
         for (int t = tile0; t < tile1 && ok; ++t) {
           for (int rb = 0; rb < units && ok; ++rb, ++u) {
             if (static_cast<int>(u & 1u) != par) continue;    // the other pair's unit
@@ -545,12 +567,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
           }
         }
         if (!ok) break;
-        if (r < p.rows) {
-          const int slots = two_blocks ? 2 : 4;
-          const int slot = two_blocks ? ch : grp;
-          const int64_t chunk = off[w.b] + w.c;
-          p.partial[((chunk * slots + slot) * p.num_kv_heads + w.h) * p.rows + r] = make_float2(m, z);
-        }
       } else {
         // thread -> key.  The pairs of groups take alternate K tiles; inside a pair the groups split the
         // window rows (columns) of a key and group ch = 1 hands its partial sum to group ch = 0.
@@ -612,6 +628,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         if (!ok) break;
       }
     }
+    if (SWEEP == 0 && ok) flush_run();                        // the CTA's last run
   }
 
   // ---- teardown
