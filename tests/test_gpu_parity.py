@@ -63,6 +63,11 @@ def test_scores_match_oracle(w):
     (16, 2, 32, 128, [1500]),             # R = 256
     (4, 4, 1, 128, [300]),                # alpha = 1
     (8, 1, 16, 128, [16 + 1, 16 + 128, 16 + 129]),   # prefix of 1, of one tile, of one tile + 1
+    (1, 1, 256, 128, [900]),              # R = 256 from one head: the widest window the tensor-core path takes
+    (2, 2, 128, 64, [700, 300]),          # R = 128 exactly, head_dim 64
+    (16, 1, 16, 128, [1000]),             # G = 16
+    (64, 2, 8, 128, [777]),               # G = 32, R = 256
+    (4, 2, 24, 128, [60 + i * 37 for i in range(64)]),   # the largest batch, short ragged sequences
 ])
 def test_scores_bf16_shapes(hq, hkv, alpha, d, lens):
     """Tensor-core score path over window sizes, group sizes, head dims and ragged tails."""
