@@ -400,7 +400,9 @@ def main():
         line["e2e"] = {"value": e_value, "unit": UNIT,
                        "h2d_bytes_per_step": pipe.h2d_bytes, "d2h_bytes_per_step": pipe.d2h_bytes,
                        "steps": args.e2e_steps, "ms_per_step": e_ms / args.e2e_steps,
-                       "note": "host side cycles %d distinct pinned layers; every layer is copied in every step" % ring}
+                       "note": "host side cycles %d distinct pinned layers; Q and K of every layer are copied in every "
+                               "step, V stays in pinned host memory and only its kept rows are read over the bus "
+                               "(counted in h2d_bytes_per_step)" % ring}
 
     if rank == 0 and not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = cpu_baseline_sample(w, layers[:16], lens, out.budgets)

@@ -94,6 +94,24 @@ typedef struct pkv_tensor {
   int64_t stride_token;  /* >= head_dim; the head dimension itself has stride 1 */
 } pkv_tensor;
 
+/*
+ * Where a pointer lives, as the CUDA runtime sees it (host only; a query, nothing is enqueued):
+ *   PKV_MEM_PAGEABLE_HOST 0   ordinary host memory: kernels cannot read it
+ *   PKV_MEM_PINNED_HOST   1   page-locked host memory mapped at the same address on the device
+ *   PKV_MEM_DEVICE        2   device memory
+ *   PKV_MEM_MANAGED       3   managed memory
+ * Returns the kind, or a negative status (-PKV_ERR_CUDA when no CUDA device answers).
+ * "device" tensors of the calls below may be of kind 1, 2 or 3.  Kind 1 makes sense for V: the path only
+ * ever touches the rows of V that are kept (Section 4.2.2: the rest is evicted), so a V that stays in pinned
+ * host memory costs a few hundred kilobytes of bus reads per layer instead of a copy of the whole tensor.
+ * K is read in full, twice, and belongs in device memory.
+ */
+#define PKV_MEM_PAGEABLE_HOST 0
+#define PKV_MEM_PINNED_HOST 1
+#define PKV_MEM_DEVICE 2
+#define PKV_MEM_MANAGED 3
+int pyramidkv_memory_kind(const void* ptr);
+
 /* Human-readable name of a status code (static string, never NULL). */
 const char* pyramidkv_strerror(int status);
 

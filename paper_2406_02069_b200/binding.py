@@ -31,7 +31,7 @@ EXPORTS = ("pyramidkv_strerror", "pyramidkv_layer_budgets", "pyramidkv_kept_coun
            "pyramidkv_compress_layer_lse", "pyramidkv_profile_layer_lse", "pyramidkv_decode_attention",
            "pyramidkv_attention_recall", "pyramidkv_pages_needed", "pyramidkv_gather_paged",
            "pyramidkv_compress_layer_paged", "pyramidkv_decode_attention_paged", "pyramidkv_shard_window_lse",
-           "pyramidkv_merge_lse", "pyramidkv_shard_scores", "pyramidkv_shard_gather")
+           "pyramidkv_merge_lse", "pyramidkv_shard_scores", "pyramidkv_shard_gather", "pyramidkv_memory_kind")
 PKV_MAX_STAGES = 8
 
 
@@ -90,6 +90,7 @@ def _load() -> ctypes.CDLL:
     lib.pyramidkv_merge_lse.argtypes = [P, I32, I64, P, P]
     lib.pyramidkv_shard_scores.argtypes = [CFG, PkvTensor, PkvTensor, P, P, P, I32, P, I64, P, SZ, P]
     lib.pyramidkv_shard_gather.argtypes = [CFG, PkvTensor, PkvTensor, P, P, I32, I32, P, P, P, P, P]
+    lib.pyramidkv_memory_kind.argtypes = [P]
     lib.pyramidkv_check_status.argtypes = [P, P, P]
     for name in EXPORTS:
         if name not in ("pyramidkv_strerror", "pyramidkv_workspace_bytes"):
@@ -102,6 +103,17 @@ _lib = _load()
 
 def library_path() -> str:
     return _build.LIB
+
+
+MEM_PAGEABLE_HOST, MEM_PINNED_HOST, MEM_DEVICE, MEM_MANAGED = 0, 1, 2, 3
+
+
+def memory_kind(t: torch.Tensor) -> int:
+    """Where the tensor's storage lives as the CUDA runtime sees it (MEM_*)."""
+    kind = _lib.pyramidkv_memory_kind(t.data_ptr())
+    if kind < 0:
+        raise PkvError(-kind, "pyramidkv_memory_kind")
+    return int(kind)
 
 
 def strerror(status: int) -> str:

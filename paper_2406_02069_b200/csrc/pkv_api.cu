@@ -548,6 +548,21 @@ using namespace pkv;
 
 extern "C" {
 
+int pyramidkv_memory_kind(const void* ptr) {
+  cudaPointerAttributes attr;
+  if (!ptr) return -PKV_ERR_INVALID_ARG;
+  if (cudaPointerGetAttributes(&attr, ptr) != cudaSuccess) {
+    cudaGetLastError();                                    // a query must not leave a sticky error behind
+    return -PKV_ERR_CUDA;
+  }
+  switch (attr.type) {
+    case cudaMemoryTypeHost: return attr.devicePointer == ptr ? PKV_MEM_PINNED_HOST : PKV_MEM_PAGEABLE_HOST;
+    case cudaMemoryTypeDevice: return PKV_MEM_DEVICE;
+    case cudaMemoryTypeManaged: return PKV_MEM_MANAGED;
+    default: return PKV_MEM_PAGEABLE_HOST;
+  }
+}
+
 const char* pyramidkv_strerror(int status) {
   switch (status) {
     case PKV_OK: return "ok";

@@ -4,7 +4,8 @@
 `compress_model_from_host` is the end-to-end form for callers whose prefill K/V
 sit in (pinned) host memory, e.g. an offloaded cache: each layer is copied to the
 device on a copy stream while the previous layer is being compressed, and the
-compact cache and its index list are copied back.  Both only marshal arguments
+compact cache and its index list are copied back.  V can stay where it is: only
+its kept rows are ever read, and the kernels can read pinned host memory.  Both only marshal arguments
 and order streams; all arithmetic is in the library's kernels.
 """
 from __future__ import annotations
@@ -40,8 +41,11 @@ class HostPipeline:
     """Double-buffered host -> device -> host pipeline for one model shape."""
 
     def __init__(self, cfg: pkv.PkvConfig, seq_lens: Sequence[int], q_shape, kv_shape, dtype: torch.dtype,
-                 device="cuda"):
+                 device="cuda", zero_copy_v: bool = True):
+        """zero_copy_v: leave V in the caller's pinned host memory and let the gather read the kept rows over
+        the bus (only they are ever needed); V is then not copied to the device at all."""
         self.cfg, self.seq_lens = cfg, list(seq_lens)
+        self.zero_copy_v = zero_copy_v
         self.budgets = pkv.layer_budgets(cfg)
         self.rows = [pkv.total_rows(cfg, kl, seq_lens) for kl in self.budgets]
         max_rows = max(self.rows)
@@ -71,20 +75,25 @@ class HostPipeline:
             with torch.cuda.stream(self.copy_in):
                 if l >= 2:
                     self.copy_in.wait_event(computed[l - 2])      # buffer free once its layer was compressed
+                direct_v = self.zero_copy_v and pkv.memory_kind(src.v) == pkv.MEM_PINNED_HOST
                 buf["q"].copy_(src.q_win, non_blocking=True)
                 buf["k"].copy_(src.k, non_blocking=True)
-                buf["v"].copy_(src.v, non_blocking=True)
+                if not direct_v:
+                    buf["v"].copy_(src.v, non_blocking=True)
                 lse = getattr(src, "window_lse", None)
                 if lse is not None:
                     buf["lse"].copy_(lse, non_blocking=True)
                 loaded[l].record(self.copy_in)
-            moved = [src.q_win, src.k, src.v] + ([lse] if lse is not None else [])
+            moved = [src.q_win, src.k] + ([] if direct_v else [src.v]) + ([lse] if lse is not None else [])
             self.h2d_bytes += sum(t.numel() * t.element_size() for t in moved)
+            if direct_v:                                          # the kept rows of V cross the bus inside the kernel
+                self.h2d_bytes += r * self.cfg.head_dim * src.v.element_size()
             with torch.cuda.stream(self.compute):
                 self.compute.wait_event(loaded[l])
                 if l >= 2:
                     self.compute.wait_event(drained[l - 2])       # outputs of this buffer were copied out
-                pkv.compress_layer(self.cfg, l, buf["q"], buf["k"], buf["v"], self.seq_lens, buf["ko"], buf["vo"],
+                pkv.compress_layer(self.cfg, l, buf["q"], buf["k"], src.v if direct_v else buf["v"], self.seq_lens,
+                                   buf["ko"], buf["vo"],
                                    buf["io"], self.workspace, stream=self.compute,
                                    window_lse=buf["lse"] if lse is not None else None)
                 computed[l].record(self.compute)

@@ -1,0 +1,65 @@
+"""GPU parity of the whole-model drivers: the host pipeline (pinned K/V/Q in, compact cache out) must give
+exactly what the device-resident calls give, with V copied to the device and with V left in pinned host
+memory and read row by row over the bus."""
+import types
+
+import pytest
+import torch
+
+import paper_2406_02069_b200 as pkv
+from paper_2406_02069_b200 import streaming, workloads
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def host_layer(x):
+    return types.SimpleNamespace(q_win=x.q_win.cpu().pin_memory(), k=x.k.cpu().pin_memory(), v=x.v.cpu().pin_memory())
+
+
+def host_out(rows, d, dtype):
+    return types.SimpleNamespace(k=torch.empty(rows, d, dtype=dtype).pin_memory(),
+                                 v=torch.empty(rows, d, dtype=dtype).pin_memory(),
+                                 idx=torch.empty(rows, dtype=torch.int32).pin_memory())
+
+
+def test_memory_kinds():
+    assert pkv.memory_kind(torch.zeros(8, device=DEV)) == pkv.binding.MEM_DEVICE
+    assert pkv.memory_kind(torch.zeros(8).pin_memory()) == pkv.binding.MEM_PINNED_HOST
+    assert pkv.memory_kind(torch.zeros(8)) == pkv.binding.MEM_PAGEABLE_HOST
+
+
+@pytest.mark.parametrize("w", [
+    workloads.scaled(workloads.LLAMA3_8B, num_layers=5, seq_len=6011, name="llama3_8b_6k"),
+    workloads.scaled(workloads.MISTRAL_RAGGED, num_layers=4, batch=3, name="mistral_b3"),
+], ids=lambda w: w.name)
+@pytest.mark.parametrize("zero_copy_v", [False, True])
+def test_host_pipeline_equals_device_resident_calls(w, zero_copy_v):
+    cfg = pkv.config_of(w)
+    lens = w.seq_lens()
+    if w.batch > 1:
+        lens = [500 + (n % 1777) for n in lens]
+    layers = [workloads.make_layer(w, l, device=DEV, seq_lens=lens) for l in range(w.num_layers)]
+    out = streaming.LayerOutputs(cfg, lens, w.torch_dtype())
+    ws = pkv.new_workspace(cfg, len(lens), max(lens), DEV)
+    streaming.compress_model(cfg, layers, lens, out, ws)
+    pkv.check_status(ws)
+
+    pipe = streaming.HostPipeline(cfg, lens, layers[0].q_win.shape, layers[0].k.shape, w.torch_dtype(),
+                                  zero_copy_v=zero_copy_v)
+    hl = [host_layer(x) for x in layers]
+    ho = [host_out(r, w.head_dim, w.torch_dtype()) for r in out.rows]
+    for rep in range(2):                                              # the second run reuses every buffer
+        pipe.run(hl, ho)
+        torch.cuda.synchronize()
+        pkv.check_status(pipe.workspace)
+        for l in range(w.num_layers):
+            assert torch.equal(ho[l].idx, out.idx[l].cpu())
+            assert torch.equal(ho[l].k, out.k[l].cpu()) and torch.equal(ho[l].v, out.v[l].cpu())
+    esz = layers[0].k.element_size()
+    qk_bytes = sum((x.k.numel() + x.q_win.numel()) * esz for x in layers)
+    v_bytes = sum(x.v.numel() * esz for x in layers)
+    if zero_copy_v:                                                  # of V only the kept rows crossed the bus
+        assert pipe.h2d_bytes == qk_bytes + sum(out.rows) * w.head_dim * esz
+    else:
+        assert pipe.h2d_bytes == qk_bytes + v_bytes
