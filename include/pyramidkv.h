@@ -173,7 +173,7 @@ int pyramidkv_score_window(const pkv_config* cfg, pkv_tensor q_win, pkv_tensor k
  * pyramidkv_score_window for callers that cannot allocate.  The paper has no
  * counterpart: this is an integration aid.  Same inputs, same scores as
  * pyramidkv_score_window, but no workspace argument: the kernels' scratch
- * (per-chunk row statistics and the row normalisers) lives in an array of
+ * (partial row statistics and the row normalisers) lives in an array of
  * PKV_STATIC_SCRATCH_BYTES (8 MiB) that is built into the library, so the call
  * and everything under it performs no cudaMalloc / cudaFree and needs no memory
  * pool.  It is meant for code that is handed only its input and output buffers:
@@ -181,10 +181,12 @@ int pyramidkv_score_window(const pkv_config* cfg, pkv_tensor q_win, pkv_tensor k
  * memory to its own pool, or a section where an allocation (which may
  * synchronise the whole device) is not acceptable.
  *   - Every GPU on which the library is loaded holds the 8 MiB until the process ends.
- *   - The problem must fit: the scratch grows with batch * H_kv * ceil(n_max / 128) *
- *     (H_q / H_kv) * alpha * 8 bytes.  Larger problems are refused with
- *     PKV_ERR_STATIC_SCRATCH before anything is enqueued; use pyramidkv_score_window
- *     with a workspace for those.
+ *   - The problem must fit.  With 16-bit inputs and (H_q / H_kv) * alpha <= 256 rows per KV head the
+ *     scratch is (256 + batch * H_kv) * 32 * (H_q / H_kv) * alpha bytes plus the row normalisers,
+ *     whatever the context length (2.2 MB for one 8-head sequence with 256 rows); other shapes run
+ *     on the fp32-pipe kernels and need batch * H_kv * ceil(n_max / 128) * (H_q / H_kv) * alpha * 16
+ *     bytes.  Larger problems are refused with PKV_ERR_STATIC_SCRATCH before anything is enqueued;
+ *     use pyramidkv_score_window with a workspace for those.
  *   - The first call made on a device looks up the array's device address
  *     (cudaGetSymbolAddress) and caches it; make that first call outside any
  *     stream capture.

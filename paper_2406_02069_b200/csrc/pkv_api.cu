@@ -83,6 +83,13 @@ struct Workspace {
   size_t bytes;
 };
 
+// Which configurations the tensor-core score kernels take (the others go to the fp32-pipe kernels).
+bool tc_eligible(const pkv_config* c) {
+  const int g = c->num_q_heads / c->num_kv_heads;
+  return (c->dtype == PKV_DTYPE_BF16 || c->dtype == PKV_DTYPE_FP16) && g * c->window <= kTcMaxRows &&
+         c->window <= 256 && g <= 256;
+}
+
 // Carves the workspace for `batch` sequences of at most max_n tokens.  base may be null (sizing only).
 Workspace carve(const pkv_config* c, int batch, int max_n, void* base) {
   Workspace w{};
@@ -95,8 +102,8 @@ Workspace carve(const pkv_config* c, int batch, int max_n, void* base) {
   w.status = reinterpret_cast<uint32_t*>(take(kAlign));
   w.lse2 = reinterpret_cast<float*>(take(heads * rows * sizeof(float)));
   // fp32-pipe sweep: 2 slots per chunk and head; tensor-core sweep: up to 4 slots per segment, one segment per
-  // run of a CTA over a head (at most CTAs + heads of them)
-  const size_t partial_slots = std::max(heads * chunks * 2, (static_cast<size_t>(kTcMaxGrid) + heads) * 4);
+  // run of a CTA over a head (at most CTAs + heads of them), whatever the context length
+  const size_t partial_slots = tc_eligible(c) ? (static_cast<size_t>(kTcMaxGrid) + heads) * 4 : heads * chunks * 2;
   w.partial = reinterpret_cast<float2*>(take(partial_slots * rows * sizeof(float2)));
   w.score_scratch_bytes = off;
   w.ld_scores = static_cast<int64_t>((static_cast<size_t>(max_n) + 63) / 64 * 64);
@@ -234,10 +241,6 @@ bool make_map(CUtensorMap* map, const pkv_tensor& t, bool fp16, int d, uint64_t 
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-bool tc_eligible(const pkv_config* c) {
-  const int g = c->num_q_heads / c->num_kv_heads;
-  return (c->dtype == PKV_DTYPE_BF16 || c->dtype == PKV_DTYPE_FP16) && g * c->window <= kTcMaxRows && c->window <= 256 && g <= 256;
-}
 
 int device_sm_count() {
   static int sms[64] = {};

@@ -50,7 +50,8 @@ def test_static_scratch_scores_equal_workspace_scores_twice_in_a_row():
 
 
 def test_problem_larger_than_the_built_in_scratch_is_refused():
-    w = workloads.LLAMA3_70B                                        # 128k tokens: needs ~17 MB of scratch
+    # 128k tokens in fp32: the fp32-pipe kernels keep statistics per 128-key chunk, ~34 MB of scratch
+    w = workloads.scaled(workloads.LLAMA3_70B, name="llama3_70b_fp32", dtype="fp32")
     cfg = pkv.config_of(w)
     assert pkv.workspace_bytes(cfg, 1, 131072) > binding.PKV_STATIC_SCRATCH_BYTES
     small = workloads.make_layer(workloads.scaled(w, num_layers=1, seq_len=256), 0, device=DEV)
