@@ -306,6 +306,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
                 const TcParams p) {
   using L = TcSmem<D>;
   constexpr int kTileKeys = SWEEP == 0 ? kTcTileKeysA : kTcTileKeysB;
+  // Sweep B walks each CTA's items and tiles from the last to the first: sweep A has just read the same keys in
+  // ascending order, so the end of every range is what the L2 still holds.
+  constexpr bool kReverse = SWEEP == 1;
   constexpr int kStageBytes = kTileKeys * D * 2;               // one K tile in shared memory
   constexpr int kKStages = kTcKBytes / kStageBytes >= 4 ? 4 : kTcKBytes / kStageBytes;
   extern __shared__ uint8_t smem_raw[];
@@ -384,7 +387,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       uint32_t it = 0, heads_loaded = 0;                       // it counts K tiles
       int cur_b = -1, cur_h = -1;
       bool ok = true;
-      for (int id = item0; id < item1 && ok; ++id) {
+      for (int ii = 0; ii < item1 - item0 && ok; ++ii) {
+        const int id = kReverse ? item1 - 1 - ii : item0 + ii;
         const TcItem w = tc_item(off, p.seq.batch, p.num_kv_heads, id);
         if (w.b != cur_b || w.h != cur_h) {
           if (heads_loaded > 0) ok = mbar_wait(q_empty, (heads_loaded - 1) & 1, abort_flag);
@@ -398,7 +402,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         const int keys = span_keys(w.b);
         const int tile0 = w.c * chunk_tiles;
         const int tile1 = min(tile0 + chunk_tiles, (keys + kTileKeys - 1) / kTileKeys);
-        for (int t = tile0; t < tile1 && ok; ++t, ++it) {
+        for (int tt = 0; tt < tile1 - tile0 && ok; ++tt, ++it) {
+          const int t = kReverse ? tile1 - 1 - tt : tile0 + tt;
           const int s = it % kKStages;
           ok = mbar_wait(k_empty(s), ((it / kKStages) & 1) ^ 1, abort_flag);
           if (!ok) break;
@@ -426,7 +431,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       bool ok = true;
       const uint32_t idesc = SWEEP == 0 ? instr_desc_16bit(128, kTcTileKeysA, p.fp16)
                                         : instr_desc_16bit(kTcTileKeysB, p.rows_pad, p.fp16);
-      for (int id = item0; id < item1 && ok; ++id) {
+      for (int ii = 0; ii < item1 - item0 && ok; ++ii) {
+        const int id = kReverse ? item1 - 1 - ii : item0 + ii;
         const TcItem w = tc_item(off, p.seq.batch, p.num_kv_heads, id);
         if (w.b != cur_b || w.h != cur_h) {
           ok = mbar_wait(q_full, heads_seen & 1, abort_flag);
@@ -435,15 +441,15 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
           cur_b = w.b; cur_h = w.h;
         }
         // does the next item belong to another head?  then Q may be overwritten after this item's MMAs
-        bool last_of_head = id + 1 >= item1;
+        bool last_of_head = ii + 1 >= item1 - item0;
         if (!last_of_head) {
-          const TcItem nx = tc_item(off, p.seq.batch, p.num_kv_heads, id + 1);
+          const TcItem nx = tc_item(off, p.seq.batch, p.num_kv_heads, kReverse ? id - 1 : id + 1);
           last_of_head = nx.b != w.b || nx.h != w.h;
         }
         const int keys = span_keys(w.b);
         const int tile0 = w.c * chunk_tiles;
         const int tile1 = min(tile0 + chunk_tiles, (keys + kTileKeys - 1) / kTileKeys);
-        for (int t = tile0; t < tile1 && ok; ++t, ++it) {
+        for (int tt = 0; tt < tile1 - tile0 && ok; ++tt, ++it) {
           const int s = it % kKStages;
           ok = mbar_wait(k_full(s), (it / kKStages) & 1, abort_flag);
           if (!ok) break;
@@ -496,7 +502,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       const int64_t seg = static_cast<int64_t>(blockIdx.x) + run_b * p.num_kv_heads + run_h;
       p.partial[(seg * slots + slot) * p.rows + r] = make_float2(m, z);
     };
-    for (int id = item0; id < item1 && ok; ++id) {
+    for (int ii = 0; ii < item1 - item0 && ok; ++ii) {
+      const int id = kReverse ? item1 - 1 - ii : item0 + ii;
       const TcItem w = tc_item(off, p.seq.batch, p.num_kv_heads, id);
       const int n = p.seq.n[w.b], alpha = p.seq.alpha, P = p.seq.prefix[w.b];
       const int keys = span_keys(w.b);
@@ -581,7 +588,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         }
         float* srow = p.scores + (static_cast<int64_t>(w.b) * p.num_kv_heads + w.h) * p.ld_scores;
         const int col0 = ch == 0 ? 0 : split_b, col1 = ch == 0 ? split_b : p.rows_pad;
-        for (int t = tile0; t < tile1 && ok; ++t, ++u) {
+        for (int tt = 0; tt < tile1 - tile0 && ok; ++tt, ++u) {
+          const int t = kReverse ? tile1 - 1 - tt : tile0 + tt;
           if (static_cast<int>(u & 1u) != par) continue;      // the other pair's tile
           if (ch == 1 && !second_half) continue;              // nothing for this group to read
           const int ts = u % t_stages;
