@@ -259,16 +259,16 @@ int launch_scores_tc(const pkv_config* c, const pkv_tensor& q, const pkv_tensor&
                      int max_n, uint32_t* status, cudaStream_t st) {
   const int sms = device_sm_count();
   if (sms <= 0) return PKV_ERR_CUDA;
-  static bool attr_done[64] = {};
+  static bool attr_done[64] = {};  // the attribute is per device; setting it twice is harmless
   int dev = 0;
-  cudaGetDevice(&dev);
-  if (!attr_done[dev]) {
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) return PKV_ERR_CUDA;
+  if (dev >= 64 || !attr_done[dev]) {
     if (cudaFuncSetAttribute(score_tc_kernel<D, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcSmem<D>::kTotal) !=
             cudaSuccess ||
         cudaFuncSetAttribute(score_tc_kernel<D, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcSmem<D>::kTotal) !=
             cudaSuccess)
       return PKV_ERR_CUDA;
-    attr_done[dev] = true;
+    if (dev < 64) attr_done[dev] = true;
   }
   alignas(64) CUtensorMap q_map, k_map_a, k_map_b;
   const bool fp16 = c->dtype == PKV_DTYPE_FP16;
