@@ -241,6 +241,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--graph", action="store_true",
                     help="replay one CUDA graph per step instead of enqueueing 4 launches per layer from the host")
+    ap.add_argument("--lanes", type=int, default=0, metavar="SMS",
+                    help="run selection + gather of a layer on SMS streaming multiprocessors of their own (a multiple "
+                         "of 8) beside the next layer's score sweeps on the rest; 0 = one stream, kernels in turn")
     ap.add_argument("--mode", default="self", choices=["self", "handoff"],
                     help="self: the library finds the row normalisers itself (two K sweeps, the graded path); "
                          "handoff: they are handed in as the prefill attention would (one K sweep)")
@@ -300,6 +303,15 @@ def main():
         streaming.compress_model(cfg, layers, lens, out, ws)
     pkv.check_status(ws)
     run_step = lambda: streaming.compress_model(cfg, layers, lens, out, ws)
+    if args.lanes:
+        if args.graph:
+            raise SystemExit("--lanes and --graph are separate experiments")
+        lanes = pkv.Lanes(select_sms=args.lanes)
+        pair = [ws, pkv.new_workspace(cfg, len(lens), max(lens))]
+        run_step = lambda: streaming.compress_model(cfg, layers, lens, out, pair, lanes=lanes)
+        for _ in range(args.warmup):
+            run_step()
+        pkv.check_status(pair[1])
     if args.graph:                                                  # the calls above warmed every first-use path
         graph = torch.cuda.CUDAGraph()
         side = torch.cuda.Stream()
@@ -370,7 +382,7 @@ def main():
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
-            "config": {"workload": w.name, "mode": args.mode, "cuda_graph": bool(args.graph), "layers": w.num_layers, "q_heads": w.num_q_heads,
+            "config": {"workload": w.name, "mode": args.mode, "cuda_graph": bool(args.graph), "select_lane_sms": args.lanes, "layers": w.num_layers, "q_heads": w.num_q_heads,
                        "kv_heads": w.num_kv_heads, "head_dim": w.head_dim, "batch": w.batch, "seq_lens": lens,
                        "window": w.window, "pool_kernel": w.pool_kernel, "avg_budget": w.avg_budget, "beta": w.beta,
                        "tokens_per_step_per_gpu": tokens, "parallelism": "replicas x%d" % world,

@@ -422,6 +422,38 @@ int pyramidkv_shard_gather(const pkv_config* cfg, pkv_tensor k_shard, pkv_tensor
                            void* k_out, void* v_out, void* stream);
 
 /*
+ * Whole-model call on two lanes.  The paper has no counterpart: this is scheduling.  Selection and gather
+ * (Section 4.2.2's last step) keep only a fraction of the GPU's SMs busy, and layers are independent, so the
+ * score sweeps of layer l + 1 can run beside the selection of layer l.  A pkv_lanes object splits the SMs of
+ * the current device into two disjoint groups (CUDA green contexts; nothing outlives the process or touches
+ * another process) with one stream on each: `select_sms` SMs (a multiple of 8, at least 8, at most half of
+ * the device) for selection and gather, the rest for the score sweeps.
+ *   pyramidkv_lanes_create    host; creates contexts, streams and events: not for a hot path.  UNSUPPORTED
+ *                             when the driver has no green contexts or cannot split as asked.
+ *   pyramidkv_lanes_destroy   host; the lanes must be idle.
+ *   pyramidkv_compress_model_lanes
+ *       layers first_layer .. first_layer + num_layers - 1 of the model, exactly as num_layers calls of
+ *       pyramidkv_compress_layer (window_lse_or_null: NULL, or one pointer per layer as for
+ *       pyramidkv_compress_layer_lse); q_win, k, v, k_out, v_out, indices are host arrays with one entry per
+ *       layer.  `workspaces` holds TWO distinct workspaces of workspace_bytes each (consecutive layers
+ *       alternate between them); each has its own status word.  The work is ordered after what `stream`
+ *       holds at the call and `stream` continues after all of it; in between it runs on the lanes' streams.
+ * Results are those of the per-layer calls bit for bit (the same kernels on the same data; only the number of
+ * CTAs of the sweeps follows the lane's SM count).  Errors: as pyramidkv_compress_layer; INVALID_ARG when the
+ * lanes belong to another device.
+ */
+typedef struct pkv_lanes pkv_lanes;
+int pyramidkv_lanes_create(int32_t select_sms, pkv_lanes** out);
+int pyramidkv_lanes_destroy(pkv_lanes* lanes);
+int pyramidkv_lanes_info(const pkv_lanes* lanes, int32_t* score_sms, int32_t* select_sms);
+int pyramidkv_compress_model_lanes(const pkv_config* cfg, pkv_lanes* lanes, int32_t first_layer, int32_t num_layers,
+                                   const pkv_tensor* q_win, const pkv_tensor* k, const pkv_tensor* v,
+                                   const float* const* window_lse_or_null,
+                                   const int32_t* seq_lens, int32_t batch,
+                                   void* const* k_out, void* const* v_out, int32_t* const* indices,
+                                   void* const* workspaces, size_t workspace_bytes, void* stream);
+
+/*
  * Synchronises `stream` and reads the workspace status word.  For tests and
  * debugging.  Returns PKV_OK, PKV_ERR_DEVICE_STATUS (a kernel gave up on a
  * bounded wait or saw an impossible state; *detail_or_null receives the word),

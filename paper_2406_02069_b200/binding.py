@@ -31,7 +31,9 @@ EXPORTS = ("pyramidkv_strerror", "pyramidkv_layer_budgets", "pyramidkv_kept_coun
            "pyramidkv_compress_layer_lse", "pyramidkv_profile_layer_lse", "pyramidkv_decode_attention",
            "pyramidkv_attention_recall", "pyramidkv_pages_needed", "pyramidkv_gather_paged",
            "pyramidkv_compress_layer_paged", "pyramidkv_decode_attention_paged", "pyramidkv_shard_window_lse",
-           "pyramidkv_merge_lse", "pyramidkv_shard_scores", "pyramidkv_shard_gather", "pyramidkv_memory_kind")
+           "pyramidkv_merge_lse", "pyramidkv_shard_scores", "pyramidkv_shard_gather", "pyramidkv_memory_kind",
+           "pyramidkv_lanes_create", "pyramidkv_lanes_destroy", "pyramidkv_lanes_info",
+           "pyramidkv_compress_model_lanes")
 PKV_MAX_STAGES = 8
 
 
@@ -91,6 +93,10 @@ def _load() -> ctypes.CDLL:
     lib.pyramidkv_shard_scores.argtypes = [CFG, PkvTensor, PkvTensor, P, P, P, I32, P, I64, P, SZ, P]
     lib.pyramidkv_shard_gather.argtypes = [CFG, PkvTensor, PkvTensor, P, P, I32, I32, P, P, P, P, P]
     lib.pyramidkv_memory_kind.argtypes = [P]
+    lib.pyramidkv_lanes_create.argtypes = [I32, ctypes.POINTER(P)]
+    lib.pyramidkv_lanes_destroy.argtypes = [P]
+    lib.pyramidkv_lanes_info.argtypes = [P, ctypes.POINTER(I32), ctypes.POINTER(I32)]
+    lib.pyramidkv_compress_model_lanes.argtypes = [CFG, P, I32, I32, P, P, P, P, P, I32, P, P, P, P, SZ, P]
     lib.pyramidkv_check_status.argtypes = [P, P, P]
     for name in EXPORTS:
         if name not in ("pyramidkv_strerror", "pyramidkv_workspace_bytes"):
@@ -407,3 +413,50 @@ def shard_gather(cfg: PkvConfig, k_shard: torch.Tensor, v_shard: torch.Tensor, i
     _check(_lib.pyramidkv_shard_gather(ctypes.byref(cfg), _tensor(k_shard), _tensor(v_shard), indices.data_ptr(), lens,
                                        batch, int(k_layer), begin, keys, k_out.data_ptr(), v_out.data_ptr(),
                                        _stream(stream)), "pyramidkv_shard_gather")
+
+
+# ----------------------------------------------------------------------------- two lanes
+class Lanes:
+    """The device's SMs split into a group for the score sweeps and a small one for selection and gather."""
+
+    def __init__(self, select_sms: int = 8):
+        handle = ctypes.c_void_p()
+        _check(_lib.pyramidkv_lanes_create(int(select_sms), ctypes.byref(handle)), "pyramidkv_lanes_create")
+        self._handle = handle
+        a, b = ctypes.c_int32(), ctypes.c_int32()
+        _check(_lib.pyramidkv_lanes_info(handle, ctypes.byref(a), ctypes.byref(b)), "pyramidkv_lanes_info")
+        self.score_sms, self.select_sms = a.value, b.value
+
+    def close(self) -> None:
+        if self._handle is not None:
+            _lib.pyramidkv_lanes_destroy(self._handle)
+            self._handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def compress_model_lanes(cfg: PkvConfig, lanes: Lanes, layers, seq_lens: Sequence[int], k_out, v_out, indices,
+                         workspaces, first_layer: int = 0, stream=None) -> None:
+    """layers: objects with .q_win/.k/.v (and optionally .window_lse, on all or none of them); k_out, v_out,
+    indices: per-layer output tensors; workspaces: two workspace tensors of one size."""
+    lens, batch = _lens(seq_lens)
+    m = len(layers)
+    if not (len(k_out) == len(v_out) == len(indices) == m) or len(workspaces) != 2:
+        raise ValueError("one output per layer and exactly two workspaces are needed")
+    if workspaces[0].numel() != workspaces[1].numel():
+        raise ValueError("the two workspaces must have one size")
+    tensors = lambda name: (PkvTensor * m)(*[_tensor(getattr(x, name)) for x in layers])
+    pointers = lambda ts: (ctypes.c_void_p * m)(*[t.data_ptr() for t in ts])
+    with_lse = [getattr(x, "window_lse", None) is not None for x in layers]
+    if any(with_lse) and not all(with_lse):
+        raise ValueError("window_lse must be given for every layer or for none")
+    lse = (ctypes.c_void_p * m)(*[_lse_ptr(x.window_lse) for x in layers]) if all(with_lse) and m else None
+    _check(_lib.pyramidkv_compress_model_lanes(
+        ctypes.byref(cfg), lanes._handle, int(first_layer), m, tensors("q_win"), tensors("k"), tensors("v"), lse, lens,
+        batch, pointers(k_out), pointers(v_out), pointers(indices),
+        (ctypes.c_void_p * 2)(workspaces[0].data_ptr(), workspaces[1].data_ptr()), workspaces[0].numel(),
+        _stream(stream)), "pyramidkv_compress_model_lanes")

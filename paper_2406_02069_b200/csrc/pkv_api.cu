@@ -242,8 +242,13 @@ bool make_map(CUtensorMap* map, const pkv_tensor& t, bool fp16, int d, uint64_t 
 }
 
 
+// SMs the persistent score kernels may count on: the device's, or fewer while a call runs them on a lane that
+// owns only a group of the SMs (pyramidkv_compress_model_lanes sets the limit for its own thread).
+thread_local int tl_sm_limit = 0;
+
 int device_sm_count() {
   static int sms[64] = {};
+  if (tl_sm_limit > 0) return tl_sm_limit;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
   if (!sms[dev]) {
@@ -1002,6 +1007,198 @@ int pyramidkv_shard_gather(const pkv_config* cfg, pkv_tensor k_shard, pkv_tensor
   launch_pdl(gather_shard_kernel, static_cast<unsigned>((threads + kShardThreads - 1) / kShardThreads), kShardThreads,
              0, static_cast<cudaStream_t>(stream), gp);
   return check_launch();
+}
+
+// ---------------------------------------------------------------------------
+// Two lanes: the SMs of the device split into two disjoint groups (CUDA green contexts), one stream on each.
+// The score sweeps of layer l + 1 then run beside the selection and gather of layer l, which by itself keeps
+// fewer than half of the SMs busy for a seventh of a layer's time.
+struct pkv_lanes {
+  CUgreenCtx ctx[2];          // [0] scores, [1] selection
+  cudaStream_t stream[2];
+  int sms[2];
+  int device;
+  cudaEvent_t start, scored[2], selected[2], done[2];
+};
+
+namespace {
+
+struct LaneApi {
+  CUresult (*device_get)(CUdevice*, int);
+  CUresult (*get_dev_resource)(CUdevice, CUdevResource*, CUdevResourceType);
+  CUresult (*split_by_count)(CUdevResource*, unsigned int*, const CUdevResource*, CUdevResource*, unsigned int,
+                             unsigned int);
+  CUresult (*generate_desc)(CUdevResourceDesc*, CUdevResource*, unsigned int);
+  CUresult (*green_create)(CUgreenCtx*, CUdevResourceDesc, CUdevice, unsigned int);
+  CUresult (*green_stream)(CUstream*, CUgreenCtx, unsigned int, int);
+  CUresult (*green_destroy)(CUgreenCtx);
+  bool ok;
+};
+
+const LaneApi& lane_api() {
+  static LaneApi api = [] {
+    LaneApi a{};
+    auto get = [](const char* name) -> void* {
+      void* sym = nullptr;
+      cudaDriverEntryPointQueryResult q;
+      if (cudaGetDriverEntryPoint(name, &sym, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess)
+        return nullptr;
+      return sym;
+    };
+    a.device_get = reinterpret_cast<decltype(a.device_get)>(get("cuDeviceGet"));
+    a.get_dev_resource = reinterpret_cast<decltype(a.get_dev_resource)>(get("cuDeviceGetDevResource"));
+    a.split_by_count = reinterpret_cast<decltype(a.split_by_count)>(get("cuDevSmResourceSplitByCount"));
+    a.generate_desc = reinterpret_cast<decltype(a.generate_desc)>(get("cuDevResourceGenerateDesc"));
+    a.green_create = reinterpret_cast<decltype(a.green_create)>(get("cuGreenCtxCreate"));
+    a.green_stream = reinterpret_cast<decltype(a.green_stream)>(get("cuGreenCtxStreamCreate"));
+    a.green_destroy = reinterpret_cast<decltype(a.green_destroy)>(get("cuGreenCtxDestroy"));
+    a.ok = a.device_get && a.get_dev_resource && a.split_by_count && a.generate_desc && a.green_create &&
+           a.green_stream && a.green_destroy;
+    cudaGetLastError();
+    return a;
+  }();
+  return api;
+}
+
+}  // namespace
+
+int pyramidkv_lanes_create(int32_t select_sms, pkv_lanes** out) {
+  if (!out || select_sms < 8) return PKV_ERR_INVALID_ARG;
+  *out = nullptr;
+  const LaneApi& api = lane_api();
+  if (!api.ok) return PKV_ERR_UNSUPPORTED;
+  int device = 0;
+  if (cudaGetDevice(&device) != cudaSuccess || cudaFree(nullptr) != cudaSuccess) return PKV_ERR_CUDA;
+  CUdevice dev;
+  CUdevResource all, group, rest;
+  unsigned int groups = 1;
+  if (api.device_get(&dev, device) != CUDA_SUCCESS ||
+      api.get_dev_resource(dev, &all, CU_DEV_RESOURCE_TYPE_SM) != CUDA_SUCCESS)
+    return PKV_ERR_UNSUPPORTED;
+  if (static_cast<unsigned>(select_sms) * 2 > all.sm.smCount) return PKV_ERR_INVALID_ARG;
+  if (api.split_by_count(&group, &groups, &all, &rest, 0, static_cast<unsigned>(select_sms)) != CUDA_SUCCESS ||
+      groups != 1 || rest.sm.smCount == 0)
+    return PKV_ERR_UNSUPPORTED;
+  pkv_lanes* l = new pkv_lanes();
+  l->device = device;
+  CUdevResource parts[2] = {rest, group};
+  bool good = true;
+  int made_ctx = 0, made_stream = 0;
+  for (int i = 0; i < 2 && good; ++i) {
+    CUdevResourceDesc desc;
+    good = api.generate_desc(&desc, &parts[i], 1) == CUDA_SUCCESS &&
+           api.green_create(&l->ctx[i], desc, dev, CU_GREEN_CTX_DEFAULT_STREAM) == CUDA_SUCCESS;
+    if (!good) break;
+    ++made_ctx;
+    CUstream s;
+    good = api.green_stream(&s, l->ctx[i], CU_STREAM_NON_BLOCKING, 0) == CUDA_SUCCESS;
+    if (!good) break;
+    ++made_stream;
+    l->stream[i] = reinterpret_cast<cudaStream_t>(s);
+    l->sms[i] = static_cast<int>(parts[i].sm.smCount);
+  }
+  cudaEvent_t* events[] = {&l->start, &l->scored[0], &l->scored[1], &l->selected[0], &l->selected[1], &l->done[0],
+                           &l->done[1]};
+  int made_events = 0;
+  for (cudaEvent_t* e : events) {
+    if (!good) break;
+    good = cudaEventCreateWithFlags(e, cudaEventDisableTiming) == cudaSuccess;
+    if (good) ++made_events;
+  }
+  if (!good) {
+    for (int i = 0; i < made_events; ++i) cudaEventDestroy(*events[i]);
+    for (int i = 0; i < made_stream; ++i) cudaStreamDestroy(l->stream[i]);
+    for (int i = 0; i < made_ctx; ++i) api.green_destroy(l->ctx[i]);
+    delete l;
+    cudaGetLastError();
+    return PKV_ERR_UNSUPPORTED;
+  }
+  *out = l;
+  return PKV_OK;
+}
+
+int pyramidkv_lanes_destroy(pkv_lanes* l) {
+  if (!l) return PKV_OK;
+  cudaEvent_t events[] = {l->start, l->scored[0], l->scored[1], l->selected[0], l->selected[1], l->done[0], l->done[1]};
+  for (cudaEvent_t e : events) cudaEventDestroy(e);
+  for (int i = 0; i < 2; ++i) cudaStreamDestroy(l->stream[i]);
+  for (int i = 0; i < 2; ++i) lane_api().green_destroy(l->ctx[i]);
+  delete l;
+  return PKV_OK;
+}
+
+int pyramidkv_lanes_info(const pkv_lanes* l, int32_t* score_sms, int32_t* select_sms) {
+  if (!l || !score_sms || !select_sms) return PKV_ERR_INVALID_ARG;
+  *score_sms = l->sms[0];
+  *select_sms = l->sms[1];
+  return PKV_OK;
+}
+
+int pyramidkv_compress_model_lanes(const pkv_config* cfg, pkv_lanes* lanes, int32_t first_layer, int32_t num_layers,
+                                   const pkv_tensor* q_win, const pkv_tensor* k, const pkv_tensor* v,
+                                   const float* const* window_lse_or_null, const int32_t* seq_lens, int32_t batch,
+                                   void* const* k_out, void* const* v_out, int32_t* const* indices,
+                                   void* const* workspaces, size_t workspace_bytes, void* stream) {
+  if (!config_ok(cfg)) return PKV_ERR_INVALID_ARG;
+  if (int rc = config_supported(cfg)) return rc;
+  if (!lanes || !q_win || !k || !v || !k_out || !v_out || !indices || !workspaces) return PKV_ERR_INVALID_ARG;
+  if (first_layer < 0 || num_layers < 1 || first_layer + num_layers > cfg->num_layers) return PKV_ERR_INVALID_ARG;
+  if (!workspaces[0] || !workspaces[1] || workspaces[0] == workspaces[1]) return PKV_ERR_INVALID_ARG;
+  int device = -1;
+  if (cudaGetDevice(&device) != cudaSuccess || device != lanes->device) return PKV_ERR_INVALID_ARG;
+  const int eb = cfg->dtype == PKV_DTYPE_FP32 ? 4 : 2;
+  for (int i = 0; i < num_layers; ++i) {
+    if (!tensor_ok(q_win[i], cfg->head_dim, eb) || !tensor_ok(k[i], cfg->head_dim, eb) ||
+        !tensor_ok(v[i], cfg->head_dim, eb) || !k_out[i] || !v_out[i] || !indices[i])
+      return PKV_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(k_out[i]) % 16 || reinterpret_cast<uintptr_t>(v_out[i]) % 16)
+      return PKV_ERR_INVALID_ARG;
+  }
+  // tables and workspaces are validated before anything is enqueued
+  int max_n = 0;
+  int64_t rows = 0;
+  Workspace ws[2];
+  {
+    SeqTable probe;
+    if (int rc = build_table(cfg, seq_lens, batch, 0, &probe, &max_n, &rows)) return rc;
+    for (int i = 0; i < 2; ++i)
+      if (int rc = workspace_check(cfg, batch, max_n, workspaces[i], workspace_bytes, &ws[i])) return rc;
+  }
+  cudaStream_t caller = static_cast<cudaStream_t>(stream), score = lanes->stream[0], select = lanes->stream[1];
+  if (cudaEventRecord(lanes->start, caller) != cudaSuccess || cudaStreamWaitEvent(score, lanes->start, 0) != cudaSuccess ||
+      cudaStreamWaitEvent(select, lanes->start, 0) != cudaSuccess)
+    return PKV_ERR_CUDA;
+  int status = PKV_OK;
+  tl_sm_limit = lanes->sms[0];
+  for (int i = 0; i < num_layers && status == PKV_OK; ++i) {
+    const int32_t k_layer = layer_budget(cfg, first_layer + i);
+    SeqTable table;
+    if ((status = build_table(cfg, seq_lens, batch, k_layer, &table, &max_n, &rows)) != PKV_OK) break;
+    const Workspace& w = ws[i & 1];
+    // the scores buffer of this workspace is free once the selection two layers back has read it
+    if (i >= 2 && cudaStreamWaitEvent(score, lanes->selected[i & 1], 0) != cudaSuccess) { status = PKV_ERR_CUDA; break; }
+    bool any_compress = false;
+    for (int b = 0; b < batch; ++b) any_compress |= table.count[b] < table.n[b];
+    if (any_compress)
+      status = run_scores(cfg, q_win[i], k[i], table, batch, w.scores, w.ld_scores, w, score,
+                          window_lse_or_null ? window_lse_or_null[i] : nullptr);
+    if (status != PKV_OK) break;
+    if (cudaEventRecord(lanes->scored[i & 1], score) != cudaSuccess ||
+        cudaStreamWaitEvent(select, lanes->scored[i & 1], 0) != cudaSuccess) { status = PKV_ERR_CUDA; break; }
+    tl_sm_limit = 0;
+    status = run_select(cfg, w.scores, w.ld_scores, table, batch, max_n, indices[i], w, select, &k[i], &v[i], k_out[i],
+                        v_out[i]);
+    tl_sm_limit = lanes->sms[0];
+    if (status != PKV_OK) break;
+    if (cudaEventRecord(lanes->selected[i & 1], select) != cudaSuccess) { status = PKV_ERR_CUDA; break; }
+  }
+  tl_sm_limit = 0;
+  // the caller's stream continues when both lanes are done, whatever happened above
+  if (cudaEventRecord(lanes->done[0], score) != cudaSuccess || cudaEventRecord(lanes->done[1], select) != cudaSuccess ||
+      cudaStreamWaitEvent(caller, lanes->done[0], 0) != cudaSuccess ||
+      cudaStreamWaitEvent(caller, lanes->done[1], 0) != cudaSuccess)
+    return status != PKV_OK ? status : PKV_ERR_CUDA;
+  return status;
 }
 
 int pyramidkv_check_status(const void* workspace, void* stream, uint32_t* detail_or_null) {

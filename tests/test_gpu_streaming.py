@@ -63,3 +63,40 @@ def test_host_pipeline_equals_device_resident_calls(w, zero_copy_v):
         assert pipe.h2d_bytes == qk_bytes + sum(out.rows) * w.head_dim * esz
     else:
         assert pipe.h2d_bytes == qk_bytes + v_bytes
+
+
+@pytest.mark.parametrize("w", [
+    workloads.scaled(workloads.LLAMA3_8B, num_layers=6, seq_len=6011, name="llama3_8b_6k"),
+    workloads.scaled(workloads.MISTRAL_RAGGED, num_layers=5, batch=3, name="mistral_b3"),
+    workloads.TINY,
+], ids=lambda w: w.name)
+def test_two_lanes_give_the_per_layer_results(w):
+    """Score sweeps of layer l + 1 beside selection and gather of layer l, on disjoint groups of SMs: the
+    outputs must be those of the per-layer calls, bit for bit, run after run."""
+    cfg = pkv.config_of(w)
+    lens = w.seq_lens()
+    if w.batch > 1:
+        lens = [500 + (n % 1777) for n in lens]
+    layers = [workloads.make_layer(w, l, device=DEV, seq_lens=lens) for l in range(w.num_layers)]
+    want = streaming.LayerOutputs(cfg, lens, w.torch_dtype())
+    ws = pkv.new_workspace(cfg, len(lens), max(lens), DEV)
+    streaming.compress_model(cfg, layers, lens, want, ws)
+    pkv.check_status(ws)
+    try:
+        lanes = pkv.Lanes(select_sms=8)
+    except pkv.PkvError as e:
+        pytest.skip("this driver cannot split the SMs: %s" % e)
+    assert lanes.select_sms == 8 and lanes.score_sms >= 8
+    pair = [pkv.new_workspace(cfg, len(lens), max(lens), DEV) for _ in range(2)]
+    for rep in range(3):
+        got = streaming.LayerOutputs(cfg, lens, w.torch_dtype())
+        for t in got.k + got.v:
+            t.fill_(-7.0)
+        streaming.compress_model(cfg, layers, lens, got, pair, lanes=lanes)
+        torch.cuda.current_stream().synchronize()          # the call joins the lanes back into this stream
+        for x in pair:
+            pkv.check_status(x)
+        for l in range(w.num_layers):
+            assert torch.equal(got.idx[l], want.idx[l]), "layer %d" % l
+            assert torch.equal(got.k[l], want.k[l]) and torch.equal(got.v[l], want.v[l])
+    lanes.close()
