@@ -10,7 +10,7 @@
 //            TMEM lane = key, so each epilogue thread owns one key and sums
 //            2^(x_ri - lse2_r) over the rows r, reading lse2 from shared memory.
 //
-// x = (q . k) * log2(e) / sqrt(d).  Operands arrive by TMA (no multicast) into
+// x = (q . k) * log2(e) / sqrt(d).  Operands arrive by plain per-CTA TMA loads into
 // 128-byte-swizzled shared memory; tcgen05.mma accumulates in TMEM (two to four
 // accumulator stages of up to 256 columns); epilogue warps read TMEM with tcgen05.ld.
 // Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner, warps 4..19 =
