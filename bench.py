@@ -346,6 +346,15 @@ def main():
     value, ms, _ = parallel.job_throughput(tokens * args.steps, ev0.elapsed_time(ev1), device="cuda")
     pkv.check_status(ws)
     ms_per_step = ms / args.steps
+    # spread of single steps: a second, shorter loop with an event after every step (this rank only)
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(min(20, args.steps) + 1)]
+    marks[0].record()
+    for e in marks[1:]:
+        run_step()
+        e.record()
+    torch.cuda.synchronize()
+    singles = sorted(a.elapsed_time(b) for a, b in zip(marks, marks[1:]))
+    step_median, step_best = singles[len(singles) // 2], singles[0]
 
     # ---- per-kernel device times (events between the launches of each layer's call), same inputs and launch shapes
     stages = {}
@@ -380,7 +389,8 @@ def main():
                          "frac_of_8TBs": path_gbs / 8000.0}}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "ms_per_step_median": step_median,
+            "ms_per_step_best": step_best, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
             "config": {"workload": w.name, "mode": args.mode, "cuda_graph": bool(args.graph), "select_lane_sms": args.lanes, "layers": w.num_layers, "q_heads": w.num_q_heads,
                        "kv_heads": w.num_kv_heads, "head_dim": w.head_dim, "batch": w.batch, "seq_lens": lens,
