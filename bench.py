@@ -381,10 +381,20 @@ def main():
         traffic = tr["bytes_per_key_row"] * sum(lens) * w.num_kv_heads
     graded = sum(graded_bytes_per_layer(w, lens, r, esz) for r in out.rows)
     path_gbs = graded / (ms_per_step * 1e-3) / 1e9
+    # the same kernel against the special-function unit: one exponential per (window row, key) and sweep;
+    # peak = 16 per clock and SM (measured: 15.98) x the SMs of the device x the maximum SM clock
+    exps = w.group * w.window * w.num_kv_heads * (sum(lens) if dominant == "rowstats_tc" else
+                                                   sum(n - w.window for n in lens))
+    sm_count = torch.cuda.get_device_properties(local).multi_processor_count
+    sfu_peak = 16.0 * sm_count * clocks["sm_max_mhz"] * 1e6 if clocks.get("sm_max_mhz") else None
+    sfu = {"unit": "exp/s", "achieved": exps / (dom_ms * 1e-3), "peak": sfu_peak,
+           "frac": exps / (dom_ms * 1e-3) / sfu_peak if sfu_peak else None,
+           "note": "16 ex2 per clock per SM at the maximum clock; the board runs power-capped below it"}
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peak["hbm_gbs"], "traffic": traffic, "peak_source": peak_kind,
                 "bytes_per_launch": dom_bytes, "ms_per_launch": dom_ms,
                 "kernels": {k: {"launches": v[0], "ms_total": v[1]} for k, v in stages.items()},
+                "special_function_unit": sfu,
                 "path": {"graded_bytes_per_step": graded, "achieved": path_gbs, "frac": path_gbs / peak["hbm_gbs"],
                          "frac_of_8TBs": path_gbs / 8000.0}}
 
