@@ -369,7 +369,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  pdl_wait();                                                  // from here on global memory is read and written
+  // Sweep B reads what the kernels before it wrote, so it waits for them here.  Sweep A reads only the caller's
+  // Q and K: it starts at once (beside the tail of the preceding kernels) and waits just before its first write.
+  if (SWEEP == 1) pdl_wait();
 
   // ---- this CTA's contiguous range of work items
   const int32_t* off = SWEEP == 0 ? p.seq.stat_off : p.seq.score_off;
@@ -497,6 +499,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     auto flush_run = [&]() {
       const int r = (two_blocks ? par * 128 : 0) + lane_row;
       if (run_b < 0 || r >= p.rows) return;
+      pdl_wait();                                             // the partials of the call before have been merged
       const int slots = two_blocks ? 2 : 4;
       const int slot = two_blocks ? ch : grp;
       const int64_t seg = static_cast<int64_t>(blockIdx.x) + run_b * p.num_kv_heads + run_h;
@@ -640,6 +643,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   }
 
   // ---- teardown
+  if (SWEEP == 0) pdl_wait();                                  // never finish before the kernels ahead in the stream
   tc_fence_before();
   __syncthreads();
   if (threadIdx.x == 0 && *abort_flag) atomicOr(p.status, kStatusWaitExpired);
