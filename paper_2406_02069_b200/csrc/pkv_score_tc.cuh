@@ -369,9 +369,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  // Sweep B reads what the kernels before it wrote, so it waits for them here.  Sweep A reads only the caller's
-  // Q and K: it starts at once (beside the tail of the preceding kernels) and waits just before its first write.
-  if (SWEEP == 1) pdl_wait();
+  // Neither sweep waits here for the kernels ahead of it in the stream: copies and MMAs touch only the caller's Q
+  // and K, so they start at once, beside the tail of those kernels.  Sweep A waits just before its first write
+  // (its partials), sweep B's epilogue just before it reads the row normalisers; both wait again before they end.
 
   // ---- this CTA's contiguous range of work items
   const int32_t* off = SWEEP == 0 ? p.seq.stat_off : p.seq.score_off;
@@ -582,6 +582,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         // window rows (columns) of a key and group ch = 1 hands its partial sum to group ch = 0.
         float* lse_s = lse_all + e * 256;                     // this warp's private copy of lse2
         if (w.b != cur_b || w.h != cur_h) {
+          pdl_wait();                                         // the normalisers are written by the kernel before
           __syncwarp();
           const float* src = p.lse2 + (static_cast<int64_t>(w.b) * p.num_kv_heads + w.h) * p.rows;
           for (int i = lane; i < 256; i += 32)       // stored negated: the epilogue adds it
@@ -643,7 +644,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   }
 
   // ---- teardown
-  if (SWEEP == 0) pdl_wait();                                  // never finish before the kernels ahead in the stream
+  pdl_wait();                                                  // never finish before the kernels ahead in the stream
   tc_fence_before();
   __syncthreads();
   if (threadIdx.x == 0 && *abort_flag) atomicOr(p.status, kStatusWaitExpired);
