@@ -25,6 +25,12 @@
  *     device to size a buffer.
  *   - Sequences of a batch are independent; each has its own length n_b.
  *     P_b = n_b - alpha is its prefix length.
+ *   - Kernels of consecutive calls on one stream overlap at their edges (programmatic dependent
+ *     launch).  In particular the score kernels begin to read q_win and k while kernels of THIS
+ *     library enqueued just before them are still running; the library orders them itself when
+ *     q_win or k lies inside a cache or page pool that one of its recent calls writes.  Work of
+ *     the caller's own (ordinary kernel launches, copies) is always finished before a kernel of
+ *     the library that follows it on the stream starts.
  *
  * Tensor layout
  *   K, V     [batch][H_kv][n_max][d]   element strides given per tensor

@@ -182,6 +182,32 @@ void mark(cudaStream_t st, const char* name) {
   cudaEventRecord(g_timer->ev[++g_timer->n], st);
 }
 
+// ---------------------------------------------------------------- outputs still in flight
+// The tensor-core sweeps start reading Q and K before the kernels ahead of them in the stream have finished.
+// That is only right for tensors those kernels do not write, so the library remembers where its last calls put
+// K/V rows (packed caches, page pools) and a sweep whose Q or K overlaps one of them waits like any other kernel.
+struct ByteRange { uintptr_t lo, hi; };
+std::mutex g_out_mutex;
+ByteRange g_recent_out[16];
+unsigned g_recent_out_next = 0;
+
+void note_output(const void* ptr, size_t bytes) {
+  if (!ptr || !bytes) return;
+  std::lock_guard<std::mutex> lock(g_out_mutex);
+  const uintptr_t lo = reinterpret_cast<uintptr_t>(ptr);
+  g_recent_out[g_recent_out_next++ % 16] = ByteRange{lo, lo + bytes};
+}
+
+bool overlaps_recent_output(const pkv_tensor& t, int batch, int heads, int tokens, int d, int elem_bytes) {
+  const int64_t last = (batch - 1) * std::max<int64_t>(t.stride_batch, 0) +
+                       (heads - 1) * std::max<int64_t>(t.stride_head, 0) + (tokens - 1) * t.stride_token + d;
+  const uintptr_t lo = reinterpret_cast<uintptr_t>(t.ptr), hi = lo + static_cast<uintptr_t>(last) * elem_bytes;
+  std::lock_guard<std::mutex> lock(g_out_mutex);
+  for (const ByteRange& r : g_recent_out)
+    if (r.hi > r.lo && lo < r.hi && r.lo < hi) return true;
+  return false;
+}
+
 // ---------------------------------------------------------------- scores
 template <typename T, int D>
 int launch_scores_generic(ScoreParams& sp, int batch, cudaStream_t st) {
@@ -289,6 +315,8 @@ int launch_scores_tc(const pkv_config* c, const pkv_tensor& q, const pkv_tensor&
   tp.rows = sp.rows;
   tp.rows_pad = (sp.rows + 31) / 32 * 32;
   tp.fp16 = fp16 ? 1 : 0;
+  tp.early = (overlaps_recent_output(q, batch, c->num_q_heads, c->window, D, 2) ||
+              overlaps_recent_output(k, batch, c->num_kv_heads, max_n, D, 2)) ? 0 : 1;
   tp.row_blocks = (sp.rows + 127) / 128;
   tp.scale_log2 = sp.scale_log2;
   tp.partial = sp.partial;
@@ -453,6 +481,13 @@ int run_select(const pkv_config* c, const float* scores, int64_t ld, const SeqTa
                     : (multi ? (wide ? pool_select_kernel<false, true, 8> : pool_select_kernel<false, true, 1>)
                              : (wide ? pool_select_kernel<false, false, 8> : pool_select_kernel<false, false, 1>));
   if (cudaLaunchKernelEx(&cfg, kernel, sp) != cudaSuccess) return PKV_ERR_CUDA;
+  if (k_out) {
+    int64_t out_rows = 0;
+    for (int b = 0; b < batch; ++b) out_rows += static_cast<int64_t>(c->num_kv_heads) * table.count[b];
+    const size_t out_bytes = static_cast<size_t>(out_rows) * c->head_dim * sp.elem_bytes;
+    note_output(k_out, out_bytes);
+    note_output(v_out, out_bytes);
+  }
   mark(st, k_out ? "pool_select_gather" : "pool_select");
   return check_launch();
 }
@@ -475,6 +510,8 @@ int run_gather(const pkv_config* c, const pkv_tensor& k, const pkv_tensor& v, co
   if (threads == 0) return PKV_OK;
   const unsigned blocks = static_cast<unsigned>((threads + kGatherThreads - 1) / kGatherThreads);
   launch_pdl(gather_rows_kernel, blocks, kGatherThreads, 0, st, gp);
+  note_output(k_out, static_cast<size_t>(total_rows) * c->head_dim * gp.elem_bytes);
+  note_output(v_out, static_cast<size_t>(total_rows) * c->head_dim * gp.elem_bytes);
   mark(st, "gather_rows");
   return check_launch();
 }
@@ -514,6 +551,9 @@ int run_gather_paged(const pkv_config* c, const pkv_tensor& k, const pkv_tensor&
   if (threads == 0) return PKV_OK;
   const unsigned blocks = static_cast<unsigned>((threads + kPagedThreads - 1) / kPagedThreads);
   launch_pdl(gather_paged_kernel, blocks, kPagedThreads, 0, st, gp);
+  const size_t pool_bytes = static_cast<size_t>(num_pages) * page_size * c->head_dim * gp.elem_bytes;
+  note_output(k_pool, pool_bytes);
+  note_output(v_pool, pool_bytes);
   mark(st, "gather_paged");
   return check_launch();
 }
@@ -1006,6 +1046,8 @@ int pyramidkv_shard_gather(const pkv_config* cfg, pkv_tensor k_shard, pkv_tensor
   if (threads == 0) return PKV_OK;
   launch_pdl(gather_shard_kernel, static_cast<unsigned>((threads + kShardThreads - 1) / kShardThreads), kShardThreads,
              0, static_cast<cudaStream_t>(stream), gp);
+  note_output(k_out, static_cast<size_t>(rows) * cfg->head_dim * eb);
+  note_output(v_out, static_cast<size_t>(rows) * cfg->head_dim * eb);
   return check_launch();
 }
 

@@ -49,6 +49,7 @@ struct TcParams {
   int32_t num_kv_heads, group, rows;      // rows = group * alpha (R)
   int32_t rows_pad;             // R rounded up to 32
   int32_t fp16;                 // 1: Q and K hold binary16, 0: bfloat16 (both operands always share the type)
+  int32_t early;                // 1: Q and K are not outputs of a library kernel that may still run: start at once
   int32_t row_blocks;           // ceil(R / 128): M-blocks of sweep A
   int32_t chunk_tiles_a;        // 256-key tiles per work item of sweep A
   int32_t chunk_tiles_b;        // 128-key tiles per work item of sweep B
@@ -372,6 +373,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   // Neither sweep waits here for the kernels ahead of it in the stream: copies and MMAs touch only the caller's Q
   // and K, so they start at once, beside the tail of those kernels.  Sweep A waits just before its first write
   // (its partials), sweep B's epilogue just before it reads the row normalisers; both wait again before they end.
+  // (When Q or K may be the output of a library kernel still in flight, e.g. a compact cache that is compressed
+  // again, the host clears `early` and the kernel waits here like any other.)
+  if (!p.early) pdl_wait();
 
   // ---- this CTA's contiguous range of work items
   const int32_t* off = SWEEP == 0 ? p.seq.stat_off : p.seq.score_off;

@@ -408,3 +408,43 @@ def test_device_errors_are_reported_not_raised_as_faults():
         pkv.score_window(cfg, x.q_win, x.k, [512], torch.zeros(1, 2, 512, device=DEV), ws[:1024])
     assert e.value.status == binding.PKV_ERR_WORKSPACE
     pkv.check_status(ws)
+
+
+def test_compressing_a_compact_cache_again_sees_the_finished_rows():
+    """The score sweeps start before the kernels ahead of them finish, which is only right for inputs those
+    kernels do not write.  Here the second call's K and V ARE the first call's outputs, back to back on one
+    stream: the library must notice and order them, so the result equals the one taken after a full stop."""
+    w = workloads.scaled(workloads.LLAMA3_8B, num_layers=2, seq_len=9000, name="llama3_8b_9k")
+    cfg = pkv.config_of(w)
+    lens = w.seq_lens()
+    kl = pkv.layer_budgets(cfg)[0]
+    x = workloads.make_layer(w, 0, device=DEV)
+    ws = pkv.new_workspace(cfg, 1, max(lens), DEV)
+    c1 = pkv.kept_count(cfg, kl, lens[0])
+    k1 = torch.empty(w.num_kv_heads * c1, w.head_dim, dtype=x.k.dtype, device=DEV)
+    v1 = torch.empty_like(k1)
+    i1 = torch.empty(w.num_kv_heads * c1, dtype=torch.int32, device=DEV)
+    # second stage: the compact cache (969 rows per head) compressed to a 128-row budget
+    cfg2 = pkv.make_config(num_layers=1, num_q_heads=w.num_q_heads, num_kv_heads=w.num_kv_heads, head_dim=w.head_dim,
+                           window=w.window, pool_kernel=w.pool_kernel, dtype="bf16", avg_budget=128, beta=1.0)
+    c2 = pkv.kept_count(cfg2, 96, c1)
+    ws2 = pkv.new_workspace(cfg2, 1, c1, DEV)
+    outs = []
+    for settle in (True, False, False, False):
+        k1.zero_(); v1.zero_()
+        k2 = torch.zeros(w.num_kv_heads * c2, w.head_dim, dtype=x.k.dtype, device=DEV)
+        v2 = torch.zeros_like(k2)
+        i2 = torch.zeros(w.num_kv_heads * c2, dtype=torch.int32, device=DEV)
+        torch.cuda.synchronize()
+        pkv.compress_layer(cfg, 0, x.q_win, x.k, x.v, lens, k1, v1, i1, ws)
+        if settle:
+            torch.cuda.synchronize()
+        pkv.compress_layer(cfg2, 0, x.q_win, k1.view(1, w.num_kv_heads, c1, w.head_dim),
+                           v1.view(1, w.num_kv_heads, c1, w.head_dim), [c1], k2, v2, i2, ws2)
+        torch.cuda.synchronize()
+        pkv.check_status(ws)
+        pkv.check_status(ws2)
+        outs.append((i2.clone(), k2.clone(), v2.clone()))
+    for got in outs[1:]:
+        assert all(torch.equal(a, b) for a, b in zip(got, outs[0]))
+    assert int(outs[0][0].max()) == c1 - 1 and (outs[0][1] != 0).any()
