@@ -100,3 +100,29 @@ def test_two_lanes_give_the_per_layer_results(w):
             assert torch.equal(got.idx[l], want.idx[l]), "layer %d" % l
             assert torch.equal(got.k[l], want.k[l]) and torch.equal(got.v[l], want.v[l])
     lanes.close()
+
+
+@pytest.mark.parametrize("w", [
+    workloads.scaled(workloads.LLAMA3_8B, num_layers=8, seq_len=9001, name="llama3_8b_9k"),
+    workloads.scaled(workloads.LLAMA2_7B, num_layers=8, seq_len=1500, name="llama2_7b_1k5"),
+], ids=lambda w: w.name)
+def test_back_to_back_passes_share_one_workspace_without_races(w):
+    """Kernels of consecutive layers overlap at their edges (the sweeps of a layer start while the selection of
+    the layer before still runs) and all layers share one workspace: many passes enqueued without a pause must
+    reproduce, in every layer, what a pass with a full stop after every layer gives."""
+    cfg = pkv.config_of(w)
+    lens = w.seq_lens()
+    layers = [workloads.make_layer(w, l, device=DEV) for l in range(w.num_layers)]
+    ws = pkv.new_workspace(cfg, len(lens), max(lens), DEV)
+    want = streaming.LayerOutputs(cfg, lens, w.torch_dtype())
+    for l, x in enumerate(layers):
+        pkv.compress_layer(cfg, l, x.q_win, x.k, x.v, lens, want.k[l], want.v[l], want.idx[l], ws)
+        torch.cuda.synchronize()
+    got = streaming.LayerOutputs(cfg, lens, w.torch_dtype())
+    for rep in range(25):
+        streaming.compress_model(cfg, layers, lens, got, ws)
+    torch.cuda.synchronize()
+    pkv.check_status(ws)
+    for l in range(w.num_layers):
+        assert torch.equal(got.idx[l], want.idx[l]), "layer %d" % l
+        assert torch.equal(got.k[l], want.k[l]) and torch.equal(got.v[l], want.v[l])
