@@ -448,3 +448,38 @@ def test_compressing_a_compact_cache_again_sees_the_finished_rows():
     for got in outs[1:]:
         assert all(torch.equal(a, b) for a, b in zip(got, outs[0]))
     assert int(outs[0][0].max()) == c1 - 1 and (outs[0][1] != 0).any()
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+def test_token_major_and_fused_layouts_give_the_contiguous_result(dtype):
+    """K/V/Q as other frameworks store them: token-major [batch][n][heads][d] and K, V interleaved in one
+    buffer.  Only the strides in the tensor descriptors differ; the outputs must not."""
+    w = workloads.scaled(workloads.LLAMA3_8B, num_layers=2, seq_len=3001, name="llama3_8b_3k", dtype=dtype)
+    cfg = pkv.config_of(w)
+    lens = [3001, 1777]
+    x = workloads.make_layer(w, 1, device=DEV, seq_lens=lens)
+    kl = pkv.layer_budgets(cfg)[1]
+    rows = pkv.total_rows(cfg, kl, lens)
+    ws = pkv.new_workspace(cfg, len(lens), max(lens), DEV)
+
+    def run(q, k, v):
+        k_out = torch.empty(rows, w.head_dim, dtype=x.k.dtype, device=DEV)
+        v_out = torch.empty_like(k_out)
+        idx = torch.empty(rows, dtype=torch.int32, device=DEV)
+        scores = torch.zeros(len(lens), w.num_kv_heads, max(lens), dtype=torch.float32, device=DEV)
+        pkv.compress_layer(cfg, 1, q, k, v, lens, k_out, v_out, idx, ws, scores=scores)
+        pkv.check_status(ws)
+        return scores.cpu(), idx.cpu(), k_out.cpu(), v_out.cpu()
+
+    want = run(x.q_win, x.k, x.v)
+    # token-major storage, viewed head-major
+    k_tm = x.k.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    v_tm = x.v.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    q_tm = x.q_win.permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    assert not k_tm.is_contiguous() and k_tm.stride(1) == w.head_dim
+    got = run(q_tm, k_tm, v_tm)
+    assert all(torch.equal(a, b) for a, b in zip(got, want))
+    # K and V interleaved per token in one buffer
+    kv = torch.stack([x.k, x.v], dim=3).contiguous()                  # [batch][H][n][2][d]
+    got = run(x.q_win, kv[:, :, :, 0], kv[:, :, :, 1])
+    assert all(torch.equal(a, b) for a, b in zip(got, want))
