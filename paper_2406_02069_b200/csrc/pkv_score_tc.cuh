@@ -151,6 +151,15 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
       : "r"(taddr)
       : "memory");
 }
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&v)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+      : "r"(taddr)
+      : "memory");
+}
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ float ex2(float x) {
   float y;
@@ -159,38 +168,23 @@ __device__ __forceinline__ float ex2(float x) {
 }
 
 // The special-function unit evaluates 16 exponentials per clock per SM, which is what bounds both
-// sweeps.  Every kTcPolyEvery-th exponential is therefore evaluated on the FMA pipe instead:
+// sweeps when every 2^x goes through it.  A fixed share of the exponentials is therefore evaluated on
+// the FMA pipe instead, two at a time with the packed fp32 instructions:
 // 2^x = 2^n * 2^f with n = round(x), f = x - n in [-0.5, 0.5]; 2^f by a cubic minimax polynomial
 // (largest relative error 7.5e-5, far inside the 2e-3 the scores are held to); 2^n by adding n to the
 // exponent field.  x is clamped to [-126, 127.5] so the exponent arithmetic cannot wrap.
-#ifndef PKV_POLY_EVERY
-#define PKV_POLY_EVERY 0
+// Of every eight consecutive pairs of values, kTcPolyPairs go this way (spread evenly over the eight).
+#ifndef PKV_POLY_PAIRS
+#define PKV_POLY_PAIRS 3
 #endif
-constexpr int kTcPolyEvery = PKV_POLY_EVERY;    // 0 = never
-
-template <bool kClampHigh>
-__device__ __forceinline__ float ex2_poly(float x) {
-  x = fmaxf(x, -126.0f);
-  if (kClampHigh) x = fminf(x, 127.5f);
-  const float t = x + 12582912.0f;              // 1.5 * 2^23: the low mantissa bits now hold round(x)
-  const float nf = t - 12582912.0f;
-  const float f = x - nf;
-  float q = fmaf(f, 0.0551716685295105f, 0.2426111251115799f);
-  q = fmaf(q, f, 0.6932609677314758f);
-  q = fmaf(q, f, 0.9999280571937561f);
-  // q * 2^n: add n to the exponent field.  The multiply-add form keeps this on the FMA pipe.
-  int bits;
-  asm("mad.lo.s32 %0, %1, 8388608, %2;" : "=r"(bits) : "r"(__float_as_int(t)), "r"(__float_as_int(q)));
-  return __int_as_float(bits);
-}
-template <bool kClampHigh>
-__device__ __forceinline__ float ex2_mixed(float x, int j) {
-  return (kTcPolyEvery > 0 && (j % (kTcPolyEvery > 0 ? kTcPolyEvery : 1)) == kTcPolyEvery - 1) ? ex2_poly<kClampHigh>(x)
-                                                                                              : ex2(x);
+constexpr int kTcPolyPairs = PKV_POLY_PAIRS;    // 0 = every exponential on the special-function unit
+__host__ __device__ constexpr bool tc_pair_is_poly(int pair) {
+  return ((pair % 8 + 1) * kTcPolyPairs) / 8 != ((pair % 8) * kTcPolyPairs) / 8;
 }
 
 // Packed pairs of fp32 (one instruction for two multiply-adds or two adds): the scale-and-shift in front
-// of each exponential and the accumulation behind it go through these, which halves their issue slots.
+// of each exponential, the polynomial and the accumulation behind it go through these, which halves
+// their issue slots.
 __device__ __forceinline__ unsigned long long pack2(float lo, float hi) {
   unsigned long long r;
   asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
@@ -210,51 +204,93 @@ __device__ __forceinline__ unsigned long long add2(unsigned long long a, unsigne
   return d;
 }
 
-// Sweep A, 32 logits of one window row: z += sum_j 2^(v_j * c2 - m).  m is a reference exponent, not
-// necessarily the running maximum: it is only moved when a group's sum is not a moderate finite
-// number (the row's first group, where m = -inf, or a logit ~60 binades above the reference).
-__device__ __forceinline__ void rowstats_group(const uint32_t (&v)[32], float c2, float& m, float& z) {
-  const unsigned long long cc = pack2(c2, c2), mm = pack2(-m, -m);
-  unsigned long long acc01 = pack2(0.f, 0.f), acc23 = acc01;
-#pragma unroll
-  for (int j = 0; j < 32; j += 4) {
-    float x0, x1, x2, x3;
-    unpack2(fma2(pack2(__uint_as_float(v[j]), __uint_as_float(v[j + 1])), cc, mm), x0, x1);
-    unpack2(fma2(pack2(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3])), cc, mm), x2, x3);
-    acc01 = add2(acc01, pack2(ex2_mixed<true>(x0, j), ex2_mixed<true>(x1, j + 1)));
-    acc23 = add2(acc23, pack2(ex2_mixed<true>(x2, j + 2), ex2_mixed<true>(x3, j + 3)));
+// 2^x0 and 2^x1 (packed) on the FMA pipe; both already clamped to [-126, 127.5].
+__device__ __forceinline__ unsigned long long ex2_poly2(float x0, float x1) {
+  const float kMagic = 12582912.0f;             // 1.5 * 2^23: adding it leaves round(x) in the low mantissa bits
+  const unsigned long long x = pack2(x0, x1);
+  const unsigned long long t = add2(x, pack2(kMagic, kMagic));
+  const unsigned long long n = add2(t, pack2(-kMagic, -kMagic));
+  const unsigned long long f = fma2(n, pack2(-1.0f, -1.0f), x);
+  unsigned long long q = fma2(f, pack2(0.0551716685295105f, 0.0551716685295105f),
+                              pack2(0.2426111251115799f, 0.2426111251115799f));
+  q = fma2(q, f, pack2(0.6932609677314758f, 0.6932609677314758f));
+  q = fma2(q, f, pack2(0.9999280571937561f, 0.9999280571937561f));
+  float t0, t1, q0, q1;
+  unpack2(t, t0, t1);
+  unpack2(q, q0, q1);
+  // q * 2^n: add n to the exponent field
+  const int r0 = __float_as_int(q0) + (__float_as_int(t0) << 23);
+  const int r1 = __float_as_int(q1) + (__float_as_int(t1) << 23);
+  return pack2(__int_as_float(r0), __int_as_float(r1));
+}
+// The pair (2^x0, 2^x1), by the unit the pair's position in its group of eight selects.
+template <bool kClampHigh>
+__device__ __forceinline__ unsigned long long ex2_pair(float x0, float x1, int pair) {
+  if (tc_pair_is_poly(pair)) {
+    x0 = fmaxf(x0, -126.0f);
+    x1 = fmaxf(x1, -126.0f);
+    if (kClampHigh) { x0 = fminf(x0, 127.5f); x1 = fminf(x1, 127.5f); }
+    return ex2_poly2(x0, x1);
   }
-  float a0, a1, a2, a3;
-  unpack2(acc01, a0, a1);
-  unpack2(acc23, a2, a3);
-  float g = (a0 + a1) + (a2 + a3);
-  if (!(g < 1.0e18f)) {
-    float gm = __uint_as_float(v[0]);
+  return pack2(ex2(x0), ex2(x1));
+}
+
+// Sweep A, N logits of one window row, fast path: acc += 2^(v_j * c2 - m) in four packed pairs of partial
+// sums.  m is a reference exponent, not necessarily the running maximum; the caller adds the partial sums up
+// once per accumulator chunk and falls back to rowstats_rescue when the total is not a moderate finite number.
+template <int N>
+__device__ __forceinline__ void rowstats_accumulate(const uint32_t (&v)[N], unsigned long long cc,
+                                                    unsigned long long mm, unsigned long long (&acc)[4]) {
 #pragma unroll
-    for (int j = 1; j < 32; ++j) gm = fmaxf(gm, __uint_as_float(v[j]));
-    const float mn = fmaxf(m, gm * c2);
-    z *= ex2(m - mn);
-    m = mn;
-    g = 0.f;
+  for (int j = 0; j < N; j += 8) {
+    float x[8];
 #pragma unroll
-    for (int j = 0; j < 32; ++j) g += ex2(fmaf(__uint_as_float(v[j]), c2, -m));
+    for (int q = 0; q < 4; ++q)
+      unpack2(fma2(pack2(__uint_as_float(v[j + 2 * q]), __uint_as_float(v[j + 2 * q + 1])), cc, mm), x[2 * q],
+              x[2 * q + 1]);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) acc[q] = add2(acc[q], ex2_pair<true>(x[2 * q], x[2 * q + 1], j / 2 + q));
   }
+}
+__device__ __forceinline__ float sum_pairs(const unsigned long long (&acc)[4]) {
+  float a[8];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) unpack2(acc[q], a[2 * q], a[2 * q + 1]);
+  return ((a[0] + a[1]) + (a[2] + a[3])) + ((a[4] + a[5]) + (a[6] + a[7]));
+}
+// Sweep A, slow path for the same N logits: moves the reference exponent to the running maximum first
+// (the row's first chunk, where m = -inf, or a logit some 60 binades above the reference).
+template <int N>
+__device__ __forceinline__ void rowstats_rescue(const uint32_t (&v)[N], float c2, float& m, float& z) {
+  float gm = __uint_as_float(v[0]);
+#pragma unroll
+  for (int j = 1; j < N; ++j) gm = fmaxf(gm, __uint_as_float(v[j]));
+  const float mn = fmaxf(m, gm * c2);
+  z *= ex2(m - mn);
+  m = mn;
+  float g = 0.f;
+#pragma unroll
+  for (int j = 0; j < N; ++j) g += ex2(fmaf(__uint_as_float(v[j]), c2, -m));
   z += g;
 }
 
-// Sweep B, 32 window rows of one key: acc += 2^(v_j * c2 + nlse_j); nlse = -lse2 sits in shared memory
-// (negated when it was loaded), acc holds two packed pairs of partial sums.
-__device__ __forceinline__ void score_group(const uint32_t (&v)[32], float c2, const float* nlse,
-                                            unsigned long long (&acc)[2]) {
-  const unsigned long long cc = pack2(c2, c2);
+// Sweep B, N window rows of one key: acc += 2^(v_j * c2 + nlse_j); nlse = -lse2 sits in shared memory
+// (negated when it was loaded), acc holds four packed pairs of partial sums.
+template <int N>
+__device__ __forceinline__ void score_group(const uint32_t (&v)[N], unsigned long long cc, const float* nlse,
+                                            unsigned long long (&acc)[4]) {
 #pragma unroll
-  for (int j = 0; j < 32; j += 4) {
-    const ulonglong2 l4 = *reinterpret_cast<const ulonglong2*>(nlse + j);     // four floats as two packed pairs
-    float x0, x1, x2, x3;
-    unpack2(fma2(pack2(__uint_as_float(v[j]), __uint_as_float(v[j + 1])), cc, l4.x), x0, x1);
-    unpack2(fma2(pack2(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3])), cc, l4.y), x2, x3);
-    acc[0] = add2(acc[0], pack2(ex2_mixed<false>(x0, j), ex2_mixed<false>(x1, j + 1)));
-    acc[1] = add2(acc[1], pack2(ex2_mixed<false>(x2, j + 2), ex2_mixed<false>(x3, j + 3)));
+  for (int j = 0; j < N; j += 8) {
+    const ulonglong2 la = *reinterpret_cast<const ulonglong2*>(nlse + j);     // eight floats as four packed pairs
+    const ulonglong2 lb = *reinterpret_cast<const ulonglong2*>(nlse + j + 4);
+    const unsigned long long l[4] = {la.x, la.y, lb.x, lb.y};
+    float x[8];
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      unpack2(fma2(pack2(__uint_as_float(v[j + 2 * q]), __uint_as_float(v[j + 2 * q + 1])), cc, l[q]), x[2 * q],
+              x[2 * q + 1]);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) acc[q] = add2(acc[q], ex2_pair<false>(x[2 * q], x[2 * q + 1], j / 2 + q));
   }
 }
 
@@ -545,11 +581,31 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
             if (!warp_has_rows) {
               // only the hand-shake below
             } else if (key_base + 127 <= min(P, n - 1)) {     // every key visible to every row: no mask
+              // fast path over the 128 columns; the sums are only looked at once, at the end
+              const unsigned long long cc = pack2(c2, c2), mm = pack2(-m, -m);
+              unsigned long long acc[4] = {pack2(0.f, 0.f), pack2(0.f, 0.f), pack2(0.f, 0.f), pack2(0.f, 0.f)};
+              // 16-column loads, double buffered: the next load is in flight while a group is evaluated
+              uint32_t va[16], vb[16];
+              tc_ld16(taddr, va);
+#pragma unroll
               for (int cg = 0; cg < 128; cg += 32) {
-                uint32_t v[32];
-                tc_ld32(taddr + cg, v);
                 tc_wait_ld();
-                rowstats_group(v, c2, m, z);
+                tc_ld16(taddr + cg + 16, vb);
+                rowstats_accumulate(va, cc, mm, acc);
+                tc_wait_ld();
+                if (cg + 32 < 128) tc_ld16(taddr + cg + 32, va);
+                rowstats_accumulate(vb, cc, mm, acc);
+              }
+              const float g = sum_pairs(acc);
+              if (g < 1.0e18f) {
+                z += g;
+              } else {                                        // rare: read the columns again, slow path
+                for (int cg = 0; cg < 128; cg += 32) {
+                  uint32_t v[32];
+                  tc_ld32(taddr + cg, v);
+                  tc_wait_ld();
+                  rowstats_rescue(v, c2, m, z);
+                }
               }
             } else {
               for (int cg = 0; cg < 128; cg += 32) {
@@ -606,20 +662,24 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
           if (!ok) break;
           tc_fence_after();
           const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + ts * stage_cols;
-          unsigned long long acc[2] = {pack2(0.f, 0.f), pack2(0.f, 0.f)};
-          for (int cg = col0; cg < col1; cg += 32) {
-            uint32_t v[32];
-            tc_ld32(taddr + cg, v);
-            tc_wait_ld();
-            score_group(v, c2, lse_s + cg, acc);
+          unsigned long long acc[4] = {pack2(0.f, 0.f), pack2(0.f, 0.f), pack2(0.f, 0.f), pack2(0.f, 0.f)};
+          const unsigned long long cc = pack2(c2, c2);
+          {
+            uint32_t va[16], vb[16];
+            tc_ld16(taddr + col0, va);
+            for (int cg = col0; cg < col1; cg += 32) {
+              tc_wait_ld();
+              tc_ld16(taddr + cg + 16, vb);
+              score_group(va, cc, lse_s + cg, acc);
+              tc_wait_ld();
+              if (cg + 32 < col1) tc_ld16(taddr + cg + 32, va);
+              score_group(vb, cc, lse_s + cg + 16, acc);
+            }
           }
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(t_empty(ts));
-          float s0, s1, s2, s3;
-          unpack2(acc[0], s0, s1);
-          unpack2(acc[1], s2, s3);
-          float sum = (s0 + s1) + (s2 + s3);
+          float sum = sum_pairs(acc);
           if (second_half) {
             if (ch == 1) {
               ok = mbar_wait(x_empty(par), (mine & 1) ^ 1, abort_flag);
