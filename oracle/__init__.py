@@ -48,6 +48,8 @@ def _load() -> ctypes.CDLL:
         lib.orc_layer_budgets.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_double,
                                           ctypes.c_void_p]
         lib.orc_layer_budgets.restype = ctypes.c_int
+        lib.orc_layer_budgets_geometric.argtypes = lib.orc_layer_budgets.argtypes
+        lib.orc_layer_budgets_geometric.restype = ctypes.c_int
         lib.orc_kept_count.argtypes = [ctypes.c_int] * 4
         lib.orc_kept_count.restype = ctypes.c_int
         lib.orc_window_scores.argtypes = [ctypes.c_void_p, ctypes.c_void_p] + [ctypes.c_int] * 6 + \
@@ -105,10 +107,13 @@ def num_threads() -> int:
     return int(_load().orc_num_threads())
 
 
-def layer_budgets(num_layers: int, avg_budget: int, alpha: int, beta: float = 20.0) -> List[int]:
-    """Eq. 1: per-layer budgets k^l (prefix rows; the alpha window rows come on top)."""
+def layer_budgets(num_layers: int, avg_budget: int, alpha: int, beta: float = 20.0,
+                  schedule: str = "linear") -> List[int]:
+    """Per-layer budgets k^l (prefix rows; the alpha window rows come on top): Eq. 1 ("linear"), or the
+    appendix's geometric decay between the same end constraints ("geometric")."""
     out = np.zeros(num_layers, dtype=np.int32)
-    rc = _load().orc_layer_budgets(num_layers, avg_budget, alpha, float(beta), out.ctypes.data)
+    fn = {"linear": _load().orc_layer_budgets, "geometric": _load().orc_layer_budgets_geometric}[schedule]
+    rc = fn(num_layers, avg_budget, alpha, float(beta), out.ctypes.data)
     if rc != 0:
         raise ValueError("budget schedule undefined for these arguments")
     return [int(x) for x in out]

@@ -7,7 +7,7 @@
 // baseline may use it.
 //
 // Steps, in the paper's order (Section 4.2):
-//   budgets   Section 4.2.1, Eq. 1   pyramidal per-layer budgets k^l
+//   budgets   Section 4.2.1, Eq. 1   pyramidal per-layer budgets k^l (and the appendix's geometric decay)
 //   logits    Section 4.2.2, Eq. 2   A^h = softmax(Q^h K^hT / sqrt(d_k)), window rows only
 //   scores    Section 4.2.2, Eq. 3   s_i = sum over window rows j of A[j][i]
 //   pool      Section 4.2.2          a pooling layer applied to the scores (max, odd width)
@@ -103,6 +103,53 @@ int orc_layer_budgets(int m, int avg_budget, int alpha, double beta, int32_t* k_
     assigned += kl;
   }
   int64_t left = k_total - assigned;                        // 0 <= left < m
+  for (int l = 0; l < m && left > 0; ++l, --left) k_out[l] += 1;
+  return 0;
+}
+
+// ---------------------------------------------------------------------------
+// Appendix "Allocation Strategies": a geometric (equivalently, exponential in the
+// layer index) decay in place of Eq. 1's arithmetic one.  The paper names the
+// strategy without a formula; the reading keeps Eq. 1's two constraints and changes
+// only the shape between them:
+//   real budgets with a constant ratio rho >= 1 between consecutive layers,
+//   x_l = x_{m-1} rho^(m-1-l),   sum_l x_l = k_total,   x_{m-1} = k_total / (beta m),
+// which makes rho the root of  1 + rho + ... + rho^(m-1) = beta m  (unique for rho >= 1;
+// beta = 1 gives rho = 1, the uniform split).  The root is found by bisection and then
+// snapped to the nearest multiple of 2^-20, so that two implementations agree on it
+// bit for bit; with the snapped rho the shares are  x_l = k_total rho^(m-1-l) / sum_j rho^j
+// (powers by repeated multiplication, the sum taken from j = 0 upward, all in double).
+// Flooring and the leftover units follow the linear schedule's rule.
+// Returns 0, or -1 for arguments the schedule is not defined for.
+int orc_layer_budgets_geometric(int m, int avg_budget, int alpha, double beta, int32_t* k_out) {
+  if (m < 1 || alpha < 1 || avg_budget < alpha || !(beta >= 1.0) || beta > 1.0e6) return -1;
+  const int64_t k_total = static_cast<int64_t>(m) * (avg_budget - alpha);
+  const int64_t bq = std::llround(beta * 1024.0);          // beta = bq / 1024
+  double rho = 1.0;
+  if (m > 1 && bq > 1024) {
+    const double target = static_cast<double>(bq) / 1024.0 * m;
+    double lo = 1.0, hi = target;                          // 1 + rho <= sum, so the root is below beta m
+    for (int it = 0; it < 200; ++it) {
+      const double mid = 0.5 * (lo + hi);
+      double sum = 0.0, pw = 1.0;
+      for (int j = 0; j < m; ++j) { sum += pw; pw *= mid; }
+      if (sum < target) lo = mid; else hi = mid;
+    }
+    rho = std::round(0.5 * (lo + hi) * 1048576.0) / 1048576.0;
+  }
+  std::vector<double> power(m);
+  double total = 0.0;
+  for (int j = 0; j < m; ++j) {
+    power[j] = j == 0 ? 1.0 : power[j - 1] * rho;
+    total += power[j];
+  }
+  int64_t assigned = 0;
+  for (int l = 0; l < m; ++l) {
+    const int64_t kl = static_cast<int64_t>(std::floor(static_cast<double>(k_total) * power[m - 1 - l] / total));
+    k_out[l] = static_cast<int32_t>(kl);
+    assigned += kl;
+  }
+  int64_t left = k_total - assigned;
   for (int l = 0; l < m && left > 0; ++l, --left) k_out[l] += 1;
   return 0;
 }

@@ -37,9 +37,17 @@ MUTANTS = [
      "out[i] = sum / static_cast<float>(std::min(P - 1, i + r) - std::max(0, i - r) + 1);"),
     ("sort_ascending", "return pooled[a] > pooled[b];", "return pooled[a] < pooled[b];"),
     ("leftover_to_top_layers", "for (int l = 0; l < m && left > 0; ++l, --left) k_out[l] += 1;",
-     "for (int l = m - 1; l >= 0 && left > 0; --l, --left) k_out[l] += 1;"),
+     "for (int l = m - 1; l >= 0 && left > 0; --l, --left) k_out[l] += 1;", 0),
+    ("geometric_leftover_to_top_layers", "for (int l = 0; l < m && left > 0; ++l, --left) k_out[l] += 1;",
+     "for (int l = m - 1; l >= 0 && left > 0; --l, --left) k_out[l] += 1;", 1),
     ("pyramid_over_whole_budget", "const int64_t k_total = static_cast<int64_t>(m) * (avg_budget - alpha);",
-     "const int64_t k_total = static_cast<int64_t>(m) * avg_budget;"),
+     "const int64_t k_total = static_cast<int64_t>(m) * avg_budget;", 0),
+    ("geometric_over_whole_budget", "const int64_t k_total = static_cast<int64_t>(m) * (avg_budget - alpha);",
+     "const int64_t k_total = static_cast<int64_t>(m) * avg_budget;", 1),
+    ("geometric_grows_with_depth", "power[m - 1 - l] / total", "power[l] / total"),
+    ("geometric_top_layer_rule", "static_cast<double>(bq) / 1024.0 * m;", "static_cast<double>(bq) / 1024.0;"),
+    ("geometric_ratio_not_snapped", "rho = std::round(0.5 * (lo + hi) * 1048576.0) / 1048576.0;",
+     "rho = std::round(0.5 * (lo + hi) * 1024.0) / 1024.0;"),
     ("slope_sign", "static_cast<__int128>(2 * bq - 2048) * l;", "static_cast<__int128>(2048 - 2 * bq) * l;"),
     ("short_context_still_compressed", "if (n <= avg_budget) return n;", "if (n <= alpha) return n;"),
     ("window_dropped", "for (int i = P; i < n; ++i) row[cnt++] = i;", "for (int i = P; i < n; ++i) row[cnt++] = P;"),
