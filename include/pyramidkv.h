@@ -75,6 +75,9 @@ extern "C" {
 #define PKV_POOL_AVG 1            /* centred mean: zeros outside the prefix, always divided by the width; float
                                      additions left to right, then one float division (it decides the top-k) */
 
+#define PKV_SCHEDULE_LINEAR 0      /* Eq. 1: arithmetic decrease from the lowest layer to the top one */
+#define PKV_SCHEDULE_GEOMETRIC 1   /* appendix "Allocation Strategies": constant ratio between consecutive layers */
+
 #define PKV_MAX_BATCH 64          /* sequences per call */
 #define PKV_MAX_STAGES 8          /* kernels one pyramidkv_compress_layer call may launch */
 #define PKV_STATIC_SCRATCH_BYTES (8u << 20)  /* built-in scratch of pyramidkv_score_window_static: 8 MiB per GPU */
@@ -89,7 +92,7 @@ typedef struct pkv_config {
   int32_t pool_kind;     /* PKV_POOL_MAX or PKV_POOL_AVG */
   int32_t dtype;         /* PKV_DTYPE_*: element type shared by K, V and Q_win */
   int32_t avg_budget;    /* B: mean rows kept per layer and KV head, window rows included; >= alpha */
-  int32_t reserved;      /* must be 0 */
+  int32_t schedule;      /* PKV_SCHEDULE_*: shape of the per-layer budgets; 0 = Eq. 1 */
   double  beta;          /* pyramid shape, >= 1 (Section 4.2.1); 1 = same size in every layer */
 } pkv_config;
 
@@ -131,6 +134,14 @@ const char* pyramidkv_strerror(int status);
  * evaluated in integers: every k^l is floored and the units lost to flooring go
  * one each to layers 0, 1, ... so that the budgets are non-increasing and sum to
  * k_total exactly.  m = 1 gives k^0 = k_total.
+ *
+ * cfg->schedule = PKV_SCHEDULE_GEOMETRIC selects the geometric (exponential in the layer index) decay that
+ * the appendix "Allocation Strategies" compares Eq. 1 with.  The paper gives it no formula; here it keeps
+ * Eq. 1's two constraints (top layer k_total / (beta m), budgets sum to k_total) and puts a constant ratio
+ * rho >= 1 between consecutive layers: rho is the root of 1 + rho + ... + rho^(m-1) = beta m, rounded to a
+ * multiple of 2^-20, and layer l gets k_total * rho^(m-1-l) / (1 + rho + ... + rho^(m-1)), floored, leftover
+ * units to layers 0, 1, ... as above.  beta = 1 is the uniform split under both schedules; with m = 2 the
+ * two schedules coincide.
  *   k_out  host, [num_layers]: rows of the prefix layer l may keep (window rows come on top).
  * Errors: PKV_ERR_INVALID_ARG for a null pointer or a config outside the ranges above.
  */
@@ -207,6 +218,15 @@ int pyramidkv_score_window_static(const pkv_config* cfg, pkv_tensor q_win, pkv_t
                                   float* scores, int64_t ld_scores, void* stream);
 
 /*
+ * pyramidkv_check_status for the built-in scratch (the paper has no counterpart): the status word of
+ * pyramidkv_score_window_static lives at the head of the library's own array, where the caller has no
+ * pointer to it.  Synchronises `stream`, copies the word out and returns PKV_OK or
+ * PKV_ERR_DEVICE_STATUS (word in *detail_or_null); PKV_ERR_CUDA if the array cannot be reached.
+ * Allocates nothing.
+ */
+int pyramidkv_check_status_static(void* stream, uint32_t* detail_or_null);
+
+/*
  * Pooling and selection, Section 4.2.2.  Per sequence and KV head:
  * pooled[i] = max of scores[i + t] over |t| <= (pool_kernel - 1)/2 clipped to [0, P_b);
  * the min(k_layer, P_b) positions with the largest pooled value are kept, ties
@@ -228,7 +248,9 @@ int pyramidkv_select_topk(const pkv_config* cfg, const float* scores, int64_t ld
  * addresses from the strides, write a new tensor).  Copies, bit for bit, row
  * indices[r] of K and of V into row r of k_out and v_out.  Out of place: k_out
  * and v_out must not overlap K or V.  v.ptr and v_out may both be NULL to move K only.
- *   indices    device int32, packed rows as written by pyramidkv_select_topk
+ *   indices    device int32, packed rows as written by pyramidkv_select_topk.  An entry outside
+ *              [0, n_b) is never turned into an address: its output row is left as it was.  (This
+ *              call has no workspace, so nothing is recorded; pyramidkv_gather_paged records it.)
  *   k_out,v_out device, [sum_b H_kv * c_b][d] elements of the config dtype, 16-byte aligned
  * Errors: INVALID_ARG, UNSUPPORTED, CUDA.
  */
@@ -296,6 +318,8 @@ int pyramidkv_decode_attention(const pkv_config* cfg, const void* q, const void*
  *     recall[b][h] = 1 - (sum of scores[b][h][i] over evicted prefix positions i) / alpha,
  * since each window row's attention sums to one and the window keys are always kept.
  *   scores, indices  device, as produced for this layer; recall  device, [batch][H_kv] floats
+ * An index entry that is no prefix position of its sequence is not used as an address; it counts as
+ * not kept.
  * Errors: INVALID_ARG, CUDA.
  */
 int pyramidkv_attention_recall(const pkv_config* cfg, const float* scores, int64_t ld_scores,
@@ -345,7 +369,8 @@ int pyramidkv_profile_layer_lse(const pkv_config* cfg, int32_t layer,
  * original position per kept row) keeps the packed layout of pyramidkv_compress_layer.
  *
  * A table entry outside [0, num_pages) is never dereferenced: the row is skipped and the workspace
- * status word gets a bit set (pyramidkv_check_status then returns PKV_ERR_DEVICE_STATUS).
+ * status word gets bit 2 set (pyramidkv_check_status then returns PKV_ERR_DEVICE_STATUS).  An entry of
+ * a caller-supplied index list outside [0, n_b) is treated the same way, with bit 3.
  */
 
 /* Host only.  Pages one KV head of a seq_len-token sequence needs; negative status on bad arguments. */
@@ -463,7 +488,10 @@ int pyramidkv_compress_model_lanes(const pkv_config* cfg, pkv_lanes* lanes, int3
  * Synchronises `stream` and reads the workspace status word.  For tests and
  * debugging.  Returns PKV_OK, PKV_ERR_DEVICE_STATUS (a kernel gave up on a
  * bounded wait or saw an impossible state; *detail_or_null receives the word),
- * or PKV_ERR_CUDA.
+ * or PKV_ERR_CUDA.  Bits of the word: 0 the selection emitted a wrong count,
+ * 1 a bounded wait ran out, 2 a block-table entry outside the pool, 3 an index
+ * entry outside its sequence.  The bits stay set until the caller zeroes the
+ * first 256 bytes of the workspace.
  */
 int pyramidkv_check_status(const void* workspace, void* stream, uint32_t* detail_or_null);
 

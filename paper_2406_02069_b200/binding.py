@@ -1,8 +1,12 @@
 """ctypes binding of libpyramidkv.so: same names as the C boundary, argument marshalling only.
 
 Every step of the path runs in the library's CUDA kernels.  torch supplies device
-memory and the stream, nothing else.  There is no CPU fallback: if the library
-cannot be loaded the import of this module fails.
+memory and the stream, nothing else.  There is no CPU fallback: the library is
+loaded (and built first when it is missing or older than its sources) by the first
+call that needs it, and that call raises if it cannot be.
+
+The wrappers check what the C side cannot see: that the tensors are as large as the
+configuration and the sequence lengths say, of the configured type, and on a device.
 """
 from __future__ import annotations
 
@@ -27,7 +31,8 @@ PKV_STATIC_SCRATCH_BYTES = 8 << 20
 EXPORTS = ("pyramidkv_strerror", "pyramidkv_layer_budgets", "pyramidkv_kept_count",
            "pyramidkv_workspace_bytes", "pyramidkv_score_window", "pyramidkv_select_topk",
            "pyramidkv_gather_compact", "pyramidkv_compress_layer", "pyramidkv_profile_layer",
-           "pyramidkv_check_status", "pyramidkv_score_window_static", "pyramidkv_score_window_lse",
+           "pyramidkv_check_status", "pyramidkv_score_window_static", "pyramidkv_check_status_static",
+           "pyramidkv_score_window_lse",
            "pyramidkv_compress_layer_lse", "pyramidkv_profile_layer_lse", "pyramidkv_decode_attention",
            "pyramidkv_attention_recall", "pyramidkv_pages_needed", "pyramidkv_gather_paged",
            "pyramidkv_compress_layer_paged", "pyramidkv_decode_attention_paged", "pyramidkv_shard_window_lse",
@@ -42,7 +47,7 @@ class PkvConfig(ctypes.Structure):
                 ("num_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32),
                 ("window", ctypes.c_int32), ("pool_kernel", ctypes.c_int32),
                 ("pool_kind", ctypes.c_int32), ("dtype", ctypes.c_int32),
-                ("avg_budget", ctypes.c_int32), ("reserved", ctypes.c_int32),
+                ("avg_budget", ctypes.c_int32), ("schedule", ctypes.c_int32),
                 ("beta", ctypes.c_double)]
 
 
@@ -58,9 +63,7 @@ class PkvError(RuntimeError):
 
 
 def _load() -> ctypes.CDLL:
-    path = _build.LIB
-    if not os.path.exists(path):
-        _build.build_library()
+    path = _build.build_library()          # compiles only when the library is missing or its sources changed
     lib = ctypes.CDLL(path)
     P, I32, I64, SZ = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
     CFG = ctypes.POINTER(PkvConfig)
@@ -98,17 +101,30 @@ def _load() -> ctypes.CDLL:
     lib.pyramidkv_lanes_info.argtypes = [P, ctypes.POINTER(I32), ctypes.POINTER(I32)]
     lib.pyramidkv_compress_model_lanes.argtypes = [CFG, P, I32, I32, P, P, P, P, P, I32, P, P, P, P, SZ, P]
     lib.pyramidkv_check_status.argtypes = [P, P, P]
+    lib.pyramidkv_check_status_static.argtypes = [P, P]
     for name in EXPORTS:
         if name not in ("pyramidkv_strerror", "pyramidkv_workspace_bytes"):
             getattr(lib, name).restype = ctypes.c_int
     return lib
 
 
-_lib = _load()
+class _LazyLibrary:
+    """Loads libpyramidkv.so on first use, so that importing the package (for its input generators, say) maps
+    no native code."""
+    _real = None
+
+    def __getattr__(self, name):
+        if _LazyLibrary._real is None:
+            _LazyLibrary._real = _load()
+        return getattr(_LazyLibrary._real, name)
+
+
+_lib = _LazyLibrary()
 
 
 def library_path() -> str:
-    return _build.LIB
+    """Path of libpyramidkv.so, built first if it is missing or older than its sources."""
+    return _build.build_library()
 
 
 MEM_PAGEABLE_HOST, MEM_PINNED_HOST, MEM_DEVICE, MEM_MANAGED = 0, 1, 2, 3
@@ -127,17 +143,19 @@ def strerror(status: int) -> str:
 
 
 def make_config(*, num_layers: int, num_q_heads: int, num_kv_heads: int, head_dim: int, window: int,
-                pool_kernel: int, dtype: str, avg_budget: int, beta: float = 20.0, pool_kind: int = 0) -> PkvConfig:
+                pool_kernel: int, dtype: str, avg_budget: int, beta: float = 20.0, pool_kind: int = 0,
+                schedule: str = "linear") -> PkvConfig:
     code = {"fp32": 0, "bf16": 1, "fp16": 2, torch.float32: 0, torch.bfloat16: 1, torch.float16: 2}[dtype]
     return PkvConfig(num_layers, num_q_heads, num_kv_heads, head_dim, window, pool_kernel, pool_kind, code,
-                     avg_budget, 0, float(beta))
+                     avg_budget, {"linear": 0, "geometric": 1}[schedule], float(beta))
 
 
 def config_of(w) -> PkvConfig:
     """Config of a workloads.Workload."""
     return make_config(num_layers=w.num_layers, num_q_heads=w.num_q_heads, num_kv_heads=w.num_kv_heads,
                        head_dim=w.head_dim, window=w.window, pool_kernel=w.pool_kernel, dtype=w.dtype,
-                       avg_budget=w.avg_budget, beta=w.beta, pool_kind={"max": 0, "avg": 1}[w.pool_kind])
+                       avg_budget=w.avg_budget, beta=w.beta, pool_kind={"max": 0, "avg": 1}[w.pool_kind],
+                       schedule=getattr(w, "schedule", "linear"))
 
 
 def _tensor(t: Optional[torch.Tensor]) -> PkvTensor:
@@ -147,6 +165,81 @@ def _tensor(t: Optional[torch.Tensor]) -> PkvTensor:
     if t.dim() != 4 or t.stride(3) != 1:
         raise ValueError("expected a [batch][head][token][d] tensor with a contiguous last dimension")
     return PkvTensor(t.data_ptr(), t.stride(0), t.stride(1), t.stride(2))
+
+
+_TORCH_DTYPE = {0: torch.float32, 1: torch.bfloat16, 2: torch.float16}
+
+
+def _on_device(t: torch.Tensor) -> bool:
+    return t.is_cuda or t.is_pinned()      # pinned host memory is mapped on the device (see memory_kind)
+
+
+def _want(ok: bool, what: str) -> None:
+    if not ok:
+        raise ValueError(what)
+
+
+def _check_kv(cfg: PkvConfig, t: torch.Tensor, name: str, batch: int, tokens: int) -> None:
+    """A K or V tensor as large as the call will read: [>= batch][H_kv][>= tokens][d], configured type."""
+    _want(t.dim() == 4 and t.stride(3) == 1, "%s must be [batch][H_kv][token][d] with a contiguous last dimension" % name)
+    _want(t.dtype == _TORCH_DTYPE[cfg.dtype], "%s has type %s, the configuration says %s" % (name, t.dtype, _TORCH_DTYPE[cfg.dtype]))
+    _want(_on_device(t), "%s must live in device memory (or pinned host memory)" % name)
+    _want(t.shape[0] >= batch and t.shape[1] == cfg.num_kv_heads and t.shape[3] == cfg.head_dim,
+          "%s has shape %s, expected [>=%d][%d][token][%d]" % (name, tuple(t.shape), batch, cfg.num_kv_heads, cfg.head_dim))
+    _want(t.shape[2] >= tokens, "%s holds %d tokens per sequence, the lengths given need %d" % (name, t.shape[2], tokens))
+    _want((batch == 1 or t.stride(0) > 0) and (cfg.num_kv_heads == 1 or t.stride(1) > 0) and t.stride(2) >= cfg.head_dim,
+          "%s: batch, head and token strides must be positive (no broadcast views)" % name)
+
+
+def _check_q(cfg: PkvConfig, q_win: torch.Tensor, batch: int) -> None:
+    _want(q_win.dim() == 4 and q_win.stride(3) == 1, "q_win must be [batch][H_q][alpha][d] with a contiguous last dimension")
+    _want(q_win.dtype == _TORCH_DTYPE[cfg.dtype], "q_win has type %s, the configuration says %s" % (q_win.dtype, _TORCH_DTYPE[cfg.dtype]))
+    _want(_on_device(q_win), "q_win must live in device memory")
+    _want(q_win.shape[0] >= batch and tuple(q_win.shape[1:]) == (cfg.num_q_heads, cfg.window, cfg.head_dim),
+          "q_win has shape %s, expected [>=%d][%d][%d][%d]" % (tuple(q_win.shape), batch, cfg.num_q_heads, cfg.window, cfg.head_dim))
+
+
+def _check_scores(cfg: PkvConfig, scores: torch.Tensor, batch: int, columns: int) -> None:
+    """scores [>= batch][H_kv][ld] float32 with ld >= columns; rows of one sequence one after another."""
+    _want(scores.dim() == 3 and scores.dtype == torch.float32 and scores.is_cuda, "scores must be a float32 [batch][H_kv][ld] device tensor")
+    _want(scores.shape[0] >= batch and scores.shape[1] == cfg.num_kv_heads and scores.shape[2] >= columns,
+          "scores has shape %s, expected [>=%d][%d][>=%d]" % (tuple(scores.shape), batch, cfg.num_kv_heads, columns))
+    _want(scores.stride(2) == 1 and scores.stride(1) >= columns and
+          (batch == 1 or scores.stride(0) == cfg.num_kv_heads * scores.stride(1)),
+          "scores: rows must be contiguous and a sequence's heads evenly spaced (stride(0) = H_kv * stride(1))")
+
+
+def _check_rows(cfg: PkvConfig, rows: int, k_out: Optional[torch.Tensor], v_out: Optional[torch.Tensor],
+                indices: Optional[torch.Tensor]) -> None:
+    """Packed outputs with room for `rows` rows."""
+    for name, t in (("k_out", k_out), ("v_out", v_out)):
+        if t is None:
+            continue
+        _want(t.is_cuda and t.is_contiguous() and t.dtype == _TORCH_DTYPE[cfg.dtype], "%s must be a contiguous device tensor of the configured type" % name)
+        _want(t.numel() >= rows * cfg.head_dim, "%s holds %d elements, %d rows need %d" % (name, t.numel(), rows, rows * cfg.head_dim))
+    if indices is not None:
+        _want(indices.is_cuda and indices.is_contiguous() and indices.dtype == torch.int32, "indices must be a contiguous int32 device tensor")
+        _want(indices.numel() >= rows, "indices holds %d entries, %d are needed" % (indices.numel(), rows))
+
+
+def _check_workspace(ws: torch.Tensor) -> None:
+    _want(ws.is_cuda and ws.dtype == torch.uint8 and ws.is_contiguous(), "the workspace must be a contiguous uint8 device tensor")
+
+
+def _check_layer_call(cfg: PkvConfig, layer: int, q_win, k, v, seq_lens, k_out, v_out, indices, workspace, scores) -> None:
+    batch = len(seq_lens)
+    _check_q(cfg, q_win, batch)
+    _check_kv(cfg, k, "k", batch, max(seq_lens))
+    _check_kv(cfg, v, "v", batch, max(seq_lens))
+    _check_rows(cfg, _layer_rows(cfg, layer, seq_lens), k_out, v_out, indices)
+    _check_workspace(workspace)
+    if scores is not None:
+        _check_scores(cfg, scores, batch, max(seq_lens) - cfg.window)
+
+
+def _layer_rows(cfg: PkvConfig, layer: int, seq_lens: Sequence[int]) -> int:
+    _want(0 <= int(layer) < cfg.num_layers, "layer %d outside [0, %d)" % (layer, cfg.num_layers))
+    return total_rows(cfg, layer_budgets(cfg)[int(layer)], seq_lens)
 
 
 def _lens(seq_lens: Sequence[int]):
@@ -213,6 +306,10 @@ def score_window(cfg: PkvConfig, q_win: torch.Tensor, k: torch.Tensor, seq_lens:
                  window_lse: Optional[torch.Tensor] = None) -> None:
     """window_lse given: the prefill's natural-log row normalisers are used and one K sweep is skipped."""
     lens, batch = _lens(seq_lens)
+    _check_q(cfg, q_win, batch)
+    _check_kv(cfg, k, "k", batch, max(seq_lens))
+    _check_scores(cfg, scores, batch, max(seq_lens) - cfg.window)
+    _check_workspace(workspace)
     if window_lse is not None:
         _check(_lib.pyramidkv_score_window_lse(ctypes.byref(cfg), _tensor(q_win), _tensor(k), _lse_ptr(window_lse),
                                                lens, batch, scores.data_ptr(), scores.stride(1),
@@ -233,14 +330,30 @@ def score_window_static(cfg: PkvConfig, q_win: torch.Tensor, k: torch.Tensor, se
     array, so keep them ordered on a stream.
     """
     lens, batch = _lens(seq_lens)
+    _check_q(cfg, q_win, batch)
+    _check_kv(cfg, k, "k", batch, max(seq_lens))
+    _check_scores(cfg, scores, batch, max(seq_lens) - cfg.window)
     _check(_lib.pyramidkv_score_window_static(ctypes.byref(cfg), _tensor(q_win), _tensor(k), lens, batch,
                                               scores.data_ptr(), scores.stride(1), _stream(stream)),
            "pyramidkv_score_window_static")
 
 
+def check_status_static(stream=None) -> int:
+    """check_status for score_window_static: synchronises the stream and reads the status word of the built-in
+    scratch; raises PkvError if a kernel flagged a failure."""
+    detail = ctypes.c_uint32(0)
+    st = _lib.pyramidkv_check_status_static(_stream(stream), ctypes.byref(detail))
+    if st != PKV_OK:
+        raise PkvError(st, "pyramidkv_check_status_static (word 0x%x)" % detail.value)
+    return 0
+
+
 def select_topk(cfg: PkvConfig, scores: torch.Tensor, seq_lens: Sequence[int], k_layer: int,
                 indices: torch.Tensor, workspace: torch.Tensor, stream=None) -> None:
     lens, batch = _lens(seq_lens)
+    _check_scores(cfg, scores, batch, max(seq_lens) - cfg.window)
+    _check_rows(cfg, total_rows(cfg, k_layer, seq_lens), None, None, indices)
+    _check_workspace(workspace)
     _check(_lib.pyramidkv_select_topk(ctypes.byref(cfg), scores.data_ptr(), scores.stride(1), lens, batch,
                                       int(k_layer), indices.data_ptr(), workspace.data_ptr(), workspace.numel(),
                                       _stream(stream)), "pyramidkv_select_topk")
@@ -250,6 +363,10 @@ def gather_compact(cfg: PkvConfig, k: torch.Tensor, v: Optional[torch.Tensor], i
                    seq_lens: Sequence[int], k_layer: int, k_out: torch.Tensor, v_out: Optional[torch.Tensor],
                    stream=None) -> None:
     lens, batch = _lens(seq_lens)
+    _check_kv(cfg, k, "k", batch, max(seq_lens))
+    if v is not None:
+        _check_kv(cfg, v, "v", batch, max(seq_lens))
+    _check_rows(cfg, total_rows(cfg, k_layer, seq_lens), k_out, v_out, indices)
     _check(_lib.pyramidkv_gather_compact(ctypes.byref(cfg), _tensor(k), _tensor(v), indices.data_ptr(), lens, batch,
                                          int(k_layer), k_out.data_ptr(),
                                          v_out.data_ptr() if v_out is not None else None, _stream(stream)),
@@ -261,6 +378,7 @@ def compress_layer(cfg: PkvConfig, layer: int, q_win: torch.Tensor, k: torch.Ten
                    workspace: torch.Tensor, scores: Optional[torch.Tensor] = None, stream=None,
                    window_lse: Optional[torch.Tensor] = None) -> None:
     lens, batch = _lens(seq_lens)
+    _check_layer_call(cfg, layer, q_win, k, v, seq_lens, k_out, v_out, indices, workspace, scores)
     if window_lse is not None:
         _check(_lib.pyramidkv_compress_layer_lse(
             ctypes.byref(cfg), int(layer), _tensor(q_win), _tensor(k), _tensor(v), _lse_ptr(window_lse), lens, batch,
@@ -281,6 +399,7 @@ def profile_layer(cfg: PkvConfig, layer: int, q_win: torch.Tensor, k: torch.Tens
                   workspace: torch.Tensor, stream=None, window_lse: Optional[torch.Tensor] = None):
     """compress_layer with per-kernel device times: returns [(kernel name, milliseconds), ...]."""
     lens, batch = _lens(seq_lens)
+    _check_layer_call(cfg, layer, q_win, k, v, seq_lens, k_out, v_out, indices, workspace, None)
     ms = (ctypes.c_float * PKV_MAX_STAGES)()
     names = ((ctypes.c_char * 32) * PKV_MAX_STAGES)()
     n = ctypes.c_int32(0)

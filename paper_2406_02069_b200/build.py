@@ -2,6 +2,7 @@
 from __future__ import annotations
 
 import glob
+import hashlib
 import os
 import subprocess
 import sys
@@ -10,20 +11,38 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libpyramidkv.so")
+STAMP = LIB + ".srchash"      # digest of the sources the library was built from (travels with the library)
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-shared"]
+
+
+def _flags():
+    """NVCC_FLAGS plus whatever PKV_NVCC_EXTRA adds (e.g. -DPKV_POLY_PAIRS=4 to move the split of the exponentials)."""
+    return NVCC_FLAGS + os.environ.get("PKV_NVCC_EXTRA", "").split()
 
 
 def sources():
     return sorted(glob.glob(os.path.join(CSRC, "*.cu")))
 
 
+def source_digest() -> str:
+    """SHA-256 over the names and contents of everything the library is compiled from."""
+    h = hashlib.sha256()
+    for f in sorted(glob.glob(os.path.join(CSRC, "*")) + glob.glob(os.path.join(ROOT, "include", "*.h"))):
+        h.update(os.path.basename(f).encode())
+        with open(f, "rb") as fh:
+            h.update(fh.read())
+    h.update(" ".join(_flags()).encode())
+    return h.hexdigest()
+
+
 def _stale() -> bool:
-    if not os.path.exists(LIB):
+    """True when the library is missing or was built from other sources.  Compared by content, not by
+    modification time: a copy of the tree to another machine does not keep the times in order."""
+    if not os.path.exists(LIB) or not os.path.exists(STAMP):
         return True
-    t = os.path.getmtime(LIB)
-    deps = glob.glob(os.path.join(CSRC, "*")) + glob.glob(os.path.join(ROOT, "include", "*.h"))
-    return any(os.path.getmtime(f) > t for f in deps)
+    with open(STAMP) as fh:
+        return fh.read().strip() != source_digest()
 
 
 def build_library(force: bool = False, verbose: bool = False) -> str:
@@ -32,12 +51,15 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
         return LIB
     nvcc = os.environ.get("NVCC", "nvcc")
     tmp = LIB + ".tmp.%d" % os.getpid()
-    cmd = [nvcc] + NVCC_FLAGS + ["-I", os.path.join(ROOT, "include"), "-I", CSRC, "-o", tmp] + sources()
+    cmd = [nvcc] + _flags() + ["-I", os.path.join(ROOT, "include"), "-I", CSRC, "-o", tmp] + sources()
     if verbose:
         cmd.insert(1, "-Xptxas=-v")
         print(" ".join(cmd), file=sys.stderr)
+    digest = source_digest()
     subprocess.check_call(cmd)
     os.replace(tmp, LIB)
+    with open(STAMP, "w") as fh:
+        fh.write(digest + "\n")
     return LIB
 
 

@@ -31,7 +31,7 @@ bool config_ok(const pkv_config* c) {
   if (c->window < 1 || c->avg_budget < c->window) return false;
   if (c->pool_kernel < 1 || (c->pool_kernel % 2) == 0) return false;
   if (!(c->beta >= 1.0) || c->beta > 1.0e6) return false;
-  if (c->reserved != 0) return false;
+  if (c->schedule != PKV_SCHEDULE_LINEAR && c->schedule != PKV_SCHEDULE_GEOMETRIC) return false;
   return true;
 }
 
@@ -46,7 +46,10 @@ int config_supported(const pkv_config* c) {
 // Eq. 1 in integers.  beta = bq / 1024.  With k_total = m (B - alpha):
 //   k^l = k_total * ((2 bq - 1024)(m - 1) - (2 bq - 2048) l) / (bq m (m - 1)),
 // floored; the units lost to flooring go to layers 0, 1, ...
+void budgets_geometric(const pkv_config* c, int32_t* out);
+
 void budgets(const pkv_config* c, int32_t* out) {
+  if (c->schedule == PKV_SCHEDULE_GEOMETRIC) { budgets_geometric(c, out); return; }
   const int m = c->num_layers;
   const long long k_total = static_cast<long long>(m) * (c->avg_budget - c->window);
   if (m == 1) { out[0] = static_cast<int32_t>(k_total); return; }
@@ -62,6 +65,46 @@ void budgets(const pkv_config* c, int32_t* out) {
     given += kl;
   }
   for (int l = 0; given < k_total; ++l, ++given) out[l] += 1;
+}
+
+// Geometric decay (appendix "Allocation Strategies"): shares k_total * rho^(m-1-l) / (1 + rho + ... + rho^(m-1)),
+// where rho >= 1 solves 1 + rho + ... + rho^(m-1) = beta * m (so that the top layer gets k_total / (beta m), as
+// in Eq. 1) and is then rounded to a multiple of 2^-20.  Doubles throughout, in a fixed order of operations:
+// the geometric sum is built term by term from rho^0 upward.
+double geometric_sum(double rho, int m, double* powers) {
+  double term = 1.0, sum = 0.0;
+  for (int j = 0; j < m; ++j) {
+    if (powers) powers[j] = term;
+    sum += term;
+    term *= rho;
+  }
+  return sum;
+}
+
+void budgets_geometric(const pkv_config* c, int32_t* out) {
+  const int m = c->num_layers;
+  const long long k_total = static_cast<long long>(m) * (c->avg_budget - c->window);
+  const double beta = static_cast<double>(std::llround(c->beta * 1024.0)) / 1024.0;
+  double rho = 1.0;
+  if (m > 1 && beta > 1.0) {
+    double below = 1.0, above = beta * m;                  // the sum is at least 1 + rho, so the root lies below beta m
+    for (int step = 0; step < 200; ++step) {
+      const double mid = 0.5 * (below + above);
+      if (geometric_sum(mid, m, nullptr) < beta * m) below = mid; else above = mid;
+    }
+    rho = std::nearbyint(0.5 * (below + above) * 1048576.0) / 1048576.0;
+  }
+  double stack_buf[512];
+  double* powers = m <= 512 ? stack_buf : new double[m];
+  const double total = geometric_sum(rho, m, powers);
+  long long given = 0;
+  for (int l = 0; l < m; ++l) {
+    const long long kl = static_cast<long long>(std::floor(static_cast<double>(k_total) * powers[m - 1 - l] / total));
+    out[l] = static_cast<int32_t>(kl);
+    given += kl;
+  }
+  for (int l = 0; given < k_total; ++l, ++given) out[l] += 1;
+  if (powers != stack_buf) delete[] powers;
 }
 
 int kept_count(const pkv_config* c, int k_layer, int n) {
@@ -101,9 +144,10 @@ Workspace carve(const pkv_config* c, int batch, int max_n, void* base) {
   const size_t chunks = (static_cast<size_t>(max_n) + kPartialChunk - 1) / kPartialChunk;
   w.status = reinterpret_cast<uint32_t*>(take(kAlign));
   w.lse2 = reinterpret_cast<float*>(take(heads * rows * sizeof(float)));
-  // fp32-pipe sweep: 2 slots per chunk and head; tensor-core sweep: up to 4 slots per segment, one segment per
-  // run of a CTA over a head (at most CTAs + heads of them), whatever the context length
-  const size_t partial_slots = tc_eligible(c) ? (static_cast<size_t>(kTcMaxGrid) + heads) * 4 : heads * chunks * 2;
+  // fp32-pipe sweep: 2 slots per chunk and head; tensor-core sweep: kTcStatSlots slots per segment, one segment
+  // per run of a CTA over a head (at most CTAs + heads of them), whatever the context length
+  const size_t partial_slots =
+      tc_eligible(c) ? (static_cast<size_t>(kTcMaxGrid) + heads) * kTcStatSlots : heads * chunks * 2;
   w.partial = reinterpret_cast<float2*>(take(partial_slots * rows * sizeof(float2)));
   w.score_scratch_bytes = off;
   w.ld_scores = static_cast<int64_t>((static_cast<size_t>(max_n) + 63) / 64 * 64);
@@ -140,9 +184,13 @@ int build_table(const pkv_config* c, const int32_t* seq_lens, int batch, int k_l
   return PKV_OK;
 }
 
-bool tensor_ok(const pkv_tensor& t, int d, int elem_bytes) {
+// A [batch][heads][token][d] view the kernels can take: 16-byte aligned base and strides, rows that do not
+// overlap, and a positive stride along every dimension that has more than one entry (a broadcast or reversed
+// view has no tensor map and would be mis-sized by the overlap test below).
+bool tensor_ok(const pkv_tensor& t, int d, int elem_bytes, int batch = 1, int heads = 1) {
   if (!t.ptr || t.stride_token < d) return false;
   if (reinterpret_cast<uintptr_t>(t.ptr) % 16) return false;
+  if ((batch > 1 && t.stride_batch <= 0) || (heads > 1 && t.stride_head <= 0)) return false;
   const int64_t q = 16 / elem_bytes;
   return t.stride_token % q == 0 && t.stride_head % q == 0 && t.stride_batch % q == 0;
 }
@@ -258,8 +306,11 @@ bool make_map(CUtensorMap* map, const pkv_tensor& t, bool fp16, int d, uint64_t 
   EncodeTiledFn fn = encode_tiled_fn();
   if (!fn) return false;
   const cuuint64_t dims[4] = {static_cast<cuuint64_t>(d), tokens, heads, batch};
-  auto bytes = [](int64_t elems) { return static_cast<cuuint64_t>(elems > 0 ? elems : 8) * 2; };
-  const cuuint64_t strides[3] = {bytes(t.stride_token), bytes(t.stride_head), bytes(t.stride_batch)};
+  // a dimension of extent 1 may come with any stride (0 included): the map then gets a harmless placeholder
+  auto bytes = [](int64_t elems, uint64_t extent) { return static_cast<cuuint64_t>(extent > 1 || elems > 0 ? elems : 8) * 2; };
+  if ((heads > 1 && t.stride_head <= 0) || (batch > 1 && t.stride_batch <= 0)) return false;
+  const cuuint64_t strides[3] = {static_cast<cuuint64_t>(t.stride_token) * 2, bytes(t.stride_head, heads),
+                                 bytes(t.stride_batch, batch)};
   const cuuint32_t box[4] = {64, box_tok, box_head, 1};
   const cuuint32_t estr[4] = {1, 1, 1, 1};
   return fn(map, fp16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(t.ptr), dims, strides, box, estr,
@@ -358,7 +409,7 @@ int launch_scores_tc(const pkv_config* c, const pkv_tensor& q, const pkv_tensor&
   tp.seq.stat_off[batch] = stat_items;
   tp.seq.score_off[batch] = score_items;
   sp.seq = tp.seq;
-  sp.slots_per_chunk = tp.row_blocks == 2 ? 2 : 4;    // partial slots each sweep-A work item writes
+  sp.slots_per_chunk = tc_stat_slots(tp.row_blocks);  // partial slots each run segment of sweep A holds
 
   const int grid_a = static_cast<int>(std::min<long long>(std::min(sms, kTcMaxGrid),
                                                           static_cast<long long>(stat_items) * sp.num_kv_heads));
@@ -646,7 +697,9 @@ static int score_window_impl(const pkv_config* cfg, pkv_tensor q_win, pkv_tensor
   if (!config_ok(cfg)) return PKV_ERR_INVALID_ARG;
   if (int rc = config_supported(cfg)) return rc;
   const int eb = cfg->dtype == PKV_DTYPE_FP32 ? 4 : 2;
-  if (!tensor_ok(q_win, cfg->head_dim, eb) || !tensor_ok(k, cfg->head_dim, eb) || !scores) return PKV_ERR_INVALID_ARG;
+  if (!tensor_ok(q_win, cfg->head_dim, eb, batch, cfg->num_q_heads) ||
+      !tensor_ok(k, cfg->head_dim, eb, batch, cfg->num_kv_heads) || !scores)
+    return PKV_ERR_INVALID_ARG;
   SeqTable table;
   int max_n;
   int64_t rows;
@@ -694,9 +747,9 @@ int pyramidkv_gather_compact(const pkv_config* cfg, pkv_tensor k, pkv_tensor v, 
   if (!config_ok(cfg)) return PKV_ERR_INVALID_ARG;
   if (int rc = config_supported(cfg)) return rc;
   const int eb = cfg->dtype == PKV_DTYPE_FP32 ? 4 : 2;
-  if (!tensor_ok(k, cfg->head_dim, eb) || !indices || !k_out) return PKV_ERR_INVALID_ARG;
+  if (!tensor_ok(k, cfg->head_dim, eb, batch, cfg->num_kv_heads) || !indices || !k_out) return PKV_ERR_INVALID_ARG;
   if ((v.ptr == nullptr) != (v_out == nullptr)) return PKV_ERR_INVALID_ARG;
-  if (v.ptr && !tensor_ok(v, cfg->head_dim, eb)) return PKV_ERR_INVALID_ARG;
+  if (v.ptr && !tensor_ok(v, cfg->head_dim, eb, batch, cfg->num_kv_heads)) return PKV_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(k_out) % 16 || reinterpret_cast<uintptr_t>(v_out) % 16) return PKV_ERR_INVALID_ARG;
   SeqTable table;
   int max_n;
@@ -723,7 +776,8 @@ static int compress_layer_impl(const pkv_config* cfg, int32_t layer, pkv_tensor 
   if (int rc = config_supported(cfg)) return rc;
   if (layer < 0 || layer >= cfg->num_layers) return PKV_ERR_INVALID_ARG;
   const int eb = cfg->dtype == PKV_DTYPE_FP32 ? 4 : 2;
-  if (!tensor_ok(q_win, cfg->head_dim, eb) || !tensor_ok(k, cfg->head_dim, eb) || !tensor_ok(v, cfg->head_dim, eb))
+  if (!tensor_ok(q_win, cfg->head_dim, eb, batch, cfg->num_q_heads) ||
+      !tensor_ok(k, cfg->head_dim, eb, batch, cfg->num_kv_heads) || !tensor_ok(v, cfg->head_dim, eb, batch, cfg->num_kv_heads))
     return PKV_ERR_INVALID_ARG;
   if (!k_out || !v_out || !indices) return PKV_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(k_out) % 16 || reinterpret_cast<uintptr_t>(v_out) % 16) return PKV_ERR_INVALID_ARG;
@@ -879,7 +933,9 @@ int pyramidkv_gather_paged(const pkv_config* cfg, pkv_tensor k, pkv_tensor v, co
   if (!config_ok(cfg)) return PKV_ERR_INVALID_ARG;
   if (int rc = config_supported(cfg)) return rc;
   const int eb = cfg->dtype == PKV_DTYPE_FP32 ? 4 : 2;
-  if (!tensor_ok(k, cfg->head_dim, eb) || !tensor_ok(v, cfg->head_dim, eb) || !indices) return PKV_ERR_INVALID_ARG;
+  if (!tensor_ok(k, cfg->head_dim, eb, batch, cfg->num_kv_heads) || !tensor_ok(v, cfg->head_dim, eb, batch, cfg->num_kv_heads) ||
+      !indices)
+    return PKV_ERR_INVALID_ARG;
   if (!paged_args_ok(block_table, page_size, num_pages, k_pool, v_pool)) return PKV_ERR_INVALID_ARG;
   if (!workspace || reinterpret_cast<uintptr_t>(workspace) % kAlign || workspace_bytes < kAlign)
     return PKV_ERR_WORKSPACE;
@@ -900,7 +956,8 @@ int pyramidkv_compress_layer_paged(const pkv_config* cfg, int32_t layer, pkv_ten
   if (int rc = config_supported(cfg)) return rc;
   if (layer < 0 || layer >= cfg->num_layers) return PKV_ERR_INVALID_ARG;
   const int eb = cfg->dtype == PKV_DTYPE_FP32 ? 4 : 2;
-  if (!tensor_ok(q_win, cfg->head_dim, eb) || !tensor_ok(k, cfg->head_dim, eb) || !tensor_ok(v, cfg->head_dim, eb))
+  if (!tensor_ok(q_win, cfg->head_dim, eb, batch, cfg->num_q_heads) ||
+      !tensor_ok(k, cfg->head_dim, eb, batch, cfg->num_kv_heads) || !tensor_ok(v, cfg->head_dim, eb, batch, cfg->num_kv_heads))
     return PKV_ERR_INVALID_ARG;
   if (!indices || !paged_args_ok(block_table, page_size, num_pages, k_pool, v_pool)) return PKV_ERR_INVALID_ARG;
   const int32_t k_layer = layer_budget(cfg, layer);
@@ -970,7 +1027,8 @@ int pyramidkv_shard_window_lse(const pkv_config* cfg, pkv_tensor q_win, pkv_tens
   if (!config_ok(cfg)) return PKV_ERR_INVALID_ARG;
   if (int rc = config_supported(cfg)) return rc;
   const int eb = cfg->dtype == PKV_DTYPE_FP32 ? 4 : 2;
-  if (!tensor_ok(q_win, cfg->head_dim, eb) || !tensor_ok(k_shard, cfg->head_dim, eb) || !lse_out)
+  if (!tensor_ok(q_win, cfg->head_dim, eb, batch, cfg->num_q_heads) ||
+      !tensor_ok(k_shard, cfg->head_dim, eb, batch, cfg->num_kv_heads) || !lse_out)
     return PKV_ERR_INVALID_ARG;
   SeqTable table;
   int max_n;
@@ -999,7 +1057,8 @@ int pyramidkv_shard_scores(const pkv_config* cfg, pkv_tensor q_win, pkv_tensor k
   if (!config_ok(cfg)) return PKV_ERR_INVALID_ARG;
   if (int rc = config_supported(cfg)) return rc;
   const int eb = cfg->dtype == PKV_DTYPE_FP32 ? 4 : 2;
-  if (!tensor_ok(q_win, cfg->head_dim, eb) || !tensor_ok(k_shard, cfg->head_dim, eb) || !window_lse || !scores)
+  if (!tensor_ok(q_win, cfg->head_dim, eb, batch, cfg->num_q_heads) ||
+      !tensor_ok(k_shard, cfg->head_dim, eb, batch, cfg->num_kv_heads) || !window_lse || !scores)
     return PKV_ERR_INVALID_ARG;
   SeqTable table;
   int max_n;
@@ -1018,7 +1077,9 @@ int pyramidkv_shard_gather(const pkv_config* cfg, pkv_tensor k_shard, pkv_tensor
   if (!config_ok(cfg)) return PKV_ERR_INVALID_ARG;
   if (int rc = config_supported(cfg)) return rc;
   const int eb = cfg->dtype == PKV_DTYPE_FP32 ? 4 : 2;
-  if (!tensor_ok(k_shard, cfg->head_dim, eb) || !tensor_ok(v_shard, cfg->head_dim, eb)) return PKV_ERR_INVALID_ARG;
+  if (!tensor_ok(k_shard, cfg->head_dim, eb, batch, cfg->num_kv_heads) ||
+      !tensor_ok(v_shard, cfg->head_dim, eb, batch, cfg->num_kv_heads))
+    return PKV_ERR_INVALID_ARG;
   if (!indices || !k_out || !v_out || !shard_begin || !shard_keys) return PKV_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(k_out) % 16 || reinterpret_cast<uintptr_t>(v_out) % 16) return PKV_ERR_INVALID_ARG;
   SeqTable table;
@@ -1190,8 +1251,9 @@ int pyramidkv_compress_model_lanes(const pkv_config* cfg, pkv_lanes* lanes, int3
   if (cudaGetDevice(&device) != cudaSuccess || device != lanes->device) return PKV_ERR_INVALID_ARG;
   const int eb = cfg->dtype == PKV_DTYPE_FP32 ? 4 : 2;
   for (int i = 0; i < num_layers; ++i) {
-    if (!tensor_ok(q_win[i], cfg->head_dim, eb) || !tensor_ok(k[i], cfg->head_dim, eb) ||
-        !tensor_ok(v[i], cfg->head_dim, eb) || !k_out[i] || !v_out[i] || !indices[i])
+    if (!tensor_ok(q_win[i], cfg->head_dim, eb, batch, cfg->num_q_heads) ||
+        !tensor_ok(k[i], cfg->head_dim, eb, batch, cfg->num_kv_heads) ||
+        !tensor_ok(v[i], cfg->head_dim, eb, batch, cfg->num_kv_heads) || !k_out[i] || !v_out[i] || !indices[i])
       return PKV_ERR_INVALID_ARG;
     if (reinterpret_cast<uintptr_t>(k_out[i]) % 16 || reinterpret_cast<uintptr_t>(v_out[i]) % 16)
       return PKV_ERR_INVALID_ARG;
@@ -1296,7 +1358,9 @@ extern "C" int pyramidkv_score_window_static(const pkv_config* cfg, pkv_tensor q
   if (!config_ok(cfg)) return PKV_ERR_INVALID_ARG;
   if (int rc = config_supported(cfg)) return rc;
   const int eb = cfg->dtype == PKV_DTYPE_FP32 ? 4 : 2;
-  if (!tensor_ok(q_win, cfg->head_dim, eb) || !tensor_ok(k, cfg->head_dim, eb) || !scores) return PKV_ERR_INVALID_ARG;
+  if (!tensor_ok(q_win, cfg->head_dim, eb, batch, cfg->num_q_heads) ||
+      !tensor_ok(k, cfg->head_dim, eb, batch, cfg->num_kv_heads) || !scores)
+    return PKV_ERR_INVALID_ARG;
   SeqTable table;
   int max_n;
   int64_t rows;
@@ -1315,4 +1379,10 @@ extern "C" int pyramidkv_score_window_static(const pkv_config* cfg, pkv_tensor q
   // statistics and normalisers are fully rewritten before they are read.
   if (cudaMemsetAsync(w.status, 0, kAlign, st) != cudaSuccess) return PKV_ERR_CUDA;
   return run_scores(cfg, q_win, k, table, batch, scores, ld_scores, w, st);
+}
+
+extern "C" int pyramidkv_check_status_static(void* stream, uint32_t* detail_or_null) {
+  void* base = static_scratch_address();
+  if (!base) return PKV_ERR_CUDA;
+  return pyramidkv_check_status(base, stream, detail_or_null);   // the status word heads the array
 }

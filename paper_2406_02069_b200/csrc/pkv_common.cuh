@@ -34,6 +34,7 @@ enum : uint32_t {
   kStatusSelectMismatch = 1u << 0,   // selection emitted a count other than k
   kStatusWaitExpired = 1u << 1,      // a bounded wait ran out
   kStatusBadPage = 1u << 2,          // a block-table entry named a page outside the pool (row skipped)
+  kStatusBadIndex = 1u << 3,         // a caller-supplied index list named a position outside its sequence (row skipped)
 };
 
 // Programmatic dependent launch: every kernel of the library is launched so that it may start while

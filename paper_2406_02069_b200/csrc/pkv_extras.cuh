@@ -108,7 +108,10 @@ __global__ void __launch_bounds__(256) attention_recall_kernel(const RecallParam
   const int32_t* idx = p.indices + p.seq.row_off[b] + static_cast<int64_t>(h) * count;
   float all = 0.f, kept = 0.f;
   for (int i = threadIdx.x; i < P; i += 256) all += s[i];
-  for (int j = threadIdx.x; j < k; j += 256) kept += s[idx[j]];
+  for (int j = threadIdx.x; j < k; j += 256) {
+    const int i = idx[j];
+    if (i >= 0 && i < P) kept += s[i];                      // an entry that is no prefix position counts as not kept
+  }
   for (int o = 16; o > 0; o >>= 1) {
     all += __shfl_xor_sync(0xffffffffu, all, o);
     kept += __shfl_xor_sync(0xffffffffu, kept, o);

@@ -3,6 +3,8 @@
 //
 // Pure data movement.  Each thread moves one 16-byte piece of a row of K and the
 // same piece of V, so a 256-byte bf16 row is one coalesced access of 16 threads.
+// The index list is the caller's: an entry outside [0, n_b) is never used as an
+// address, its output row is left untouched.
 #pragma once
 
 #include "pkv_common.cuh"
@@ -34,6 +36,7 @@ __global__ void __launch_bounds__(kGatherThreads) gather_rows_kernel(const Gathe
   while (b + 1 < p.seq.batch && row >= p.seq.row_off[b + 1]) ++b;
   const int h = static_cast<int>((row - p.seq.row_off[b]) / p.seq.count[b]);
   const int pos = p.indices[row];
+  if (pos < 0 || pos >= p.seq.n[b]) return;                 // not a position of this sequence: nothing is read
   const int64_t dst = row * p.pieces + piece;
   {
     const char* src = static_cast<const char*>(p.k.ptr) +

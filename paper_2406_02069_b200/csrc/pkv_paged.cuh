@@ -5,7 +5,8 @@
 // sequence and inside a sequence head after head, the pages of that head's kept list: row r of the list
 // sits in page table[r / page_size] at slot r % page_size.  The caller's allocator fills the table; the
 // kernels only follow it.  A table entry outside [0, num_pages) is never dereferenced: the kernel records
-// kStatusBadPage in the status word and skips that row.
+// kStatusBadPage in the status word and skips that row.  The same goes for an entry of the index list
+// outside [0, n_b): kStatusBadIndex, row skipped.
 #pragma once
 
 #include "pkv_common.cuh"
@@ -62,6 +63,10 @@ __global__ void __launch_bounds__(kPagedThreads) gather_paged_kernel(const Gathe
     return;
   }
   const int pos = p.indices[row];
+  if (pos < 0 || pos >= p.seq.n[b]) {
+    if (piece == 0) atomicOr(p.status, kStatusBadIndex);
+    return;
+  }
   const int64_t dst = slot * p.pieces + piece;
   const char* ksrc = static_cast<const char*>(p.k.ptr) +
                      (b * p.k.sb + h * p.k.sh + static_cast<int64_t>(pos) * p.k.st) * p.elem_bytes;

@@ -43,6 +43,10 @@ constexpr int kTcKBytes = 128 * 1024;   // shared memory given to K stages (2 x 
 constexpr int kTcMaxGrid = 256;         // CTAs of a sweep at most (the workspace holds a partial segment per CTA)
 constexpr int kTcMaxRows = 256;         // window rows (G * alpha) the tensor-core path takes
 constexpr long long kTcWaitCycles = 1ll << 31;   // bound of any one wait, in SM clocks
+constexpr int kTcStatSlots = 4;         // partial (reference, sum) slots per run segment and row in sweep A, at most
+// ... and how many of them a sweep with `row_blocks` blocks of 128 window rows writes (one per epilogue warp
+// group that works on a row)
+__host__ __device__ constexpr int tc_stat_slots(int row_blocks) { return row_blocks == 2 ? 2 : 4; }
 
 struct TcParams {
   SeqTable seq;                 // stat_off / score_off count CHUNKS of chunk_tiles tiles
@@ -89,15 +93,17 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Hardware-suspended wait for a barrier phase; returns false when the hardware's own time limit ran out.
+// Hardware-suspended wait for a barrier phase: the thread sleeps until the phase completes or the time hint (in
+// nanoseconds) has passed, whichever comes first; returns false in the second case.  The hint matters: with the
+// default (short) limit the waiting warps of this kernel spent a fifth of all issued instructions on re-trying.
 __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
-      : "r"(bar), "r"(parity)
+      : "r"(bar), "r"(parity), "r"(20000u)
       : "memory");
   return ok != 0;
 }
@@ -108,8 +114,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   if (mbar_try(bar, parity)) return true;
   const long long start = clock64();
   for (;;) {
-    for (int i = 0; i < 32; ++i)
-      if (mbar_try(bar, parity)) return true;
+    if (mbar_try(bar, parity)) return true;
     if (*abort_flag) return false;
     if (clock64() - start > kTcWaitCycles) break;
   }
@@ -139,18 +144,6 @@ __device__ __forceinline__ void tc_mma_f16kind(uint32_t d_tmem, uint64_t a_desc,
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
-        "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
-        "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-      : "r"(taddr)
-      : "memory");
-}
 __device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&v)[16]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
@@ -169,13 +162,10 @@ __device__ __forceinline__ float ex2(float x) {
 
 // The special-function unit evaluates 16 exponentials per clock per SM, which is what bounds both
 // sweeps when every 2^x goes through it.  A fixed share of the exponentials is therefore evaluated on
-// the FMA pipe instead, two at a time with the packed fp32 instructions:
-// 2^x = 2^n * 2^f with n = round(x), f = x - n in [-0.5, 0.5]; 2^f by a cubic minimax polynomial
-// (largest relative error 7.5e-5, far inside the 2e-3 the scores are held to); 2^n by adding n to the
-// exponent field.  x is clamped to [-126, 127.5] so the exponent arithmetic cannot wrap.
-// Of every eight consecutive pairs of values, kTcPolyPairs go this way (spread evenly over the eight).
+// the FMA pipe instead, two at a time with the packed fp32 instructions.  Of every eight consecutive
+// pairs of values (16 accumulator columns), kTcPolyPairs go this way, spread evenly over the eight.
 #ifndef PKV_POLY_PAIRS
-#define PKV_POLY_PAIRS 3
+#define PKV_POLY_PAIRS 2
 #endif
 constexpr int kTcPolyPairs = PKV_POLY_PAIRS;    // 0 = every exponential on the special-function unit
 __host__ __device__ constexpr bool tc_pair_is_poly(int pair) {
@@ -203,54 +193,57 @@ __device__ __forceinline__ unsigned long long add2(unsigned long long a, unsigne
   asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
   return d;
 }
+__device__ __forceinline__ float fma_sat(float a, float b, float c) {   // a * b + c clamped to [0, 1]
+  float d;
+  asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
 
-// 2^x0 and 2^x1 (packed) on the FMA pipe; both already clamped to [-126, 127.5].
-__device__ __forceinline__ unsigned long long ex2_poly2(float x0, float x1) {
-  const float kMagic = 12582912.0f;             // 1.5 * 2^23: adding it leaves round(x) in the low mantissa bits
-  const unsigned long long x = pack2(x0, x1);
-  const unsigned long long t = add2(x, pack2(kMagic, kMagic));
-  const unsigned long long n = add2(t, pack2(-kMagic, -kMagic));
-  const unsigned long long f = fma2(n, pack2(-1.0f, -1.0f), x);
+// acc + (2^x0, 2^x1), evaluated on the FMA pipe.
+//   y = sat((x + 126) / 253)            one instruction rescales x and clamps it to [-126, 127], so that the
+//                                       exponent arithmetic below cannot wrap (-inf and NaN give y = 0)
+//   t = 253 y + (1.5 * 2^23 + 1)        rounds to an integer: the low mantissa bits of t hold n + 127, n = round(x)
+//   f = 253 y + (1.5 * 2^23 + 1 - t)    = x - n in [-0.5, 0.5]
+//   2^f by a cubic minimax polynomial (largest relative error 7.5e-5, far inside the 2e-3 the scores are held to);
+//   2^n is the float whose exponent field is n + 127, i.e. t << 23;  result = acc + 2^f * 2^n.
+__device__ __forceinline__ unsigned long long ex2_poly_add(float x0, float x1, unsigned long long acc) {
+  const float kMagic1 = 12582913.0f;
+  const float y0 = fma_sat(x0, 1.0f / 253.0f, 126.0f / 253.0f), y1 = fma_sat(x1, 1.0f / 253.0f, 126.0f / 253.0f);
+  const unsigned long long y = pack2(y0, y1), k253 = pack2(253.0f, 253.0f), km = pack2(kMagic1, kMagic1);
+  const unsigned long long t = fma2(y, k253, km);
+  const unsigned long long g = fma2(t, pack2(-1.0f, -1.0f), km);
+  const unsigned long long f = fma2(y, k253, g);
   unsigned long long q = fma2(f, pack2(0.0551716685295105f, 0.0551716685295105f),
                               pack2(0.2426111251115799f, 0.2426111251115799f));
   q = fma2(q, f, pack2(0.6932609677314758f, 0.6932609677314758f));
   q = fma2(q, f, pack2(0.9999280571937561f, 0.9999280571937561f));
-  float t0, t1, q0, q1;
+  float t0, t1;
   unpack2(t, t0, t1);
-  unpack2(q, q0, q1);
-  // q * 2^n: add n to the exponent field
-  const int r0 = __float_as_int(q0) + (__float_as_int(t0) << 23);
-  const int r1 = __float_as_int(q1) + (__float_as_int(t1) << 23);
-  return pack2(__int_as_float(r0), __int_as_float(r1));
-}
-// The pair (2^x0, 2^x1), by the unit the pair's position in its group of eight selects.
-template <bool kClampHigh>
-__device__ __forceinline__ unsigned long long ex2_pair(float x0, float x1, int pair) {
-  if (tc_pair_is_poly(pair)) {
-    x0 = fmaxf(x0, -126.0f);
-    x1 = fmaxf(x1, -126.0f);
-    if (kClampHigh) { x0 = fminf(x0, 127.5f); x1 = fminf(x1, 127.5f); }
-    return ex2_poly2(x0, x1);
-  }
-  return pack2(ex2(x0), ex2(x1));
+  const unsigned long long scale = pack2(__int_as_float(__float_as_int(t0) << 23), __int_as_float(__float_as_int(t1) << 23));
+  return fma2(q, scale, acc);
 }
 
-// Sweep A, N logits of one window row, fast path: acc += 2^(v_j * c2 - m) in four packed pairs of partial
-// sums.  m is a reference exponent, not necessarily the running maximum; the caller adds the partial sums up
-// once per accumulator chunk and falls back to rowstats_rescue when the total is not a moderate finite number.
-template <int N>
-__device__ __forceinline__ void rowstats_accumulate(const uint32_t (&v)[N], unsigned long long cc,
-                                                    unsigned long long mm, unsigned long long (&acc)[4]) {
+// acc[j % 4] += (2^x0, 2^x1) for the eight packed pairs xs[j] of one 16-column chunk, each pair by the unit its
+// position selects.
+__device__ __forceinline__ void ex2_accumulate8(const unsigned long long (&xs)[8], unsigned long long (&acc)[4]) {
 #pragma unroll
-  for (int j = 0; j < N; j += 8) {
-    float x[8];
-#pragma unroll
-    for (int q = 0; q < 4; ++q)
-      unpack2(fma2(pack2(__uint_as_float(v[j + 2 * q]), __uint_as_float(v[j + 2 * q + 1])), cc, mm), x[2 * q],
-              x[2 * q + 1]);
-#pragma unroll
-    for (int q = 0; q < 4; ++q) acc[q] = add2(acc[q], ex2_pair<true>(x[2 * q], x[2 * q + 1], j / 2 + q));
+  for (int j = 0; j < 8; ++j) {
+    float x0, x1;
+    unpack2(xs[j], x0, x1);
+    if (tc_pair_is_poly(j)) acc[j & 3] = ex2_poly_add(x0, x1, acc[j & 3]);
+    else acc[j & 3] = add2(acc[j & 3], pack2(ex2(x0), ex2(x1)));
   }
+}
+
+// Sweep A, 16 logits of one window row, fast path: acc += 2^(v_j * c2 - m) in four packed pairs of partial sums.
+// m is a reference exponent, not necessarily the running maximum; the caller adds the partial sums up once per
+// unit and falls back to rowstats_rescue when the total is not a moderate finite number.
+__device__ __forceinline__ void rowstats_accumulate(const uint32_t (&v)[16], unsigned long long cc,
+                                                    unsigned long long mm, unsigned long long (&acc)[4]) {
+  unsigned long long xs[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) xs[j] = fma2(pack2(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1])), cc, mm);
+  ex2_accumulate8(xs, acc);
 }
 __device__ __forceinline__ float sum_pairs(const unsigned long long (&acc)[4]) {
   float a[8];
@@ -258,40 +251,35 @@ __device__ __forceinline__ float sum_pairs(const unsigned long long (&acc)[4]) {
   for (int q = 0; q < 4; ++q) unpack2(acc[q], a[2 * q], a[2 * q + 1]);
   return ((a[0] + a[1]) + (a[2] + a[3])) + ((a[4] + a[5]) + (a[6] + a[7]));
 }
-// Sweep A, slow path for the same N logits: moves the reference exponent to the running maximum first
-// (the row's first chunk, where m = -inf, or a logit some 60 binades above the reference).
-template <int N>
-__device__ __forceinline__ void rowstats_rescue(const uint32_t (&v)[N], float c2, float& m, float& z) {
+// Sweep A, slow path for the same 16 logits: moves the reference exponent up to a whole number at or above the
+// running maximum first (the row's first chunk, where m = -inf, or a logit some 60 binades above the reference).
+// `live` is false for threads that only keep the warp's loads aligned.
+__device__ __forceinline__ void rowstats_rescue(const uint32_t (&v)[16], float c2, bool live, float& m, float& z) {
+  if (!live) return;
   float gm = __uint_as_float(v[0]);
 #pragma unroll
-  for (int j = 1; j < N; ++j) gm = fmaxf(gm, __uint_as_float(v[j]));
-  const float mn = fmaxf(m, gm * c2);
+  for (int j = 1; j < 16; ++j) gm = fmaxf(gm, __uint_as_float(v[j]));
+  const float mn = fmaxf(m, ceilf(gm * c2));
   z *= ex2(m - mn);
   m = mn;
   float g = 0.f;
 #pragma unroll
-  for (int j = 0; j < N; ++j) g += ex2(fmaf(__uint_as_float(v[j]), c2, -m));
+  for (int j = 0; j < 16; ++j) g += ex2(fmaf(__uint_as_float(v[j]), c2, -m));
   z += g;
 }
 
-// Sweep B, N window rows of one key: acc += 2^(v_j * c2 + nlse_j); nlse = -lse2 sits in shared memory
+// Sweep B, 16 window rows of one key: acc += 2^(v_j * c2 + nlse_j); nlse = -lse2 sits in shared memory
 // (negated when it was loaded), acc holds four packed pairs of partial sums.
-template <int N>
-__device__ __forceinline__ void score_group(const uint32_t (&v)[N], unsigned long long cc, const float* nlse,
+__device__ __forceinline__ void score_group(const uint32_t (&v)[16], unsigned long long cc, const float* nlse,
                                             unsigned long long (&acc)[4]) {
+  unsigned long long xs[8];
 #pragma unroll
-  for (int j = 0; j < N; j += 8) {
-    const ulonglong2 la = *reinterpret_cast<const ulonglong2*>(nlse + j);     // eight floats as four packed pairs
-    const ulonglong2 lb = *reinterpret_cast<const ulonglong2*>(nlse + j + 4);
-    const unsigned long long l[4] = {la.x, la.y, lb.x, lb.y};
-    float x[8];
-#pragma unroll
-    for (int q = 0; q < 4; ++q)
-      unpack2(fma2(pack2(__uint_as_float(v[j + 2 * q]), __uint_as_float(v[j + 2 * q + 1])), cc, l[q]), x[2 * q],
-              x[2 * q + 1]);
-#pragma unroll
-    for (int q = 0; q < 4; ++q) acc[q] = add2(acc[q], ex2_pair<false>(x[2 * q], x[2 * q + 1], j / 2 + q));
+  for (int j = 0; j < 8; j += 2) {
+    const ulonglong2 l = *reinterpret_cast<const ulonglong2*>(nlse + 2 * j);   // four floats as two packed pairs
+    xs[j] = fma2(pack2(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1])), cc, l.x);
+    xs[j + 1] = fma2(pack2(__uint_as_float(v[2 * j + 2]), __uint_as_float(v[2 * j + 3])), cc, l.y);
   }
+  ex2_accumulate8(xs, acc);
 }
 
 // Shared-memory matrix descriptor of a K-major bf16 operand whose rows are 128 bytes wide and
@@ -540,7 +528,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       const int r = (two_blocks ? par * 128 : 0) + lane_row;
       if (run_b < 0 || r >= p.rows) return;
       pdl_wait();                                             // the partials of the call before have been merged
-      const int slots = two_blocks ? 2 : 4;
+      const int slots = tc_stat_slots(p.row_blocks);
       const int slot = two_blocks ? ch : grp;
       const int64_t seg = static_cast<int64_t>(blockIdx.x) + run_b * p.num_kv_heads + run_h;
       p.partial[(seg * slots + slot) * p.rows + r] = make_float2(m, z);
@@ -584,7 +572,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
               // fast path over the 128 columns; the sums are only looked at once, at the end
               const unsigned long long cc = pack2(c2, c2), mm = pack2(-m, -m);
               unsigned long long acc[4] = {pack2(0.f, 0.f), pack2(0.f, 0.f), pack2(0.f, 0.f), pack2(0.f, 0.f)};
-              // 16-column loads, double buffered: the next load is in flight while a group is evaluated
+              // 16-column loads, double buffered: the next load is in flight while a chunk is evaluated
               uint32_t va[16], vb[16];
               tc_ld16(taddr, va);
 #pragma unroll
@@ -597,36 +585,35 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
                 rowstats_accumulate(vb, cc, mm, acc);
               }
               const float g = sum_pairs(acc);
-              if (g < 1.0e18f) {
-                z += g;
-              } else {                                        // rare: read the columns again, slow path
-                for (int cg = 0; cg < 128; cg += 32) {
-                  uint32_t v[32];
-                  tc_ld32(taddr + cg, v);
+              const bool good = g < 1.0e18f;                  // false for inf and NaN too
+              if (good) z += g;
+              if (!__all_sync(0xffffffffu, good)) {           // rare: the warp reads its columns again, slow path
+                for (int cg = 0; cg < 128; cg += 16) {
+                  tc_ld16(taddr + cg, va);
                   tc_wait_ld();
-                  rowstats_rescue(v, c2, m, z);
+                  rowstats_rescue(va, c2, !good, m, z);
                 }
               }
             } else {
-              for (int cg = 0; cg < 128; cg += 32) {
-                uint32_t v[32];
-                tc_ld32(taddr + cg, v);
+              for (int cg = 0; cg < 128; cg += 16) {
+                uint32_t v[16];
+                tc_ld16(taddr + cg, v);
                 tc_wait_ld();
                 float gm = -INFINITY;
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
+                for (int j = 0; j < 16; ++j) {
                   const bool vis = key_base + cg + j <= last_visible;
                   const float x = vis ? __uint_as_float(v[j]) * c2 : -INFINITY;
                   v[j] = __float_as_uint(x);
                   gm = fmaxf(gm, x);
                 }
                 if (gm > -INFINITY) {
-                  const float mn = fmaxf(m, gm);
+                  const float mn = fmaxf(m, ceilf(gm));
                   z *= ex2(m - mn);
                   m = mn;
                   float a0 = 0.f;
 #pragma unroll
-                  for (int j = 0; j < 32; ++j) a0 += ex2(__uint_as_float(v[j]) - m);
+                  for (int j = 0; j < 16; ++j) a0 += ex2(__uint_as_float(v[j]) - m);
                   z += a0;
                 }
               }

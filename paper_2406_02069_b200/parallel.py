@@ -107,7 +107,13 @@ def compress_layer_sharded(cfg, layer: int, q_win: torch.Tensor, k_shard: torch.
     this rank's key range of each sequence.  On return every rank holds the layer's packed compact cache
     (k_out, v_out), its index list and the full score rows scores [batch][H_kv][>= max prefix].
     `ops` is the kernel binding (tests may pass a stand-in with the same functions).
+    With `stream` given, the whole layer (the kernels, torch's copies and fills, and the collectives, which
+    follow torch's current stream) runs on that stream.
     """
+    if stream is not None and q_win.is_cuda:
+        with torch.cuda.stream(stream):
+            return compress_layer_sharded(cfg, layer, q_win, k_shard, v_shard, seq_lens, k_out, v_out, indices,
+                                          scores, workspace, exchange, ops=ops, stream=None)
     if ops is None:
         from . import binding as ops
     world, rank = exchange.world, exchange.rank

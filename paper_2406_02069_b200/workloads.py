@@ -55,6 +55,7 @@ class Workload:
     seed: int = 0
     pool_kind: str = "max"   # "max" | "avg" (the mean-pool variant)
     needle_depth: float = -1.0   # in [0, 1]: where the planted block starts in the prefix; < 0: drawn from the seed
+    schedule: str = "linear"     # "linear" | "geometric": shape of the per-layer budgets (a configuration label only)
 
     @property
     def group(self) -> int:

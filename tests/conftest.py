@@ -20,3 +20,15 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+def pytest_terminal_summary(terminalreporter):
+    """How the kept lists of this run compared with the oracle's (see helpers.assert_indices_match)."""
+    try:
+        from helpers import INDEX_LOG
+    except ImportError:
+        return
+    if INDEX_LOG["lists"]:
+        terminalreporter.write_line("kept lists compared with the oracle: %d, identical: %d, largest distance of a "
+                                    "differing entry from the threshold: %.3f tolerances"
+                                    % (INDEX_LOG["lists"], INDEX_LOG["identical"], INDEX_LOG["worst"]))

@@ -5,6 +5,11 @@ import torch
 import oracle
 
 RTOL, ATOL = 2e-3, 1e-5     # score tolerance: |gpu - oracle| <= RTOL * |oracle| + ATOL (fp32)
+INDEX_SLACK = 1.0           # index sets may differ where the oracle's pooled score is within this many score
+                            # tolerances of its k-th pooled value
+# Every kept list compared in this session: [lists, identical lists, largest |pooled - kth| / tolerance among the
+# lists that differed].  tests/conftest.py prints it at the end of a run.
+INDEX_LOG = {"lists": 0, "identical": 0, "worst": 0.0}
 
 
 def assert_scores_close(got: np.ndarray, want: np.ndarray, what=""):
@@ -25,7 +30,9 @@ def assert_indices_match(got_row: np.ndarray, want_row: np.ndarray, oracle_score
     # window block and ordering are exact requirements
     assert np.array_equal(got_row[len(got_row) - alpha:], want_row[len(want_row) - alpha:]), what + " window block"
     assert np.all(np.diff(got_row) > 0), what + " not strictly ascending"
+    INDEX_LOG["lists"] += 1
     if np.array_equal(got_row, want_row):
+        INDEX_LOG["identical"] += 1
         return True
     P = oracle_scores_row.shape[0]
     pool = oracle.pool_avg if pool_kind == "avg" else oracle.pool_max
@@ -36,8 +43,9 @@ def assert_indices_match(got_row: np.ndarray, want_row: np.ndarray, oracle_score
     assert diff.size > 0 and diff.max() < P
     slack = RTOL * abs(kth) + ATOL
     worst = np.max(np.abs(pooled[diff] - kth))
-    assert worst <= 2 * slack, "%s: index sets differ away from the threshold (|pooled - kth| = %g, slack %g)" % (
-        what, worst, slack)
+    INDEX_LOG["worst"] = max(INDEX_LOG["worst"], float(worst / slack))
+    assert worst <= INDEX_SLACK * slack, "%s: index sets differ away from the threshold (|pooled - kth| = %g, " \
+                                         "tolerance %g)" % (what, worst, slack)
     return False
 
 

@@ -123,7 +123,7 @@ def test_single_sweep_with_prefill_lse_matches_oracle(w):
         outs.append((idx.cpu().numpy(), k_out.cpu(), v_out.cpu()))
     counts = [pkv.kept_count(cfg, kl, n) for n in lens]
     heads = [np.array_equal(outs[0][0][sl], outs[1][0][sl]) for _, _, sl in packed_rows(counts, w.num_kv_heads)]
-    assert np.mean(heads) >= 0.9, "only %d of %d heads keep the same list in both modes" % (sum(heads), len(heads))
+    assert np.mean(heads) >= 0.95, "only %d of %d heads keep the same list in both modes" % (sum(heads), len(heads))
     if all(heads):
         assert torch.equal(outs[0][1], outs[1][1]) and torch.equal(outs[0][2], outs[1][2])
 
@@ -227,7 +227,7 @@ def test_compress_layer_matches_oracle(w):
             if kl >= w.pool_kernel * len(planted) and lens[b] > w.avg_budget:
                 assert set(planted) <= set(got_idx[sl].tolist()), "planted tokens evicted"
         total = len(ref["counts"]) * w.num_kv_heads
-        assert identical >= 0.9 * total, "only %d of %d index lists identical" % (identical, total)
+        assert identical >= 0.95 * total, "only %d of %d index lists identical" % (identical, total)
 
 
 @pytest.mark.parametrize("w,layers", [
@@ -262,7 +262,7 @@ def test_full_size_layers_match_oracle(w, layers):
                                                    w.window, "%s layer %d b %d h %d" % (w.name, layer, b, h)))
             sel = idx[sl].long()
             assert torch.equal(k_out[sl], x.k[b, h, sel]) and torch.equal(v_out[sl], x.v[b, h, sel])
-        assert identical >= 0.9 * len(ref["counts"]) * w.num_kv_heads
+        assert identical >= 0.95 * len(ref["counts"]) * w.num_kv_heads
         del x, k_out, v_out, scores
         torch.cuda.empty_cache()
 
@@ -395,17 +395,27 @@ def test_edge_cases(n, B, alpha, G):
 
 
 def test_device_errors_are_reported_not_raised_as_faults():
-    """Bad arguments come back as status codes even with real device buffers."""
+    """Bad arguments with real device buffers: the Python wrapper refuses a mis-sized tensor before the call,
+    and the C side (reached directly here, as a C caller would) answers with a status code."""
+    import ctypes
     w = workloads.TINY
     cfg = pkv.config_of(w)
     x = workloads.make_layer(w, 0, device=DEV)
     ws = pkv.new_workspace(cfg, 1, 512, DEV)
-    scores = torch.zeros(1, w.num_kv_heads, 100, dtype=torch.float32, device=DEV)      # ld too small
-    with pytest.raises(pkv.PkvError) as e:
+    scores = torch.zeros(1, w.num_kv_heads, 100, dtype=torch.float32, device=DEV)      # 100 columns for 504 keys
+    with pytest.raises(ValueError):
         pkv.score_window(cfg, x.q_win, x.k, [512], scores, ws)
-    assert e.value.status == binding.PKV_ERR_INVALID_ARG
+    with pytest.raises(ValueError):                                                     # K shorter than the length given
+        pkv.score_window(cfg, x.q_win, x.k[:, :, :300], [512], torch.zeros(1, 2, 512, device=DEV), ws)
+    with pytest.raises(ValueError):                                                     # wrong element type
+        pkv.score_window(cfg, x.q_win.half(), x.k.half(), [512], torch.zeros(1, 2, 512, device=DEV), ws)
+    lens = (ctypes.c_int32 * 1)(512)
+    full = torch.zeros(1, 2, 512, device=DEV)
+    rc = binding._lib.pyramidkv_score_window(ctypes.byref(cfg), binding._tensor(x.q_win), binding._tensor(x.k), lens, 1,
+                                             full.data_ptr(), 100, ws.data_ptr(), ws.numel(), 0)   # ld too small
+    assert rc == binding.PKV_ERR_INVALID_ARG
     with pytest.raises(pkv.PkvError) as e:
-        pkv.score_window(cfg, x.q_win, x.k, [512], torch.zeros(1, 2, 512, device=DEV), ws[:1024])
+        pkv.score_window(cfg, x.q_win, x.k, [512], full, ws[:1024])
     assert e.value.status == binding.PKV_ERR_WORKSPACE
     pkv.check_status(ws)
 

@@ -110,7 +110,7 @@ def test_emulated_ranks_reproduce_the_unsharded_layer(w, ragged, world):
                                                alpha, "%s b %d h %d" % (w.name, b, h)))
         sel = idx[sl].long()
         assert torch.equal(k_all[sl], x.k[b, h, sel]) and torch.equal(v_all[sl], x.v[b, h, sel])
-    assert identical >= 0.9 * len(ref["counts"]) * w.num_kv_heads
+    assert identical >= 0.95 * len(ref["counts"]) * w.num_kv_heads
 
 
 def _free_port():
