@@ -415,12 +415,18 @@ int launch_scores_tc(const pkv_config* c, const pkv_tensor& q, const pkv_tensor&
                                                           static_cast<long long>(stat_items) * sp.num_kv_heads));
   sp.stat_grid = grid_a;
   const int grid_b = static_cast<int>(std::min<long long>(sms, static_cast<long long>(score_items) * sp.num_kv_heads));
-  if (sp.lse_in == sp.lse2) {                    // normalisers not supplied: sweep A and its merge
+  tp.stat_grid = grid_a;
+  tp.log2_group = std::log2(static_cast<float>(sp.group));
+  if (sp.lse_in == sp.lse2) {                    // normalisers not supplied: sweep A
     launch_pdl(score_tc_kernel<D, 0>, grid_a, kTcThreads, TcSmem<D>::kTotal, st, q_map, k_map_a, tp);
     mark(st, "rowstats_tc");
-    launch_pdl(combine_stats_kernel, dim3((sp.rows + 31) / 32, sp.num_kv_heads, batch), kCombineThreads, 0, st, sp,
-               std::log2(static_cast<float>(sp.group)));
-    mark(st, "combine_stats");
+    if (sp.stats_only) {                         // the normalisers themselves are wanted: merge kernel
+      launch_pdl(combine_stats_kernel, dim3((sp.rows + 31) / 32, sp.num_kv_heads, batch), kCombineThreads, 0, st, sp,
+                 tp.log2_group);
+      mark(st, "combine_stats");
+    } else {
+      tp.merge = 1;                              // sweep B merges the partials of its heads itself
+    }
   }
   if (sp.stats_only) return check_launch();
   launch_pdl(score_tc_kernel<D, 1>, grid_b, kTcThreads, TcSmem<D>::kTotal, st, q_map, k_map_b, tp);

@@ -64,6 +64,10 @@ struct TcParams {
   const float* lse2;            // sweep B in:  [batch][H_kv][R] row normalisers (log of the row's sum of exps)
   float lse_scale, lse_add;     // lse2_r = lse2[r] * lse_scale + lse_add: (1, 0) for the library's own sweep A,
                                 // (log2 e, log2 G) for natural-log normalisers handed in by the caller
+  int32_t merge;                // sweep B: 1 = lse2 is not read; every CTA merges the partials of sweep A for the
+                                // heads it works on (no merge kernel between the sweeps)
+  int32_t stat_grid;            // CTAs sweep A ran with (which segments belong to a head follows from it)
+  float log2_group;             // log2 G, added to the merged normalisers
   float* scores;                // sweep B out: [batch][H_kv][ld]
   int64_t ld_scores;
   uint32_t* status;
@@ -343,11 +347,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   uint8_t* misc = smem + L::kMiscOff;
   uint64_t* bars = reinterpret_cast<uint64_t*>(misc);          // [0..3] k_full, [4..7] k_empty, [8..11] t_full,
                                                                // [12..15] t_empty, [16] q_full, [17] q_empty,
-                                                               // [18..19] x_full, [20..21] x_empty
+                                                               // [18..19] x_full, [20..21] x_empty, [22] lse_full
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 256);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 260);
   float* xch = reinterpret_cast<float*>(misc + 1024);          // sweep B: [2][128] partial sums handed between groups
-  float* lse_all = reinterpret_cast<float*>(misc + 4096);      // sweep B: [16 warps][256] lse2 of the current head
+  float* lse_all = reinterpret_cast<float*>(misc + 4096);      // sweep B: [2][256] -lse2 of the current / next head
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t bar0 = smem_u32(bars);
@@ -358,6 +362,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
   const uint32_t q_full = bar0 + 8u * 16, q_empty = bar0 + 8u * 17;
   auto x_full = [&](int s) { return bar0 + 8u * (18 + s); };
   auto x_empty = [&](int s) { return bar0 + 8u * (20 + s); };
+  const uint32_t lse_full = bar0 + 8u * 22;
 
   // Accumulator stages.  Sweep A: 256 key columns per unit (one row block x one K tile): two stages.
   // Sweep B: rows_pad columns per unit (one K tile), rounded up to a power of two: two to four stages.
@@ -379,6 +384,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     mbar_init(q_full, 1);
     mbar_init(q_empty, 1);
     for (int s = 0; s < 2; ++s) { mbar_init(x_full(s), 4); mbar_init(x_empty(s), 4); }
+    mbar_init(lse_full, kTcEpiWarps);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -516,6 +522,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
     const int lane_row = quarter * 32 + lane;   // TMEM lane of this thread
     const float c2 = p.scale_log2;
     uint32_t u = 0, mine = 0;                   // units seen by the CTA / units this group's pair has read
+    uint32_t heads_seen = 0;                    // sweep B: (sequence, head) changes so far
+    const float* lse_s = lse_all;               // sweep B: the current head's -lse2
     int cur_b = -1, cur_h = -1;
     bool ok = true;
     // Sweep A: a thread's (reference, sum) runs on over consecutive work items of one (sequence, head) and is
@@ -627,14 +635,67 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
       } else {
         // thread -> key.  The pairs of groups take alternate K tiles; inside a pair the groups split the
         // window rows (columns) of a key and group ch = 1 hands its partial sum to group ch = 0.
-        float* lse_s = lse_all + e * 256;                     // this warp's private copy of lse2
+        // The head's normalisers, negated (the epilogue adds them), in one of two buffers that alternate from
+        // head to head.  The sixteen warps fill a buffer together (512 threads over the rows, 2 to 16 lanes per
+        // row), then meet at a barrier; a buffer is written again only after every warp has passed the barrier of
+        // the head in between, i.e. after all of them are done with it.  The values come either from the caller
+        // (or the merge kernel), or straight from sweep A's partial (reference, sum) pairs of this head, which
+        // every CTA that works on the head merges for itself, always in the same order.
         if (w.b != cur_b || w.h != cur_h) {
-          pdl_wait();                                         // the normalisers are written by the kernel before
+          pdl_wait();                                         // normalisers and partials are written by kernels before
+          float* dst = lse_all + (heads_seen & 1u) * 256;
+          const int rows_p2 = p.rows_pad <= 32 ? 32 : (p.rows_pad <= 64 ? 64 : (p.rows_pad <= 128 ? 128 : 256));
+          const int per_row = (kTcEpiWarps * 32) / rows_p2;   // lanes that share a row: 2, 4, 8 or 16
+          const int r = (e * 32 + lane) / per_row, part = (e * 32 + lane) % per_row;
+          float val = -INFINITY;
+          if (p.merge) {
+            // sweep A's CTAs took contiguous item ranges (items ordered sequence, head, chunk): the first `rem`
+            // CTAs per + 1 items, the others per; this head's items fell to CTAs c0..c1, one segment each
+            const int nc = p.seq.stat_off[w.b + 1] - p.seq.stat_off[w.b];
+            const int total_a = p.num_kv_heads * p.seq.stat_off[p.seq.batch];
+            const int per_a = total_a / p.stat_grid, rem_a = total_a % p.stat_grid, edge = rem_a * (per_a + 1);
+            const int i0 = p.num_kv_heads * p.seq.stat_off[w.b] + w.h * nc, i1 = i0 + nc - 1;
+            const int c0 = i0 < edge ? i0 / (per_a + 1) : rem_a + (i0 - edge) / per_a;
+            const int c1 = i1 < edge ? i1 / (per_a + 1) : rem_a + (i1 - edge) / per_a;
+            const int hg = w.b * p.num_kv_heads + w.h, slots = tc_stat_slots(p.row_blocks);
+            const int t0 = (c0 + hg) * slots, t1 = (c1 + hg + 1) * slots;
+            float m = -INFINITY, z = 0.f;
+            if (r < p.rows) {
+              const float2* base = p.partial + r;
+              for (int t = t0 + part; t < t1; t += 4 * per_row) {
+                float2 pz[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                  pz[q] = t + q * per_row < t1 ? __ldcg(base + static_cast<int64_t>(t + q * per_row) * p.rows)
+                                               : make_float2(-INFINITY, 0.f);
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                  if (pz[q].x > -INFINITY) {                  // (-inf, 0) marks a slot that saw no key of this row
+                    const float mn = fmaxf(m, pz[q].x);
+                    z = z * ex2(m - mn) + pz[q].y * ex2(pz[q].x - mn);
+                    m = mn;
+                  }
+              }
+            }
+            for (int o = 1; o < per_row; o <<= 1) {           // the lanes of a row meet pairwise; both partners of a
+              const float m2 = __shfl_xor_sync(0xffffffffu, m, o), z2 = __shfl_xor_sync(0xffffffffu, z, o);   // pair
+              const float mm = fmaxf(m, m2);                                        // compute the same merged value
+              z = (m > -INFINITY ? z * ex2(m - mm) : 0.f) + (m2 > -INFINITY ? z2 * ex2(m2 - mm) : 0.f);
+              m = mm;
+            }
+            if (r < p.rows) val = -(m + __log2f(z) + p.log2_group);
+          } else if (r < p.rows) {
+            const float* src = p.lse2 + (static_cast<int64_t>(w.b) * p.num_kv_heads + w.h) * p.rows;
+            val = -fmaf(src[r], p.lse_scale, p.lse_add);
+          }
+          if (part == 0) dst[r] = val;
           __syncwarp();
-          const float* src = p.lse2 + (static_cast<int64_t>(w.b) * p.num_kv_heads + w.h) * p.rows;
-          for (int i = lane; i < 256; i += 32)       // stored negated: the epilogue adds it
-            lse_s[i] = i < p.rows ? -fmaf(src[i], p.lse_scale, p.lse_add) : -INFINITY;
-          __syncwarp();
+          if (lane == 0) mbar_arrive(lse_full);
+          ok = mbar_wait(lse_full, heads_seen & 1u, abort_flag);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          lse_s = dst;
+          ++heads_seen;
           cur_b = w.b; cur_h = w.h;
         }
         float* srow = p.scores + (static_cast<int64_t>(w.b) * p.num_kv_heads + w.h) * p.ld_scores;
