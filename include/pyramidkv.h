@@ -26,11 +26,11 @@
  *   - Sequences of a batch are independent; each has its own length n_b.
  *     P_b = n_b - alpha is its prefix length.
  *   - Kernels of consecutive calls on one stream overlap at their edges (programmatic dependent
- *     launch).  In particular the score kernels begin to read q_win and k while kernels of THIS
- *     library enqueued just before them are still running; the library orders them itself when
- *     q_win or k lies inside a cache or page pool that one of its recent calls writes.  Work of
- *     the caller's own (ordinary kernel launches, copies) is always finished before a kernel of
- *     the library that follows it on the stream starts.
+ *     launch): a kernel of the library does its set-up while its predecessor drains, and waits for the
+ *     predecessor's completion before it touches global memory.  The one exception is opt-in: with
+ *     PKV_FLAG_INPUTS_FINAL in cfg->flags the score kernels read q_win and k without that wait (see the
+ *     flag).  Even then the library orders them itself when q_win or k lies inside a cache or page pool
+ *     that one of its own recent calls writes.
  *
  * Tensor layout
  *   K, V     [batch][H_kv][n_max][d]   element strides given per tensor
@@ -78,6 +78,14 @@ extern "C" {
 #define PKV_SCHEDULE_LINEAR 0      /* Eq. 1: arithmetic decrease from the lowest layer to the top one */
 #define PKV_SCHEDULE_GEOMETRIC 1   /* appendix "Allocation Strategies": constant ratio between consecutive layers */
 
+/* cfg->flags.  PKV_FLAG_INPUTS_FINAL: the caller promises that q_win and k are complete in memory by the time
+ * the kernels ahead of the call on its stream have been ALLOWED TO LET THEIR DEPENDENTS START, not merely by the
+ * time they finish: nothing still running on the stream writes them.  The score kernels then begin to read them
+ * at once, beside the tail of whatever runs before them (about 5 % on short contexts).  Without the flag they
+ * wait until everything ahead of them on the stream has completed and flushed its writes, which is always right,
+ * also when the producer of K is a kernel that signals its dependents early (programmatic dependent launch). */
+#define PKV_FLAG_INPUTS_FINAL 1u
+
 #define PKV_MAX_BATCH 64          /* sequences per call */
 #define PKV_MAX_STAGES 8          /* kernels one pyramidkv_compress_layer call may launch */
 #define PKV_STATIC_SCRATCH_BYTES (8u << 20)  /* built-in scratch of pyramidkv_score_window_static: 8 MiB per GPU */
@@ -94,6 +102,8 @@ typedef struct pkv_config {
   int32_t avg_budget;    /* B: mean rows kept per layer and KV head, window rows included; >= alpha */
   int32_t schedule;      /* PKV_SCHEDULE_*: shape of the per-layer budgets; 0 = Eq. 1 */
   double  beta;          /* pyramid shape, >= 1 (Section 4.2.1); 1 = same size in every layer */
+  uint32_t flags;        /* PKV_FLAG_* bits, 0 by default */
+  uint32_t reserved;     /* must be 0 */
 } pkv_config;
 
 typedef struct pkv_tensor {
@@ -483,6 +493,22 @@ int pyramidkv_compress_model_lanes(const pkv_config* cfg, pkv_lanes* lanes, int3
                                    const int32_t* seq_lens, int32_t batch,
                                    void* const* k_out, void* const* v_out, int32_t* const* indices,
                                    void* const* workspaces, size_t workspace_bytes, void* stream);
+
+/*
+ * Test aids; the paper has no counterpart.
+ *
+ * pyramidkv_test_hooks: process-wide knobs read by the calls that follow.  wait_clocks > 0 replaces the bound
+ * of every wait inside the tensor-core score kernels (default 2^31 SM clocks) ; withhold_tile != 0 makes the
+ * copy engine thread of the first CTA of the row-statistics sweep leave out its last K tile, so that the
+ * waits for that tile run out, the kernel gives up in an orderly way (every role leaves its loop, the
+ * accumulator memory is released, the status word gets bit 1) and returns.  (0, 0) restores normal operation.
+ *
+ * pyramidkv_test_slow_copy: copies `bytes` (a multiple of 16) from src to dst with one small CTA that lets
+ * its dependents start at once and then copies in `steps` pieces with a pause after each: a stand-in for a
+ * caller's kernel that produces K and signals early.
+ */
+int pyramidkv_test_hooks(int64_t wait_clocks, int32_t withhold_tile);
+int pyramidkv_test_slow_copy(void* dst, const void* src, size_t bytes, int32_t steps, void* stream);
 
 /*
  * Synchronises `stream` and reads the workspace status word.  For tests and

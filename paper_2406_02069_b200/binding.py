@@ -38,7 +38,7 @@ EXPORTS = ("pyramidkv_strerror", "pyramidkv_layer_budgets", "pyramidkv_kept_coun
            "pyramidkv_compress_layer_paged", "pyramidkv_decode_attention_paged", "pyramidkv_shard_window_lse",
            "pyramidkv_merge_lse", "pyramidkv_shard_scores", "pyramidkv_shard_gather", "pyramidkv_memory_kind",
            "pyramidkv_lanes_create", "pyramidkv_lanes_destroy", "pyramidkv_lanes_info",
-           "pyramidkv_compress_model_lanes")
+           "pyramidkv_compress_model_lanes", "pyramidkv_test_hooks", "pyramidkv_test_slow_copy")
 PKV_MAX_STAGES = 8
 
 
@@ -48,7 +48,7 @@ class PkvConfig(ctypes.Structure):
                 ("window", ctypes.c_int32), ("pool_kernel", ctypes.c_int32),
                 ("pool_kind", ctypes.c_int32), ("dtype", ctypes.c_int32),
                 ("avg_budget", ctypes.c_int32), ("schedule", ctypes.c_int32),
-                ("beta", ctypes.c_double)]
+                ("beta", ctypes.c_double), ("flags", ctypes.c_uint32), ("reserved", ctypes.c_uint32)]
 
 
 class PkvTensor(ctypes.Structure):
@@ -101,6 +101,8 @@ def _load() -> ctypes.CDLL:
     lib.pyramidkv_lanes_info.argtypes = [P, ctypes.POINTER(I32), ctypes.POINTER(I32)]
     lib.pyramidkv_compress_model_lanes.argtypes = [CFG, P, I32, I32, P, P, P, P, P, I32, P, P, P, P, SZ, P]
     lib.pyramidkv_check_status.argtypes = [P, P, P]
+    lib.pyramidkv_test_hooks.argtypes = [I64, I32]
+    lib.pyramidkv_test_slow_copy.argtypes = [P, P, SZ, I32, P]
     lib.pyramidkv_check_status_static.argtypes = [P, P]
     for name in EXPORTS:
         if name not in ("pyramidkv_strerror", "pyramidkv_workspace_bytes"):
@@ -144,18 +146,20 @@ def strerror(status: int) -> str:
 
 def make_config(*, num_layers: int, num_q_heads: int, num_kv_heads: int, head_dim: int, window: int,
                 pool_kernel: int, dtype: str, avg_budget: int, beta: float = 20.0, pool_kind: int = 0,
-                schedule: str = "linear") -> PkvConfig:
+                schedule: str = "linear", inputs_final: bool = False) -> PkvConfig:
+    """inputs_final sets PKV_FLAG_INPUTS_FINAL: nothing still running on the stream writes q_win or k when a call is
+    enqueued, so the score kernels may read them before the kernels ahead of them have finished."""
     code = {"fp32": 0, "bf16": 1, "fp16": 2, torch.float32: 0, torch.bfloat16: 1, torch.float16: 2}[dtype]
     return PkvConfig(num_layers, num_q_heads, num_kv_heads, head_dim, window, pool_kernel, pool_kind, code,
-                     avg_budget, {"linear": 0, "geometric": 1}[schedule], float(beta))
+                     avg_budget, {"linear": 0, "geometric": 1}[schedule], float(beta), 1 if inputs_final else 0, 0)
 
 
-def config_of(w) -> PkvConfig:
+def config_of(w, inputs_final: bool = False) -> PkvConfig:
     """Config of a workloads.Workload."""
     return make_config(num_layers=w.num_layers, num_q_heads=w.num_q_heads, num_kv_heads=w.num_kv_heads,
                        head_dim=w.head_dim, window=w.window, pool_kernel=w.pool_kernel, dtype=w.dtype,
                        avg_budget=w.avg_budget, beta=w.beta, pool_kind={"max": 0, "avg": 1}[w.pool_kind],
-                       schedule=getattr(w, "schedule", "linear"))
+                       schedule=getattr(w, "schedule", "linear"), inputs_final=inputs_final)
 
 
 def _tensor(t: Optional[torch.Tensor]) -> PkvTensor:
@@ -237,9 +241,21 @@ def _check_layer_call(cfg: PkvConfig, layer: int, q_win, k, v, seq_lens, k_out, 
         _check_scores(cfg, scores, batch, max(seq_lens) - cfg.window)
 
 
+_budget_cache = {}
+
+
 def _layer_rows(cfg: PkvConfig, layer: int, seq_lens: Sequence[int]) -> int:
+    """Packed output rows of a layer (host arithmetic, remembered per configuration and lengths: the per-layer call
+    is on the hot path of short configurations)."""
     _want(0 <= int(layer) < cfg.num_layers, "layer %d outside [0, %d)" % (layer, cfg.num_layers))
-    return total_rows(cfg, layer_budgets(cfg)[int(layer)], seq_lens)
+    key = (cfg.num_layers, cfg.num_kv_heads, cfg.window, cfg.avg_budget, cfg.schedule, cfg.beta, tuple(seq_lens))
+    rows = _budget_cache.get(key)
+    if rows is None:
+        rows = [total_rows(cfg, kl, seq_lens) for kl in layer_budgets(cfg)]
+        if len(_budget_cache) > 64:
+            _budget_cache.clear()
+        _budget_cache[key] = rows
+    return rows[int(layer)]
 
 
 def _lens(seq_lens: Sequence[int]):
@@ -336,6 +352,22 @@ def score_window_static(cfg: PkvConfig, q_win: torch.Tensor, k: torch.Tensor, se
     _check(_lib.pyramidkv_score_window_static(ctypes.byref(cfg), _tensor(q_win), _tensor(k), lens, batch,
                                               scores.data_ptr(), scores.stride(1), _stream(stream)),
            "pyramidkv_score_window_static")
+
+
+def test_hooks(wait_clocks: int = 0, withhold_tile: bool = False) -> None:
+    """Test aid: bound of the waits inside the tensor-core score kernels (0 = default) and the withheld K tile."""
+    _check(_lib.pyramidkv_test_hooks(int(wait_clocks), 1 if withhold_tile else 0), "pyramidkv_test_hooks")
+
+
+test_hooks.__test__ = False      # not a test case, whatever its name says to a collector
+
+
+def slow_copy(dst: torch.Tensor, src: torch.Tensor, steps: int = 64, stream=None) -> None:
+    """Test aid: dst <- src by a deliberately slow kernel that lets the kernels behind it on the stream start early."""
+    if dst.numel() * dst.element_size() != src.numel() * src.element_size() or not (dst.is_contiguous() and src.is_contiguous()):
+        raise ValueError("slow_copy takes two contiguous tensors of one size")
+    _check(_lib.pyramidkv_test_slow_copy(dst.data_ptr(), src.data_ptr(), dst.numel() * dst.element_size(), int(steps),
+                                         _stream(stream)), "pyramidkv_test_slow_copy")
 
 
 def check_status_static(stream=None) -> int:

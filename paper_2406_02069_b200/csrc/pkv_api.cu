@@ -5,6 +5,7 @@
 #include <cstdio>
 #include <algorithm>
 #include <cstring>
+#include <atomic>
 #include <mutex>
 #include <utility>
 
@@ -19,6 +20,10 @@
 namespace pkv {
 namespace {
 
+// Test knobs (pyramidkv_test_hooks): bound of the waits inside the tensor-core kernels, and the withheld tile.
+std::atomic<long long> g_test_wait_clocks{0};
+std::atomic<int> g_test_withhold{0};
+
 constexpr size_t kAlign = 256;
 constexpr int kPartialChunk = 128;   // smallest key chunk any row-statistics kernel uses (sizes the workspace)
 
@@ -32,6 +37,7 @@ bool config_ok(const pkv_config* c) {
   if (c->pool_kernel < 1 || (c->pool_kernel % 2) == 0) return false;
   if (!(c->beta >= 1.0) || c->beta > 1.0e6) return false;
   if (c->schedule != PKV_SCHEDULE_LINEAR && c->schedule != PKV_SCHEDULE_GEOMETRIC) return false;
+  if ((c->flags & ~PKV_FLAG_INPUTS_FINAL) != 0 || c->reserved != 0) return false;
   return true;
 }
 
@@ -366,8 +372,14 @@ int launch_scores_tc(const pkv_config* c, const pkv_tensor& q, const pkv_tensor&
   tp.rows = sp.rows;
   tp.rows_pad = (sp.rows + 31) / 32 * 32;
   tp.fp16 = fp16 ? 1 : 0;
-  tp.early = (overlaps_recent_output(q, batch, c->num_q_heads, c->window, D, 2) ||
-              overlaps_recent_output(k, batch, c->num_kv_heads, max_n, D, 2)) ? 0 : 1;
+  // An early start needs the caller's word that nothing on the stream still writes Q or K, and the library's own
+  // knowledge that none of its recent outputs is among them.
+  tp.early = (c->flags & PKV_FLAG_INPUTS_FINAL) != 0 &&
+             !(overlaps_recent_output(q, batch, c->num_q_heads, c->window, D, 2) ||
+               overlaps_recent_output(k, batch, c->num_kv_heads, max_n, D, 2));
+  const long long test_wait = g_test_wait_clocks.load();
+  tp.wait_clocks = test_wait > 0 ? test_wait : kTcWaitCycles;
+  tp.withhold = g_test_withhold.load();
   tp.row_blocks = (sp.rows + 127) / 128;
   tp.scale_log2 = sp.scale_log2;
   tp.partial = sp.partial;
@@ -1391,4 +1403,37 @@ extern "C" int pyramidkv_check_status_static(void* stream, uint32_t* detail_or_n
   void* base = static_scratch_address();
   if (!base) return PKV_ERR_CUDA;
   return pyramidkv_check_status(base, stream, detail_or_null);   // the status word heads the array
+}
+
+// ---------------------------------------------------------------------------
+// Test aids (no counterpart in the paper).
+namespace pkv {
+// One small CTA: lets the kernels behind it in the stream start at once, then copies 16-byte pieces in `steps`
+// rounds with a pause after each round, as a slow producer of K that signals its dependents early would.
+__global__ void __launch_bounds__(256) slow_copy_kernel(uint4* dst, const uint4* src, size_t pieces, int steps) {
+  pdl_trigger();
+  const size_t per = (pieces + steps - 1) / steps;
+  for (int s = 0; s < steps; ++s) {
+    const size_t lo = s * per, hi = lo + per < pieces ? lo + per : pieces;
+    for (size_t i = lo + threadIdx.x; i < hi; i += blockDim.x) dst[i] = src[i];
+    __syncthreads();
+    __nanosleep(20000);
+  }
+}
+}  // namespace pkv
+
+extern "C" int pyramidkv_test_hooks(int64_t wait_clocks, int32_t withhold_tile) {
+  if (wait_clocks < 0) return PKV_ERR_INVALID_ARG;
+  g_test_wait_clocks.store(wait_clocks);
+  g_test_withhold.store(withhold_tile ? 1 : 0);
+  return PKV_OK;
+}
+
+extern "C" int pyramidkv_test_slow_copy(void* dst, const void* src, size_t bytes, int32_t steps, void* stream) {
+  if (!dst || !src || bytes % 16 || steps < 1) return PKV_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(dst) % 16 || reinterpret_cast<uintptr_t>(src) % 16) return PKV_ERR_INVALID_ARG;
+  if (bytes == 0) return PKV_OK;
+  slow_copy_kernel<<<1, 256, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<uint4*>(dst),
+                                                                     static_cast<const uint4*>(src), bytes / 16, steps);
+  return cudaPeekAtLastError() == cudaSuccess ? PKV_OK : PKV_ERR_CUDA;
 }

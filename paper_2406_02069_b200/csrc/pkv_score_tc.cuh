@@ -53,7 +53,10 @@ struct TcParams {
   int32_t num_kv_heads, group, rows;      // rows = group * alpha (R)
   int32_t rows_pad;             // R rounded up to 32
   int32_t fp16;                 // 1: Q and K hold binary16, 0: bfloat16 (both operands always share the type)
-  int32_t early;                // 1: Q and K are not outputs of a library kernel that may still run: start at once
+  int32_t early;                // 1: the caller vouches for Q and K (PKV_FLAG_INPUTS_FINAL) and they are not outputs
+                                // of a library kernel that may still run: start reading them at once
+  int32_t withhold;             // test aid: CTA 0 of sweep A never loads its last K tile (its waits then run out)
+  long long wait_clocks;        // bound of any one wait, in SM clocks
   int32_t row_blocks;           // ceil(R / 128): M-blocks of sweep A
   int32_t chunk_tiles_a;        // 256-key tiles per work item of sweep A
   int32_t chunk_tiles_b;        // 128-key tiles per work item of sweep B
@@ -112,15 +115,15 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait.  The thread is suspended by the hardware between checks (no sleeping in software, which
-// would add its wake-up latency to every hand-off of the pipeline).  Gives up after kTcWaitCycles SM
-// clocks (of the order of a second) or when another thread gave up (abort flag); returns false then.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+// would add its wake-up latency to every hand-off of the pipeline).  Gives up after `limit` SM
+// clocks (kTcWaitCycles, of the order of a second, unless a test lowers it) or when another thread gave up (abort flag); returns false then.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long limit) {
   if (mbar_try(bar, parity)) return true;
   const long long start = clock64();
   for (;;) {
     if (mbar_try(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (clock64() - start > kTcWaitCycles) break;
+    if (clock64() - start > limit) break;
   }
   *abort_flag = 1;
   return false;
@@ -427,7 +430,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         const int id = kReverse ? item1 - 1 - ii : item0 + ii;
         const TcItem w = tc_item(off, p.seq.batch, p.num_kv_heads, id);
         if (w.b != cur_b || w.h != cur_h) {
-          if (heads_loaded > 0) ok = mbar_wait(q_empty, (heads_loaded - 1) & 1, abort_flag);
+          if (heads_loaded > 0) ok = mbar_wait(q_empty, (heads_loaded - 1) & 1, abort_flag, p.wait_clocks);
           if (!ok) break;
           mbar_expect_tx(q_full, static_cast<uint32_t>(p.rows) * D * 2);
           for (int half = 0; half < L::kHalves; ++half)
@@ -441,8 +444,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         for (int tt = 0; tt < tile1 - tile0 && ok; ++tt, ++it) {
           const int t = kReverse ? tile1 - 1 - tt : tile0 + tt;
           const int s = it % kKStages;
-          ok = mbar_wait(k_empty(s), ((it / kKStages) & 1) ^ 1, abort_flag);
+          ok = mbar_wait(k_empty(s), ((it / kKStages) & 1) ^ 1, abort_flag, p.wait_clocks);
           if (!ok) break;
+          if (SWEEP == 0 && p.withhold && blockIdx.x == 0 && ii + 1 == item1 - item0 && tt + 1 == tile1 - tile0)
+            continue;                                       // test aid: this tile never arrives
           mbar_expect_tx(k_full(s), kStageBytes);
           for (int half = 0; half < L::kHalves; ++half)
             tma_load_4d(smem_u32(k_s) + s * kStageBytes + half * kTileKeys * 128, &k_map, k_full(s), half * 64,
@@ -471,7 +476,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         const int id = kReverse ? item1 - 1 - ii : item0 + ii;
         const TcItem w = tc_item(off, p.seq.batch, p.num_kv_heads, id);
         if (w.b != cur_b || w.h != cur_h) {
-          ok = mbar_wait(q_full, heads_seen & 1, abort_flag);
+          ok = mbar_wait(q_full, heads_seen & 1, abort_flag, p.wait_clocks);
           if (!ok) break;
           ++heads_seen;
           cur_b = w.b; cur_h = w.h;
@@ -487,14 +492,14 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
         const int tile1 = min(tile0 + chunk_tiles, (keys + kTileKeys - 1) / kTileKeys);
         for (int tt = 0; tt < tile1 - tile0 && ok; ++tt, ++it) {
           const int s = it % kKStages;
-          ok = mbar_wait(k_full(s), (it / kKStages) & 1, abort_flag);
+          ok = mbar_wait(k_full(s), (it / kKStages) & 1, abort_flag, p.wait_clocks);
           if (!ok) break;
           const uint32_t k_addr = smem_u32(k_s) + s * kStageBytes;
           const uint32_t q_addr = smem_u32(q_s);
           const int units = SWEEP == 0 ? p.row_blocks : 1;
           for (int rb = 0; rb < units && ok; ++rb, ++u) {
             const int ts = u % t_stages;
-            ok = mbar_wait(t_empty(ts), ((u / t_stages) & 1) ^ 1, abort_flag);
+            ok = mbar_wait(t_empty(ts), ((u / t_stages) & 1) ^ 1, abort_flag, p.wait_clocks);
             if (!ok) break;
             tc_fence_after();
             const uint32_t d_addr = tmem_base + ts * stage_cols;
@@ -568,7 +573,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
           for (int rb = 0; rb < units && ok; ++rb, ++u) {
             if (static_cast<int>(u & 1u) != par) continue;    // the other pair's unit
             const int ts = u & 1;
-            ok = mbar_wait(t_full(ts), (u >> 1) & 1, abort_flag);
+            ok = mbar_wait(t_full(ts), (u >> 1) & 1, abort_flag, p.wait_clocks);
             ok = __all_sync(0xffffffffu, ok);                 // whole warp proceeds together or not at all
             if (!ok) break;
             tc_fence_after();
@@ -691,7 +696,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
           if (part == 0) dst[r] = val;
           __syncwarp();
           if (lane == 0) mbar_arrive(lse_full);
-          ok = mbar_wait(lse_full, heads_seen & 1u, abort_flag);
+          ok = mbar_wait(lse_full, heads_seen & 1u, abort_flag, p.wait_clocks);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           lse_s = dst;
@@ -705,7 +710,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
           if (static_cast<int>(u & 1u) != par) continue;      // the other pair's tile
           if (ch == 1 && !second_half) continue;              // nothing for this group to read
           const int ts = u % t_stages;
-          ok = mbar_wait(t_full(ts), (u / t_stages) & 1, abort_flag);
+          ok = mbar_wait(t_full(ts), (u / t_stages) & 1, abort_flag, p.wait_clocks);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
           tc_fence_after();
@@ -730,14 +735,14 @@ score_tc_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant
           float sum = sum_pairs(acc);
           if (second_half) {
             if (ch == 1) {
-              ok = mbar_wait(x_empty(par), (mine & 1) ^ 1, abort_flag);
+              ok = mbar_wait(x_empty(par), (mine & 1) ^ 1, abort_flag, p.wait_clocks);
               ok = __all_sync(0xffffffffu, ok);
               if (!ok) break;
               xch[par * 128 + lane_row] = sum;
               __syncwarp();
               if (lane == 0) mbar_arrive(x_full(par));
             } else {
-              ok = mbar_wait(x_full(par), mine & 1, abort_flag);
+              ok = mbar_wait(x_full(par), mine & 1, abort_flag, p.wait_clocks);
               ok = __all_sync(0xffffffffu, ok);
               if (!ok) break;
               sum += xch[par * 128 + lane_row];

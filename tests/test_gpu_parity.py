@@ -493,3 +493,66 @@ def test_token_major_and_fused_layouts_give_the_contiguous_result(dtype):
     kv = torch.stack([x.k, x.v], dim=3).contiguous()                  # [batch][H][n][2][d]
     got = run(x.q_win, kv[:, :, :, 0], kv[:, :, :, 1])
     assert all(torch.equal(a, b) for a, b in zip(got, want))
+
+
+def test_keys_written_by_a_kernel_that_signals_early_are_read_complete():
+    """A producer of K that lets its dependents start at once and then takes its time: the score sweeps that follow
+    it on the stream (default flags) must still see the finished K.  Same result as with a full stop in between, and
+    as the promised-final path after a full stop."""
+    w = workloads.scaled(workloads.LLAMA3_8B, num_layers=2, seq_len=9000, name="llama3_8b_9k_slow_producer")
+    lens = w.seq_lens()
+    x = workloads.make_layer(w, 0, device=DEV)
+    results = []
+    for mode in ("back_to_back", "full_stop", "full_stop_inputs_final"):
+        cfg = pkv.config_of(w, inputs_final=mode == "full_stop_inputs_final")
+        kl = pkv.layer_budgets(cfg)[0]
+        rows = pkv.total_rows(cfg, kl, lens)
+        ws = pkv.new_workspace(cfg, 1, max(lens), DEV)
+        k_live = torch.zeros_like(x.k)                       # filled on the stream, right before the call
+        k_out = torch.empty(rows, w.head_dim, dtype=x.k.dtype, device=DEV)
+        v_out = torch.empty_like(k_out)
+        idx = torch.empty(rows, dtype=torch.int32, device=DEV)
+        scores = torch.zeros(1, w.num_kv_heads, max(lens), dtype=torch.float32, device=DEV)
+        torch.cuda.synchronize()
+        binding.slow_copy(k_live, x.k, steps=64)
+        if mode != "back_to_back":
+            torch.cuda.synchronize()
+        pkv.compress_layer(cfg, 0, x.q_win, k_live, x.v, lens, k_out, v_out, idx, ws, scores=scores)
+        pkv.check_status(ws)
+        assert torch.equal(k_live, x.k)
+        results.append((scores.clone(), idx.clone(), k_out.clone(), v_out.clone()))
+    for other in results[1:]:
+        for a, b in zip(results[0], other):
+            assert torch.equal(a, b)
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_workspace_stays_usable():
+    """Every wait inside the tensor-core kernels is bounded.  Here one K tile of one CTA is never loaded and the bound
+    is lowered to about a millisecond: the waits for that tile give up, the kernel winds down by itself (all roles
+    leave, accumulator memory released), the status word says so, and the next ordinary call on the same workspace
+    gives exactly what a fresh workspace gives."""
+    w = workloads.scaled(workloads.LLAMA3_8B, num_layers=2, seq_len=7000 + 5, name="llama3_8b_7k_expired_wait")
+    cfg = pkv.config_of(w)
+    lens = w.seq_lens()
+    x = workloads.make_layer(w, 1, device=DEV)
+    ws = pkv.new_workspace(cfg, 1, max(lens), DEV)
+    scores = torch.zeros(1, w.num_kv_heads, max(lens), dtype=torch.float32, device=DEV)
+    try:
+        binding.test_hooks(wait_clocks=1 << 21, withhold_tile=True)
+        pkv.score_window(cfg, x.q_win, x.k, lens, scores, ws)
+        with pytest.raises(pkv.PkvError) as e:
+            pkv.check_status(ws)
+        assert e.value.status == binding.PKV_ERR_DEVICE_STATUS and "0x2" in str(e.value)
+    finally:
+        binding.test_hooks(0, False)
+    ws[:256].zero_()
+    again = torch.zeros_like(scores)
+    pkv.score_window(cfg, x.q_win, x.k, lens, again, ws)
+    pkv.check_status(ws)
+    fresh_ws = pkv.new_workspace(cfg, 1, max(lens), DEV)
+    fresh = torch.zeros_like(scores)
+    pkv.score_window(cfg, x.q_win, x.k, lens, fresh, fresh_ws)
+    pkv.check_status(fresh_ws)
+    assert torch.equal(again, fresh)
+    want, _ = oracle.window_scores(x.q_win[0].cpu(), x.k[0, :, : lens[0]].cpu())
+    assert_scores_close(again[0, :, : lens[0] - w.window].cpu().numpy(), want, "after the expired wait")
