@@ -36,9 +36,10 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
 # kernel name, valid only while the kernel's source files have the digest given: a change voids them.
 TC_SOURCES = ("pkv_score_tc.cuh", "pkv_common.cuh")
 NCU_TRAFFIC = {
-    # profiles/score_tc_llama3_70b_128k.md: (read + written) bytes / (n * H_kv) key rows
-    "rowstats_tc": {"sources": TC_SOURCES, "digest": "8e99f49500089722", "bytes_per_key_row": 260.1},
-    "scores_tc": {"sources": TC_SOURCES, "digest": "8e99f49500089722", "bytes_per_key_row": 179.9},
+    # profiles/score_tc_llama3_70b_128k.md: (read + written) bytes / (n * H_kv) key rows, caches flushed by ncu
+    # before the launch (in the step itself sweep B finds about a third of K still in the L2)
+    "rowstats_tc": {"sources": TC_SOURCES, "digest": "45e260642c6f852a", "bytes_per_key_row": 260.1},
+    "scores_tc": {"sources": TC_SOURCES, "digest": "45e260642c6f852a", "bytes_per_key_row": 263.3},
 }
 
 
@@ -224,6 +225,42 @@ class HostOut:
         return o
 
 
+def time_decode(w):
+    """One new token per sequence attends to layer 0's compact cache: microseconds per call, CUDA events around a
+    loop of calls (the cache of one layer is a few megabytes and stays in the L2: a warm number, said so)."""
+    import paper_2406_02069_b200 as pkv
+    from paper_2406_02069_b200 import workloads
+    torch.cuda.set_device(0)
+    cfg = pkv.config_of(w, inputs_final=True)
+    lens = w.seq_lens()
+    kl = pkv.layer_budgets(cfg)[0]
+    x = workloads.make_layer(w, 0, device="cuda")
+    ws = pkv.new_workspace(cfg, len(lens), max(lens))
+    rows = pkv.total_rows(cfg, kl, lens)
+    k_out = torch.empty(rows, w.head_dim, dtype=x.k.dtype, device="cuda")
+    v_out = torch.empty_like(k_out)
+    idx = torch.empty(rows, dtype=torch.int32, device="cuda")
+    pkv.compress_layer(cfg, 0, x.q_win, x.k, x.v, lens, k_out, v_out, idx, ws)
+    pkv.check_status(ws)
+    q = torch.randn(len(lens), w.num_q_heads, w.head_dim, device="cuda").to(x.k.dtype)
+    out = torch.zeros(len(lens), w.num_q_heads, w.head_dim, dtype=torch.float32, device="cuda")
+    for _ in range(10):
+        pkv.decode_attention(cfg, q, k_out, v_out, lens, kl, out)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps = 200
+    e0.record()
+    for _ in range(reps):
+        pkv.decode_attention(cfg, q, k_out, v_out, lens, kl, out)
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) / reps * 1e3
+    cache_bytes = 2 * rows * w.head_dim * x.k.element_size()
+    print(json.dumps({"kernel": "decode_attention", "workload": w.name, "avg_budget": w.avg_budget,
+                      "rows_per_head_layer0": kl + w.window, "q_heads": w.num_q_heads, "batch": len(lens),
+                      "us_per_call": us, "cache_bytes": cache_bytes, "gbs": cache_bytes / us / 1e3,
+                      "note": "back-to-back calls on one layer's cache: L2-warm"}))
+
+
 def time_other(pkv, streaming, workloads, parallel, name, budget, peak, barrier, target_ms=400.0):
     """ms per step, tokens/s and the path's HBM fraction of another configuration: all layers resident, three
     warm-up steps, then a loop of about target_ms between two CUDA events."""
@@ -282,6 +319,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-others", action="store_true", help="skip the short timings of the other configurations")
+    ap.add_argument("--time-decode", action="store_true",
+                    help="instead of the compression path, time pyramidkv_decode_attention (a consumer of the compact "
+                         "cache, not part of the metric) on layer 0 of the workload with --budget rows per head")
     ap.add_argument("--graph", action="store_true",
                     help="replay one CUDA graph per step instead of enqueueing 4 launches per layer from the host")
     ap.add_argument("--lanes", type=int, default=0, metavar="SMS",
@@ -306,6 +346,9 @@ def main():
                                                                 args.seq_len or w.seq_len_hi))
     if args.impl == "reference":
         run_reference(args, w)
+        return
+    if args.time_decode:
+        time_decode(w)
         return
 
     import paper_2406_02069_b200 as pkv
@@ -483,6 +526,8 @@ def main():
                                "step, V stays in pinned host memory and only its kept rows are read over the bus "
                                "(counted in h2d_bytes_per_step)" % ring}
 
+    if rank == 0 and not args.no_cpu_baseline and world == 1:
+        line["cpu_baseline"] = cpu_baseline_sample(w, layers[:16], lens, out.budgets)
     # ---- the other configurations, timed the same way (device-resident, CUDA events), one short loop each
     if args.workload == "llama3_70b_128k" and not (args.layers or args.seq_len or args.budget or args.graph or
                                                     args.lanes or args.no_others) and args.mode == "self":
@@ -492,8 +537,6 @@ def main():
                           for name, budget in (("llama2_7b_4k", None), ("llama3_8b_32k", None),
                                                ("mistral_7b_ragged", 512), ("tiny_fp32", None))]
 
-    if rank == 0 and not args.no_cpu_baseline and world == 1:
-        line["cpu_baseline"] = cpu_baseline_sample(w, layers[:16], lens, out.budgets)
     if rank == 0:
         print(json.dumps(line))
     if dist is not None:
