@@ -498,10 +498,11 @@ int pyramidkv_compress_model_lanes(const pkv_config* cfg, pkv_lanes* lanes, int3
  * Test aids; the paper has no counterpart.
  *
  * pyramidkv_test_hooks: process-wide knobs read by the calls that follow.  wait_clocks > 0 replaces the bound
- * of every wait inside the tensor-core score kernels (default 2^31 SM clocks) ; withhold_tile != 0 makes the
- * copy engine thread of the first CTA of the row-statistics sweep leave out its last K tile, so that the
- * waits for that tile run out, the kernel gives up in an orderly way (every role leaves its loop, the
- * accumulator memory is released, the status word gets bit 1) and returns.  (0, 0) restores normal operation.
+ * of every wait inside the tensor-core score kernels (default 2^31 SM clocks).  Bit 0 of withhold_tile makes the
+ * copy engine thread of the first CTA of the row-statistics sweep leave out its last K tile, so that the waits
+ * for that tile run out, the kernel gives up in an orderly way (every role leaves its loop, the accumulator
+ * memory is released, the status word gets bit 1) and returns.  Bit 1 keeps short contexts on the two-sweep
+ * kernels instead of the single-sweep one (same scores within rounding).  (0, 0) restores normal operation.
  *
  * pyramidkv_test_slow_copy: copies `bytes` (a multiple of 16) from src to dst with one small CTA that lets
  * its dependents start at once and then copies in `steps` pieces with a pause after each: a stand-in for a

@@ -354,9 +354,11 @@ def score_window_static(cfg: PkvConfig, q_win: torch.Tensor, k: torch.Tensor, se
            "pyramidkv_score_window_static")
 
 
-def test_hooks(wait_clocks: int = 0, withhold_tile: bool = False) -> None:
-    """Test aid: bound of the waits inside the tensor-core score kernels (0 = default) and the withheld K tile."""
-    _check(_lib.pyramidkv_test_hooks(int(wait_clocks), 1 if withhold_tile else 0), "pyramidkv_test_hooks")
+def test_hooks(wait_clocks: int = 0, withhold_tile: bool = False, two_sweeps: bool = False) -> None:
+    """Test aid: bound of the waits inside the tensor-core score kernels (0 = default), the withheld K tile, and
+    short contexts kept on the two-sweep kernels."""
+    _check(_lib.pyramidkv_test_hooks(int(wait_clocks), (1 if withhold_tile else 0) | (2 if two_sweeps else 0)),
+           "pyramidkv_test_hooks")
 
 
 test_hooks.__test__ = False      # not a test case, whatever its name says to a collector

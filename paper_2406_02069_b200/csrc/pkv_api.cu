@@ -14,6 +14,7 @@
 #include "pkv_gather.cuh"
 #include "pkv_score_generic.cuh"
 #include "pkv_score_tc.cuh"
+#include "pkv_score_resident.cuh"
 #include "pkv_select.cuh"
 #include "pkv_shard.cuh"
 
@@ -23,6 +24,7 @@ namespace {
 // Test knobs (pyramidkv_test_hooks): bound of the waits inside the tensor-core kernels, and the withheld tile.
 std::atomic<long long> g_test_wait_clocks{0};
 std::atomic<int> g_test_withhold{0};
+std::atomic<int> g_test_two_sweeps{0};     // 1: never take the single-sweep kernel for short contexts
 
 constexpr size_t kAlign = 256;
 constexpr int kPartialChunk = 128;   // smallest key chunk any row-statistics kernel uses (sizes the workspace)
@@ -351,7 +353,9 @@ int launch_scores_tc(const pkv_config* c, const pkv_tensor& q, const pkv_tensor&
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) return PKV_ERR_CUDA;
   if (dev >= 64 || !attr_done[dev]) {
-    if (cudaFuncSetAttribute(score_tc_kernel<D, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcSmem<D>::kTotal) !=
+    if (cudaFuncSetAttribute(score_resident_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             RsSmem<D>::kTotal) != cudaSuccess ||
+        cudaFuncSetAttribute(score_tc_kernel<D, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcSmem<D>::kTotal) !=
             cudaSuccess ||
         cudaFuncSetAttribute(score_tc_kernel<D, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcSmem<D>::kTotal) !=
             cudaSuccess)
@@ -429,6 +433,34 @@ int launch_scores_tc(const pkv_config* c, const pkv_tensor& q, const pkv_tensor&
   const int grid_b = static_cast<int>(std::min<long long>(sms, static_cast<long long>(score_items) * sp.num_kv_heads));
   tp.stat_grid = grid_a;
   tp.log2_group = std::log2(static_cast<float>(sp.group));
+  // Short contexts with few window rows: the logits of a head fit in the tensor memory of a cluster, one sweep.
+  const int tiles_max = (max_n + kRsTileKeys - 1) / kRsTileKeys;
+  if (sp.lse_in == sp.lse2 && !sp.stats_only && sp.rows <= kRsRows && tiles_max <= kRsMaxCluster * kRsMaxTiles &&
+      !g_test_two_sweeps.load()) {
+    int cluster = 1;
+    while (cluster * kRsMaxTiles < tiles_max) cluster *= 2;
+    // more CTAs per head while they still all fit on the device at once and keep at least two tiles each
+    while (2 * cluster <= kRsMaxCluster && static_cast<long long>(2 * cluster) * sp.num_kv_heads * batch <= sms &&
+           tiles_max >= 4 * cluster)
+      cluster *= 2;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(cluster * sp.num_kv_heads, batch);
+    cfg.blockDim = dim3(kRsThreads);
+    cfg.dynamicSmemBytes = RsSmem<D>::kTotal;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    if (cudaLaunchKernelEx(&cfg, score_resident_kernel<D>, q_map, k_map_b, tp) != cudaSuccess) return PKV_ERR_CUDA;
+    mark(st, "scores_resident");
+    return check_launch();
+  }
   if (sp.lse_in == sp.lse2) {                    // normalisers not supplied: sweep A
     launch_pdl(score_tc_kernel<D, 0>, grid_a, kTcThreads, TcSmem<D>::kTotal, st, q_map, k_map_a, tp);
     mark(st, "rowstats_tc");
@@ -1425,7 +1457,8 @@ __global__ void __launch_bounds__(256) slow_copy_kernel(uint4* dst, const uint4*
 extern "C" int pyramidkv_test_hooks(int64_t wait_clocks, int32_t withhold_tile) {
   if (wait_clocks < 0) return PKV_ERR_INVALID_ARG;
   g_test_wait_clocks.store(wait_clocks);
-  g_test_withhold.store(withhold_tile ? 1 : 0);
+  g_test_withhold.store((withhold_tile & 1) ? 1 : 0);
+  g_test_two_sweeps.store((withhold_tile & 2) ? 1 : 0);
   return PKV_OK;
 }
 

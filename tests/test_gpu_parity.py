@@ -556,3 +556,40 @@ def test_a_wait_that_runs_out_is_reported_and_the_workspace_stays_usable():
     assert torch.equal(again, fresh)
     want, _ = oracle.window_scores(x.q_win[0].cpu(), x.k[0, :, : lens[0]].cpu())
     assert_scores_close(again[0, :, : lens[0] - w.window].cpu().numpy(), want, "after the expired wait")
+
+
+@pytest.mark.parametrize("hq,hkv,alpha,d,dtype,lens", [
+    (8, 8, 32, 128, "bf16", [4096]),                    # the multi-head 4k shape: two tiles per CTA, clusters of 8 ... 4
+    (6, 2, 8, 64, "fp16", [41, 3000, 257]),             # 24 window rows of 3 query heads, ragged: some CTAs hold no tile
+    (4, 4, 16, 128, "bf16", [16384, 9000]),             # the longest context the kernel takes: 16 tiles per CTA
+    (2, 2, 32, 128, "bf16", [2049 + 32]),               # a ragged last tile
+])
+def test_single_sweep_kernel_for_short_contexts(hq, hkv, alpha, d, dtype, lens):
+    """Up to 32 window rows per KV head and 16384 keys: the logits of a head stay in tensor memory across a
+    thread-block cluster and K is swept once.  Against the oracle, and against the two-sweep kernels on the same
+    inputs (a test switch keeps the call on them): equal within twice the score tolerance."""
+    tdt = {"bf16": torch.bfloat16, "fp16": torch.float16}[dtype]
+    cfg = pkv.make_config(num_layers=1, num_q_heads=hq, num_kv_heads=hkv, head_dim=d, window=alpha, pool_kernel=7,
+                          dtype=dtype, avg_budget=alpha + 8)
+    g = torch.Generator(device="cpu").manual_seed(hq * 1000 + alpha + len(lens))
+    n_max = max(lens)
+    q = (torch.randn(len(lens), hq, alpha, d, generator=g) * 1.5).to(tdt)
+    k = torch.randn(len(lens), hkv, n_max, d, generator=g).to(tdt)
+    k[:, :, 0] *= 3.0                                          # a sink
+    qd, kd = q.to(DEV), k.to(DEV)
+    ws = pkv.new_workspace(cfg, len(lens), n_max, DEV)
+    both = []
+    for two in (False, True):
+        scores = torch.full((len(lens), hkv, n_max), -1.0, dtype=torch.float32, device=DEV)
+        try:
+            binding.test_hooks(two_sweeps=two)
+            pkv.score_window(cfg, qd, kd, lens, scores, ws)
+            pkv.check_status(ws)
+        finally:
+            binding.test_hooks()
+        both.append(scores.cpu().numpy())
+    for b, n in enumerate(lens):
+        want, _ = oracle.window_scores(q[b], k[b, :, :n])
+        assert_scores_close(both[0][b, :, : n - alpha], want, "single sweep, seq %d" % b)
+        assert_scores_close(both[1][b, :, : n - alpha], want, "two sweeps, seq %d" % b)
+        assert (both[0][b, :, n - alpha:] == -1.0).all()       # nothing written beyond the prefix
