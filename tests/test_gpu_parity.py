@@ -593,3 +593,66 @@ def test_single_sweep_kernel_for_short_contexts(hq, hkv, alpha, d, dtype, lens):
         assert_scores_close(both[0][b, :, : n - alpha], want, "single sweep, seq %d" % b)
         assert_scores_close(both[1][b, :, : n - alpha], want, "two sweeps, seq %d" % b)
         assert (both[0][b, :, n - alpha:] == -1.0).all()       # nothing written beyond the prefix
+
+
+@pytest.mark.parametrize("case", ["mha_4k_layer0", "mha_4k_top_layer", "ragged_with_short", "ties", "mean_pool",
+                                  "wide_pool", "alpha8_gqa3"])
+def test_short_context_layer_equals_three_calls(case):
+    """Short multi-head contexts go through the single-sweep cluster kernel.  The fused per-layer call against the
+    three separate calls on the same inputs: identical scores, lists and rows, bit for bit; and the lists are the
+    oracle's selection on those scores (max and mean pool, ties everywhere, a batch with a sequence short enough to
+    be kept whole, 24 window rows of a 3:1 group)."""
+    base = workloads.scaled(workloads.LLAMA2_7B, num_layers=4, num_q_heads=8, num_kv_heads=8, name="tail_" + case)
+    layer, lens, same_keys = 0, None, False
+    if case == "mha_4k_layer0":
+        w = base
+    elif case == "mha_4k_top_layer":
+        w, layer = base, 3
+    elif case == "ragged_with_short":
+        w, lens = workloads.scaled(base, batch=4), [4096, 100, 1333, 16384]      # 100 <= B: kept whole
+    elif case == "ties":
+        w, lens, same_keys = base, [3000], True
+    elif case == "mean_pool":
+        w = workloads.scaled(base, pool_kind="avg", seq_len=2500)
+    elif case == "wide_pool":
+        w = workloads.scaled(base, pool_kernel=13, seq_len=5000)
+    else:
+        w = workloads.scaled(base, num_q_heads=6, num_kv_heads=2, window=8, avg_budget=40, seq_len=7777)
+    cfg = pkv.config_of(w)
+    lens = lens or w.seq_lens()
+    kl = pkv.layer_budgets(cfg)[layer]
+    x = workloads.make_layer(w, layer, device=DEV, seq_lens=lens)
+    if same_keys:
+        x.k[:, :, : min(lens) - w.window] = x.k[:, :, :1]        # every prefix key the same: the ties decide
+    ws = pkv.new_workspace(cfg, len(lens), max(lens), DEV)
+    rows = pkv.total_rows(cfg, kl, lens)
+    outs = []
+    for fused in (True, False):
+        k_out = torch.zeros(rows, w.head_dim, dtype=x.k.dtype, device=DEV)
+        v_out = torch.zeros_like(k_out)
+        idx = torch.full((rows,), -5, dtype=torch.int32, device=DEV)
+        scores = torch.zeros(len(lens), w.num_kv_heads, max(lens), dtype=torch.float32, device=DEV)
+        if fused:
+            pkv.compress_layer(cfg, layer, x.q_win, x.k, x.v, lens, k_out, v_out, idx, ws, scores=scores)
+        else:
+            pkv.score_window(cfg, x.q_win, x.k, lens, scores, ws)
+            pkv.select_topk(cfg, scores, lens, kl, idx, ws)
+            pkv.gather_compact(cfg, x.k, x.v, idx, lens, kl, k_out, v_out)
+        pkv.check_status(ws)
+        outs.append((scores, idx, k_out, v_out))
+    for a, b in zip(*outs):
+        assert torch.equal(a, b)
+    scores, idx = outs[0][0].cpu().numpy(), outs[0][1].cpu().numpy()
+    pool = oracle.pool_avg if w.pool_kind == "avg" else oracle.pool_max
+    off = 0
+    for b, n in enumerate(lens):
+        c = pkv.kept_count(cfg, kl, n)
+        for h in range(w.num_kv_heads):
+            got = idx[off + h * c: off + (h + 1) * c]
+            if c < n:
+                want = oracle.select_topk(pool(scores[b, h, : n - w.window], w.pool_kernel), c - w.window)
+                assert np.array_equal(got[: c - w.window], want)
+                assert np.array_equal(got[c - w.window:], np.arange(n - w.window, n))
+            else:
+                assert np.array_equal(got, np.arange(n))
+        off += w.num_kv_heads * c
