@@ -18,7 +18,7 @@
 
 namespace pkv {
 
-constexpr int kGenChunk = 256;       // keys per rowstats CTA
+constexpr int kGenChunk = 128;       // keys per rowstats CTA (= the chunk the workspace is sized for)
 constexpr int kGenKeyTile = 16;      // keys staged in shared memory at a time
 constexpr int kGenRowBlock = 256;    // window rows per rowstats CTA pass (= its thread count)
 constexpr int kGenScoreKeys = 128;   // keys (= threads) per scores CTA
