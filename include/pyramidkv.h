@@ -272,7 +272,7 @@ int pyramidkv_gather_compact(const pkv_config* cfg, pkv_tensor k, pkv_tensor v,
  * The whole step for one layer (Section 4.2): scores, pool, top-k with the
  * budget of `layer`, window retention, gather; the same results as the three
  * calls above issued in order.
- *   layer          0 <= layer < num_layers; its budget is taken from the Eq. 1 schedule
+ *   layer          0 <= layer < num_layers; its budget is taken from the schedule cfg->schedule names (Eq. 1 by default)
  *   scores_or_null device [batch][H_kv][ld_scores] to receive the scores, or NULL
  *                  (then ld_scores is ignored and scores live in the workspace)
  * Errors: as above.

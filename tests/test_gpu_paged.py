@@ -161,3 +161,58 @@ def test_a_page_outside_the_pool_is_reported_and_never_written():
         pkv.pages_needed(cfg, kl, lens[0], 0)
     with pytest.raises(ValueError):
         pkv.gather_paged(cfg, x.k, x.v, idx, lens, kl, table.to(DEV).long(), k_pool, v_pool, ws)
+
+
+def test_an_index_outside_its_sequence_is_never_used_as_an_address():
+    """Index lists may come from the caller.  An entry below 0 or beyond the sequence is skipped by the gather kernels
+    (its output row keeps what it held), the other rows are copied bit for bit, the paged gather records it in the
+    status word (bit 3), and the recall diagnostic counts it as not kept."""
+    w = workloads.scaled(workloads.LLAMA3_8B, num_layers=2, seq_len=700, avg_budget=64, name="bad_index")
+    cfg = pkv.config_of(w)
+    lens = w.seq_lens()
+    kl = pkv.layer_budgets(cfg)[0]
+    x = workloads.make_layer(w, 0, device=DEV)
+    ws = pkv.new_workspace(cfg, len(lens), max(lens), DEV)
+    rows = pkv.total_rows(cfg, kl, lens)
+    good = torch.empty(rows, dtype=torch.int32, device=DEV)
+    scores = torch.zeros(1, w.num_kv_heads, max(lens), dtype=torch.float32, device=DEV)
+    k_ref = torch.empty(rows, w.head_dim, dtype=x.k.dtype, device=DEV)
+    v_ref = torch.empty_like(k_ref)
+    pkv.compress_layer(cfg, 0, x.q_win, x.k, x.v, lens, k_ref, v_ref, good, ws, scores=scores)
+    pkv.check_status(ws)
+    bad = good.clone()
+    bad_rows = [3, 17, rows - 1]
+    bad[3], bad[17], bad[rows - 1] = -1, lens[0], 2 ** 30      # below, one past the end, far beyond
+    ok_rows = torch.ones(rows, dtype=torch.bool, device=DEV)
+    ok_rows[bad_rows] = False
+    # stand-alone gather: no workspace, so nothing to record; the rows are simply left alone
+    k_out = torch.full((rows, w.head_dim), -3.0, dtype=x.k.dtype, device=DEV)
+    v_out = torch.full_like(k_out, -5.0)
+    pkv.gather_compact(cfg, x.k, x.v, bad, lens, kl, k_out, v_out)
+    torch.cuda.synchronize()
+    assert torch.equal(k_out[ok_rows], k_ref[ok_rows]) and torch.equal(v_out[ok_rows], v_ref[ok_rows])
+    assert (k_out[bad_rows] == -3.0).all() and (v_out[bad_rows] == -5.0).all()
+    # paged gather: the same, and the status word says so
+    page_size = 16
+    pages, table, num_pages = make_tables(cfg, lens, kl, page_size, w.num_kv_heads, seed=3, spare=2)
+    k_pool = torch.full((num_pages, page_size, w.head_dim), -3.0, dtype=x.k.dtype, device=DEV)
+    v_pool = torch.full_like(k_pool, -5.0)
+    pkv.gather_paged(cfg, x.k, x.v, bad, lens, kl, table.to(DEV), k_pool, v_pool, ws)
+    with pytest.raises(pkv.PkvError) as e:
+        pkv.check_status(ws)
+    assert e.value.status == binding.PKV_ERR_DEVICE_STATUS and "0x8" in str(e.value)
+    ws[:256].zero_()
+    k_pool2 = torch.full_like(k_pool, -3.0)
+    v_pool2 = torch.full_like(v_pool, -5.0)
+    pkv.gather_paged(cfg, x.k, x.v, good, lens, kl, table.to(DEV), k_pool2, v_pool2, ws)
+    pkv.check_status(ws)
+    differ = (k_pool != k_pool2).any(dim=2).sum().item()
+    assert differ == len(bad_rows)                              # exactly the three skipped slots
+    # recall: a bad entry is not a kept position
+    rec_good = torch.zeros(1, w.num_kv_heads, dtype=torch.float32, device=DEV)
+    rec_bad = torch.zeros_like(rec_good)
+    pkv.attention_recall(cfg, scores, good, lens, kl, rec_good)
+    pkv.attention_recall(cfg, scores, bad, lens, kl, rec_bad)
+    torch.cuda.synchronize()
+    assert rec_bad[0, 0] < rec_good[0, 0]                      # rows 3 and 17 belong to head 0: two kept keys fewer
+    assert torch.equal(rec_bad[0, 1:], rec_good[0, 1:])        # the last bad entry sits in a window slot: not counted
