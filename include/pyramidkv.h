@@ -337,6 +337,34 @@ int pyramidkv_attention_recall(const pkv_config* cfg, const float* scores, int64
                                int32_t k_layer, float* recall, void* stream);
 
 /*
+ * The window rows' attention together with the scores (Section 4.1, Section 4.2.2 Eq. 2 and Eq. 3: the scores
+ * are column sums of the attention matrix of the last alpha queries, whose rows times V are what the prefill
+ * attention returns for those queries).  One kernel forms the softmax probabilities of the window rows once and
+ * uses them twice: summed over rows and query heads they are the scores, multiplied by V they are the attention
+ * output.  A prefill that calls this for its last alpha rows gets their output and the compression from the same
+ * pass over K; the row normalisers still come from the row-statistics sweep that runs first.
+ *   attn_out  device, [batch][H_q][alpha][d] floats, contiguous, 16-byte aligned:
+ *             attn_out[b][g][j] = sum over keys i <= P_b + j of softmax_i(q_gj . k_i / sqrt(d)) * v_i
+ *   scores    pyramidkv_attend_window: required, device [batch][H_kv][ld_scores] (the P_b prefix positions of
+ *             each row are written); pyramidkv_attend_compress_layer: optional as in pyramidkv_compress_layer
+ * The probabilities are rounded to the inputs' 16-bit type before they multiply V, as V itself is.  Rows of V
+ * behind a sequence's length are never used, whatever they hold.  Everything else as pyramidkv_score_window /
+ * pyramidkv_compress_layer; the scores agree with theirs to rounding.
+ * Errors: as those calls; UNSUPPORTED unless the inputs are 16-bit, head_dim is 128 and (H_q / H_kv) * window
+ * <= 256.  The workspace is the one pyramidkv_workspace_bytes sizes.
+ */
+int pyramidkv_attend_window(const pkv_config* cfg, pkv_tensor q_win, pkv_tensor k, pkv_tensor v,
+                            const int32_t* seq_lens, int32_t batch, float* attn_out,
+                            float* scores, int64_t ld_scores,
+                            void* workspace, size_t workspace_bytes, void* stream);
+int pyramidkv_attend_compress_layer(const pkv_config* cfg, int32_t layer,
+                                    pkv_tensor q_win, pkv_tensor k, pkv_tensor v,
+                                    const int32_t* seq_lens, int32_t batch, float* attn_out,
+                                    void* k_out, void* v_out, int32_t* indices,
+                                    float* scores_or_null, int64_t ld_scores,
+                                    void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Measuring aid; the paper has no counterpart.  Same arguments and results as
  * pyramidkv_compress_layer, but a CUDA event is recorded after every kernel the
  * call launches, the stream is synchronised, and the device time of each kernel

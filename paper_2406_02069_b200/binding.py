@@ -38,7 +38,8 @@ EXPORTS = ("pyramidkv_strerror", "pyramidkv_layer_budgets", "pyramidkv_kept_coun
            "pyramidkv_compress_layer_paged", "pyramidkv_decode_attention_paged", "pyramidkv_shard_window_lse",
            "pyramidkv_merge_lse", "pyramidkv_shard_scores", "pyramidkv_shard_gather", "pyramidkv_memory_kind",
            "pyramidkv_lanes_create", "pyramidkv_lanes_destroy", "pyramidkv_lanes_info",
-           "pyramidkv_compress_model_lanes", "pyramidkv_test_hooks", "pyramidkv_test_slow_copy")
+           "pyramidkv_compress_model_lanes", "pyramidkv_test_hooks", "pyramidkv_test_slow_copy",
+           "pyramidkv_attend_window", "pyramidkv_attend_compress_layer")
 PKV_MAX_STAGES = 8
 
 
@@ -84,6 +85,9 @@ def _load() -> ctypes.CDLL:
     lib.pyramidkv_compress_layer_lse.argtypes = [CFG, I32, PkvTensor, PkvTensor, PkvTensor, P, P, I32, P, P, P, P,
                                                  I64, P, SZ, P]
     lib.pyramidkv_profile_layer_lse.argtypes = lib.pyramidkv_compress_layer_lse.argtypes + [P, P, P]
+    lib.pyramidkv_attend_window.argtypes = [CFG, PkvTensor, PkvTensor, PkvTensor, P, I32, P, P, I64, P, SZ, P]
+    lib.pyramidkv_attend_compress_layer.argtypes = [CFG, I32, PkvTensor, PkvTensor, PkvTensor, P, I32, P, P, P, P, P,
+                                                    I64, P, SZ, P]
     lib.pyramidkv_decode_attention.argtypes = [CFG, P, P, P, P, I32, I32, P, P]
     lib.pyramidkv_attention_recall.argtypes = [CFG, P, I64, P, P, I32, I32, P, P]
     lib.pyramidkv_pages_needed.argtypes = [CFG, I32, I32, I32]
@@ -426,6 +430,43 @@ def compress_layer(cfg: PkvConfig, layer: int, q_win: torch.Tensor, k: torch.Ten
                                          scores.stride(1) if scores is not None else 0,
                                          workspace.data_ptr(), workspace.numel(), _stream(stream)),
            "pyramidkv_compress_layer")
+
+
+def _check_attn_out(cfg: PkvConfig, attn_out: torch.Tensor, batch: int) -> None:
+    _want(attn_out.is_cuda and attn_out.dtype == torch.float32 and attn_out.is_contiguous() and
+          tuple(attn_out.shape) == (batch, cfg.num_q_heads, cfg.window, cfg.head_dim),
+          "attn_out must be a contiguous float32 device tensor [batch][H_q][window][d]")
+
+
+def attend_window(cfg: PkvConfig, q_win: torch.Tensor, k: torch.Tensor, v: torch.Tensor, seq_lens: Sequence[int],
+                  attn_out: torch.Tensor, scores: torch.Tensor, workspace: torch.Tensor, stream=None) -> None:
+    """The window rows' attention output and the window scores from one fused pass."""
+    lens, batch = _lens(seq_lens)
+    _check_q(cfg, q_win, batch)
+    _check_kv(cfg, k, "k", batch, max(seq_lens))
+    _check_kv(cfg, v, "v", batch, max(seq_lens))
+    _check_attn_out(cfg, attn_out, batch)
+    _check_scores(cfg, scores, batch, max(seq_lens) - cfg.window)
+    _check_workspace(workspace)
+    _check(_lib.pyramidkv_attend_window(ctypes.byref(cfg), _tensor(q_win), _tensor(k), _tensor(v), lens, batch,
+                                        attn_out.data_ptr(), scores.data_ptr(), scores.stride(1),
+                                        workspace.data_ptr(), workspace.numel(), _stream(stream)),
+           "pyramidkv_attend_window")
+
+
+def attend_compress_layer(cfg: PkvConfig, layer: int, q_win: torch.Tensor, k: torch.Tensor, v: torch.Tensor,
+                          seq_lens: Sequence[int], attn_out: torch.Tensor, k_out: torch.Tensor, v_out: torch.Tensor,
+                          indices: torch.Tensor, workspace: torch.Tensor, scores: Optional[torch.Tensor] = None,
+                          stream=None) -> None:
+    """compress_layer that also returns the window rows' attention output."""
+    lens, batch = _lens(seq_lens)
+    _check_layer_call(cfg, layer, q_win, k, v, seq_lens, k_out, v_out, indices, workspace, scores)
+    _check_attn_out(cfg, attn_out, batch)
+    _check(_lib.pyramidkv_attend_compress_layer(
+        ctypes.byref(cfg), int(layer), _tensor(q_win), _tensor(k), _tensor(v), lens, batch, attn_out.data_ptr(),
+        k_out.data_ptr(), v_out.data_ptr(), indices.data_ptr(),
+        scores.data_ptr() if scores is not None else None, scores.stride(1) if scores is not None else 0,
+        workspace.data_ptr(), workspace.numel(), _stream(stream)), "pyramidkv_attend_compress_layer")
 
 
 def profile_layer(cfg: PkvConfig, layer: int, q_win: torch.Tensor, k: torch.Tensor, v: torch.Tensor,

@@ -15,6 +15,7 @@
 #include "pkv_score_generic.cuh"
 #include "pkv_score_tc.cuh"
 #include "pkv_score_resident.cuh"
+#include "pkv_attend.cuh"
 #include "pkv_select.cuh"
 #include "pkv_shard.cuh"
 
@@ -130,6 +131,7 @@ struct Workspace {
   uint2* sel_cand;           // selection: candidate (key, position) pairs, [heads][sel_cand_stride]
   int64_t sel_cand_stride;
   uint32_t* sel_cnt;         // selection: pairs per cluster rank, [heads][kSelMaxCluster]
+  float* o_partial;          // window attention: per-segment accumulators [kAtMaxGrid + heads][R][d], or null
   size_t score_scratch_bytes;   // bytes of the leading regions that the score kernels alone need
   size_t bytes;
 };
@@ -140,6 +142,10 @@ bool tc_eligible(const pkv_config* c) {
   return (c->dtype == PKV_DTYPE_BF16 || c->dtype == PKV_DTYPE_FP16) && g * c->window <= kTcMaxRows &&
          c->window <= 256 && g <= 256;
 }
+
+// Which configurations the fused window-attention kernel takes.
+bool attend_eligible(const pkv_config* c) { return tc_eligible(c) && c->head_dim == kAtD; }
+constexpr int kAtMaxGrid = 160;      // CTAs of the window-attention kernel at most (sizes its partial accumulators)
 
 // Carves the workspace for `batch` sequences of at most max_n tokens.  base may be null (sizing only).
 Workspace carve(const pkv_config* c, int batch, int max_n, void* base) {
@@ -163,6 +169,8 @@ Workspace carve(const pkv_config* c, int batch, int max_n, void* base) {
   w.sel_cand_stride = static_cast<int64_t>(max_n) + 32 * kSelMaxCluster;   // cluster * slice never exceeds this
   w.sel_cand = reinterpret_cast<uint2*>(take(heads * w.sel_cand_stride * sizeof(uint2)));
   w.sel_cnt = reinterpret_cast<uint32_t*>(take(heads * kSelMaxCluster * sizeof(uint32_t)));
+  if (attend_eligible(c))
+    w.o_partial = reinterpret_cast<float*>(take((static_cast<size_t>(kAtMaxGrid) + heads) * rows * kAtD * sizeof(float)));
   w.bytes = off;
   return w;
 }
@@ -512,6 +520,72 @@ int run_scores(const pkv_config* c, const pkv_tensor& q, const pkv_tensor& k, co
                              : launch_scores_generic<__half, 128>(sp, batch, st);
   return c->head_dim == 64 ? launch_scores_generic<__nv_bfloat16, 64>(sp, batch, st)
                            : launch_scores_generic<__nv_bfloat16, 128>(sp, batch, st);
+}
+
+// ---------------------------------------------------------------- window attention fused with the scores
+// Needs the row normalisers in w.lse2 (run_scores with stats_only).  Writes the scores of the prefix positions and
+// attn_out[batch][H_q][alpha][d].
+int run_attend(const pkv_config* c, const pkv_tensor& q, const pkv_tensor& k, const pkv_tensor& v, const SeqTable& table,
+               int batch, int max_n, float* scores, int64_t ld, float* attn_out, const Workspace& w, cudaStream_t st) {
+  const int sms = device_sm_count();
+  if (sms <= 0) return PKV_ERR_CUDA;
+  static bool attr_done[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) return PKV_ERR_CUDA;
+  if (dev >= 64 || !attr_done[dev]) {
+    if (cudaFuncSetAttribute(window_attend_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kAtSmemBytes) !=
+        cudaSuccess)
+      return PKV_ERR_CUDA;
+    if (dev < 64) attr_done[dev] = true;
+  }
+  const bool fp16 = c->dtype == PKV_DTYPE_FP16;
+  const int group = c->num_q_heads / c->num_kv_heads;
+  alignas(64) CUtensorMap q_map, k_map, v_map;
+  if (!make_map(&q_map, q, fp16, kAtD, c->window, c->num_q_heads, batch, c->window, group) ||
+      !make_map(&k_map, k, fp16, kAtD, max_n, c->num_kv_heads, batch, kAtTileKeys, 1) ||
+      !make_map(&v_map, v, fp16, kAtD, max_n, c->num_kv_heads, batch, kAtTileKeys, 1))
+    return PKV_ERR_CUDA;
+  AtParams ap{};
+  ap.seq = table;
+  ap.num_kv_heads = c->num_kv_heads;
+  ap.group = group;
+  ap.rows = group * c->window;
+  ap.rows_pad = (ap.rows + 31) / 32 * 32;
+  ap.fp16 = fp16 ? 1 : 0;
+  const long long test_wait = g_test_wait_clocks.load();
+  ap.wait_clocks = test_wait > 0 ? test_wait : kTcWaitCycles;
+  ap.scale_log2 = static_cast<float>(1.4426950408889634 / std::sqrt(static_cast<double>(c->head_dim)));
+  ap.lse2 = w.lse2;
+  ap.scores = scores;
+  ap.ld_scores = ld;
+  ap.o_partial = w.o_partial;
+  ap.out = attn_out;
+  ap.status = w.status;
+  const int grid_cap = std::min(sms, kAtMaxGrid);
+  // Key tiles per work item: the largest power of two that still spreads the items evenly over the SMs.
+  auto items_for = [&](int ct) {
+    long long items = 0;
+    for (int b = 0; b < batch; ++b) items += ((table.n[b] + kAtTileKeys - 1) / kAtTileKeys + ct - 1) / ct;
+    return items * c->num_kv_heads;
+  };
+  int ct = 16;
+  for (; ct > 1; ct /= 2) {
+    const long long items = items_for(ct), waves = (items + grid_cap - 1) / grid_cap;
+    if (items >= grid_cap && static_cast<double>(items) / static_cast<double>(waves * grid_cap) >= 0.93) break;
+  }
+  ap.chunk_tiles = ct;
+  int items = 0;
+  for (int b = 0; b < batch; ++b) {
+    ap.seq.score_off[b] = items;
+    items += ((table.n[b] + kAtTileKeys - 1) / kAtTileKeys + ct - 1) / ct;
+  }
+  ap.seq.score_off[batch] = items;
+  ap.grid = static_cast<int>(std::min<long long>(grid_cap, static_cast<long long>(items) * c->num_kv_heads));
+  launch_pdl(window_attend_kernel, ap.grid, kAtThreads, kAtSmemBytes, st, q_map, k_map, v_map, ap);
+  mark(st, "window_attend");
+  launch_pdl(window_attend_reduce_kernel, dim3(ap.rows, c->num_kv_heads, batch), kAtD, 0, st, ap);
+  mark(st, "window_attend_reduce");
+  return check_launch();
 }
 
 // ---------------------------------------------------------------- select
@@ -865,6 +939,60 @@ int pyramidkv_compress_layer_lse(const pkv_config* cfg, int32_t layer, pkv_tenso
   if (!window_lse) return PKV_ERR_INVALID_ARG;
   return compress_layer_impl(cfg, layer, q_win, k, v, window_lse, seq_lens, batch, k_out, v_out, indices,
                              scores_or_null, ld_scores, workspace, workspace_bytes, stream);
+}
+
+// Window attention fused with the scores: row statistics sweep, merge, then the fused pass; with a layer
+// (layer >= 0) the selection and the gather follow as in pyramidkv_compress_layer.
+static int attend_impl(const pkv_config* cfg, int32_t layer, pkv_tensor q_win, pkv_tensor k, pkv_tensor v,
+                       const int32_t* seq_lens, int32_t batch, float* attn_out, void* k_out, void* v_out,
+                       int32_t* indices, float* scores_or_null, int64_t ld_scores, void* workspace,
+                       size_t workspace_bytes, void* stream) {
+  if (!config_ok(cfg)) return PKV_ERR_INVALID_ARG;
+  if (int rc = config_supported(cfg)) return rc;
+  if (!attend_eligible(cfg)) return PKV_ERR_UNSUPPORTED;
+  const bool compress = layer >= 0;
+  if (compress && layer >= cfg->num_layers) return PKV_ERR_INVALID_ARG;
+  if (!tensor_ok(q_win, cfg->head_dim, 2, batch, cfg->num_q_heads) ||
+      !tensor_ok(k, cfg->head_dim, 2, batch, cfg->num_kv_heads) || !tensor_ok(v, cfg->head_dim, 2, batch, cfg->num_kv_heads))
+    return PKV_ERR_INVALID_ARG;
+  if (!attn_out || reinterpret_cast<uintptr_t>(attn_out) % 16) return PKV_ERR_INVALID_ARG;
+  if (compress) {
+    if (!k_out || !v_out || !indices) return PKV_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(k_out) % 16 || reinterpret_cast<uintptr_t>(v_out) % 16) return PKV_ERR_INVALID_ARG;
+  } else if (!scores_or_null) {
+    return PKV_ERR_INVALID_ARG;
+  }
+  const int32_t k_layer = compress ? layer_budget(cfg, layer) : 0;
+  SeqTable table;
+  int max_n;
+  int64_t rows;
+  if (int rc = build_table(cfg, seq_lens, batch, k_layer, &table, &max_n, &rows)) return rc;
+  Workspace w;
+  if (int rc = workspace_check(cfg, batch, max_n, workspace, workspace_bytes, &w)) return rc;
+  float* scores = scores_or_null ? scores_or_null : w.scores;
+  const int64_t ld = scores_or_null ? ld_scores : w.ld_scores;
+  if (ld < max_n - cfg->window) return PKV_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (int rc = run_scores(cfg, q_win, k, table, batch, scores, ld, w, st, nullptr, /*stats_only=*/true)) return rc;
+  if (int rc = run_attend(cfg, q_win, k, v, table, batch, max_n, scores, ld, attn_out, w, st)) return rc;
+  if (!compress) return PKV_OK;
+  return run_select(cfg, scores, ld, table, batch, max_n, indices, w, st, &k, &v, k_out, v_out);
+}
+
+int pyramidkv_attend_window(const pkv_config* cfg, pkv_tensor q_win, pkv_tensor k, pkv_tensor v,
+                            const int32_t* seq_lens, int32_t batch, float* attn_out, float* scores,
+                            int64_t ld_scores, void* workspace, size_t workspace_bytes, void* stream) {
+  return attend_impl(cfg, -1, q_win, k, v, seq_lens, batch, attn_out, nullptr, nullptr, nullptr, scores, ld_scores,
+                     workspace, workspace_bytes, stream);
+}
+
+int pyramidkv_attend_compress_layer(const pkv_config* cfg, int32_t layer, pkv_tensor q_win, pkv_tensor k, pkv_tensor v,
+                                    const int32_t* seq_lens, int32_t batch, float* attn_out, void* k_out,
+                                    void* v_out, int32_t* indices, float* scores_or_null, int64_t ld_scores,
+                                    void* workspace, size_t workspace_bytes, void* stream) {
+  if (layer < 0) return PKV_ERR_INVALID_ARG;
+  return attend_impl(cfg, layer, q_win, k, v, seq_lens, batch, attn_out, k_out, v_out, indices, scores_or_null,
+                     ld_scores, workspace, workspace_bytes, stream);
 }
 
 static int profile_layer_impl(const pkv_config* cfg, int32_t layer, pkv_tensor q_win, pkv_tensor k, pkv_tensor v,

@@ -1,0 +1,481 @@
+// The window rows' attention and the window scores from one pass over K and V (Section 4.1 and
+// Section 4.2.2, Eq. 2 and Eq. 3): the scores of Eq. 3 are column sums of the very attention matrix
+// whose rows, multiplied by V, are what the prefill attention returns for the last alpha queries.
+// This kernel is that attention for those rows (all query heads of a KV head at once) and emits the
+// scores from inside it:
+//
+//   S[key i][row r]   = K Q^T                       tcgen05.mma, TMEM lane = key   (as the score sweep)
+//   e_ri              = 2^(x_ri - lse2_r + 15)      x = S * log2(e) / sqrt(d); lse2 = the row's final
+//                                                   normaliser (from the row-statistics sweep) + log2 G
+//   score_i           = 2^-15 * sum_r e_ri          Eq. 3 (mean over the group's query heads)
+//   O^T[c][row r]    += sum_i V[i][c] * e_ri        tcgen05.mma, A = V tile (d-major), B = e rounded to the
+//                                                   inputs' 16-bit type in shared memory (row-major per key)
+//   out[r][c]         = G * 2^-15 * O^T[c][r]       summed over the CTAs that share a head (reduce kernel)
+//
+// The normalisers are final before the pass starts, so the accumulators are never rescaled.  The factor
+// 2^15 keeps binary16 probabilities of long contexts out of the subnormal range; it is exact.
+//
+// Warp roles: 0 = TMA producer of Q and K, 1 = MMA issuer and TMEM owner, 2 = TMA producer of V,
+// 4..11 = epilogue in two groups of four warps (TMEM lane quarter = warp % 4).  An accumulator unit
+// is one K tile x (up to) 128 window rows; unit u lives in S stage u % 2 and is evaluated by group
+// u % 2, which writes the unit's e values to its own P buffer.  The issuer queues S(u + 1) before
+// P x V of unit u, so the tensor pipe works on the next logits while a group evaluates exponentials.
+// TMEM: columns 0..255 two S stages, 256..511 O^T (lane = channel c, column = window row).
+//
+// Every wait on an mbarrier is bounded, as in the score sweeps: a wait that runs out sets the abort
+// flag, all roles leave their loops, copies in flight are drained, TMEM is released.
+#pragma once
+
+#include "pkv_score_tc.cuh"
+
+namespace pkv {
+
+constexpr int kAtThreads = 384;
+constexpr int kAtEpiWarp0 = 4;
+constexpr int kAtEpiWarps = 8;
+constexpr int kAtTileKeys = 128;
+constexpr int kAtD = 128;                // head dimension this kernel is built for
+constexpr int kAtKStages = 2;
+constexpr int kAtShift = 15;             // e values carry a factor 2^15
+constexpr int kAtTileBytes = kAtTileKeys * kAtD * 2;        // a K or V tile, or one P buffer (128 keys x 128 rows)
+constexpr int kAtQOff = 0;
+constexpr int kAtQBytes = kTcMaxRows * kAtD * 2;
+constexpr int kAtKOff = kAtQOff + kAtQBytes;
+constexpr int kAtVOff = kAtKOff + kAtKStages * kAtTileBytes;
+constexpr int kAtPOff = kAtVOff + kAtTileBytes;
+constexpr int kAtMiscOff = kAtPOff + 2 * kAtTileBytes;
+constexpr int kAtMiscBytes = 3072;       // barriers 0.., TMEM slot 256, abort flag 260, exchange 512.., -lse2 1024..
+constexpr int kAtSmemBytes = kAtMiscOff + kAtMiscBytes;     // 227 KB: all a CTA can have
+static_assert(kAtSmemBytes <= 232448, "shared memory of the window-attention kernel");
+
+struct AtParams {
+  SeqTable seq;                 // score_off counts this kernel's work items: chunks of chunk_tiles tiles over ALL n keys
+  int32_t num_kv_heads, group, rows, rows_pad, fp16;
+  int32_t chunk_tiles;
+  long long wait_clocks;
+  float scale_log2;             // log2(e) / sqrt(d)
+  const float* lse2;            // [batch][H_kv][R]: log2 of the row's sum of 2^x, plus log2 G
+  float* scores;                // [batch][H_kv][ld]: the prefix positions are written
+  int64_t ld_scores;
+  float* o_partial;             // [segment][R][d]: a segment is one CTA's run over one (sequence, head)
+  float* out;                   // reduce kernel: [batch][H_q][alpha][d]
+  int32_t grid;                 // CTAs the attention kernel runs with (the reduce kernel finds a head's segments from it)
+  uint32_t* status;
+};
+
+// Shared-memory matrix descriptor of a 16-bit operand stored M/N-major (the 64 elements that are contiguous run
+// along M or N, one 128-byte line per contraction index, 128-byte swizzle): groups of 8 contraction indices are
+// 1024 bytes apart, blocks of 64 elements along M/N `block_bytes` apart.  `addr` advances by 2048 bytes per
+// 16-step of the contraction.
+__device__ __forceinline__ uint64_t smem_desc_mn_sw128(uint32_t addr, uint32_t block_bytes) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((addr & 0x3FFFFu) >> 4);
+  d |= static_cast<uint64_t>(block_bytes >> 4) << 16;
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;
+  d |= static_cast<uint64_t>(1) << 46;
+  d |= static_cast<uint64_t>(2) << 61;
+  return d;
+}
+
+__device__ __forceinline__ uint32_t pack_16bit(float lo, float hi, int fp16) {
+  if (fp16) {
+    const __half2 h = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&h);
+  }
+  const __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&h);
+}
+
+__global__ void __launch_bounds__(kAtThreads, 1)
+window_attend_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
+                     const __grid_constant__ CUtensorMap v_map, const AtParams p) {
+  extern __shared__ __align__(1024) uint8_t at_smem[];
+  uint8_t* smem = at_smem;
+  pdl_trigger();
+  if (smem_u32(smem) & 1023u) {                                // the carve-up below needs this; never seen otherwise
+    if (threadIdx.x == 0) atomicOr(p.status, kStatusWaitExpired);
+    return;
+  }
+  uint8_t* q_s = smem + kAtQOff;
+  uint8_t* k_s = smem + kAtKOff;
+  uint8_t* v_s = smem + kAtVOff;
+  uint8_t* p_s = smem + kAtPOff;
+  uint8_t* misc = smem + kAtMiscOff;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(misc);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 256);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 260);
+  float* xch = reinterpret_cast<float*>(misc + 512);           // [128] partial score sums, group 1 -> group 0
+  float* lse_all = reinterpret_cast<float*>(misc + 1024);      // [2][256] shifted -lse2 of the current / next head
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t bar0 = smem_u32(bars);
+  auto k_full = [&](int s) { return bar0 + 8u * s; };
+  auto k_empty = [&](int s) { return bar0 + 8u * (2 + s); };
+  const uint32_t v_full = bar0 + 8u * 4, v_empty = bar0 + 8u * 5;
+  auto s_full = [&](int s) { return bar0 + 8u * (6 + s); };
+  auto s_empty = [&](int s) { return bar0 + 8u * (8 + s); };
+  auto p_full = [&](int s) { return bar0 + 8u * (10 + s); };
+  auto p_empty = [&](int s) { return bar0 + 8u * (12 + s); };
+  const uint32_t q_full = bar0 + 8u * 14, q_empty = bar0 + 8u * 15;
+  const uint32_t o_full = bar0 + 8u * 16, o_empty = bar0 + 8u * 17;
+  const uint32_t x_full = bar0 + 8u * 18, x_empty = bar0 + 8u * 19;
+  const uint32_t lse_full = bar0 + 8u * 20;
+
+  const int halves = p.rows_pad > 128 ? 2 : 1;                 // units per K tile
+  const int n_s = halves == 2 ? 128 : p.rows_pad;              // window rows (columns) of one S unit
+  const int n_pv = n_s < 64 ? 64 : n_s;                        // ... and of its P x V product (whole 64-row blocks)
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(k_full(s), 1); mbar_init(k_empty(s), 1);
+      mbar_init(s_full(s), 1); mbar_init(s_empty(s), 4);
+      mbar_init(p_full(s), 4); mbar_init(p_empty(s), 1);
+    }
+    mbar_init(v_full, 1); mbar_init(v_empty, 1);
+    mbar_init(q_full, 1); mbar_init(q_empty, 1);
+    mbar_init(o_full, 1); mbar_init(o_empty, kAtEpiWarps);
+    mbar_init(x_full, 4); mbar_init(x_empty, 4);
+    mbar_init(lse_full, kAtEpiWarps);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  // Q rows beyond R and P rows beyond the unit's width stay zero for the whole kernel
+  for (int i = threadIdx.x; i < kAtQBytes / 16; i += kAtThreads) reinterpret_cast<uint4*>(q_s)[i] = make_uint4(0, 0, 0, 0);
+  for (int i = threadIdx.x; i < 2 * kAtTileBytes / 16; i += kAtThreads) reinterpret_cast<uint4*>(p_s)[i] = make_uint4(0, 0, 0, 0);
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();                                                  // the normalisers come from the kernels before
+
+  const int32_t* off = p.seq.score_off;
+  const int total = p.num_kv_heads * off[p.seq.batch];
+  const int per = total / gridDim.x, rem = total % gridDim.x;
+  const int item0 = blockIdx.x * per + min(static_cast<int>(blockIdx.x), rem);
+  const int item1 = item0 + per + (static_cast<int>(blockIdx.x) < rem ? 1 : 0);
+  auto tiles_of = [&](const TcItem& w, int& tile0, int& tile1) {
+    tile0 = w.c * p.chunk_tiles;
+    tile1 = min(tile0 + p.chunk_tiles, (p.seq.n[w.b] + kAtTileKeys - 1) / kAtTileKeys);
+  };
+
+  if (warp == 0) {
+    // =========================================================== TMA producer: Q per head, K per tile
+    if (lane == 0) {
+      uint32_t it = 0, heads_loaded = 0;
+      int cur_b = -1, cur_h = -1;
+      bool ok = true;
+      for (int id = item0; id < item1 && ok; ++id) {
+        const TcItem w = tc_item(off, p.seq.batch, p.num_kv_heads, id);
+        if (w.b != cur_b || w.h != cur_h) {
+          if (heads_loaded > 0) ok = mbar_wait(q_empty, (heads_loaded - 1) & 1, abort_flag, p.wait_clocks);
+          if (!ok) break;
+          mbar_expect_tx(q_full, static_cast<uint32_t>(p.rows) * kAtD * 2);
+          for (int half = 0; half < 2; ++half)
+            tma_load_4d(smem_u32(q_s) + half * kTcMaxRows * 128, &q_map, q_full, half * 64, 0, w.h * p.group, w.b);
+          ++heads_loaded;
+          cur_b = w.b; cur_h = w.h;
+        }
+        int tile0, tile1;
+        tiles_of(w, tile0, tile1);
+        for (int t = tile0; t < tile1 && ok; ++t, ++it) {
+          const int s = it % kAtKStages;
+          ok = mbar_wait(k_empty(s), ((it / kAtKStages) & 1) ^ 1, abort_flag, p.wait_clocks);
+          if (!ok) break;
+          mbar_expect_tx(k_full(s), kAtTileBytes);
+          for (int half = 0; half < 2; ++half)
+            tma_load_4d(smem_u32(k_s) + s * kAtTileBytes + half * kAtTileKeys * 128, &k_map, k_full(s), half * 64,
+                        t * kAtTileKeys, w.h, w.b);
+        }
+      }
+      if (!ok) {
+        const uint32_t first = it > kAtKStages ? it - kAtKStages : 0;
+        for (uint32_t j = first; j < it; ++j)
+          for (uint32_t spin = 0; spin < (1u << 16) && !mbar_test(k_full(j % kAtKStages), (j / kAtKStages) & 1); ++spin)
+            __nanosleep(64);
+        if (heads_loaded > 0)
+          for (uint32_t spin = 0; spin < (1u << 16) && !mbar_test(q_full, (heads_loaded - 1) & 1); ++spin) __nanosleep(64);
+      }
+    }
+  } else if (warp == 2) {
+    // =========================================================== TMA producer: V per tile (one stage)
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int id = item0; id < item1 && ok; ++id) {
+        const TcItem w = tc_item(off, p.seq.batch, p.num_kv_heads, id);
+        int tile0, tile1;
+        tiles_of(w, tile0, tile1);
+        for (int t = tile0; t < tile1 && ok; ++t, ++it) {
+          ok = mbar_wait(v_empty, (it & 1) ^ 1, abort_flag, p.wait_clocks);
+          if (!ok) break;
+          mbar_expect_tx(v_full, kAtTileBytes);
+          for (int half = 0; half < 2; ++half)
+            tma_load_4d(smem_u32(v_s) + half * kAtTileKeys * 128, &v_map, v_full, half * 64, t * kAtTileKeys, w.h, w.b);
+        }
+      }
+      if (!ok && it > 0)
+        for (uint32_t spin = 0; spin < (1u << 16) && !mbar_test(v_full, (it - 1) & 1); ++spin) __nanosleep(64);
+    }
+  } else if (warp == 1) {
+    // =========================================================== MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc_s = instr_desc_16bit(kAtTileKeys, n_s, p.fp16);
+      const uint32_t idesc_pv = instr_desc_16bit(kAtD, n_pv, p.fp16) | (1u << 15) | (1u << 16);   // A and B M/N-major
+      uint32_t it = 0, u = 0, heads_seen = 0, runs = 0;
+      int cur_b = -1, cur_h = -1;
+      bool ok = true, fresh[2] = {true, true}, wait_o = false;
+      struct Unit { bool valid; uint32_t u, it; int hf; bool last; } pend = {false, 0, 0, 0, false};
+      auto issue_pv = [&](const Unit& q) -> bool {
+        const int st = q.u & 1;
+        if (!mbar_wait(p_full(st), (q.u >> 1) & 1, abort_flag, p.wait_clocks)) return false;
+        if (q.hf == 0 && !mbar_wait(v_full, q.it & 1, abort_flag, p.wait_clocks)) return false;
+        if (wait_o) {                                          // the epilogue has read the accumulators of the run before
+          if (!mbar_wait(o_empty, (runs - 1) & 1, abort_flag, p.wait_clocks)) return false;
+          wait_o = false;
+        }
+        tc_fence_after();
+        const uint32_t d_addr = tmem_base + 256 + q.hf * 128;
+        const uint32_t v_addr = smem_u32(v_s), p_addr = smem_u32(p_s) + st * kAtTileBytes;
+#pragma unroll
+        for (int kk = 0; kk < kAtTileKeys / 16; ++kk)
+          tc_mma_f16kind(d_addr, smem_desc_mn_sw128(v_addr + kk * 2048, kAtTileKeys * 128),
+                         smem_desc_mn_sw128(p_addr + kk * 2048, kAtTileKeys * 128), idesc_pv,
+                         (fresh[q.hf] && kk == 0) ? 0u : 1u);
+        fresh[q.hf] = false;
+        tc_commit(p_empty(st));
+        if (q.last) tc_commit(v_empty);
+        return true;
+      };
+      auto end_run = [&]() -> bool {
+        if (pend.valid && !issue_pv(pend)) return false;
+        pend.valid = false;
+        tc_commit(o_full);
+        ++runs;
+        wait_o = true;
+        fresh[0] = fresh[1] = true;
+        return true;
+      };
+      for (int id = item0; id < item1 && ok; ++id) {
+        const TcItem w = tc_item(off, p.seq.batch, p.num_kv_heads, id);
+        if (w.b != cur_b || w.h != cur_h) {
+          if (cur_b >= 0) ok = end_run();
+          if (!ok) break;
+          ok = mbar_wait(q_full, heads_seen & 1, abort_flag, p.wait_clocks);
+          if (!ok) break;
+          ++heads_seen;
+          cur_b = w.b; cur_h = w.h;
+        }
+        bool last_of_head = id + 1 >= item1;
+        if (!last_of_head) {
+          const TcItem nx = tc_item(off, p.seq.batch, p.num_kv_heads, id + 1);
+          last_of_head = nx.b != w.b || nx.h != w.h;
+        }
+        int tile0, tile1;
+        tiles_of(w, tile0, tile1);
+        for (int t = tile0; t < tile1 && ok; ++t, ++it) {
+          const int s = it % kAtKStages;
+          ok = mbar_wait(k_full(s), (it / kAtKStages) & 1, abort_flag, p.wait_clocks);
+          if (!ok) break;
+          const uint32_t k_addr = smem_u32(k_s) + s * kAtTileBytes, q_addr = smem_u32(q_s);
+          for (int hf = 0; hf < halves && ok; ++hf, ++u) {
+            const int st = u & 1;
+            ok = mbar_wait(s_empty(st), ((u >> 1) & 1) ^ 1, abort_flag, p.wait_clocks);
+            if (!ok) break;
+            tc_fence_after();
+#pragma unroll
+            for (int kk = 0; kk < kAtD / 16; ++kk) {
+              const uint32_t ka = k_addr + (kk / 4) * kAtTileKeys * 128 + (kk % 4) * 32;
+              const uint32_t qa = q_addr + (kk / 4) * kTcMaxRows * 128 + hf * 128 * 128 + (kk % 4) * 32;
+              tc_mma_f16kind(tmem_base + st * 128, smem_desc_sw128(ka), smem_desc_sw128(qa), idesc_s, kk > 0);
+            }
+            tc_commit(s_full(st));
+            if (hf == halves - 1) tc_commit(k_empty(s));
+            if (pend.valid) ok = issue_pv(pend);
+            pend = Unit{true, u, it, hf, hf == halves - 1};
+          }
+        }
+        if (ok && last_of_head) tc_commit(q_empty);
+      }
+      if (ok && cur_b >= 0) end_run();
+    }
+  } else if (warp >= kAtEpiWarp0) {
+    // =========================================================== epilogue
+    const int e = warp - kAtEpiWarp0;
+    const int quarter = warp & 3, grp = e >> 2;
+    const int lane_row = quarter * 32 + lane;                  // TMEM lane: key of a tile in S, channel in O^T
+    const uint32_t lanes = static_cast<uint32_t>(quarter * 32) << 16;
+    const float c2 = p.scale_log2;
+    const float unshift = 1.0f / static_cast<float>(1 << kAtShift);
+    uint32_t it = 0, u = 0, heads_seen = 0, runs = 0;
+    const float* nl = lse_all;
+    int cur_b = -1, cur_h = -1;
+    bool ok = true;
+    // Hands the accumulators of the run that ends to global memory (raw: the reduce kernel scales).
+    auto flush_o = [&]() -> bool {
+      bool good = mbar_wait(o_full, runs & 1, abort_flag, p.wait_clocks);
+      good = __all_sync(0xffffffffu, good);
+      if (!good) return false;
+      tc_fence_after();
+      const int ncols = halves == 2 ? 256 : n_pv;
+      const int64_t seg = static_cast<int64_t>(blockIdx.x) + cur_b * p.num_kv_heads + cur_h;
+      float* dst = p.o_partial + seg * p.rows * kAtD + lane_row;
+      for (int cg = grp * (ncols / 2); cg < (grp + 1) * (ncols / 2); cg += 16) {
+        uint32_t v[16];
+        tc_ld16(tmem_base + lanes + 256 + cg, v);
+        tc_wait_ld();
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+          if (cg + j < p.rows) dst[static_cast<int64_t>(cg + j) * kAtD] = __uint_as_float(v[j]);
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(o_empty);
+      ++runs;
+      return true;
+    };
+    for (int id = item0; id < item1 && ok; ++id) {
+      const TcItem w = tc_item(off, p.seq.batch, p.num_kv_heads, id);
+      const int n = p.seq.n[w.b], alpha = p.seq.alpha, P = p.seq.prefix[w.b];
+      if (w.b != cur_b || w.h != cur_h) {
+        if (cur_b >= 0) ok = flush_o();
+        if (!ok) break;
+        // the head's normalisers, negated and shifted, in one of two buffers that alternate from head to head
+        float* dst = lse_all + (heads_seen & 1u) * 256;
+        const int r = e * 32 + lane;
+        const float* src = p.lse2 + (static_cast<int64_t>(w.b) * p.num_kv_heads + w.h) * p.rows;
+        dst[r] = r < p.rows ? static_cast<float>(kAtShift) - src[r] : -INFINITY;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(lse_full);
+        ok = mbar_wait(lse_full, heads_seen & 1u, abort_flag, p.wait_clocks);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        nl = dst;
+        ++heads_seen;
+        cur_b = w.b; cur_h = w.h;
+      }
+      float* srow = p.scores + (static_cast<int64_t>(w.b) * p.num_kv_heads + w.h) * p.ld_scores;
+      int tile0, tile1;
+      tiles_of(w, tile0, tile1);
+      for (int t = tile0; t < tile1 && ok; ++t, ++it) {
+        for (int hf = 0; hf < halves && ok; ++hf, ++u) {
+          if (static_cast<int>(u & 1u) != grp) continue;       // the other group's unit
+          const int st = u & 1;
+          ok = mbar_wait(s_full(st), (u >> 1) & 1, abort_flag, p.wait_clocks);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          ok = mbar_wait(p_empty(st), ((u >> 1) & 1) ^ 1, abort_flag, p.wait_clocks);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          tc_fence_after();
+          const int i = t * kAtTileKeys + lane_row;
+          const bool in_seq = i < n;
+          const int jp = i - P;                                // window key P + jp is seen by rows j >= jp
+          const uint32_t taddr = tmem_base + lanes + st * 128;
+          uint8_t* prow = p_s + st * kAtTileBytes + lane_row * 128;
+          const float* nlr = nl + hf * 128;
+          float sum = 0.f;
+          for (int cg = 0; cg < n_s; cg += 16) {
+            uint32_t v[16];
+            tc_ld16(taddr + cg, v);
+            tc_wait_ld();
+            float ev[16];
+            if (!in_seq) {
+#pragma unroll
+              for (int j = 0; j < 16; ++j) ev[j] = 0.f;
+            } else if (jp <= 0) {
+#pragma unroll
+              for (int j = 0; j < 16; ++j) ev[j] = ex2(fmaf(__uint_as_float(v[j]), c2, nlr[cg + j]));
+            } else {
+#pragma unroll
+              for (int j = 0; j < 16; ++j) {
+                const float x = ex2(fmaf(__uint_as_float(v[j]), c2, nlr[cg + j]));
+                ev[j] = (hf * 128 + cg + j) % alpha >= jp ? x : 0.f;
+              }
+            }
+            uint32_t pk[8];
+#pragma unroll
+            for (int j = 0; j < 16; j += 2) {
+              sum += ev[j] + ev[j + 1];
+              pk[j >> 1] = pack_16bit(ev[j], ev[j + 1], p.fp16);
+            }
+            const int nb = cg >> 6, c0 = (cg & 63) >> 3;       // 64-row block and first 16-byte chunk inside it
+            uint8_t* blk = prow + nb * (kAtTileKeys * 128);
+            *reinterpret_cast<uint4*>(blk + ((c0 ^ (lane_row & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            *reinterpret_cast<uint4*>(blk + (((c0 + 1) ^ (lane_row & 7)) << 4)) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+          }
+          if (hf == 0 && (t + 1) * kAtTileKeys > n) {
+            // last tile of a sequence: what lies behind the sequence in V may be anything, and 0 x NaN is NaN
+            ok = mbar_wait(v_full, it & 1, abort_flag, p.wait_clocks);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            if (!in_seq)
+              for (int half = 0; half < 2; ++half)
+#pragma unroll
+                for (int c = 0; c < 8; ++c)
+                  reinterpret_cast<uint4*>(v_s + half * kAtTileKeys * 128 + lane_row * 128)[c] = make_uint4(0, 0, 0, 0);
+          }
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) { mbar_arrive(p_full(st)); mbar_arrive(s_empty(st)); }
+          if (halves == 2) {
+            if (hf == 1) {
+              ok = mbar_wait(x_empty, (it & 1) ^ 1, abort_flag, p.wait_clocks);
+              ok = __all_sync(0xffffffffu, ok);
+              if (!ok) break;
+              xch[lane_row] = sum;
+              __syncwarp();
+              if (lane == 0) mbar_arrive(x_full);
+            } else {
+              ok = mbar_wait(x_full, it & 1, abort_flag, p.wait_clocks);
+              ok = __all_sync(0xffffffffu, ok);
+              if (!ok) break;
+              sum += xch[lane_row];
+              __syncwarp();
+              if (lane == 0) mbar_arrive(x_empty);
+            }
+          }
+          if (hf == 0 && i < P) srow[i] = sum * unshift;
+        }
+      }
+    }
+    if (ok && cur_b >= 0) flush_o();
+  }
+
+  // ---- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag) atomicOr(p.status, kStatusWaitExpired);
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+  }
+}
+
+// out[b][h * G + g][j][c] = G * 2^-15 * sum over the head's segments of o_partial[segment][g * alpha + j][c].
+// grid (R, H_kv, batch), block d.
+__global__ void __launch_bounds__(kAtD) window_attend_reduce_kernel(const AtParams p) {
+  pdl_trigger();
+  pdl_wait();
+  const int r = blockIdx.x, h = blockIdx.y, b = blockIdx.z, c = threadIdx.x;
+  const int nc = p.seq.score_off[b + 1] - p.seq.score_off[b];
+  const int total = p.num_kv_heads * p.seq.score_off[p.seq.batch];
+  const int per = total / p.grid, rem = total % p.grid, edge = rem * (per + 1);
+  const int i0 = p.num_kv_heads * p.seq.score_off[b] + h * nc, i1 = i0 + nc - 1;
+  const int c0 = i0 < edge ? i0 / (per + 1) : rem + (i0 - edge) / per;
+  const int c1 = i1 < edge ? i1 / (per + 1) : rem + (i1 - edge) / per;
+  const int hg = b * p.num_kv_heads + h;
+  float acc = 0.f;
+  for (int s = c0 + hg; s <= c1 + hg; ++s) acc += __ldcg(p.o_partial + (static_cast<int64_t>(s) * p.rows + r) * kAtD + c);
+  const int alpha = p.seq.alpha, g = r / alpha, j = r % alpha;
+  const int64_t hq = static_cast<int64_t>(b) * p.num_kv_heads * p.group + h * p.group + g;
+  p.out[(hq * alpha + j) * kAtD + c] = acc * static_cast<float>(p.group) / static_cast<float>(1 << kAtShift);
+}
+
+}  // namespace pkv
