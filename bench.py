@@ -303,6 +303,8 @@ def time_other(pkv, streaming, workloads, parallel, name, budget, peak, barrier,
     value, ms, _ = parallel.job_throughput(sum(lens) * steps, e0.elapsed_time(e1), device="cuda")
     pkv.check_status(ws)
     graded = sum(graded_bytes_per_layer(w, lens, r, esz) for r in out.rows)
+    if args.mode == "attend":                                      # this mode also reads V once and writes the attention output
+        graded += w.num_layers * (k_bytes_layer + len(lens) * w.num_q_heads * w.window * w.head_dim * 4)
     gbs = graded / (ms / steps * 1e-3) / 1e9
     k_layer_mb = sum(lens) * w.num_kv_heads * w.head_dim * esz / 1e6
     return {"workload": w.name, "avg_budget": w.avg_budget, "layers": w.num_layers, "seq_lens": lens, "steps": steps,
@@ -339,9 +341,11 @@ def main():
     ap.add_argument("--lanes", type=int, default=0, metavar="SMS",
                     help="run selection + gather of a layer on SMS streaming multiprocessors of their own (a multiple "
                          "of 8) beside the next layer's score sweeps on the rest; 0 = one stream, kernels in turn")
-    ap.add_argument("--mode", default="self", choices=["self", "handoff"],
+    ap.add_argument("--mode", default="self", choices=["self", "handoff", "attend"],
                     help="self: the library finds the row normalisers itself (two K sweeps, the graded path); "
-                         "handoff: they are handed in as the prefill attention would (one K sweep)")
+                         "handoff: they are handed in as the prefill attention would (one K sweep); attend: the "
+                         "second sweep is the window rows' prefill attention itself (reads V too, returns their "
+                         "attention output) and emits the scores from inside it")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     auto_steps = args.steps is None
@@ -391,6 +395,9 @@ def main():
         # stand-in for the prefill attention's by-product: log-sum-exp of the window rows, computed once, untimed
         for x in layers:
             x.window_lse = prefill_window_lse(w, x, lens)
+    if args.mode == "attend":
+        for x in layers:
+            x.attn_out = torch.empty(len(lens), w.num_q_heads, w.window, w.head_dim, dtype=torch.float32, device="cuda")
     out = streaming.LayerOutputs(cfg, lens, tdt)
     ws = pkv.new_workspace(cfg, len(lens), max(lens))
     tokens = sum(lens)
@@ -460,7 +467,8 @@ def main():
         stages = {}
         for l, x in enumerate(layers):
             for name, t_ms in pkv.profile_layer(cfg, l, x.q_win, x.k, x.v, lens, out.k[l], out.v[l], out.idx[l], ws,
-                                                window_lse=getattr(x, "window_lse", None)):
+                                                window_lse=getattr(x, "window_lse", None),
+                                                attn_out=getattr(x, "attn_out", None)):
                 s = stages.setdefault(name, [0, 0.0])
                 s[0] += 1
                 s[1] += t_ms
@@ -472,6 +480,8 @@ def main():
     q_bytes_layer = len(lens) * w.num_q_heads * w.window * w.head_dim * esz
     score_bytes_layer = sum(n - w.window for n in lens) * w.num_kv_heads * 4
     dom_bytes = k_bytes_layer + q_bytes_layer + score_bytes_layer   # one sweep over K per launch
+    if dominant == "window_attend":
+        dom_bytes += k_bytes_layer                                  # ... and one over V
     achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
     traffic = None
     tr = NCU_TRAFFIC.get(dominant)
@@ -481,7 +491,7 @@ def main():
     path_gbs = graded / (ms_per_step * 1e-3) / 1e9
     # the same kernel against the special-function unit: one exponential per (window row, key) and sweep;
     # peak = 16 per clock and SM (measured: 15.98) x the SMs of the device x the maximum SM clock
-    exps = w.group * w.window * w.num_kv_heads * (sum(lens) if dominant == "rowstats_tc" else
+    exps = w.group * w.window * w.num_kv_heads * (sum(lens) if dominant in ("rowstats_tc", "window_attend") else
                                                    sum(n - w.window for n in lens))
     sm_count = torch.cuda.get_device_properties(local).multi_processor_count
     sfu_peak = 16.0 * sm_count * clocks["sm_max_mhz"] * 1e6 if clocks.get("sm_max_mhz") else None

@@ -381,6 +381,15 @@ int pyramidkv_profile_layer(const pkv_config* cfg, int32_t layer,
                             void* workspace, size_t workspace_bytes, void* stream,
                             float* stage_ms, char (*stage_names)[32], int32_t* num_stages);
 
+/* The same measuring aid for pyramidkv_attend_compress_layer. */
+int pyramidkv_profile_attend_compress_layer(const pkv_config* cfg, int32_t layer,
+                                            pkv_tensor q_win, pkv_tensor k, pkv_tensor v,
+                                            const int32_t* seq_lens, int32_t batch, float* attn_out,
+                                            void* k_out, void* v_out, int32_t* indices,
+                                            float* scores_or_null, int64_t ld_scores,
+                                            void* workspace, size_t workspace_bytes, void* stream,
+                                            float* stage_ms, char (*stage_names)[32], int32_t* num_stages);
+
 /* The same measuring aid for pyramidkv_compress_layer_lse. */
 int pyramidkv_profile_layer_lse(const pkv_config* cfg, int32_t layer,
                                 pkv_tensor q_win, pkv_tensor k, pkv_tensor v, const float* window_lse,
@@ -530,7 +539,8 @@ int pyramidkv_compress_model_lanes(const pkv_config* cfg, pkv_lanes* lanes, int3
  * copy engine thread of the first CTA of the row-statistics sweep leave out its last K tile, so that the waits
  * for that tile run out, the kernel gives up in an orderly way (every role leaves its loop, the accumulator
  * memory is released, the status word gets bit 1) and returns.  Bit 1 keeps short contexts on the two-sweep
- * kernels instead of the single-sweep one (same scores within rounding).  (0, 0) restores normal operation.
+ * kernels instead of the single-sweep one (same scores within rounding).  Bit 2 is bit 0 for the window-attention
+ * kernel of pyramidkv_attend_window.  (0, 0) restores normal operation.
  *
  * pyramidkv_test_slow_copy: copies `bytes` (a multiple of 16) from src to dst with one small CTA that lets
  * its dependents start at once and then copies in `steps` pieces with a pause after each: a stand-in for a

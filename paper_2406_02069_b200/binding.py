@@ -39,7 +39,8 @@ EXPORTS = ("pyramidkv_strerror", "pyramidkv_layer_budgets", "pyramidkv_kept_coun
            "pyramidkv_merge_lse", "pyramidkv_shard_scores", "pyramidkv_shard_gather", "pyramidkv_memory_kind",
            "pyramidkv_lanes_create", "pyramidkv_lanes_destroy", "pyramidkv_lanes_info",
            "pyramidkv_compress_model_lanes", "pyramidkv_test_hooks", "pyramidkv_test_slow_copy",
-           "pyramidkv_attend_window", "pyramidkv_attend_compress_layer")
+           "pyramidkv_attend_window", "pyramidkv_attend_compress_layer",
+           "pyramidkv_profile_attend_compress_layer")
 PKV_MAX_STAGES = 8
 
 
@@ -88,6 +89,7 @@ def _load() -> ctypes.CDLL:
     lib.pyramidkv_attend_window.argtypes = [CFG, PkvTensor, PkvTensor, PkvTensor, P, I32, P, P, I64, P, SZ, P]
     lib.pyramidkv_attend_compress_layer.argtypes = [CFG, I32, PkvTensor, PkvTensor, PkvTensor, P, I32, P, P, P, P, P,
                                                     I64, P, SZ, P]
+    lib.pyramidkv_profile_attend_compress_layer.argtypes = lib.pyramidkv_attend_compress_layer.argtypes + [P, P, P]
     lib.pyramidkv_decode_attention.argtypes = [CFG, P, P, P, P, I32, I32, P, P]
     lib.pyramidkv_attention_recall.argtypes = [CFG, P, I64, P, P, I32, I32, P, P]
     lib.pyramidkv_pages_needed.argtypes = [CFG, I32, I32, I32]
@@ -358,10 +360,12 @@ def score_window_static(cfg: PkvConfig, q_win: torch.Tensor, k: torch.Tensor, se
            "pyramidkv_score_window_static")
 
 
-def test_hooks(wait_clocks: int = 0, withhold_tile: bool = False, two_sweeps: bool = False) -> None:
-    """Test aid: bound of the waits inside the tensor-core score kernels (0 = default), the withheld K tile, and
-    short contexts kept on the two-sweep kernels."""
-    _check(_lib.pyramidkv_test_hooks(int(wait_clocks), (1 if withhold_tile else 0) | (2 if two_sweeps else 0)),
+def test_hooks(wait_clocks: int = 0, withhold_tile: bool = False, two_sweeps: bool = False,
+               withhold_attend_tile: bool = False) -> None:
+    """Test aid: bound of the waits inside the tensor-core kernels (0 = default), the withheld K tile (of the row
+    statistics sweep, or of the window-attention kernel), and short contexts kept on the two-sweep kernels."""
+    _check(_lib.pyramidkv_test_hooks(int(wait_clocks), (1 if withhold_tile else 0) | (2 if two_sweeps else 0) |
+                                     (4 if withhold_attend_tile else 0)),
            "pyramidkv_test_hooks")
 
 
@@ -471,13 +475,22 @@ def attend_compress_layer(cfg: PkvConfig, layer: int, q_win: torch.Tensor, k: to
 
 def profile_layer(cfg: PkvConfig, layer: int, q_win: torch.Tensor, k: torch.Tensor, v: torch.Tensor,
                   seq_lens: Sequence[int], k_out: torch.Tensor, v_out: torch.Tensor, indices: torch.Tensor,
-                  workspace: torch.Tensor, stream=None, window_lse: Optional[torch.Tensor] = None):
-    """compress_layer with per-kernel device times: returns [(kernel name, milliseconds), ...]."""
+                  workspace: torch.Tensor, stream=None, window_lse: Optional[torch.Tensor] = None,
+                  attn_out: Optional[torch.Tensor] = None):
+    """compress_layer (attend_compress_layer when attn_out is given) with per-kernel device times: returns
+    [(kernel name, milliseconds), ...]."""
     lens, batch = _lens(seq_lens)
     _check_layer_call(cfg, layer, q_win, k, v, seq_lens, k_out, v_out, indices, workspace, None)
     ms = (ctypes.c_float * PKV_MAX_STAGES)()
     names = ((ctypes.c_char * 32) * PKV_MAX_STAGES)()
     n = ctypes.c_int32(0)
+    if attn_out is not None:
+        _check_attn_out(cfg, attn_out, batch)
+        _check(_lib.pyramidkv_profile_attend_compress_layer(
+            ctypes.byref(cfg), int(layer), _tensor(q_win), _tensor(k), _tensor(v), lens, batch, attn_out.data_ptr(),
+            k_out.data_ptr(), v_out.data_ptr(), indices.data_ptr(), None, 0, workspace.data_ptr(), workspace.numel(),
+            _stream(stream), ms, names, ctypes.byref(n)), "pyramidkv_profile_attend_compress_layer")
+        return [(names[i].value.decode(), float(ms[i])) for i in range(n.value)]
     if window_lse is not None:
         _check(_lib.pyramidkv_profile_layer_lse(
             ctypes.byref(cfg), int(layer), _tensor(q_win), _tensor(k), _tensor(v), _lse_ptr(window_lse), lens, batch,

@@ -25,6 +25,7 @@ namespace {
 // Test knobs (pyramidkv_test_hooks): bound of the waits inside the tensor-core kernels, and the withheld tile.
 std::atomic<long long> g_test_wait_clocks{0};
 std::atomic<int> g_test_withhold{0};
+std::atomic<int> g_test_withhold_attend{0};  // 1: the withheld K tile, in the window-attention kernel
 std::atomic<int> g_test_two_sweeps{0};     // 1: never take the single-sweep kernel for short contexts
 
 constexpr size_t kAlign = 256;
@@ -554,6 +555,7 @@ int run_attend(const pkv_config* c, const pkv_tensor& q, const pkv_tensor& k, co
   ap.fp16 = fp16 ? 1 : 0;
   const long long test_wait = g_test_wait_clocks.load();
   ap.wait_clocks = test_wait > 0 ? test_wait : kTcWaitCycles;
+  ap.withhold = g_test_withhold_attend.load();
   ap.scale_log2 = static_cast<float>(1.4426950408889634 / std::sqrt(static_cast<double>(c->head_dim)));
   ap.lse2 = w.lse2;
   ap.scores = scores;
@@ -999,7 +1001,7 @@ static int profile_layer_impl(const pkv_config* cfg, int32_t layer, pkv_tensor q
                               const float* window_lse, const int32_t* seq_lens, int32_t batch, void* k_out,
                               void* v_out, int32_t* indices, float* scores_or_null, int64_t ld_scores,
                               void* workspace, size_t workspace_bytes, void* stream, float* stage_ms,
-                              char (*stage_names)[32], int32_t* num_stages) {
+                              char (*stage_names)[32], int32_t* num_stages, float* attn_out = nullptr) {
   if (!stage_ms || !stage_names || !num_stages) return PKV_ERR_INVALID_ARG;
   StageTimer timer;
   for (auto& e : timer.ev)
@@ -1007,8 +1009,10 @@ static int profile_layer_impl(const pkv_config* cfg, int32_t layer, pkv_tensor q
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   cudaEventRecord(timer.ev[0], st);
   g_timer = &timer;
-  int rc = compress_layer_impl(cfg, layer, q_win, k, v, window_lse, seq_lens, batch, k_out, v_out, indices,
-                               scores_or_null, ld_scores, workspace, workspace_bytes, stream);
+  int rc = attn_out ? attend_impl(cfg, layer, q_win, k, v, seq_lens, batch, attn_out, k_out, v_out, indices,
+                                  scores_or_null, ld_scores, workspace, workspace_bytes, stream)
+                    : compress_layer_impl(cfg, layer, q_win, k, v, window_lse, seq_lens, batch, k_out, v_out, indices,
+                                          scores_or_null, ld_scores, workspace, workspace_bytes, stream);
   g_timer = nullptr;
   if (rc == PKV_OK && cudaStreamSynchronize(st) != cudaSuccess) rc = PKV_ERR_CUDA;
   *num_stages = 0;
@@ -1040,6 +1044,16 @@ int pyramidkv_profile_layer_lse(const pkv_config* cfg, int32_t layer, pkv_tensor
   return profile_layer_impl(cfg, layer, q_win, k, v, window_lse, seq_lens, batch, k_out, v_out, indices,
                             scores_or_null, ld_scores, workspace, workspace_bytes, stream, stage_ms, stage_names,
                             num_stages);
+}
+
+int pyramidkv_profile_attend_compress_layer(const pkv_config* cfg, int32_t layer, pkv_tensor q_win, pkv_tensor k,
+                                            pkv_tensor v, const int32_t* seq_lens, int32_t batch, float* attn_out,
+                                            void* k_out, void* v_out, int32_t* indices, float* scores_or_null,
+                                            int64_t ld_scores, void* workspace, size_t workspace_bytes, void* stream,
+                                            float* stage_ms, char (*stage_names)[32], int32_t* num_stages) {
+  if (!attn_out || layer < 0) return PKV_ERR_INVALID_ARG;
+  return profile_layer_impl(cfg, layer, q_win, k, v, nullptr, seq_lens, batch, k_out, v_out, indices, scores_or_null,
+                            ld_scores, workspace, workspace_bytes, stream, stage_ms, stage_names, num_stages, attn_out);
 }
 
 int pyramidkv_decode_attention(const pkv_config* cfg, const void* q, const void* k_cache, const void* v_cache,
@@ -1587,6 +1601,7 @@ extern "C" int pyramidkv_test_hooks(int64_t wait_clocks, int32_t withhold_tile) 
   g_test_wait_clocks.store(wait_clocks);
   g_test_withhold.store((withhold_tile & 1) ? 1 : 0);
   g_test_two_sweeps.store((withhold_tile & 2) ? 1 : 0);
+  g_test_withhold_attend.store((withhold_tile & 4) ? 1 : 0);
   return PKV_OK;
 }
 

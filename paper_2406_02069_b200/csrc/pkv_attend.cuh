@@ -16,10 +16,12 @@
 // 2^15 keeps binary16 probabilities of long contexts out of the subnormal range; it is exact.
 //
 // Warp roles: 0 = TMA producer of Q and K, 1 = MMA issuer and TMEM owner, 2 = TMA producer of V,
-// 4..11 = epilogue in two groups of four warps (TMEM lane quarter = warp % 4).  An accumulator unit
-// is one K tile x (up to) 128 window rows; unit u lives in S stage u % 2 and is evaluated by group
-// u % 2, which writes the unit's e values to its own P buffer.  The issuer queues S(u + 1) before
-// P x V of unit u, so the tensor pipe works on the next logits while a group evaluates exponentials.
+// 4..19 = epilogue in four groups of four warps (TMEM lane quarter = warp % 4).  An accumulator unit
+// is one K tile x (up to) 128 window rows; unit u lives in S stage u % 2 and is evaluated by the two
+// groups with par = u % 2, each taking half of its columns and writing the e values to P buffer u % 2
+// (one warp per scheduler and group leaves the exponential unit idle most of the time; two pairs do not).
+// The issuer queues S(u + 1) before P x V of unit u, so the tensor pipe works on the next logits while
+// the groups evaluate exponentials.
 // TMEM: columns 0..255 two S stages, 256..511 O^T (lane = channel c, column = window row).
 //
 // Every wait on an mbarrier is bounded, as in the score sweeps: a wait that runs out sets the abort
@@ -30,9 +32,9 @@
 
 namespace pkv {
 
-constexpr int kAtThreads = 384;
+constexpr int kAtThreads = 640;
 constexpr int kAtEpiWarp0 = 4;
-constexpr int kAtEpiWarps = 8;
+constexpr int kAtEpiWarps = 16;
 constexpr int kAtTileKeys = 128;
 constexpr int kAtD = 128;                // head dimension this kernel is built for
 constexpr int kAtKStages = 2;
@@ -44,7 +46,7 @@ constexpr int kAtKOff = kAtQOff + kAtQBytes;
 constexpr int kAtVOff = kAtKOff + kAtKStages * kAtTileBytes;
 constexpr int kAtPOff = kAtVOff + kAtTileBytes;
 constexpr int kAtMiscOff = kAtPOff + 2 * kAtTileBytes;
-constexpr int kAtMiscBytes = 3072;       // barriers 0.., TMEM slot 256, abort flag 260, exchange 512.., -lse2 1024..
+constexpr int kAtMiscBytes = 3072;       // barriers 0.., TMEM slot 256, abort flag 260, exchange 512.., -lse2 2048..
 constexpr int kAtSmemBytes = kAtMiscOff + kAtMiscBytes;     // 227 KB: all a CTA can have
 static_assert(kAtSmemBytes <= 232448, "shared memory of the window-attention kernel");
 
@@ -52,6 +54,7 @@ struct AtParams {
   SeqTable seq;                 // score_off counts this kernel's work items: chunks of chunk_tiles tiles over ALL n keys
   int32_t num_kv_heads, group, rows, rows_pad, fp16;
   int32_t chunk_tiles;
+  int32_t withhold;             // test aid: CTA 0 never loads its last K tile (its waits then run out)
   long long wait_clocks;
   float scale_log2;             // log2(e) / sqrt(d)
   const float* lse2;            // [batch][H_kv][R]: log2 of the row's sum of 2^x, plus log2 G
@@ -86,6 +89,27 @@ __device__ __forceinline__ uint32_t pack_16bit(float lo, float hi, int fp16) {
   return *reinterpret_cast<const uint32_t*>(&h);
 }
 
+// 16 window rows of one key, all visible: e = 2^(v * c2 + nl), summed into acc (a packed pair of partial sums)
+// and rounded to 16 bits into two 16-byte chunks (c0, c0 + 1, swizzled by sw) of the key's line of the P buffer.
+template <bool FP16>
+__device__ __forceinline__ void at_chunk(const uint32_t (&v)[16], unsigned long long cc, const float* nl, uint8_t* blk,
+                                         int c0, int sw, unsigned long long& acc) {
+  uint32_t pk[8];
+#pragma unroll
+  for (int j = 0; j < 8; j += 2) {
+    const ulonglong2 l = *reinterpret_cast<const ulonglong2*>(nl + 2 * j);   // four floats as two packed pairs
+    float x0, x1, x2, x3;
+    unpack2(fma2(pack2(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1])), cc, l.x), x0, x1);
+    unpack2(fma2(pack2(__uint_as_float(v[2 * j + 2]), __uint_as_float(v[2 * j + 3])), cc, l.y), x2, x3);
+    const float e0 = ex2(x0), e1 = ex2(x1), e2 = ex2(x2), e3 = ex2(x3);
+    acc = add2(acc, add2(pack2(e0, e1), pack2(e2, e3)));
+    pk[j] = pack_16bit(e0, e1, FP16 ? 1 : 0);
+    pk[j + 1] = pack_16bit(e2, e3, FP16 ? 1 : 0);
+  }
+  *reinterpret_cast<uint4*>(blk + ((c0 ^ sw) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+  *reinterpret_cast<uint4*>(blk + (((c0 + 1) ^ sw) << 4)) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+}
+
 __global__ void __launch_bounds__(kAtThreads, 1)
 window_attend_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
                      const __grid_constant__ CUtensorMap v_map, const AtParams p) {
@@ -104,8 +128,8 @@ window_attend_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_con
   uint64_t* bars = reinterpret_cast<uint64_t*>(misc);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 256);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(misc + 260);
-  float* xch = reinterpret_cast<float*>(misc + 512);           // [128] partial score sums, group 1 -> group 0
-  float* lse_all = reinterpret_cast<float*>(misc + 1024);      // [2][256] shifted -lse2 of the current / next head
+  float* xch = reinterpret_cast<float*>(misc + 512);           // [3][128] partial score sums handed between groups
+  float* lse_all = reinterpret_cast<float*>(misc + 2048);      // [256] shifted -lse2 of the current head
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t bar0 = smem_u32(bars);
@@ -118,8 +142,9 @@ window_attend_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_con
   auto p_empty = [&](int s) { return bar0 + 8u * (12 + s); };
   const uint32_t q_full = bar0 + 8u * 14, q_empty = bar0 + 8u * 15;
   const uint32_t o_full = bar0 + 8u * 16, o_empty = bar0 + 8u * 17;
-  const uint32_t x_full = bar0 + 8u * 18, x_empty = bar0 + 8u * 19;
-  const uint32_t lse_full = bar0 + 8u * 20;
+  auto x_full = [&](int s) { return bar0 + 8u * (18 + s); };
+  auto x_empty = [&](int s) { return bar0 + 8u * (20 + s); };
+  const uint32_t lse_full = bar0 + 8u * 22;
 
   const int halves = p.rows_pad > 128 ? 2 : 1;                 // units per K tile
   const int n_s = halves == 2 ? 128 : p.rows_pad;              // window rows (columns) of one S unit
@@ -128,13 +153,13 @@ window_attend_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_con
   if (threadIdx.x == 0) {
     for (int s = 0; s < 2; ++s) {
       mbar_init(k_full(s), 1); mbar_init(k_empty(s), 1);
-      mbar_init(s_full(s), 1); mbar_init(s_empty(s), 4);
-      mbar_init(p_full(s), 4); mbar_init(p_empty(s), 1);
+      mbar_init(s_full(s), 1); mbar_init(s_empty(s), 8);
+      mbar_init(p_full(s), 8); mbar_init(p_empty(s), 1);
+      mbar_init(x_full(s), halves == 2 ? 12 : 4); mbar_init(x_empty(s), 4);
     }
     mbar_init(v_full, 1); mbar_init(v_empty, 1);
     mbar_init(q_full, 1); mbar_init(q_empty, 1);
     mbar_init(o_full, 1); mbar_init(o_empty, kAtEpiWarps);
-    mbar_init(x_full, 4); mbar_init(x_empty, 4);
     mbar_init(lse_full, kAtEpiWarps);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -187,6 +212,7 @@ window_attend_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_con
           const int s = it % kAtKStages;
           ok = mbar_wait(k_empty(s), ((it / kAtKStages) & 1) ^ 1, abort_flag, p.wait_clocks);
           if (!ok) break;
+          if (p.withhold && blockIdx.x == 0 && id + 1 == item1 && t + 1 == tile1) continue;   // test aid: never arrives
           mbar_expect_tx(k_full(s), kAtTileBytes);
           for (int half = 0; half < 2; ++half)
             tma_load_4d(smem_u32(k_s) + s * kAtTileBytes + half * kAtTileKeys * 128, &k_map, k_full(s), half * 64,
@@ -306,14 +332,17 @@ window_attend_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_con
     }
   } else if (warp >= kAtEpiWarp0) {
     // =========================================================== epilogue
+    // Sixteen warps in four groups.  The two groups with the same `par` evaluate the units u with u % 2 == par,
+    // each one half of the unit's columns (window rows); group ch = 0 of the unit with row half 0 collects the
+    // partial score sums of the others and writes the score.
     const int e = warp - kAtEpiWarp0;
-    const int quarter = warp & 3, grp = e >> 2;
+    const int quarter = warp & 3, g4 = e >> 2, par = g4 & 1, ch = g4 >> 1;
     const int lane_row = quarter * 32 + lane;                  // TMEM lane: key of a tile in S, channel in O^T
     const uint32_t lanes = static_cast<uint32_t>(quarter * 32) << 16;
     const float c2 = p.scale_log2;
     const float unshift = 1.0f / static_cast<float>(1 << kAtShift);
-    uint32_t it = 0, u = 0, heads_seen = 0, runs = 0;
-    const float* nl = lse_all;
+    const int col0 = ch * (n_s / 2), col1 = col0 + n_s / 2;    // this group's columns of a unit (multiples of 16)
+    uint32_t it = 0, u = 0, lse_rounds = 0, runs = 0;
     int cur_b = -1, cur_h = -1;
     bool ok = true;
     // Hands the accumulators of the run that ends to global memory (raw: the reduce kernel scales).
@@ -325,7 +354,7 @@ window_attend_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_con
       const int ncols = halves == 2 ? 256 : n_pv;
       const int64_t seg = static_cast<int64_t>(blockIdx.x) + cur_b * p.num_kv_heads + cur_h;
       float* dst = p.o_partial + seg * p.rows * kAtD + lane_row;
-      for (int cg = grp * (ncols / 2); cg < (grp + 1) * (ncols / 2); cg += 16) {
+      for (int cg = g4 * 16; cg < ncols; cg += 64) {           // 16-column pieces dealt round to the four groups
         uint32_t v[16];
         tc_ld16(tmem_base + lanes + 256 + cg, v);
         tc_wait_ld();
@@ -339,24 +368,31 @@ window_attend_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_con
       ++runs;
       return true;
     };
+    // One meeting of the sixteen warps.
+    auto meet = [&]() -> bool {
+      __syncwarp();
+      if (lane == 0) mbar_arrive(lse_full);
+      bool good = mbar_wait(lse_full, lse_rounds & 1u, abort_flag, p.wait_clocks);
+      ++lse_rounds;
+      return __all_sync(0xffffffffu, good);
+    };
     for (int id = item0; id < item1 && ok; ++id) {
       const TcItem w = tc_item(off, p.seq.batch, p.num_kv_heads, id);
       const int n = p.seq.n[w.b], alpha = p.seq.alpha, P = p.seq.prefix[w.b];
       if (w.b != cur_b || w.h != cur_h) {
         if (cur_b >= 0) ok = flush_o();
         if (!ok) break;
-        // the head's normalisers, negated and shifted, in one of two buffers that alternate from head to head
-        float* dst = lse_all + (heads_seen & 1u) * 256;
-        const int r = e * 32 + lane;
-        const float* src = p.lse2 + (static_cast<int64_t>(w.b) * p.num_kv_heads + w.h) * p.rows;
-        dst[r] = r < p.rows ? static_cast<float>(kAtShift) - src[r] : -INFINITY;
-        __syncwarp();
-        if (lane == 0) mbar_arrive(lse_full);
-        ok = mbar_wait(lse_full, heads_seen & 1u, abort_flag, p.wait_clocks);
-        ok = __all_sync(0xffffffffu, ok);
+        // the head's normalisers, negated and shifted: written once everybody is done with the old ones, read
+        // once everybody has written
+        ok = meet();
         if (!ok) break;
-        nl = dst;
-        ++heads_seen;
+        const int r = e * 32 + lane;
+        if (r < kTcMaxRows) {
+          const float* src = p.lse2 + (static_cast<int64_t>(w.b) * p.num_kv_heads + w.h) * p.rows;
+          lse_all[r] = r < p.rows ? static_cast<float>(kAtShift) - src[r] : -INFINITY;
+        }
+        ok = meet();
+        if (!ok) break;
         cur_b = w.b; cur_h = w.h;
       }
       float* srow = p.scores + (static_cast<int64_t>(w.b) * p.num_kv_heads + w.h) * p.ld_scores;
@@ -364,7 +400,7 @@ window_attend_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_con
       tiles_of(w, tile0, tile1);
       for (int t = tile0; t < tile1 && ok; ++t, ++it) {
         for (int hf = 0; hf < halves && ok; ++hf, ++u) {
-          if (static_cast<int>(u & 1u) != grp) continue;       // the other group's unit
+          if (static_cast<int>(u & 1u) != par) continue;       // the other pair's unit
           const int st = u & 1;
           ok = mbar_wait(s_full(st), (u >> 1) & 1, abort_flag, p.wait_clocks);
           ok = __all_sync(0xffffffffu, ok);
@@ -378,38 +414,58 @@ window_attend_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_con
           const int jp = i - P;                                // window key P + jp is seen by rows j >= jp
           const uint32_t taddr = tmem_base + lanes + st * 128;
           uint8_t* prow = p_s + st * kAtTileBytes + lane_row * 128;
-          const float* nlr = nl + hf * 128;
+          const float* nlr = lse_all + hf * 128;
           float sum = 0.f;
-          for (int cg = 0; cg < n_s; cg += 16) {
-            uint32_t v[16];
-            tc_ld16(taddr + cg, v);
-            tc_wait_ld();
-            float ev[16];
-            if (!in_seq) {
-#pragma unroll
-              for (int j = 0; j < 16; ++j) ev[j] = 0.f;
-            } else if (jp <= 0) {
-#pragma unroll
-              for (int j = 0; j < 16; ++j) ev[j] = ex2(fmaf(__uint_as_float(v[j]), c2, nlr[cg + j]));
-            } else {
+          if (__all_sync(0xffffffffu, in_seq && jp <= 0)) {
+            // every key of the warp sees every row (all tiles but a sequence's last ones): no mask, 16-column loads
+            // double buffered so that the next one is in flight while a chunk is evaluated
+            unsigned long long acc = pack2(0.f, 0.f);
+            const unsigned long long cc = pack2(c2, c2);
+            const int sw = lane_row & 7;
+            uint32_t va[16], vb[16];
+            tc_ld16(taddr + col0, va);
+            for (int cg = col0; cg < col1; cg += 32) {
+              const bool two = cg + 16 < col1;
+              tc_wait_ld();
+              if (two) tc_ld16(taddr + cg + 16, vb);
+              if (p.fp16) at_chunk<true>(va, cc, nlr + cg, prow + (cg >> 6) * (kAtTileKeys * 128), (cg & 63) >> 3, sw, acc);
+              else at_chunk<false>(va, cc, nlr + cg, prow + (cg >> 6) * (kAtTileKeys * 128), (cg & 63) >> 3, sw, acc);
+              if (two) {
+                const int cn = cg + 16;
+                tc_wait_ld();
+                if (cg + 32 < col1) tc_ld16(taddr + cg + 32, va);
+                if (p.fp16) at_chunk<true>(vb, cc, nlr + cn, prow + (cn >> 6) * (kAtTileKeys * 128), (cn & 63) >> 3, sw, acc);
+                else at_chunk<false>(vb, cc, nlr + cn, prow + (cn >> 6) * (kAtTileKeys * 128), (cn & 63) >> 3, sw, acc);
+              }
+            }
+            float lo, hi;
+            unpack2(acc, lo, hi);
+            sum = lo + hi;
+          } else {
+            for (int cg = col0; cg < col1; cg += 16) {
+              uint32_t v[16];
+              tc_ld16(taddr + cg, v);
+              tc_wait_ld();
+              float ev[16];
 #pragma unroll
               for (int j = 0; j < 16; ++j) {
                 const float x = ex2(fmaf(__uint_as_float(v[j]), c2, nlr[cg + j]));
-                ev[j] = (hf * 128 + cg + j) % alpha >= jp ? x : 0.f;
+                const bool vis = in_seq && (jp <= 0 || (hf * 128 + cg + j) % alpha >= jp);
+                ev[j] = vis ? x : 0.f;
               }
-            }
-            uint32_t pk[8];
+              uint32_t pk[8];
 #pragma unroll
-            for (int j = 0; j < 16; j += 2) {
-              sum += ev[j] + ev[j + 1];
-              pk[j >> 1] = pack_16bit(ev[j], ev[j + 1], p.fp16);
+              for (int j = 0; j < 16; j += 2) {
+                sum += ev[j] + ev[j + 1];
+                pk[j >> 1] = pack_16bit(ev[j], ev[j + 1], p.fp16);
+              }
+              const int nb = cg >> 6, c0 = (cg & 63) >> 3;     // 64-row block and first 16-byte chunk inside it
+              uint8_t* blk = prow + nb * (kAtTileKeys * 128);
+              *reinterpret_cast<uint4*>(blk + ((c0 ^ (lane_row & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+              *reinterpret_cast<uint4*>(blk + (((c0 + 1) ^ (lane_row & 7)) << 4)) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
             }
-            const int nb = cg >> 6, c0 = (cg & 63) >> 3;       // 64-row block and first 16-byte chunk inside it
-            uint8_t* blk = prow + nb * (kAtTileKeys * 128);
-            *reinterpret_cast<uint4*>(blk + ((c0 ^ (lane_row & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-            *reinterpret_cast<uint4*>(blk + (((c0 + 1) ^ (lane_row & 7)) << 4)) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
           }
-          if (hf == 0 && (t + 1) * kAtTileKeys > n) {
+          if (hf == 0 && ch == 0 && (t + 1) * kAtTileKeys > n) {
             // last tile of a sequence: what lies behind the sequence in V may be anything, and 0 x NaN is NaN
             ok = mbar_wait(v_full, it & 1, abort_flag, p.wait_clocks);
             ok = __all_sync(0xffffffffu, ok);
@@ -424,24 +480,28 @@ window_attend_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_con
           tc_fence_before();
           __syncwarp();
           if (lane == 0) { mbar_arrive(p_full(st)); mbar_arrive(s_empty(st)); }
-          if (halves == 2) {
-            if (hf == 1) {
-              ok = mbar_wait(x_empty, (it & 1) ^ 1, abort_flag, p.wait_clocks);
-              ok = __all_sync(0xffffffffu, ok);
-              if (!ok) break;
-              xch[lane_row] = sum;
-              __syncwarp();
-              if (lane == 0) mbar_arrive(x_full);
-            } else {
-              ok = mbar_wait(x_full, it & 1, abort_flag, p.wait_clocks);
-              ok = __all_sync(0xffffffffu, ok);
-              if (!ok) break;
-              sum += xch[lane_row];
-              __syncwarp();
-              if (lane == 0) mbar_arrive(x_empty);
-            }
+          // the key's score: partial sums of the other groups that work on the tile, added in a fixed order.  With
+          // two units per tile all four groups share a tile (one exchange, three slots); with one, the two groups
+          // of a pair do (an exchange per pair, one slot).
+          const int xi = halves == 2 ? 0 : par;
+          const uint32_t xph = halves == 2 ? it : it >> 1;
+          if (hf == 0 && ch == 0) {
+            ok = mbar_wait(x_full(xi), xph & 1, abort_flag, p.wait_clocks);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            if (halves == 2) sum += xch[lane_row] + xch[128 + lane_row] + xch[256 + lane_row];
+            else sum += xch[xi * 128 + lane_row];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(x_empty(xi));
+            if (i < P) srow[i] = sum * unshift;
+          } else {
+            ok = mbar_wait(x_empty(xi), (xph & 1) ^ 1, abort_flag, p.wait_clocks);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            xch[(halves == 2 ? hf * 2 + ch - 1 : xi) * 128 + lane_row] = sum;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(x_full(xi));
           }
-          if (hf == 0 && i < P) srow[i] = sum * unshift;
         }
       }
     }

@@ -31,13 +31,18 @@ class LayerOutputs:
 def compress_model(cfg: pkv.PkvConfig, layers, seq_lens: Sequence[int], out: LayerOutputs,
                    workspace, stream: Optional[torch.cuda.Stream] = None, lanes=None) -> None:
     """layers: sequence of objects with .q_win, .k, .v device tensors, one per layer; a layer that also
-    has .window_lse (the prefill's log-sum-exp of the window rows) is scored in a single K sweep.
+    has .window_lse (the prefill's log-sum-exp of the window rows) is scored in a single K sweep; one that has
+    .attn_out ([batch][H_q][window][d] float32) also gets the window rows' attention output written there.
     With `lanes` (binding.Lanes) and `workspace` a pair of workspaces, the score sweeps of a layer run beside
     the selection and gather of the layer before it, each on its own group of SMs."""
     if lanes is not None:
         pkv.compress_model_lanes(cfg, lanes, layers, seq_lens, out.k, out.v, out.idx, workspace, stream=stream)
         return
     for l, x in enumerate(layers):
+        if getattr(x, "attn_out", None) is not None:       # the window rows' attention output is wanted too
+            pkv.attend_compress_layer(cfg, l, x.q_win, x.k, x.v, seq_lens, x.attn_out, out.k[l], out.v[l], out.idx[l],
+                                      workspace, stream=stream)
+            continue
         pkv.compress_layer(cfg, l, x.q_win, x.k, x.v, seq_lens, out.k[l], out.v[l], out.idx[l], workspace,
                            stream=stream, window_lse=getattr(x, "window_lse", None))
 

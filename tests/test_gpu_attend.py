@@ -13,7 +13,7 @@ import torch
 
 import oracle
 import paper_2406_02069_b200 as pkv
-from paper_2406_02069_b200 import workloads
+from paper_2406_02069_b200 import binding, workloads
 from helpers import assert_indices_match, assert_scores_close, packed_rows
 
 pytestmark = pytest.mark.gpu
@@ -38,13 +38,16 @@ def make_inputs(hq, hkv, alpha, lens, dtype, seed, pad_value=None):
     return q, k, v
 
 
-def check_attention(got_out, q, k, v, lens, alpha, hq, hkv):
+def check_attention(got_out, q, k, v, lens, alpha, hq, hkv, sample=None):
+    """sample: None = every query head, else the (KV head, member of its group) pairs to check."""
     G = hq // hkv
     for b, n in enumerate(lens):
         pos = np.arange(n)
         for h in range(hkv):
             kb, vb = k[b, h, :n], v[b, h, :n]
             for g in range(G):
+                if sample is not None and (h, g) not in sample:
+                    continue
                 want = oracle.window_attention(q[b, h * G + g], kb, vb, pos, n)
                 bound = oracle.window_attention(q[b, h * G + g], kb, vb.abs(), pos, n)
                 err = np.abs(got_out[b, h * G + g].astype(np.float64) - want)
@@ -136,6 +139,40 @@ def test_fused_layer_call_matches_the_oracle(base, kw):
                         w.num_kv_heads)
 
 
+@pytest.mark.parametrize("w,layer,sample", [
+    (workloads.LLAMA3_70B, 79, {(0, 0), (3, 5), (7, 7)}),
+    (workloads.LLAMA2_7B, 0, {(0, 0), (13, 0), (31, 0)}),
+    (workloads.MISTRAL_RAGGED, 0, {(0, 0), (2, 3), (7, 1)}),
+], ids=lambda x: getattr(x, "name", None))
+def test_full_size_layer_with_attention(w, layer, sample):
+    """The configurations at their full sizes, in the launch shapes `bench.py --mode attend` times: every score and
+    every kept list of the layer against the oracle, the attention output of sampled query heads."""
+    cfg = pkv.config_of(w)
+    lens = w.seq_lens()
+    kl = pkv.layer_budgets(cfg)[layer]
+    ws = pkv.new_workspace(cfg, len(lens), max(lens), DEV)
+    x = workloads.make_layer(w, layer, device=DEV)
+    rows = pkv.total_rows(cfg, kl, lens)
+    k_out = torch.empty(rows, w.head_dim, dtype=x.k.dtype, device=DEV)
+    v_out = torch.empty_like(k_out)
+    idx = torch.empty(rows, dtype=torch.int32, device=DEV)
+    scores = torch.full((len(lens), w.num_kv_heads, max(lens)), -1.0, dtype=torch.float32, device=DEV)
+    out = torch.empty(len(lens), w.num_q_heads, w.window, w.head_dim, dtype=torch.float32, device=DEV)
+    pkv.attend_compress_layer(cfg, layer, x.q_win, x.k, x.v, lens, out, k_out, v_out, idx, ws, scores=scores)
+    pkv.check_status(ws)
+    qc, kc, vc = x.q_win.cpu(), x.k.cpu(), x.v.cpu()
+    ref = oracle.compress_batch(qc, kc, vc, lens, pool_kernel=w.pool_kernel, avg_budget=w.avg_budget, k_layer=kl)
+    got_scores, got_idx = scores.cpu().numpy(), idx.cpu().numpy()
+    for b, n in enumerate(lens):
+        assert_scores_close(got_scores[b, :, : n - w.window], ref["scores"][b], "%s seq %d" % (w.name, b))
+    for b, h, sl in packed_rows(ref["counts"], w.num_kv_heads):
+        assert_indices_match(got_idx[sl], ref["indices"][sl], ref["scores"][b][h], w.pool_kernel, w.window,
+                             "%s b %d h %d" % (w.name, b, h))
+        sel = idx[sl].long()
+        assert torch.equal(k_out[sl], x.k[b, h, sel]) and torch.equal(v_out[sl], x.v[b, h, sel])
+    check_attention(out.cpu().numpy(), qc, kc, vc, lens, w.window, w.num_q_heads, w.num_kv_heads, sample=sample)
+
+
 def test_shapes_the_kernel_does_not_take_are_refused():
     cfg = pkv.make_config(num_layers=1, num_q_heads=4, num_kv_heads=2, head_dim=64, window=8, pool_kernel=5,
                           dtype="bf16", avg_budget=8, beta=1.0)
@@ -147,3 +184,34 @@ def test_shapes_the_kernel_does_not_take_are_refused():
     with pytest.raises(pkv.PkvError) as err:
         pkv.attend_window(cfg, q, k, k, [100], out, scores, ws)
     assert err.value.status == 2      # PKV_ERR_UNSUPPORTED: head_dim 64
+
+
+def test_a_wait_that_runs_out_in_the_attention_kernel_is_reported():
+    """One K tile of one CTA of the window-attention kernel is never loaded and the bound of the waits is lowered to
+    about a millisecond: the kernel winds down by itself (every role leaves, accumulator memory released), the status
+    word says so, and the next ordinary call on the same workspace gives what a fresh workspace gives."""
+    hq, hkv, alpha, lens = 16, 2, 32, [5000]
+    cfg = pkv.make_config(num_layers=1, num_q_heads=hq, num_kv_heads=hkv, head_dim=128, window=alpha, pool_kernel=7,
+                          dtype="bf16", avg_budget=alpha, beta=1.0)
+    q, k, v = (t.to(DEV) for t in make_inputs(hq, hkv, alpha, lens, torch.bfloat16, seed=3))
+    ws = pkv.new_workspace(cfg, 1, max(lens), DEV)
+    scores = torch.zeros(1, hkv, max(lens), dtype=torch.float32, device=DEV)
+    out = torch.zeros(1, hq, alpha, 128, dtype=torch.float32, device=DEV)
+    try:
+        binding.test_hooks(wait_clocks=1 << 21, withhold_attend_tile=True)
+        pkv.attend_window(cfg, q, k, v, lens, out, scores, ws)
+        with pytest.raises(pkv.PkvError) as e:
+            pkv.check_status(ws)
+        assert e.value.status == binding.PKV_ERR_DEVICE_STATUS and "0x2" in str(e.value)
+    finally:
+        binding.test_hooks(0, False)
+    ws[:256].zero_()
+    again_s, again_o = torch.zeros_like(scores), torch.zeros_like(out)
+    pkv.attend_window(cfg, q, k, v, lens, again_o, again_s, ws)
+    pkv.check_status(ws)
+    fresh_ws = pkv.new_workspace(cfg, 1, max(lens), DEV)
+    fresh_s, fresh_o = torch.zeros_like(scores), torch.zeros_like(out)
+    pkv.attend_window(cfg, q, k, v, lens, fresh_o, fresh_s, fresh_ws)
+    pkv.check_status(fresh_ws)
+    assert torch.equal(again_s, fresh_s) and torch.equal(again_o, fresh_o)
+    check_attention(again_o.cpu().numpy(), q.cpu(), k.cpu(), v.cpu(), lens, alpha, hq, hkv)
