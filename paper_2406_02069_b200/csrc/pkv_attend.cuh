@@ -80,6 +80,28 @@ __device__ __forceinline__ uint64_t smem_desc_mn_sw128(uint32_t addr, uint32_t b
   return d;
 }
 
+// The MMA issuer is one thread and this kernel issues 32 MMAs per K tile (two units of 8 + 8), so the descriptors
+// are split into their 32-bit halves: the high half (strides, version, swizzle) is a constant, the low half (start
+// address and leading offset) is formed once per unit and advanced by a compile-time constant per MMA.  (Measured:
+// an MMA of this shape, 128 x 128 x 16, still takes the issuer about 100 clocks, whatever it costs in instructions;
+// with 32 of them per tile that, not the exponentials, sets the pace of the kernel.)
+constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);   // stride 1024 B, version 1, 128-byte swizzle
+__device__ __forceinline__ uint32_t desc_lo_k_major(uint32_t addr) { return ((addr & 0x3FFFFu) >> 4) | (1u << 16); }
+__device__ __forceinline__ uint32_t desc_lo_mn_major(uint32_t addr, uint32_t block_bytes) {
+  return ((addr & 0x3FFFFu) >> 4) | ((block_bytes >> 4) << 16);
+}
+template <bool ACC>
+__device__ __forceinline__ void tc_mma_halves(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "mov.b64 da, {%1, %3};\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(kDescHi), "r"(idesc), "n"(ACC ? 1 : 0)
+      : "memory");
+}
+
 __device__ __forceinline__ uint32_t pack_16bit(float lo, float hi, int fp16) {
   if (fp16) {
     const __half2 h = __floats2half2_rn(lo, hi);
@@ -267,12 +289,13 @@ window_attend_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_con
         }
         tc_fence_after();
         const uint32_t d_addr = tmem_base + 256 + q.hf * 128;
-        const uint32_t v_addr = smem_u32(v_s), p_addr = smem_u32(p_s) + st * kAtTileBytes;
+        const uint32_t v_lo = desc_lo_mn_major(smem_u32(v_s), kAtTileKeys * 128);
+        const uint32_t p_lo = desc_lo_mn_major(smem_u32(p_s) + st * kAtTileBytes, kAtTileKeys * 128);
+        if (fresh[q.hf]) tc_mma_halves<false>(d_addr, v_lo, p_lo, idesc_pv);
+        else tc_mma_halves<true>(d_addr, v_lo, p_lo, idesc_pv);
 #pragma unroll
-        for (int kk = 0; kk < kAtTileKeys / 16; ++kk)
-          tc_mma_f16kind(d_addr, smem_desc_mn_sw128(v_addr + kk * 2048, kAtTileKeys * 128),
-                         smem_desc_mn_sw128(p_addr + kk * 2048, kAtTileKeys * 128), idesc_pv,
-                         (fresh[q.hf] && kk == 0) ? 0u : 1u);
+        for (int kk = 1; kk < kAtTileKeys / 16; ++kk)          // 16 keys further: 2048 bytes in both operands
+          tc_mma_halves<true>(d_addr, v_lo + kk * (2048 >> 4), p_lo + kk * (2048 >> 4), idesc_pv);
         fresh[q.hf] = false;
         tc_commit(p_empty(st));
         if (q.last) tc_commit(v_empty);
@@ -314,11 +337,13 @@ window_attend_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_con
             ok = mbar_wait(s_empty(st), ((u >> 1) & 1) ^ 1, abort_flag, p.wait_clocks);
             if (!ok) break;
             tc_fence_after();
+            const uint32_t k_lo = desc_lo_k_major(k_addr), q_lo = desc_lo_k_major(q_addr + hf * 128 * 128);
+            tc_mma_halves<false>(tmem_base + st * 128, k_lo, q_lo, idesc_s);
 #pragma unroll
-            for (int kk = 0; kk < kAtD / 16; ++kk) {
-              const uint32_t ka = k_addr + (kk / 4) * kAtTileKeys * 128 + (kk % 4) * 32;
-              const uint32_t qa = q_addr + (kk / 4) * kTcMaxRows * 128 + hf * 128 * 128 + (kk % 4) * 32;
-              tc_mma_f16kind(tmem_base + st * 128, smem_desc_sw128(ka), smem_desc_sw128(qa), idesc_s, kk > 0);
+            for (int kk = 1; kk < kAtD / 16; ++kk) {           // 16 channels further: 32 bytes, the next 64-channel block
+              constexpr int kBlock = kAtTileKeys * 128 >> 4, kQBlock = kTcMaxRows * 128 >> 4;      // after four steps
+              tc_mma_halves<true>(tmem_base + st * 128, k_lo + (kk / 4) * kBlock + (kk % 4) * 2,
+                                  q_lo + (kk / 4) * kQBlock + (kk % 4) * 2, idesc_s);
             }
             tc_commit(s_full(st));
             if (hf == halves - 1) tc_commit(k_empty(s));
