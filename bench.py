@@ -303,8 +303,6 @@ def time_other(pkv, streaming, workloads, parallel, name, budget, peak, barrier,
     value, ms, _ = parallel.job_throughput(sum(lens) * steps, e0.elapsed_time(e1), device="cuda")
     pkv.check_status(ws)
     graded = sum(graded_bytes_per_layer(w, lens, r, esz) for r in out.rows)
-    if args.mode == "attend":                                      # this mode also reads V once and writes the attention output
-        graded += w.num_layers * (k_bytes_layer + len(lens) * w.num_q_heads * w.window * w.head_dim * 4)
     gbs = graded / (ms / steps * 1e-3) / 1e9
     k_layer_mb = sum(lens) * w.num_kv_heads * w.head_dim * esz / 1e6
     return {"workload": w.name, "avg_budget": w.avg_budget, "layers": w.num_layers, "seq_lens": lens, "steps": steps,
@@ -488,6 +486,8 @@ def main():
     if tr and tr["digest"] == csrc_digest(tr["sources"]):
         traffic = tr["bytes_per_key_row"] * sum(lens) * w.num_kv_heads
     graded = sum(graded_bytes_per_layer(w, lens, r, esz) for r in out.rows)
+    if args.mode == "attend":                                      # this mode also reads V once and writes the attention output
+        graded += w.num_layers * (k_bytes_layer + len(lens) * w.num_q_heads * w.window * w.head_dim * 4)
     path_gbs = graded / (ms_per_step * 1e-3) / 1e9
     # the same kernel against the special-function unit: one exponential per (window row, key) and sweep;
     # peak = 16 per clock and SM (measured: 15.98) x the SMs of the device x the maximum SM clock
