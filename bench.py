@@ -35,6 +35,10 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from ncu captures, keyed by
 # kernel name, valid only while the kernel's source files have the digest given: a change voids them.
 TC_SOURCES = ("pkv_score_tc.cuh", "pkv_common.cuh")
+# CUDA streams the independent layers of a step are spread over (measured per configuration: the batch-8 ragged
+# shape keeps every SM busy from one stream and gains nothing)
+LAYER_STREAMS = {"llama3_70b_128k": 2, "llama3_8b_32k": 3, "llama2_7b_4k": 3}
+
 NCU_TRAFFIC = {
     # profiles/score_tc_llama3_70b_128k.md: (read + written) bytes / (n * H_kv) key rows, caches flushed by ncu
     # before the launch (in the step itself sweep B finds about a third of K still in the L2)
@@ -273,8 +277,10 @@ def time_other(pkv, streaming, workloads, parallel, name, budget, peak, barrier,
     layers = [workloads.make_layer(w, l, device="cuda") for l in range(w.num_layers)]
     out = streaming.LayerOutputs(cfg, lens, w.torch_dtype())
     ws = pkv.new_workspace(cfg, len(lens), max(lens))
+    n_streams = LAYER_STREAMS.get(name, 1)
+    ls = streaming.LayerStreams(cfg, lens, n_streams) if n_streams > 1 else None
     for _ in range(3):
-        streaming.compress_model(cfg, layers, lens, out, ws)
+        streaming.compress_model(cfg, layers, lens, out, ws, layer_streams=ls)
     pkv.check_status(ws)
     # these configurations spend 40-110 us per layer on the device, of the order of what the host needs to enqueue
     # a layer's launches: the step is captured once in a CUDA graph and replayed (the per-layer call allocates nothing
@@ -283,7 +289,7 @@ def time_other(pkv, streaming, workloads, parallel, name, budget, peak, barrier,
     side = torch.cuda.Stream()
     with torch.cuda.stream(side):
         with torch.cuda.graph(graph, stream=side):
-            streaming.compress_model(cfg, layers, lens, out, ws)
+            streaming.compress_model(cfg, layers, lens, out, ws, layer_streams=ls)
     torch.cuda.synchronize()
     for _ in range(3):
         graph.replay()
@@ -302,11 +308,13 @@ def time_other(pkv, streaming, workloads, parallel, name, budget, peak, barrier,
     barrier()
     value, ms, _ = parallel.job_throughput(sum(lens) * steps, e0.elapsed_time(e1), device="cuda")
     pkv.check_status(ws)
+    if ls is not None:
+        ls.check_status()
     graded = sum(graded_bytes_per_layer(w, lens, r, esz) for r in out.rows)
     gbs = graded / (ms / steps * 1e-3) / 1e9
     k_layer_mb = sum(lens) * w.num_kv_heads * w.head_dim * esz / 1e6
     return {"workload": w.name, "avg_budget": w.avg_budget, "layers": w.num_layers, "seq_lens": lens, "steps": steps,
-            "cuda_graph": True,
+            "cuda_graph": True, "layer_streams": n_streams,
             "ms_per_step": ms / steps, "value": value, "unit": UNIT,
             "path": {"graded_bytes_per_step": graded, "achieved": gbs, "frac": gbs / peak["hbm_gbs"]},
             "l2": "one layer's K is %.1f MB; %d distinct layers (%.1f GB of K and V) are cycled, so a layer is "
@@ -339,6 +347,10 @@ def main():
     ap.add_argument("--lanes", type=int, default=0, metavar="SMS",
                     help="run selection + gather of a layer on SMS streaming multiprocessors of their own (a multiple "
                          "of 8) beside the next layer's score sweeps on the rest; 0 = one stream, kernels in turn")
+    ap.add_argument("--streams", type=int, default=None, metavar="N",
+                    help="enqueue the (independent) layers round robin on N CUDA streams with a workspace each, so that "
+                         "a layer's selection and the tails of its sweeps run beside the next layers' sweeps; default: "
+                         "what LAYER_STREAMS names for the workload, else 1")
     ap.add_argument("--mode", default="self", choices=["self", "handoff", "attend"],
                     help="self: the library finds the row normalisers itself (two K sweeps, the graded path); "
                          "handoff: they are handed in as the prefill attention would (one K sweep); attend: the "
@@ -405,7 +417,15 @@ def main():
     for _ in range(args.warmup):
         streaming.compress_model(cfg, layers, lens, out, ws)
     pkv.check_status(ws)
-    run_step = lambda: streaming.compress_model(cfg, layers, lens, out, ws)
+    n_streams = args.streams if args.streams is not None else LAYER_STREAMS.get(args.workload, 1)
+    if args.lanes:
+        n_streams = 1
+    ls = streaming.LayerStreams(cfg, lens, n_streams) if n_streams > 1 else None
+    run_step = lambda: streaming.compress_model(cfg, layers, lens, out, ws, layer_streams=ls)
+    if ls is not None:
+        for _ in range(args.warmup):
+            run_step()
+        ls.check_status()
     if args.lanes:
         if args.graph:
             raise SystemExit("--lanes and --graph are separate experiments")
@@ -420,7 +440,7 @@ def main():
         side = torch.cuda.Stream()
         with torch.cuda.stream(side):
             with torch.cuda.graph(graph, stream=side):
-                streaming.compress_model(cfg, layers, lens, out, ws)
+                streaming.compress_model(cfg, layers, lens, out, ws, layer_streams=ls)
         torch.cuda.synchronize()
         run_step = graph.replay
     if auto_steps:                                                  # size the timed region to about a second
@@ -448,6 +468,8 @@ def main():
     # whole-job rate: tokens of all ranks over the slowest rank's device time
     value, ms, _ = parallel.job_throughput(tokens * args.steps, ev0.elapsed_time(ev1), device="cuda")
     pkv.check_status(ws)
+    if ls is not None:
+        ls.check_status()
     ms_per_step = ms / args.steps
     # spread of single steps: a second, shorter loop with an event after every step (this rank only)
     marks = [torch.cuda.Event(enable_timing=True) for _ in range(min(20, args.steps) + 1)]
@@ -514,7 +536,8 @@ def main():
             "warmup": args.warmup, "ms_per_step": ms_per_step, "ms_per_step_median": step_median,
             "ms_per_step_best": step_best, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
-            "config": {"workload": w.name, "mode": args.mode, "cuda_graph": bool(args.graph), "select_lane_sms": args.lanes, "layers": w.num_layers, "q_heads": w.num_q_heads,
+            "config": {"workload": w.name, "mode": args.mode, "cuda_graph": bool(args.graph), "select_lane_sms": args.lanes,
+                       "layer_streams": n_streams, "layers": w.num_layers, "q_heads": w.num_q_heads,
                        "kv_heads": w.num_kv_heads, "head_dim": w.head_dim, "batch": w.batch, "seq_lens": lens,
                        "window": w.window, "pool_kernel": w.pool_kernel, "avg_budget": w.avg_budget, "beta": w.beta,
                        "tokens_per_step_per_gpu": tokens, "parallelism": "replicas x%d" % world,

@@ -28,23 +28,62 @@ class LayerOutputs:
         self.idx = [torch.empty(r, dtype=torch.int32, device=device) for r in self.rows]
 
 
+class LayerStreams:
+    """A few CUDA streams with a workspace each.  The layers of a model are independent of one another, so
+    `compress_model` can enqueue them round robin on these streams: the short kernels of one layer (selection and
+    gather, the tails of the sweeps) then run beside the sweeps of the next layers instead of leaving SMs idle."""
+
+    def __init__(self, cfg: pkv.PkvConfig, seq_lens: Sequence[int], count: int, device="cuda"):
+        if count < 1:
+            raise ValueError("at least one stream")
+        self.streams = [torch.cuda.Stream(device=device) for _ in range(count)]
+        self.workspaces = [pkv.new_workspace(cfg, len(seq_lens), max(seq_lens), device) for _ in range(count)]
+        self.fork = torch.cuda.Event()
+        self.joins = [torch.cuda.Event() for _ in range(count)]
+
+    def check_status(self) -> None:
+        for ws in self.workspaces:
+            pkv.check_status(ws)
+
+
 def compress_model(cfg: pkv.PkvConfig, layers, seq_lens: Sequence[int], out: LayerOutputs,
-                   workspace, stream: Optional[torch.cuda.Stream] = None, lanes=None) -> None:
+                   workspace, stream: Optional[torch.cuda.Stream] = None, lanes=None,
+                   layer_streams: Optional[LayerStreams] = None) -> None:
     """layers: sequence of objects with .q_win, .k, .v device tensors, one per layer; a layer that also
     has .window_lse (the prefill's log-sum-exp of the window rows) is scored in a single K sweep; one that has
     .attn_out ([batch][H_q][window][d] float32) also gets the window rows' attention output written there.
     With `lanes` (binding.Lanes) and `workspace` a pair of workspaces, the score sweeps of a layer run beside
-    the selection and gather of the layer before it, each on its own group of SMs."""
+    the selection and gather of the layer before it, each on its own group of SMs.
+    With `layer_streams` (`workspace` is then not used) layer l runs on stream l mod count with that stream's
+    workspace; the streams start after the work already enqueued on `stream` (the current stream if None) and
+    `stream` continues after all of them: to the caller the call is ordered like the single-stream one, and its
+    results are the same bit for bit."""
     if lanes is not None:
         pkv.compress_model_lanes(cfg, lanes, layers, seq_lens, out.k, out.v, out.idx, workspace, stream=stream)
         return
+    if layer_streams is not None:
+        cur = stream if stream is not None else torch.cuda.current_stream()
+        layer_streams.fork.record(cur)
+        for s in layer_streams.streams:
+            s.wait_event(layer_streams.fork)
+        count = len(layer_streams.streams)
+        for l, x in enumerate(layers):
+            _compress_one(cfg, l, x, seq_lens, out, layer_streams.workspaces[l % count], layer_streams.streams[l % count])
+        for s, e in zip(layer_streams.streams, layer_streams.joins):
+            e.record(s)
+            cur.wait_event(e)
+        return
     for l, x in enumerate(layers):
-        if getattr(x, "attn_out", None) is not None:       # the window rows' attention output is wanted too
-            pkv.attend_compress_layer(cfg, l, x.q_win, x.k, x.v, seq_lens, x.attn_out, out.k[l], out.v[l], out.idx[l],
-                                      workspace, stream=stream)
-            continue
-        pkv.compress_layer(cfg, l, x.q_win, x.k, x.v, seq_lens, out.k[l], out.v[l], out.idx[l], workspace,
-                           stream=stream, window_lse=getattr(x, "window_lse", None))
+        _compress_one(cfg, l, x, seq_lens, out, workspace, stream)
+
+
+def _compress_one(cfg, l, x, seq_lens, out, workspace, stream) -> None:
+    if getattr(x, "attn_out", None) is not None:           # the window rows' attention output is wanted too
+        pkv.attend_compress_layer(cfg, l, x.q_win, x.k, x.v, seq_lens, x.attn_out, out.k[l], out.v[l], out.idx[l],
+                                  workspace, stream=stream)
+        return
+    pkv.compress_layer(cfg, l, x.q_win, x.k, x.v, seq_lens, out.k[l], out.v[l], out.idx[l], workspace,
+                       stream=stream, window_lse=getattr(x, "window_lse", None))
 
 
 class HostPipeline:
