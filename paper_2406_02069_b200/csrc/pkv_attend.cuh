@@ -16,13 +16,15 @@
 // 2^15 keeps binary16 probabilities of long contexts out of the subnormal range; it is exact.
 //
 // Warp roles: 0 = TMA producer of Q and K, 1 = MMA issuer and TMEM owner, 2 = TMA producer of V,
-// 4..19 = epilogue in four groups of four warps (TMEM lane quarter = warp % 4).  An accumulator unit
-// is one K tile x (up to) 128 window rows; unit u lives in S stage u % 2 and is evaluated by the two
-// groups with par = u % 2, each taking half of its columns and writing the e values to P buffer u % 2
-// (one warp per scheduler and group leaves the exponential unit idle most of the time; two pairs do not).
-// The issuer queues S(u + 1) before P x V of unit u, so the tensor pipe works on the next logits while
-// the groups evaluate exponentials.
-// TMEM: columns 0..255 two S stages, 256..511 O^T (lane = channel c, column = window row).
+// 4..19 = epilogue in four groups of four warps (TMEM lane quarter = warp % 4), all on the same K tile.
+// Per tile the issuer queues ONE product K Q^T over all window rows (N up to 256: an MMA costs the issuing
+// thread about 100 clocks whatever its width, so few wide ones) into the single 256-column S stage; the
+// epilogue takes the rows in halves of (up to) 128: it loads a half's logits into registers, and once the last
+// half is loaded gives the S stage back, so the next tile's K Q^T runs beside the exponentials; each half's e
+// values go to their own P buffer and V^T P of a half is queued when the buffer is full, behind the next tile's
+// K Q^T.
+// TMEM: columns 0..255 the S stage, 256..511 O^T (lane = channel c, column = window row).
+// Shared memory: Q 64 KB, one K tile, two V tiles, two P buffers of 32 KB each (128 keys x 128 rows).
 //
 // Every wait on an mbarrier is bounded, as in the score sweeps: a wait that runs out sets the abort
 // flag, all roles leave their loops, copies in flight are drained, TMEM is released.
@@ -37,14 +39,14 @@ constexpr int kAtEpiWarp0 = 4;
 constexpr int kAtEpiWarps = 16;
 constexpr int kAtTileKeys = 128;
 constexpr int kAtD = 128;                // head dimension this kernel is built for
-constexpr int kAtKStages = 2;
+constexpr int kAtVStages = 2;            // V tiles in shared memory (one K tile: it is free again as soon as K Q^T ran)
 constexpr int kAtShift = 15;             // e values carry a factor 2^15
 constexpr int kAtTileBytes = kAtTileKeys * kAtD * 2;        // a K or V tile, or one P buffer (128 keys x 128 rows)
 constexpr int kAtQOff = 0;
 constexpr int kAtQBytes = kTcMaxRows * kAtD * 2;
 constexpr int kAtKOff = kAtQOff + kAtQBytes;
-constexpr int kAtVOff = kAtKOff + kAtKStages * kAtTileBytes;
-constexpr int kAtPOff = kAtVOff + kAtTileBytes;
+constexpr int kAtVOff = kAtKOff + kAtTileBytes;
+constexpr int kAtPOff = kAtVOff + kAtVStages * kAtTileBytes;
 constexpr int kAtMiscOff = kAtPOff + 2 * kAtTileBytes;
 constexpr int kAtMiscBytes = 3072;       // barriers 0.., TMEM slot 256, abort flag 260, exchange 512.., -lse2 2048..
 constexpr int kAtSmemBytes = kAtMiscOff + kAtMiscBytes;     // 227 KB: all a CTA can have
@@ -80,11 +82,10 @@ __device__ __forceinline__ uint64_t smem_desc_mn_sw128(uint32_t addr, uint32_t b
   return d;
 }
 
-// The MMA issuer is one thread and this kernel issues 32 MMAs per K tile (two units of 8 + 8), so the descriptors
-// are split into their 32-bit halves: the high half (strides, version, swizzle) is a constant, the low half (start
-// address and leading offset) is formed once per unit and advanced by a compile-time constant per MMA.  (Measured:
-// an MMA of this shape, 128 x 128 x 16, still takes the issuer about 100 clocks, whatever it costs in instructions;
-// with 32 of them per tile that, not the exponentials, sets the pace of the kernel.)
+// The MMA issuer is one thread and this kernel issues 24 MMAs per K tile, so the descriptors are split into their
+// 32-bit halves: the high half (strides, version, swizzle) is a constant, the low half (start address and leading
+// offset) is formed once per product and advanced by a compile-time constant per MMA.  (Measured: an MMA still takes
+// the issuer about 100 clocks at N = 128 and 90 at N = 256, whatever it costs in instructions; hence few, wide MMAs.)
 constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);   // stride 1024 B, version 1, 128-byte swizzle
 __device__ __forceinline__ uint32_t desc_lo_k_major(uint32_t addr) { return ((addr & 0x3FFFFu) >> 4) | (1u << 16); }
 __device__ __forceinline__ uint32_t desc_lo_mn_major(uint32_t addr, uint32_t block_bytes) {
@@ -155,38 +156,36 @@ window_attend_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_con
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t bar0 = smem_u32(bars);
-  auto k_full = [&](int s) { return bar0 + 8u * s; };
-  auto k_empty = [&](int s) { return bar0 + 8u * (2 + s); };
-  const uint32_t v_full = bar0 + 8u * 4, v_empty = bar0 + 8u * 5;
-  auto s_full = [&](int s) { return bar0 + 8u * (6 + s); };
-  auto s_empty = [&](int s) { return bar0 + 8u * (8 + s); };
-  auto p_full = [&](int s) { return bar0 + 8u * (10 + s); };
-  auto p_empty = [&](int s) { return bar0 + 8u * (12 + s); };
-  const uint32_t q_full = bar0 + 8u * 14, q_empty = bar0 + 8u * 15;
-  const uint32_t o_full = bar0 + 8u * 16, o_empty = bar0 + 8u * 17;
-  auto x_full = [&](int s) { return bar0 + 8u * (18 + s); };
-  auto x_empty = [&](int s) { return bar0 + 8u * (20 + s); };
-  const uint32_t lse_full = bar0 + 8u * 22;
+  const uint32_t k_full = bar0, k_empty = bar0 + 8u;
+  auto v_full = [&](int s) { return bar0 + 8u * (2 + s); };
+  auto v_empty = [&](int s) { return bar0 + 8u * (4 + s); };
+  const uint32_t s_full = bar0 + 8u * 6, s_empty = bar0 + 8u * 7;
+  auto p_full = [&](int s) { return bar0 + 8u * (8 + s); };
+  auto p_empty = [&](int s) { return bar0 + 8u * (10 + s); };
+  const uint32_t q_full = bar0 + 8u * 12, q_empty = bar0 + 8u * 13;
+  const uint32_t o_full = bar0 + 8u * 14, o_empty = bar0 + 8u * 15;
+  const uint32_t x_full = bar0 + 8u * 16, x_empty = bar0 + 8u * 17;
+  const uint32_t lse_full = bar0 + 8u * 18;
 
-  const int halves = p.rows_pad > 128 ? 2 : 1;                 // units per K tile
-  const int n_s = halves == 2 ? 128 : p.rows_pad;              // window rows (columns) of one S unit
-  const int n_pv = n_s < 64 ? 64 : n_s;                        // ... and of its P x V product (whole 64-row blocks)
+  const int halves = p.rows_pad > 128 ? 2 : 1;                 // row halves the epilogue takes a tile in
+  const int n_half = halves == 2 ? 128 : p.rows_pad;           // window rows (columns) of one half
+  const int n_pv = n_half < 64 ? 64 : n_half;                  // ... and of its P x V product (whole 64-row blocks)
 
   if (threadIdx.x == 0) {
+    mbar_init(k_full, 1); mbar_init(k_empty, 1);
+    mbar_init(s_full, 1); mbar_init(s_empty, kAtEpiWarps);
     for (int s = 0; s < 2; ++s) {
-      mbar_init(k_full(s), 1); mbar_init(k_empty(s), 1);
-      mbar_init(s_full(s), 1); mbar_init(s_empty(s), 8);
-      mbar_init(p_full(s), 8); mbar_init(p_empty(s), 1);
-      mbar_init(x_full(s), halves == 2 ? 12 : 4); mbar_init(x_empty(s), 4);
+      mbar_init(v_full(s), 1); mbar_init(v_empty(s), 1);
+      mbar_init(p_full(s), kAtEpiWarps); mbar_init(p_empty(s), 1);
     }
-    mbar_init(v_full, 1); mbar_init(v_empty, 1);
     mbar_init(q_full, 1); mbar_init(q_empty, 1);
     mbar_init(o_full, 1); mbar_init(o_empty, kAtEpiWarps);
+    mbar_init(x_full, 12); mbar_init(x_empty, 4);
     mbar_init(lse_full, kAtEpiWarps);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  // Q rows beyond R and P rows beyond the unit's width stay zero for the whole kernel
+  // Q rows beyond R and P rows beyond a half's width stay zero for the whole kernel
   for (int i = threadIdx.x; i < kAtQBytes / 16; i += kAtThreads) reinterpret_cast<uint4*>(q_s)[i] = make_uint4(0, 0, 0, 0);
   for (int i = threadIdx.x; i < 2 * kAtTileBytes / 16; i += kAtThreads) reinterpret_cast<uint4*>(p_s)[i] = make_uint4(0, 0, 0, 0);
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -231,27 +230,23 @@ window_attend_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_con
         int tile0, tile1;
         tiles_of(w, tile0, tile1);
         for (int t = tile0; t < tile1 && ok; ++t, ++it) {
-          const int s = it % kAtKStages;
-          ok = mbar_wait(k_empty(s), ((it / kAtKStages) & 1) ^ 1, abort_flag, p.wait_clocks);
+          ok = mbar_wait(k_empty, (it & 1) ^ 1, abort_flag, p.wait_clocks);
           if (!ok) break;
           if (p.withhold && blockIdx.x == 0 && id + 1 == item1 && t + 1 == tile1) continue;   // test aid: never arrives
-          mbar_expect_tx(k_full(s), kAtTileBytes);
+          mbar_expect_tx(k_full, kAtTileBytes);
           for (int half = 0; half < 2; ++half)
-            tma_load_4d(smem_u32(k_s) + s * kAtTileBytes + half * kAtTileKeys * 128, &k_map, k_full(s), half * 64,
-                        t * kAtTileKeys, w.h, w.b);
+            tma_load_4d(smem_u32(k_s) + half * kAtTileKeys * 128, &k_map, k_full, half * 64, t * kAtTileKeys, w.h, w.b);
         }
       }
       if (!ok) {
-        const uint32_t first = it > kAtKStages ? it - kAtKStages : 0;
-        for (uint32_t j = first; j < it; ++j)
-          for (uint32_t spin = 0; spin < (1u << 16) && !mbar_test(k_full(j % kAtKStages), (j / kAtKStages) & 1); ++spin)
-            __nanosleep(64);
+        if (it > 0)
+          for (uint32_t spin = 0; spin < (1u << 16) && !mbar_test(k_full, (it - 1) & 1); ++spin) __nanosleep(64);
         if (heads_loaded > 0)
           for (uint32_t spin = 0; spin < (1u << 16) && !mbar_test(q_full, (heads_loaded - 1) & 1); ++spin) __nanosleep(64);
       }
     }
   } else if (warp == 2) {
-    // =========================================================== TMA producer: V per tile (one stage)
+    // =========================================================== TMA producer: V per tile
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
@@ -260,54 +255,63 @@ window_attend_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_con
         int tile0, tile1;
         tiles_of(w, tile0, tile1);
         for (int t = tile0; t < tile1 && ok; ++t, ++it) {
-          ok = mbar_wait(v_empty, (it & 1) ^ 1, abort_flag, p.wait_clocks);
+          const int s = it & 1;
+          ok = mbar_wait(v_empty(s), ((it >> 1) & 1) ^ 1, abort_flag, p.wait_clocks);
           if (!ok) break;
-          mbar_expect_tx(v_full, kAtTileBytes);
+          mbar_expect_tx(v_full(s), kAtTileBytes);
           for (int half = 0; half < 2; ++half)
-            tma_load_4d(smem_u32(v_s) + half * kAtTileKeys * 128, &v_map, v_full, half * 64, t * kAtTileKeys, w.h, w.b);
+            tma_load_4d(smem_u32(v_s) + s * kAtTileBytes + half * kAtTileKeys * 128, &v_map, v_full(s), half * 64,
+                        t * kAtTileKeys, w.h, w.b);
         }
       }
-      if (!ok && it > 0)
-        for (uint32_t spin = 0; spin < (1u << 16) && !mbar_test(v_full, (it - 1) & 1); ++spin) __nanosleep(64);
+      if (!ok) {
+        const uint32_t first = it > 2 ? it - 2 : 0;
+        for (uint32_t j = first; j < it; ++j)
+          for (uint32_t spin = 0; spin < (1u << 16) && !mbar_test(v_full(j & 1), (j >> 1) & 1); ++spin) __nanosleep(64);
+      }
     }
   } else if (warp == 1) {
     // =========================================================== MMA issuer
     if (lane == 0) {
-      const uint32_t idesc_s = instr_desc_16bit(kAtTileKeys, n_s, p.fp16);
+      // all window rows at once; with two halves always 256 columns, so that the second half holds zeros (Q rows
+      // beyond R are zero) rather than what the stage held before
+      const uint32_t idesc_s = instr_desc_16bit(kAtTileKeys, halves == 2 ? 256 : p.rows_pad, p.fp16);
       const uint32_t idesc_pv = instr_desc_16bit(kAtD, n_pv, p.fp16) | (1u << 15) | (1u << 16);   // A and B M/N-major
-      uint32_t it = 0, u = 0, heads_seen = 0, runs = 0;
+      uint32_t it = 0, heads_seen = 0, runs = 0;
       int cur_b = -1, cur_h = -1;
-      bool ok = true, fresh[2] = {true, true}, wait_o = false;
-      struct Unit { bool valid; uint32_t u, it; int hf; bool last; } pend = {false, 0, 0, 0, false};
-      auto issue_pv = [&](const Unit& q) -> bool {
-        const int st = q.u & 1;
-        if (!mbar_wait(p_full(st), (q.u >> 1) & 1, abort_flag, p.wait_clocks)) return false;
-        if (q.hf == 0 && !mbar_wait(v_full, q.it & 1, abort_flag, p.wait_clocks)) return false;
+      bool ok = true, fresh = true, wait_o = false, pend = false;   // pend: the products V^T P of tile it - 1 are still to be queued
+      // V^T P of both row halves of tile j, each as soon as its P buffer is full
+      auto issue_pv = [&](uint32_t j) -> bool {
+        const int vs = j & 1;
+        if (!mbar_wait(v_full(vs), (j >> 1) & 1, abort_flag, p.wait_clocks)) return false;
         if (wait_o) {                                          // the epilogue has read the accumulators of the run before
           if (!mbar_wait(o_empty, (runs - 1) & 1, abort_flag, p.wait_clocks)) return false;
           wait_o = false;
         }
-        tc_fence_after();
-        const uint32_t d_addr = tmem_base + 256 + q.hf * 128;
-        const uint32_t v_lo = desc_lo_mn_major(smem_u32(v_s), kAtTileKeys * 128);
-        const uint32_t p_lo = desc_lo_mn_major(smem_u32(p_s) + st * kAtTileBytes, kAtTileKeys * 128);
-        if (fresh[q.hf]) tc_mma_halves<false>(d_addr, v_lo, p_lo, idesc_pv);
-        else tc_mma_halves<true>(d_addr, v_lo, p_lo, idesc_pv);
+        const uint32_t v_lo = desc_lo_mn_major(smem_u32(v_s) + vs * kAtTileBytes, kAtTileKeys * 128);
+        for (int hf = 0; hf < halves; ++hf) {
+          if (!mbar_wait(p_full(hf), j & 1, abort_flag, p.wait_clocks)) return false;
+          tc_fence_after();
+          const uint32_t d_addr = tmem_base + 256 + hf * 128;
+          const uint32_t p_lo = desc_lo_mn_major(smem_u32(p_s) + hf * kAtTileBytes, kAtTileKeys * 128);
+          if (fresh) tc_mma_halves<false>(d_addr, v_lo, p_lo, idesc_pv);
+          else tc_mma_halves<true>(d_addr, v_lo, p_lo, idesc_pv);
 #pragma unroll
-        for (int kk = 1; kk < kAtTileKeys / 16; ++kk)          // 16 keys further: 2048 bytes in both operands
-          tc_mma_halves<true>(d_addr, v_lo + kk * (2048 >> 4), p_lo + kk * (2048 >> 4), idesc_pv);
-        fresh[q.hf] = false;
-        tc_commit(p_empty(st));
-        if (q.last) tc_commit(v_empty);
+          for (int kk = 1; kk < kAtTileKeys / 16; ++kk)        // 16 keys further: 2048 bytes in both operands
+            tc_mma_halves<true>(d_addr, v_lo + kk * (2048 >> 4), p_lo + kk * (2048 >> 4), idesc_pv);
+          tc_commit(p_empty(hf));
+        }
+        fresh = false;
+        tc_commit(v_empty(vs));
         return true;
       };
       auto end_run = [&]() -> bool {
-        if (pend.valid && !issue_pv(pend)) return false;
-        pend.valid = false;
+        if (pend && !issue_pv(it - 1)) return false;
+        pend = false;
         tc_commit(o_full);
         ++runs;
         wait_o = true;
-        fresh[0] = fresh[1] = true;
+        fresh = true;
         return true;
       };
       for (int id = item0; id < item1 && ok; ++id) {
@@ -328,28 +332,25 @@ window_attend_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_con
         int tile0, tile1;
         tiles_of(w, tile0, tile1);
         for (int t = tile0; t < tile1 && ok; ++t, ++it) {
-          const int s = it % kAtKStages;
-          ok = mbar_wait(k_full(s), (it / kAtKStages) & 1, abort_flag, p.wait_clocks);
+          ok = mbar_wait(k_full, it & 1, abort_flag, p.wait_clocks);
           if (!ok) break;
-          const uint32_t k_addr = smem_u32(k_s) + s * kAtTileBytes, q_addr = smem_u32(q_s);
-          for (int hf = 0; hf < halves && ok; ++hf, ++u) {
-            const int st = u & 1;
-            ok = mbar_wait(s_empty(st), ((u >> 1) & 1) ^ 1, abort_flag, p.wait_clocks);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t k_lo = desc_lo_k_major(k_addr), q_lo = desc_lo_k_major(q_addr + hf * 128 * 128);
-            tc_mma_halves<false>(tmem_base + st * 128, k_lo, q_lo, idesc_s);
+          ok = mbar_wait(s_empty, (it & 1) ^ 1, abort_flag, p.wait_clocks);   // the tile before is in registers
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t k_lo = desc_lo_k_major(smem_u32(k_s)), q_lo = desc_lo_k_major(smem_u32(q_s));
+          tc_mma_halves<false>(tmem_base, k_lo, q_lo, idesc_s);
 #pragma unroll
-            for (int kk = 1; kk < kAtD / 16; ++kk) {           // 16 channels further: 32 bytes, the next 64-channel block
-              constexpr int kBlock = kAtTileKeys * 128 >> 4, kQBlock = kTcMaxRows * 128 >> 4;      // after four steps
-              tc_mma_halves<true>(tmem_base + st * 128, k_lo + (kk / 4) * kBlock + (kk % 4) * 2,
-                                  q_lo + (kk / 4) * kQBlock + (kk % 4) * 2, idesc_s);
-            }
-            tc_commit(s_full(st));
-            if (hf == halves - 1) tc_commit(k_empty(s));
-            if (pend.valid) ok = issue_pv(pend);
-            pend = Unit{true, u, it, hf, hf == halves - 1};
+          for (int kk = 1; kk < kAtD / 16; ++kk) {             // 16 channels further: 32 bytes, the next 64-channel block
+            constexpr int kBlock = kAtTileKeys * 128 >> 4, kQBlock = kTcMaxRows * 128 >> 4;        // after four steps
+            tc_mma_halves<true>(tmem_base, k_lo + (kk / 4) * kBlock + (kk % 4) * 2, q_lo + (kk / 4) * kQBlock + (kk % 4) * 2,
+                                idesc_s);
           }
+          tc_commit(s_full);
+          tc_commit(k_empty);
+          // the products of the tile before come behind this tile's logits in the queue: the logits are what the
+          // epilogue waits for next
+          if (pend) ok = issue_pv(it - 1);
+          pend = true;
         }
         if (ok && last_of_head) tc_commit(q_empty);
       }
@@ -357,17 +358,18 @@ window_attend_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_con
     }
   } else if (warp >= kAtEpiWarp0) {
     // =========================================================== epilogue
-    // Sixteen warps in four groups.  The two groups with the same `par` evaluate the units u with u % 2 == par,
-    // each one half of the unit's columns (window rows); group ch = 0 of the unit with row half 0 collects the
-    // partial score sums of the others and writes the score.
+    // Sixteen warps, all on the same tile.  A half's 16-column pieces are dealt round to the four groups (a group
+    // = the four warps that cover the 128 TMEM lanes).  A thread carries its key's partial score sum through the
+    // halves; group 0 then collects the other groups' sums and writes the score.
     const int e = warp - kAtEpiWarp0;
-    const int quarter = warp & 3, g4 = e >> 2, par = g4 & 1, ch = g4 >> 1;
+    const int quarter = warp & 3, g4 = e >> 2;
     const int lane_row = quarter * 32 + lane;                  // TMEM lane: key of a tile in S, channel in O^T
     const uint32_t lanes = static_cast<uint32_t>(quarter * 32) << 16;
     const float c2 = p.scale_log2;
     const float unshift = 1.0f / static_cast<float>(1 << kAtShift);
-    const int col0 = ch * (n_s / 2), col1 = col0 + n_s / 2;    // this group's columns of a unit (multiples of 16)
-    uint32_t it = 0, u = 0, lse_rounds = 0, runs = 0;
+    const int cg_a = g4 * 16, cg_b = cg_a + 64;                // this group's pieces of a half
+    const bool has_a = cg_a < n_half, has_b = cg_b < n_half;
+    uint32_t it = 0, lse_rounds = 0, runs = 0;
     int cur_b = -1, cur_h = -1;
     bool ok = true;
     // Hands the accumulators of the run that ends to global memory (raw: the reduce kernel scales).
@@ -424,53 +426,52 @@ window_attend_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_con
       int tile0, tile1;
       tiles_of(w, tile0, tile1);
       for (int t = tile0; t < tile1 && ok; ++t, ++it) {
-        for (int hf = 0; hf < halves && ok; ++hf, ++u) {
-          if (static_cast<int>(u & 1u) != par) continue;       // the other pair's unit
-          const int st = u & 1;
-          ok = mbar_wait(s_full(st), (u >> 1) & 1, abort_flag, p.wait_clocks);
+        const int i = t * kAtTileKeys + lane_row;
+        const bool in_seq = i < n;
+        const int jp = i - P;                                  // window key P + jp is seen by rows j >= jp
+        const bool plain = __all_sync(0xffffffffu, in_seq && jp <= 0);   // no mask anywhere in this warp's keys
+        ok = mbar_wait(s_full, it & 1, abort_flag, p.wait_clocks);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+        float sum = 0.f;
+        for (int hf = 0; hf < halves && ok; ++hf) {
+          const uint32_t taddr = tmem_base + lanes + hf * 128;
+          uint32_t va[16], vb[16];
+          if (has_a) tc_ld16(taddr + cg_a, va);
+          if (has_b) tc_ld16(taddr + cg_b, vb);
+          tc_wait_ld();
+          if (hf == halves - 1) {                              // this tile's logits are in registers: the stage is free
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(s_empty);
+          }
+          ok = mbar_wait(p_empty(hf), (it & 1) ^ 1, abort_flag, p.wait_clocks);   // V^T P of the tile before has read the buffer
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) break;
-          ok = mbar_wait(p_empty(st), ((u >> 1) & 1) ^ 1, abort_flag, p.wait_clocks);
-          ok = __all_sync(0xffffffffu, ok);
-          if (!ok) break;
-          tc_fence_after();
-          const int i = t * kAtTileKeys + lane_row;
-          const bool in_seq = i < n;
-          const int jp = i - P;                                // window key P + jp is seen by rows j >= jp
-          const uint32_t taddr = tmem_base + lanes + st * 128;
-          uint8_t* prow = p_s + st * kAtTileBytes + lane_row * 128;
+          uint8_t* prow = p_s + hf * kAtTileBytes + lane_row * 128;
           const float* nlr = lse_all + hf * 128;
-          float sum = 0.f;
-          if (__all_sync(0xffffffffu, in_seq && jp <= 0)) {
-            // every key of the warp sees every row (all tiles but a sequence's last ones): no mask, 16-column loads
-            // double buffered so that the next one is in flight while a chunk is evaluated
+          if (plain) {
             unsigned long long acc = pack2(0.f, 0.f);
             const unsigned long long cc = pack2(c2, c2);
             const int sw = lane_row & 7;
-            uint32_t va[16], vb[16];
-            tc_ld16(taddr + col0, va);
-            for (int cg = col0; cg < col1; cg += 32) {
-              const bool two = cg + 16 < col1;
-              tc_wait_ld();
-              if (two) tc_ld16(taddr + cg + 16, vb);
-              if (p.fp16) at_chunk<true>(va, cc, nlr + cg, prow + (cg >> 6) * (kAtTileKeys * 128), (cg & 63) >> 3, sw, acc);
-              else at_chunk<false>(va, cc, nlr + cg, prow + (cg >> 6) * (kAtTileKeys * 128), (cg & 63) >> 3, sw, acc);
-              if (two) {
-                const int cn = cg + 16;
-                tc_wait_ld();
-                if (cg + 32 < col1) tc_ld16(taddr + cg + 32, va);
-                if (p.fp16) at_chunk<true>(vb, cc, nlr + cn, prow + (cn >> 6) * (kAtTileKeys * 128), (cn & 63) >> 3, sw, acc);
-                else at_chunk<false>(vb, cc, nlr + cn, prow + (cn >> 6) * (kAtTileKeys * 128), (cn & 63) >> 3, sw, acc);
-              }
+            if (has_a) {
+              if (p.fp16) at_chunk<true>(va, cc, nlr + cg_a, prow, cg_a >> 3, sw, acc);
+              else at_chunk<false>(va, cc, nlr + cg_a, prow, cg_a >> 3, sw, acc);
+            }
+            if (has_b) {
+              if (p.fp16) at_chunk<true>(vb, cc, nlr + cg_b, prow + kAtTileKeys * 128, (cg_b & 63) >> 3, sw, acc);
+              else at_chunk<false>(vb, cc, nlr + cg_b, prow + kAtTileKeys * 128, (cg_b & 63) >> 3, sw, acc);
             }
             float lo, hi;
             unpack2(acc, lo, hi);
-            sum = lo + hi;
+            sum += lo + hi;
           } else {
-            for (int cg = col0; cg < col1; cg += 16) {
-              uint32_t v[16];
-              tc_ld16(taddr + cg, v);
-              tc_wait_ld();
+#pragma unroll
+            for (int piece = 0; piece < 2; ++piece) {
+              if (piece == 0 ? !has_a : !has_b) continue;
+              const int cg = piece == 0 ? cg_a : cg_b;
+              const uint32_t (&v)[16] = piece == 0 ? va : vb;
               float ev[16];
 #pragma unroll
               for (int j = 0; j < 16; ++j) {
@@ -490,43 +491,39 @@ window_attend_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_con
               *reinterpret_cast<uint4*>(blk + (((c0 + 1) ^ (lane_row & 7)) << 4)) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
             }
           }
-          if (hf == 0 && ch == 0 && (t + 1) * kAtTileKeys > n) {
+          if (hf == 0 && g4 == 0 && (t + 1) * kAtTileKeys > n) {
             // last tile of a sequence: what lies behind the sequence in V may be anything, and 0 x NaN is NaN
-            ok = mbar_wait(v_full, it & 1, abort_flag, p.wait_clocks);
+            ok = mbar_wait(v_full(it & 1), (it >> 1) & 1, abort_flag, p.wait_clocks);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             if (!in_seq)
               for (int half = 0; half < 2; ++half)
 #pragma unroll
                 for (int c = 0; c < 8; ++c)
-                  reinterpret_cast<uint4*>(v_s + half * kAtTileKeys * 128 + lane_row * 128)[c] = make_uint4(0, 0, 0, 0);
+                  reinterpret_cast<uint4*>(v_s + (it & 1) * kAtTileBytes + half * kAtTileKeys * 128 + lane_row * 128)[c] =
+                      make_uint4(0, 0, 0, 0);
           }
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-          tc_fence_before();
           __syncwarp();
-          if (lane == 0) { mbar_arrive(p_full(st)); mbar_arrive(s_empty(st)); }
-          // the key's score: partial sums of the other groups that work on the tile, added in a fixed order.  With
-          // two units per tile all four groups share a tile (one exchange, three slots); with one, the two groups
-          // of a pair do (an exchange per pair, one slot).
-          const int xi = halves == 2 ? 0 : par;
-          const uint32_t xph = halves == 2 ? it : it >> 1;
-          if (hf == 0 && ch == 0) {
-            ok = mbar_wait(x_full(xi), xph & 1, abort_flag, p.wait_clocks);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            if (halves == 2) sum += xch[lane_row] + xch[128 + lane_row] + xch[256 + lane_row];
-            else sum += xch[xi * 128 + lane_row];
-            __syncwarp();
-            if (lane == 0) mbar_arrive(x_empty(xi));
-            if (i < P) srow[i] = sum * unshift;
-          } else {
-            ok = mbar_wait(x_empty(xi), (xph & 1) ^ 1, abort_flag, p.wait_clocks);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            xch[(halves == 2 ? hf * 2 + ch - 1 : xi) * 128 + lane_row] = sum;
-            __syncwarp();
-            if (lane == 0) mbar_arrive(x_full(xi));
-          }
+          if (lane == 0) mbar_arrive(p_full(hf));
+        }
+        if (!ok) break;
+        // the key's score: the other groups' partial sums, added in a fixed order
+        if (g4 == 0) {
+          ok = mbar_wait(x_full, it & 1, abort_flag, p.wait_clocks);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          sum += xch[lane_row] + xch[128 + lane_row] + xch[256 + lane_row];
+          __syncwarp();
+          if (lane == 0) mbar_arrive(x_empty);
+          if (i < P) srow[i] = sum * unshift;
+        } else {
+          ok = mbar_wait(x_empty, (it & 1) ^ 1, abort_flag, p.wait_clocks);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          xch[(g4 - 1) * 128 + lane_row] = sum;
+          __syncwarp();
+          if (lane == 0) mbar_arrive(x_full);
         }
       }
     }
