@@ -53,6 +53,11 @@ MUTANTS = [
     ("window_dropped", "for (int i = P; i < n; ++i) row[cnt++] = i;", "for (int i = P; i < n; ++i) row[cnt++] = P;"),
     ("v_copied_from_k", "static_cast<const char*>(v) + src, d * esz);", "static_cast<const char*>(k) + src, d * esz);"),
     ("fp16_bias", "e - 15);", "e - 16);"),
+    ("attention_mask_off_by_one", "if (pos[r] > P + j) {", "if (pos[r] >= P + j) {"),
+    ("attention_not_normalised", "o += (w[r] / z) * elem(vc,", "o += w[r] * elem(vc,", 0),
+    ("attention_values_from_k", "o += (w[r] / z) * elem(vc,", "o += (w[r] / z) * elem(kc,", 0),
+    ("attention_no_scale", "w[r] = dot * scale;\n      mx = std::max(mx, w[r]);\n    }\n    double z = 0.0;\n    for (int r = 0; r < c; ++r) { w[r] = std::exp(w[r] - mx); z += w[r]; }\n    for (int t = 0; t < d; ++t) {\n      double o = 0.0;",
+     "w[r] = dot;\n      mx = std::max(mx, w[r]);\n    }\n    double z = 0.0;\n    for (int r = 0; r < c; ++r) { w[r] = std::exp(w[r] - mx); z += w[r]; }\n    for (int t = 0; t < d; ++t) {\n      double o = 0.0;"),
     ("page_slot", "* page_size + (r % page_size)) * row_bytes;\n    std::memcpy(static_cast<char*>(pool) + dst",
      "* page_size + (r / page_size)) * row_bytes;\n    std::memcpy(static_cast<char*>(pool) + dst"),
 ]
