@@ -47,3 +47,34 @@ def test_layers_on_several_streams_give_the_single_stream_result(base, kw, count
     for l, (k, v, i) in enumerate(copies):
         assert torch.equal(i, ref.idx[l].cpu()), "layer %d: kept list" % l
         assert torch.equal(k, ref.k[l].cpu()) and torch.equal(v, ref.v[l].cpu()), "layer %d: rows" % l
+
+
+def test_a_step_on_several_streams_can_be_captured_in_one_cuda_graph():
+    """Fork and join are events, so a whole step on several streams is one graph; replaying it gives the same cache."""
+    w = workloads.scaled(workloads.LLAMA3_8B, name="llama3_8b_streams_graph", num_layers=5, seq_len=4000 + 3)
+    cfg = pkv.config_of(w)
+    lens = w.seq_lens()
+    layers = [workloads.make_layer(w, l, device=DEV) for l in range(w.num_layers)]
+    ref = streaming.LayerOutputs(cfg, lens, w.torch_dtype(), DEV)
+    ws = pkv.new_workspace(cfg, len(lens), max(lens), DEV)
+    streaming.compress_model(cfg, layers, lens, ref, ws)
+    pkv.check_status(ws)
+    got = streaming.LayerOutputs(cfg, lens, w.torch_dtype(), DEV)
+    ls = streaming.LayerStreams(cfg, lens, 3, DEV)
+    streaming.compress_model(cfg, layers, lens, got, None, layer_streams=ls)      # warms every first-use path
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            streaming.compress_model(cfg, layers, lens, got, None, layer_streams=ls)
+    for t in got.k + got.v:
+        t.zero_()
+    for t in got.idx:
+        t.fill_(-1)
+    graph.replay()
+    graph.replay()
+    torch.cuda.synchronize()
+    ls.check_status()
+    for l in range(w.num_layers):
+        assert torch.equal(got.idx[l], ref.idx[l]) and torch.equal(got.k[l], ref.k[l]) and torch.equal(got.v[l], ref.v[l])
