@@ -31,6 +31,10 @@
  *     PKV_FLAG_INPUTS_FINAL in cfg->flags the score kernels read q_win and k without that wait (see the
  *     flag).  Even then the library orders them itself when q_win or k lies inside a cache or page pool
  *     that one of its own recent calls writes.
+ *   - Calls on different streams may run at the same time as long as each has a workspace of its own (a
+ *     call keeps its intermediate results there); the layers of a model are independent of one another, so a
+ *     caller may spread them over a few streams to keep the device busy during the short kernels of a layer.
+ *     Ordering between streams (a call that reads what a call on another stream writes) is the caller's, by events.
  *
  * Tensor layout
  *   K, V     [batch][H_kv][n_max][d]   element strides given per tensor
