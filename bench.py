@@ -37,7 +37,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
 TC_SOURCES = ("pkv_score_tc.cuh", "pkv_common.cuh")
 # CUDA streams the independent layers of a step are spread over (measured per configuration: the batch-8 ragged
 # shape keeps every SM busy from one stream and gains nothing)
-LAYER_STREAMS = {"llama3_70b_128k": 2, "llama3_8b_32k": 3, "llama2_7b_4k": 3}
+LAYER_STREAMS = {"llama3_70b_128k": 2, "llama3_8b_32k": 3, "llama2_7b_4k": 4}
 
 NCU_TRAFFIC = {
     # profiles/score_tc_llama3_70b_128k.md: (read + written) bytes / (n * H_kv) key rows, caches flushed by ncu

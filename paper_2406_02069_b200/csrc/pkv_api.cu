@@ -362,8 +362,10 @@ int launch_scores_tc(const pkv_config* c, const pkv_tensor& q, const pkv_tensor&
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) return PKV_ERR_CUDA;
   if (dev >= 64 || !attr_done[dev]) {
-    if (cudaFuncSetAttribute(score_resident_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             RsSmem<D>::kTotal) != cudaSuccess ||
+    if (cudaFuncSetAttribute(score_resident_kernel<D, kRsStages>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             RsSmem<D, kRsStages>::kTotal) != cudaSuccess ||
+        cudaFuncSetAttribute(score_resident_kernel<D, kRsStagesShort>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             RsSmem<D, kRsStagesShort>::kTotal) != cudaSuccess ||
         cudaFuncSetAttribute(score_tc_kernel<D, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcSmem<D>::kTotal) !=
             cudaSuccess ||
         cudaFuncSetAttribute(score_tc_kernel<D, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcSmem<D>::kTotal) !=
@@ -455,7 +457,9 @@ int launch_scores_tc(const pkv_config* c, const pkv_tensor& q, const pkv_tensor&
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(cluster * sp.num_kv_heads, batch);
     cfg.blockDim = dim3(kRsThreads);
-    cfg.dynamicSmemBytes = RsSmem<D>::kTotal;
+    // at most 8 tiles per CTA: three K stages and 256 TMEM columns do, and two such CTAs fit on an SM
+    const bool small = (tiles_max + cluster - 1) / cluster <= 8;
+    cfg.dynamicSmemBytes = small ? RsSmem<D, kRsStagesShort>::kTotal : RsSmem<D, kRsStages>::kTotal;
     cfg.stream = st;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -466,7 +470,9 @@ int launch_scores_tc(const pkv_config* c, const pkv_tensor& q, const pkv_tensor&
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    if (cudaLaunchKernelEx(&cfg, score_resident_kernel<D>, q_map, k_map_b, tp) != cudaSuccess) return PKV_ERR_CUDA;
+    if ((small ? cudaLaunchKernelEx(&cfg, score_resident_kernel<D, kRsStagesShort>, q_map, k_map_b, tp)
+               : cudaLaunchKernelEx(&cfg, score_resident_kernel<D, kRsStages>, q_map, k_map_b, tp)) != cudaSuccess)
+      return PKV_ERR_CUDA;
     mark(st, "scores_resident");
     return check_launch();
   }

@@ -31,15 +31,17 @@ constexpr int kRsRows = 32;                 // window rows (columns of a tile's 
 constexpr int kRsTileKeys = 128;
 constexpr int kRsMaxTiles = 512 / kRsRows;  // tiles a CTA keeps in its 512 TMEM columns
 constexpr int kRsMaxCluster = 8;
-constexpr int kRsStages = 6;                // K tiles in flight per CTA
+constexpr int kRsStages = 6;                // K tiles in flight per CTA ...
+constexpr int kRsStagesShort = 3;           // ... or 3 when a CTA has at most 8 tiles: half the shared memory and (with 256 TMEM
+                                            // columns) room for two CTAs per SM, so that two layers' kernels can share the device
 
-template <int D>
+template <int D, int STAGES>
 struct RsSmem {
   static constexpr int kStageBytes = kRsTileKeys * D * 2;
   static constexpr int kQBytes = kRsRows * D * 2;
   static constexpr int kQOff = 0;
   static constexpr int kKOff = 8192;                          // Q takes at most 8 KB
-  static constexpr int kMiscOff = kKOff + kRsStages * kStageBytes;
+  static constexpr int kMiscOff = kKOff + STAGES * kStageBytes;
   static constexpr int kMiscBytes = 4096;
   static constexpr int kTotal = kMiscOff + kMiscBytes + 1024;  // + slack for manual 1024-byte alignment
 };
@@ -57,15 +59,15 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
       : "memory");
 }
 
-// grid (cluster * H_kv, batch), cluster (cluster, 1, 1), block kRsThreads, dynamic shared memory RsSmem<D>::kTotal.
+// grid (cluster * H_kv, batch), cluster (cluster, 1, 1), block kRsThreads, dynamic shared memory RsSmem<D, STAGES>::kTotal.
 // Uses of TcParams: seq (n, prefix, alpha), num_kv_heads, group, rows (<= 32), fp16, early, scale_log2, log2_group,
 // scores, ld_scores, status, wait_clocks.
-template <int D>
+template <int D, int STAGES>
 __global__ void __launch_bounds__(kRsThreads, 1)
 score_resident_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_constant__ CUtensorMap k_map,
                       const TcParams p) {
   namespace cg = cooperative_groups;
-  using L = RsSmem<D>;
+  using L = RsSmem<D, STAGES>;
   constexpr int kHalves = D / 64;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -85,9 +87,9 @@ score_resident_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_co
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t bar0 = smem_u32(bars);
   auto k_full = [&](int s) { return bar0 + 8u * s; };
-  auto k_empty = [&](int s) { return bar0 + 8u * (kRsStages + s); };
-  const uint32_t q_full = bar0 + 8u * (2 * kRsStages);
-  auto t_full = [&](int t) { return bar0 + 8u * (2 * kRsStages + 1 + t); };
+  auto k_empty = [&](int s) { return bar0 + 8u * (STAGES + s); };
+  const uint32_t q_full = bar0 + 8u * (2 * STAGES);
+  auto t_full = [&](int t) { return bar0 + 8u * (2 * STAGES + 1 + t); };
 
   // this CTA's tiles of the sequence: tiles_per consecutive ones from rank * tiles_per on
   const int n = p.seq.n[b], alpha = p.seq.alpha, P = p.seq.prefix[b];
@@ -95,11 +97,14 @@ score_resident_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_co
   const int tiles_per = (ntiles + C - 1) / C;                  // <= kRsMaxTiles (the host checks)
   const int tile0 = min(ntiles, rank * tiles_per), tile1 = min(ntiles, tile0 + tiles_per);
   const int T = tile1 - tile0;
+  // TMEM columns: 32 per tile, a power of two; CTAs that need 256 or fewer leave room for a second CTA on the SM
+  uint32_t tmem_cols = 32;
+  while (tmem_cols < static_cast<uint32_t>(tiles_per * kRsRows)) tmem_cols <<= 1;
 
   // ---- set-up (shared memory and TMEM only: it may overlap the tail of the preceding kernel)
   pdl_trigger();
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kRsStages; ++s) { mbar_init(k_full(s), 1); mbar_init(k_empty(s), 1); }
+    for (int s = 0; s < STAGES; ++s) { mbar_init(k_full(s), 1); mbar_init(k_empty(s), 1); }
     mbar_init(q_full, 1);
     for (int t = 0; t < kRsMaxTiles; ++t) mbar_init(t_full(t), 1);
     *abort_flag = 0;
@@ -109,7 +114,7 @@ score_resident_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_co
   for (int i = threadIdx.x; i < L::kQBytes / 16; i += kRsThreads) reinterpret_cast<uint4*>(q_s)[i] = make_uint4(0, 0, 0, 0);
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512)
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(tmem_cols)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -128,8 +133,8 @@ score_resident_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_co
       bool ok = true;
       int issued = 0;
       for (int t = 0; t < T && ok; ++t) {
-        const int s = t % kRsStages;
-        ok = mbar_wait(k_empty(s), ((t / kRsStages) & 1) ^ 1, abort_flag, p.wait_clocks);
+        const int s = t % STAGES;
+        ok = mbar_wait(k_empty(s), ((t / STAGES) & 1) ^ 1, abort_flag, p.wait_clocks);
         if (!ok) break;
         mbar_expect_tx(k_full(s), L::kStageBytes);
         for (int half = 0; half < kHalves; ++half)
@@ -139,8 +144,8 @@ score_resident_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_co
       }
       if (!ok) {
         // drain: wait (bounded) for the copies still in flight before shared memory is given up
-        for (int j = max(0, issued - kRsStages); j < issued; ++j)
-          for (uint32_t spin = 0; spin < (1u << 16) && !mbar_test(k_full(j % kRsStages), (j / kRsStages) & 1); ++spin)
+        for (int j = max(0, issued - STAGES); j < issued; ++j)
+          for (uint32_t spin = 0; spin < (1u << 16) && !mbar_test(k_full(j % STAGES), (j / STAGES) & 1); ++spin)
             __nanosleep(64);
         for (uint32_t spin = 0; spin < (1u << 16) && !mbar_test(q_full, 0); ++spin) __nanosleep(64);
       }
@@ -151,8 +156,8 @@ score_resident_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_co
       const uint32_t idesc = instr_desc_16bit(kRsTileKeys, kRsRows, p.fp16);
       bool ok = mbar_wait(q_full, 0, abort_flag, p.wait_clocks);
       for (int t = 0; t < T && ok; ++t) {
-        const int s = t % kRsStages;
-        ok = mbar_wait(k_full(s), (t / kRsStages) & 1, abort_flag, p.wait_clocks);
+        const int s = t % STAGES;
+        ok = mbar_wait(k_full(s), (t / STAGES) & 1, abort_flag, p.wait_clocks);
         if (!ok) break;
         tc_fence_after();
         const uint32_t k_addr = smem_u32(k_s) + s * L::kStageBytes, q_addr = smem_u32(q_s);
@@ -290,7 +295,7 @@ score_resident_kernel(const __grid_constant__ CUtensorMap q_map, const __grid_co
   if (threadIdx.x == 0 && *abort_flag) atomicOr(p.status, kStatusWaitExpired);
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
   }
 }
 
