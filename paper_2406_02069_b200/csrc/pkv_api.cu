@@ -634,7 +634,9 @@ int run_select(const pkv_config* c, const float* scores, int64_t ld, const SeqTa
     for (auto kernel : {pool_select_kernel<false, false, 1>, pool_select_kernel<true, false, 1>,
                         pool_select_kernel<false, true, 1>, pool_select_kernel<true, true, 1>,
                         pool_select_kernel<false, false, 8>, pool_select_kernel<true, false, 8>,
-                        pool_select_kernel<false, true, 8>, pool_select_kernel<true, true, 8>})
+                        pool_select_kernel<false, true, 8>, pool_select_kernel<true, true, 8>,
+                        pool_select_kernel<false, false, 1, kSelThreadsSmall>, pool_select_kernel<true, false, 1, kSelThreadsSmall>,
+                        pool_select_kernel<false, false, 8, kSelThreadsSmall>, pool_select_kernel<true, false, 8, kSelThreadsSmall>})
       if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                kSelSliceCap * 6 + 8 * kSelHalo) != cudaSuccess)
         return PKV_ERR_CUDA;
@@ -642,7 +644,11 @@ int run_select(const pkv_config* c, const float* scores, int64_t ld, const SeqTa
   }
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(cluster * c->num_kv_heads, batch);
-  cfg.blockDim = dim3(kSelThreads);
+  // short slices (at most 8 positions per thread): the 512-thread instance, of which two fit on an SM, or one beside
+  // another layer's single-sweep score CTA.  (It could take 8192 positions, but at 16 per thread it is slower than
+  // 1024 threads at 8: measured +6 % per step on the 32k and batch-8 shapes.)
+  const bool small_cta = slice <= 4096;
+  cfg.blockDim = dim3(small_cta ? kSelThreadsSmall : kSelThreads);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
   cudaLaunchAttribute attr[2];
@@ -663,6 +669,9 @@ int run_select(const pkv_config* c, const float* scores, int64_t ld, const SeqTa
                              : (wide ? pool_select_kernel<true, false, 8> : pool_select_kernel<true, false, 1>))
                     : (multi ? (wide ? pool_select_kernel<false, true, 8> : pool_select_kernel<false, true, 1>)
                              : (wide ? pool_select_kernel<false, false, 8> : pool_select_kernel<false, false, 1>));
+  if (small_cta)                                    // never multi: a slice of 8192 positions is one round
+    kernel = avg ? (wide ? pool_select_kernel<true, false, 8, kSelThreadsSmall> : pool_select_kernel<true, false, 1, kSelThreadsSmall>)
+                 : (wide ? pool_select_kernel<false, false, 8, kSelThreadsSmall> : pool_select_kernel<false, false, 1, kSelThreadsSmall>);
   if (cudaLaunchKernelEx(&cfg, kernel, sp) != cudaSuccess) return PKV_ERR_CUDA;
   if (k_out) {
     int64_t out_rows = 0;

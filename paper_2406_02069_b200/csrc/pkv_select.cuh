@@ -37,6 +37,7 @@ namespace pkv {
 namespace cg = cooperative_groups;
 
 constexpr int kSelThreads = 1024;
+constexpr int kSelThreadsSmall = 512;      // the instance for short slices (it can take up to 8192 positions)
 constexpr int kSelWarps = kSelThreads / 32;
 constexpr int kSelMaxCluster = 8;
 constexpr int kSelBins = 2048;
@@ -141,12 +142,19 @@ __device__ __noinline__ void gather_listed_rows(const int32_t* out, const char* 
 // MULTI: some CTA's slice is longer than kSelSliceCap and is taken in several rounds.
 // GROUPS: maxima each thread keeps for the lower bound of step 2 (1 for small budgets, 8 when k nears or
 // passes the thread count, so that the bound stays tight).
-template <bool AVG, bool MULTI, int GROUPS>
-__global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectParams p) {
+template <bool AVG, bool MULTI, int GROUPS, int THREADS = kSelThreads>
+__global__ void __launch_bounds__(THREADS, THREADS == kSelThreads ? 1 : 2) pool_select_kernel(const SelectParams p) {
+  // THREADS = 512 is the instance for short slices (at most 8192 positions): half the registers of an SM, so that
+  // two such CTAs, or one and a CTA of another layer's score kernel, share an SM
+  constexpr int WARPS = THREADS / 32;
+  constexpr int CAP = kSelSliceCap / (kSelThreads / THREADS);   // positions a CTA holds per round
+  constexpr int PER_LANE = kSelPerLane;
+  constexpr int BPT = kSelBins / THREADS;                        // histogram bins every thread scans: 2 or 4
+  static_assert(BPT == 2 || BPT == 4, "thread count of the selection kernel");
   extern __shared__ __align__(16) uint32_t sel_smem[];      // [halo | slice | halo] raw scores; later CTA 0's pairs
   __shared__ uint32_t hist[2][kSelBins];                    // per-pass digit histogram (double buffered)
-  __shared__ uint32_t warp_sum[kSelWarps];
-  __shared__ uint32_t warp_gt[kSelWarps], warp_eq[kSelWarps];
+  __shared__ uint32_t warp_sum[WARPS];
+  __shared__ uint32_t warp_gt[WARPS], warp_eq[WARPS];
   __shared__ uint32_t sel_digit, sel_above, bound_digit;
 
   pdl_trigger();
@@ -166,16 +174,16 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
 
   // The window positions close the list (Section 4.2.1: always retained).
   if (rank == 0)
-    for (int j = tid; j < alpha; j += kSelThreads) out[k + j] = P + j;
+    for (int j = tid; j < alpha; j += THREADS) out[k + j] = P + j;
   if (k >= P) {                                             // nothing to evict: identity list
-    for (int i = rank * kSelThreads + tid; i < P; i += C * kSelThreads) out[i] = i;
+    for (int i = rank * THREADS + tid; i < P; i += C * THREADS) out[i] = i;
   }
 
   const int64_t head = static_cast<int64_t>(b) * p.num_kv_heads + h;
   const int slice = ((P + C - 1) / C + 31) & ~31;           // multiple of 32 positions per CTA
   uint2* regions = p.cand + head * p.cand_stride;           // region of CTA c starts at c * slice
   uint32_t* counts = p.cand_cnt + head * kSelMaxCluster;
-  for (int i = tid; i < 2 * kSelBins; i += kSelThreads) (&hist[0][0])[i] = 0;
+  for (int i = tid; i < 2 * kSelBins; i += THREADS) (&hist[0][0])[i] = 0;
   // A cluster of one keeps its candidates in shared memory when they fit: no trip through global memory.
   bool local_pairs = false;
   int local_count = 0;
@@ -186,26 +194,26 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
     const int radius = p.pool_radius;
     uint2* region = regions + static_cast<int64_t>(rank) * slice;
     if (p.cached) {                                         // the pool's reach fits the staged halo
-      // The slice is taken in rounds of at most kSelSliceCap positions (one round up to 131072 keys per head
+      // The slice is taken in rounds of at most CAP positions (one round up to 131072 keys per head
       // with a cluster of 8).  Round: stage raw scores with a halo (outside the prefix: -inf for the max, 0
       // for the mean), pool them into one key per lane and step.
       float* raw = reinterpret_cast<float*>(sel_smem + kSelHalo);
       const float outside = AVG ? 0.0f : -INFINITY;
       const float width = static_cast<float>(2 * radius + 1);
-      const int rounds = MULTI ? (hi - lo + kSelSliceCap - 1) / kSelSliceCap : 1;
-      const int run = ((min(slice, kSelSliceCap) / kSelWarps) + 31) & ~31;   // positions per warp and round
-      uint32_t pk[kSelPerLane];
+      const int rounds = MULTI ? (hi - lo + CAP - 1) / CAP : 1;
+      const int run = ((min(slice, CAP) / WARPS) + 31) & ~31;   // positions per warp and round
+      uint32_t pk[PER_LANE];
       int wlo = hi, whi = hi;
       auto pool_round = [&](int r) {
-        const int rlo = lo + r * kSelSliceCap, rhi = min(hi, rlo + kSelSliceCap);
+        const int rlo = lo + r * CAP, rhi = min(hi, rlo + CAP);
         if (MULTI) __syncthreads();                         // the previous round's readers are done
-        for (int i = rlo - kSelHalo + tid; i < rhi + kSelHalo; i += kSelThreads)
+        for (int i = rlo - kSelHalo + tid; i < rhi + kSelHalo; i += THREADS)
           raw[i - rlo] = (i >= 0 && i < P) ? s[i] : outside;
         __syncthreads();
         wlo = min(rhi, rlo + warp * run);
         whi = min(rhi, wlo + run);
 #pragma unroll
-        for (int it = 0; it < kSelPerLane; ++it) {
+        for (int it = 0; it < PER_LANE; ++it) {
           const int i = wlo + it * 32 + lane;
           pk[it] = 0;
           if (i < whi) {
@@ -228,11 +236,11 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
 #pragma unroll
       for (int g = 0; g < GROUPS; ++g) tmax[g] = 0;
 #pragma unroll
-      for (int it = 0; it < kSelPerLane; ++it) pk[it] = 0;
+      for (int it = 0; it < PER_LANE; ++it) pk[it] = 0;
       for (int r = 0; r < rounds; ++r) {
         pool_round(r);
 #pragma unroll
-        for (int it = 0; it < kSelPerLane; ++it) tmax[it % GROUPS] = max(tmax[it % GROUPS], pk[it]);
+        for (int it = 0; it < PER_LANE; ++it) tmax[it % GROUPS] = max(tmax[it % GROUPS], pk[it]);
       }
       // ---- 2. lower bound of the k-th largest key: the k-th largest of these maxima (maxima of disjoint
       //         groups of positions, so at least k keys are no smaller), resolved to its top 22 bits by two
@@ -248,8 +256,12 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
           if (digit < kSelBins && lane == __ffs(peers) - 1) atomicAdd(&hist[1][digit], __popc(peers));
         }
         __syncthreads();
-        const uint2 v = reinterpret_cast<const uint2*>(hist[1])[tid];
-        const uint32_t mine = v.x + v.y;
+        uint32_t bins[BPT];                                 // every thread owns BPT adjacent digits
+#pragma unroll
+        for (int j = 0; j < BPT; ++j) bins[j] = hist[1][BPT * tid + j];
+        uint32_t mine = 0;
+#pragma unroll
+        for (int j = 0; j < BPT; ++j) mine += bins[j];
         uint32_t incl = mine;
         for (int off = 1; off < 32; off <<= 1) {
           const uint32_t u = __shfl_down_sync(0xffffffffu, incl, off);
@@ -259,14 +271,18 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
         if (tid == 0) { bound_digit = kSelBins; sel_above = 0; }   // kSelBins: fewer than brem maxima in play
         __syncthreads();
         uint32_t higher = incl - mine;
-        for (int w2 = warp + 1; w2 < kSelWarps; ++w2) higher += warp_sum[w2];
+        for (int w2 = warp + 1; w2 < WARPS; ++w2) higher += warp_sum[w2];
         if (higher < brem && brem <= higher + mine) {
-          const bool upper = higher + v.y >= brem;
-          bound_digit = upper ? 2 * tid + 1 : 2 * tid;
-          sel_above = upper ? higher : higher + v.y;
+          uint32_t above = higher;                          // from the thread's highest digit down
+#pragma unroll
+          for (int j = BPT - 1; j >= 0; --j) {
+            if (above < brem && brem <= above + bins[j]) { bound_digit = BPT * tid + j; sel_above = above; }
+            above += bins[j];
+          }
         }
         __syncthreads();
-        reinterpret_cast<uint2*>(hist[1])[tid] = make_uint2(0, 0);
+#pragma unroll
+        for (int j = 0; j < BPT; ++j) hist[1][BPT * tid + j] = 0;
         const uint32_t bd = bound_digit;
         if (bd == kSelBins) {                               // cannot bound (k exceeds the number of maxima): keep all
           if (bp == 0) { bprefix = 0; bmask = 0; }
@@ -285,21 +301,21 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
         if (MULTI) pool_round(r);                           // a single round still holds its keys in registers
         uint32_t wc = 0;
 #pragma unroll
-        for (int it = 0; it < kSelPerLane; ++it) {
+        for (int it = 0; it < PER_LANE; ++it) {
           const int i = wlo + it * 32 + lane;
           wc += __popc(__ballot_sync(0xffffffffu, i < whi && pk[it] >= bound));
         }
         if (lane == 0) warp_gt[warp] = wc;
         __syncthreads();
         uint32_t base = filled, all_cand = 0;
-        for (int w2 = 0; w2 < kSelWarps; ++w2) {
+        for (int w2 = 0; w2 < WARPS; ++w2) {
           if (w2 < warp) base += warp_gt[w2];
           all_cand += warp_gt[w2];
         }
         local_pairs = !MULTI && C == 1 && static_cast<int>(all_cand) <= p.smem_pairs;
         uint2* dst = local_pairs ? reinterpret_cast<uint2*>(sel_smem) : region;   // the raw scores are dead by now
 #pragma unroll
-        for (int it = 0; it < kSelPerLane; ++it) {
+        for (int it = 0; it < PER_LANE; ++it) {
           const int i = wlo + it * 32 + lane;
           const bool c = i < whi && pk[it] >= bound;
           const uint32_t bal = __ballot_sync(0xffffffffu, c);
@@ -312,7 +328,7 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
       if (tid == 0) counts[rank] = filled;
     } else {
       // a very wide pool: every position is a candidate
-      for (int i = lo + tid; i < hi; i += kSelThreads) region[i - lo] = make_uint2(pooled_key(s, i, P, radius, AVG ? 1 : 0), i);
+      for (int i = lo + tid; i < hi; i += THREADS) region[i - lo] = make_uint2(pooled_key(s, i, P, radius, AVG ? 1 : 0), i);
       if (tid == 0) counts[rank] = hi - lo;
     }
   }
@@ -334,7 +350,7 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
     uint2* flat = reinterpret_cast<uint2*>(sel_smem);
     const int held = min(N, p.smem_pairs);
     if (!local_pairs) {
-      for (int j = tid; j < held; j += kSelThreads) flat[j] = fetch(j);
+      for (int j = tid; j < held; j += THREADS) flat[j] = fetch(j);
       __syncthreads();
     }
     auto item = [&](int j) -> uint2 { return j < held ? flat[j] : fetch(j); };
@@ -344,7 +360,7 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
       const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
       const uint32_t dmask = pass == 2 ? 1023u : 2047u;
       uint32_t* hcur = hist[pass & 1];
-      for (int j0 = warp * 32; j0 < N; j0 += kSelThreads) {
+      for (int j0 = warp * 32; j0 < N; j0 += THREADS) {
         const int j = j0 + lane;
         uint32_t digit = kSelBins;                          // kSelBins = does not take part
         if (j < N) {
@@ -355,10 +371,15 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
         if (digit < kSelBins && lane == __ffs(peers) - 1) atomicAdd(&hcur[digit], __popc(peers));
       }
       __syncthreads();
-      const uint2 v = reinterpret_cast<const uint2*>(hcur)[tid];           // every thread owns two adjacent digits
-      reinterpret_cast<uint2*>(hist[(pass + 1) & 1])[tid] = make_uint2(0, 0);   // next pass's buffer
-      const uint32_t mine = v.x + v.y;
-      uint32_t incl = mine;                                 // keys in this and the higher pairs of the warp
+      uint32_t bins[BPT];                                   // every thread owns BPT adjacent digits
+      uint32_t mine = 0;
+#pragma unroll
+      for (int j = 0; j < BPT; ++j) {
+        bins[j] = hcur[BPT * tid + j];
+        hist[(pass + 1) & 1][BPT * tid + j] = 0;            // next pass's buffer
+        mine += bins[j];
+      }
+      uint32_t incl = mine;                                 // keys in this and the higher threads of the warp
       for (int off = 1; off < 32; off <<= 1) {
         const uint32_t u = __shfl_down_sync(0xffffffffu, incl, off);
         if (lane + off < 32) incl += u;
@@ -366,10 +387,14 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
       if (lane == 0) warp_sum[warp] = incl;
       __syncthreads();
       uint32_t higher = incl - mine;
-      for (int w2 = warp + 1; w2 < kSelWarps; ++w2) higher += warp_sum[w2];
-      if (higher < remaining && remaining <= higher + mine) {  // exactly one thread: the k-th key is in its pair
-        if (higher + v.y >= remaining) { sel_digit = 2 * tid + 1; sel_above = higher; }
-        else { sel_digit = 2 * tid; sel_above = higher + v.y; }
+      for (int w2 = warp + 1; w2 < WARPS; ++w2) higher += warp_sum[w2];
+      if (higher < remaining && remaining <= higher + mine) {  // exactly one thread: the k-th key is in its digits
+        uint32_t above = higher;                            // from the thread's highest digit down
+#pragma unroll
+        for (int j = BPT - 1; j >= 0; --j) {
+          if (above < remaining && remaining <= above + bins[j]) { sel_digit = BPT * tid + j; sel_above = above; }
+          above += bins[j];
+        }
       }
       __syncthreads();
       prefix |= sel_digit << shift;
@@ -381,7 +406,7 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
     const uint32_t need_eq = remaining;                     // ties at T to take, from the left
 
     // keys above / at the threshold, warp by warp over contiguous chunks of the concatenation
-    const int chunk = (((N + kSelWarps - 1) / kSelWarps) + 31) & ~31;
+    const int chunk = (((N + WARPS - 1) / WARPS) + 31) & ~31;
     const int j_lo = min(N, warp * chunk), j_hi = min(N, j_lo + chunk);
     uint32_t ngt = 0, neq = 0;
     for (int j0 = j_lo; j0 < j_hi; j0 += 32) {
@@ -394,7 +419,7 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
     __syncthreads();
     uint32_t gt_before = 0, eq_before = 0;
     for (int w2 = 0; w2 < warp; ++w2) { gt_before += warp_gt[w2]; eq_before += warp_eq[w2]; }
-    if (tid == kSelThreads - 1) {                           // the last thread can see the grand total
+    if (tid == THREADS - 1) {                           // the last thread can see the grand total
       if (gt_before + ngt + min(eq_before + neq, need_eq) != static_cast<uint32_t>(k))
         atomicOr(p.status, kStatusSelectMismatch);
     }
@@ -417,12 +442,12 @@ __global__ void __launch_bounds__(kSelThreads) pool_select_kernel(const SelectPa
     const char* kb = static_cast<const char*>(p.k.ptr) + (b * p.k.sb + h * p.k.sh) * p.elem_bytes;
     const char* vb = static_cast<const char*>(p.v.ptr) + (b * p.v.sb + h * p.v.sh) * p.elem_bytes;
     const int64_t row0 = p.seq.row_off[b] + static_cast<int64_t>(h) * count;
-    const int total = count * p.pieces, stride = C * kSelThreads;
+    const int total = count * p.pieces, stride = C * THREADS;
     if (total >= 8 * stride) {                              // a long list: the batched copy
       gather_listed_rows(out, kb, vb, p.k.st * p.elem_bytes, p.v.st * p.elem_bytes, static_cast<uint4*>(p.k_out),
-                         static_cast<uint4*>(p.v_out), row0, total, p.pieces, rank * kSelThreads + tid, stride);
+                         static_cast<uint4*>(p.v_out), row0, total, p.pieces, rank * THREADS + tid, stride);
     } else {
-      for (int g = rank * kSelThreads + tid; g < total; g += stride) {
+      for (int g = rank * THREADS + tid; g < total; g += stride) {
         const int row = g / p.pieces, piece = g - row * p.pieces;
         const int pos = __ldcg(out + row);                  // written by other CTAs of the cluster: skip L1
         const int64_t dst = (row0 + row) * p.pieces + piece;
