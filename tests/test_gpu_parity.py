@@ -130,7 +130,7 @@ def test_single_sweep_with_prefill_lse_matches_oracle(w):
 
 @pytest.mark.parametrize("P,k,w", [(1, 1, 1), (5, 2, 7), (33, 32, 3), (100, 0, 5), (100, 100, 5), (100, 250, 5),
                                    (1000, 37, 7), (4064, 188, 7), (8193, 500, 7), (20000, 4, 7), (40000, 937, 7),
-                                   (131040, 188, 7), (70001, 2016, 1), (131073 + 4, 188, 7), (262144 + 5, 300, 7),
+                                   (131040, 188, 7), (4000, 900, 7), (2500, 2000, 5), (4096, 513, 7), (70001, 2016, 1), (131073 + 4, 188, 7), (262144 + 5, 300, 7),
                                    (1048576 + 77, 2016, 7)])
 def test_select_is_bit_exact_on_oracle_scores(P, k, w):
     """Selection alone: same scores in, identical index lists out, ties included."""
