@@ -37,7 +37,11 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
 TC_SOURCES = ("pkv_score_tc.cuh", "pkv_common.cuh")
 # CUDA streams the independent layers of a step are spread over (measured per configuration: the batch-8 ragged
 # shape keeps every SM busy from one stream and gains nothing)
-LAYER_STREAMS = {"llama3_70b_128k": 2, "llama3_8b_32k": 3, "llama2_7b_4k": 4}
+LAYER_STREAMS = {"llama3_70b_128k": 2, "llama3_8b_32k": 4, "llama2_7b_4k": 4, "mistral_7b_ragged": 4}
+# ... and the CTAs each call's persistent score sweeps are capped to (pkv_config.sweep_ctas; 0 = one per SM), so that
+# two layers' sweeps run side by side: on the 32k and batch-8 shapes half the SMs each is 10-15 % faster than
+# full-width sweeps that take turns; the 128k shape gains nothing from it
+SWEEP_CTAS = {"llama3_8b_32k": 74, "mistral_7b_ragged": 74}
 
 NCU_TRAFFIC = {
     # profiles/score_tc_llama3_70b_128k.md: (read + written) bytes / (n * H_kv) key rows, caches flushed by ncu
@@ -271,13 +275,13 @@ def time_other(pkv, streaming, workloads, parallel, name, budget, peak, barrier,
     w = workloads.WORKLOADS[name]
     if budget:
         w = workloads.with_budget(w, budget)
-    cfg = pkv.config_of(w, inputs_final=True)
+    n_streams = LAYER_STREAMS.get(name, 1)
+    cfg = pkv.config_of(w, inputs_final=True, sweep_ctas=SWEEP_CTAS.get(name, 0) if n_streams > 1 else 0)
     lens = w.seq_lens()
     esz = 4 if w.dtype == "fp32" else 2
     layers = [workloads.make_layer(w, l, device="cuda") for l in range(w.num_layers)]
     out = streaming.LayerOutputs(cfg, lens, w.torch_dtype())
     ws = pkv.new_workspace(cfg, len(lens), max(lens))
-    n_streams = LAYER_STREAMS.get(name, 1)
     ls = streaming.LayerStreams(cfg, lens, n_streams) if n_streams > 1 else None
     for _ in range(3):
         streaming.compress_model(cfg, layers, lens, out, ws, layer_streams=ls)
@@ -314,7 +318,7 @@ def time_other(pkv, streaming, workloads, parallel, name, budget, peak, barrier,
     gbs = graded / (ms / steps * 1e-3) / 1e9
     k_layer_mb = sum(lens) * w.num_kv_heads * w.head_dim * esz / 1e6
     return {"workload": w.name, "avg_budget": w.avg_budget, "layers": w.num_layers, "seq_lens": lens, "steps": steps,
-            "cuda_graph": True, "layer_streams": n_streams,
+            "cuda_graph": True, "layer_streams": n_streams, "sweep_ctas": cfg.sweep_ctas,
             "ms_per_step": ms / steps, "value": value, "unit": UNIT,
             "path": {"graded_bytes_per_step": graded, "achieved": gbs, "frac": gbs / peak["hbm_gbs"]},
             "l2": "one layer's K is %.1f MB; %d distinct layers (%.1f GB of K and V) are cycled, so a layer is "
@@ -351,6 +355,9 @@ def main():
                     help="enqueue the (independent) layers round robin on N CUDA streams with a workspace each, so that "
                          "a layer's selection and the tails of its sweeps run beside the next layers' sweeps; default: "
                          "what LAYER_STREAMS names for the workload, else 1")
+    ap.add_argument("--sweep-ctas", type=int, default=None, metavar="N",
+                    help="cap the CTAs of each call's persistent score sweeps (pkv_config.sweep_ctas); default: what "
+                         "SWEEP_CTAS names for the workload when it runs on several streams, else 0 = one per SM")
     ap.add_argument("--mode", default="self", choices=["self", "handoff", "attend"],
                     help="self: the library finds the row normalisers itself (two K sweeps, the graded path); "
                          "handoff: they are handed in as the prefill attention would (one K sweep); attend: the "
@@ -396,7 +403,12 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    cfg = pkv.config_of(w, inputs_final=True)           # every layer's Q and K are resident before the timed region
+    n_streams = args.streams if args.streams is not None else LAYER_STREAMS.get(args.workload, 1)
+    if args.lanes:
+        n_streams = 1
+    sweep_ctas = args.sweep_ctas if args.sweep_ctas is not None else (SWEEP_CTAS.get(args.workload, 0) if n_streams > 1 else 0)
+    # every layer's Q and K are resident before the timed region
+    cfg = pkv.config_of(w, inputs_final=True, sweep_ctas=sweep_ctas)
     lens = w.seq_lens()
     esz = 2 if w.dtype == "bf16" else 4
     tdt = w.torch_dtype()
@@ -417,9 +429,6 @@ def main():
     for _ in range(args.warmup):
         streaming.compress_model(cfg, layers, lens, out, ws)
     pkv.check_status(ws)
-    n_streams = args.streams if args.streams is not None else LAYER_STREAMS.get(args.workload, 1)
-    if args.lanes:
-        n_streams = 1
     ls = streaming.LayerStreams(cfg, lens, n_streams) if n_streams > 1 else None
     run_step = lambda: streaming.compress_model(cfg, layers, lens, out, ws, layer_streams=ls)
     if ls is not None:
@@ -547,7 +556,7 @@ def main():
             "ms_per_step_best": step_best, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
             "config": {"workload": w.name, "mode": args.mode, "cuda_graph": bool(args.graph), "select_lane_sms": args.lanes,
-                       "layer_streams": n_streams, "layers": w.num_layers, "q_heads": w.num_q_heads,
+                       "layer_streams": n_streams, "sweep_ctas": sweep_ctas, "layers": w.num_layers, "q_heads": w.num_q_heads,
                        "kv_heads": w.num_kv_heads, "head_dim": w.head_dim, "batch": w.batch, "seq_lens": lens,
                        "window": w.window, "pool_kernel": w.pool_kernel, "avg_budget": w.avg_budget, "beta": w.beta,
                        "tokens_per_step_per_gpu": tokens, "parallelism": "replicas x%d" % world,

@@ -107,7 +107,10 @@ typedef struct pkv_config {
   int32_t schedule;      /* PKV_SCHEDULE_*: shape of the per-layer budgets; 0 = Eq. 1 */
   double  beta;          /* pyramid shape, >= 1 (Section 4.2.1); 1 = same size in every layer */
   uint32_t flags;        /* PKV_FLAG_* bits, 0 by default */
-  uint32_t reserved;     /* must be 0 */
+  uint32_t sweep_ctas;   /* CTAs the persistent score sweeps of a call launch: 0 = one per SM (default), else at
+                            most this many (<= 1024).  A caller that runs independent layers on several streams
+                            gives each call a share of the SMs this way, so that two layers' sweeps run side by
+                            side instead of one after the other; results do not depend on it beyond rounding. */
 } pkv_config;
 
 typedef struct pkv_tensor {

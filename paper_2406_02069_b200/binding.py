@@ -50,7 +50,7 @@ class PkvConfig(ctypes.Structure):
                 ("window", ctypes.c_int32), ("pool_kernel", ctypes.c_int32),
                 ("pool_kind", ctypes.c_int32), ("dtype", ctypes.c_int32),
                 ("avg_budget", ctypes.c_int32), ("schedule", ctypes.c_int32),
-                ("beta", ctypes.c_double), ("flags", ctypes.c_uint32), ("reserved", ctypes.c_uint32)]
+                ("beta", ctypes.c_double), ("flags", ctypes.c_uint32), ("sweep_ctas", ctypes.c_uint32)]
 
 
 class PkvTensor(ctypes.Structure):
@@ -152,20 +152,21 @@ def strerror(status: int) -> str:
 
 def make_config(*, num_layers: int, num_q_heads: int, num_kv_heads: int, head_dim: int, window: int,
                 pool_kernel: int, dtype: str, avg_budget: int, beta: float = 20.0, pool_kind: int = 0,
-                schedule: str = "linear", inputs_final: bool = False) -> PkvConfig:
+                schedule: str = "linear", inputs_final: bool = False, sweep_ctas: int = 0) -> PkvConfig:
     """inputs_final sets PKV_FLAG_INPUTS_FINAL: nothing still running on the stream writes q_win or k when a call is
-    enqueued, so the score kernels may read them before the kernels ahead of them have finished."""
+    enqueued, so the score kernels may read them before the kernels ahead of them have finished.  sweep_ctas > 0
+    caps the CTAs of the persistent score sweeps (a share of the SMs for callers that run layers on several streams)."""
     code = {"fp32": 0, "bf16": 1, "fp16": 2, torch.float32: 0, torch.bfloat16: 1, torch.float16: 2}[dtype]
     return PkvConfig(num_layers, num_q_heads, num_kv_heads, head_dim, window, pool_kernel, pool_kind, code,
-                     avg_budget, {"linear": 0, "geometric": 1}[schedule], float(beta), 1 if inputs_final else 0, 0)
+                     avg_budget, {"linear": 0, "geometric": 1}[schedule], float(beta), 1 if inputs_final else 0, int(sweep_ctas))
 
 
-def config_of(w, inputs_final: bool = False) -> PkvConfig:
+def config_of(w, inputs_final: bool = False, sweep_ctas: int = 0) -> PkvConfig:
     """Config of a workloads.Workload."""
     return make_config(num_layers=w.num_layers, num_q_heads=w.num_q_heads, num_kv_heads=w.num_kv_heads,
                        head_dim=w.head_dim, window=w.window, pool_kernel=w.pool_kernel, dtype=w.dtype,
                        avg_budget=w.avg_budget, beta=w.beta, pool_kind={"max": 0, "avg": 1}[w.pool_kind],
-                       schedule=getattr(w, "schedule", "linear"), inputs_final=inputs_final)
+                       schedule=getattr(w, "schedule", "linear"), inputs_final=inputs_final, sweep_ctas=sweep_ctas)
 
 
 def _tensor(t: Optional[torch.Tensor]) -> PkvTensor:

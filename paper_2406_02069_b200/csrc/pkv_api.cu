@@ -41,7 +41,7 @@ bool config_ok(const pkv_config* c) {
   if (c->pool_kernel < 1 || (c->pool_kernel % 2) == 0) return false;
   if (!(c->beta >= 1.0) || c->beta > 1.0e6) return false;
   if (c->schedule != PKV_SCHEDULE_LINEAR && c->schedule != PKV_SCHEDULE_GEOMETRIC) return false;
-  if ((c->flags & ~PKV_FLAG_INPUTS_FINAL) != 0 || c->reserved != 0) return false;
+  if ((c->flags & ~PKV_FLAG_INPUTS_FINAL) != 0 || c->sweep_ctas > 1024) return false;
   return true;
 }
 
@@ -356,8 +356,9 @@ int device_sm_count() {
 template <int D>
 int launch_scores_tc(const pkv_config* c, const pkv_tensor& q, const pkv_tensor& k, ScoreParams& sp, int batch,
                      int max_n, uint32_t* status, cudaStream_t st) {
-  const int sms = device_sm_count();
+  int sms = device_sm_count();
   if (sms <= 0) return PKV_ERR_CUDA;
+  if (c->sweep_ctas > 0) sms = std::min(sms, static_cast<int>(c->sweep_ctas));   // the caller's share of the SMs
   static bool attr_done[64] = {};  // the attribute is per device; setting it twice is harmless
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) return PKV_ERR_CUDA;
@@ -569,7 +570,7 @@ int run_attend(const pkv_config* c, const pkv_tensor& q, const pkv_tensor& k, co
   ap.o_partial = w.o_partial;
   ap.out = attn_out;
   ap.status = w.status;
-  const int grid_cap = std::min(sms, kAtMaxGrid);
+  const int grid_cap = std::min(c->sweep_ctas > 0 ? std::min(sms, static_cast<int>(c->sweep_ctas)) : sms, kAtMaxGrid);
   // Key tiles per work item: the largest power of two that still spreads the items evenly over the SMs.
   auto items_for = [&](int ct) {
     long long items = 0;

@@ -78,3 +78,53 @@ def test_a_step_on_several_streams_can_be_captured_in_one_cuda_graph():
     ls.check_status()
     for l in range(w.num_layers):
         assert torch.equal(got.idx[l], ref.idx[l]) and torch.equal(got.k[l], ref.k[l]) and torch.equal(got.v[l], ref.v[l])
+
+
+@pytest.mark.parametrize("sweep_ctas", [1, 37, 74, 1024])
+def test_a_share_of_the_sms_for_the_sweeps_changes_nothing_but_rounding(sweep_ctas):
+    """pkv_config.sweep_ctas caps the CTAs of the persistent score sweeps (a caller's way to let two layers' sweeps run
+    side by side).  Whatever the cap, down to a single CTA that walks every head, the scores stay within the
+    tolerance of the oracle and the kept lists match it; the window-attention call honours the cap too."""
+    import numpy as np
+    import oracle
+    from helpers import assert_indices_match, assert_scores_close, packed_rows
+    w = workloads.scaled(workloads.MISTRAL_RAGGED, name="mistral_sweep_ctas", num_layers=2, batch=3)
+    lens = [300 + (n % 1500) for n in w.seq_lens()]
+    cfg = pkv.config_of(w, sweep_ctas=sweep_ctas)
+    assert cfg.sweep_ctas == sweep_ctas
+    layer = 1
+    kl = pkv.layer_budgets(cfg)[layer]
+    x = workloads.make_layer(w, layer, device=DEV, seq_lens=lens)
+    ws = pkv.new_workspace(cfg, len(lens), max(lens), DEV)
+    rows = pkv.total_rows(cfg, kl, lens)
+    k_out = torch.empty(rows, w.head_dim, dtype=x.k.dtype, device=DEV)
+    v_out = torch.empty_like(k_out)
+    idx = torch.empty(rows, dtype=torch.int32, device=DEV)
+    scores = torch.zeros(len(lens), w.num_kv_heads, max(lens), dtype=torch.float32, device=DEV)
+    pkv.compress_layer(cfg, layer, x.q_win, x.k, x.v, lens, k_out, v_out, idx, ws, scores=scores)
+    pkv.check_status(ws)
+    ref = oracle.compress_batch(x.q_win.cpu(), x.k.cpu(), x.v.cpu(), lens, pool_kernel=w.pool_kernel,
+                                avg_budget=w.avg_budget, k_layer=kl)
+    got_scores, got_idx = scores.cpu().numpy(), idx.cpu().numpy()
+    for b, n in enumerate(lens):
+        assert_scores_close(got_scores[b, :, : n - w.window], ref["scores"][b], "seq %d" % b)
+    for b, h, sl in packed_rows(ref["counts"], w.num_kv_heads):
+        assert_indices_match(got_idx[sl], ref["indices"][sl], ref["scores"][b][h], w.pool_kernel, w.window,
+                             "b %d h %d" % (b, h))
+    # the fused attention call under the same cap
+    out = torch.empty(len(lens), w.num_q_heads, w.window, w.head_dim, dtype=torch.float32, device=DEV)
+    scores2 = torch.zeros_like(scores)
+    pkv.attend_window(cfg, x.q_win, x.k, x.v, lens, out, scores2, ws)
+    pkv.check_status(ws)
+    got2 = scores2.cpu().numpy()
+    for b, n in enumerate(lens):
+        assert_scores_close(got2[b, :, : n - w.window], ref["scores"][b], "attend seq %d" % b)
+    assert np.isfinite(out.cpu().numpy()).all()
+
+
+def test_a_cap_above_the_limit_is_refused():
+    w = workloads.scaled(workloads.LLAMA3_8B, name="cap", num_layers=1, seq_len=500)
+    cfg = pkv.config_of(w, sweep_ctas=1025)
+    with pytest.raises(pkv.PkvError) as err:
+        pkv.layer_budgets(cfg)
+    assert err.value.status == 1      # PKV_ERR_INVALID_ARG
