@@ -68,20 +68,6 @@ struct AtParams {
   uint32_t* status;
 };
 
-// Shared-memory matrix descriptor of a 16-bit operand stored M/N-major (the 64 elements that are contiguous run
-// along M or N, one 128-byte line per contraction index, 128-byte swizzle): groups of 8 contraction indices are
-// 1024 bytes apart, blocks of 64 elements along M/N `block_bytes` apart.  `addr` advances by 2048 bytes per
-// 16-step of the contraction.
-__device__ __forceinline__ uint64_t smem_desc_mn_sw128(uint32_t addr, uint32_t block_bytes) {
-  uint64_t d = 0;
-  d |= static_cast<uint64_t>((addr & 0x3FFFFu) >> 4);
-  d |= static_cast<uint64_t>(block_bytes >> 4) << 16;
-  d |= static_cast<uint64_t>(1024 >> 4) << 32;
-  d |= static_cast<uint64_t>(1) << 46;
-  d |= static_cast<uint64_t>(2) << 61;
-  return d;
-}
-
 // The MMA issuer is one thread and this kernel issues 24 MMAs per K tile, so the descriptors are split into their
 // 32-bit halves: the high half (strides, version, swizzle) is a constant, the low half (start address and leading
 // offset) is formed once per product and advanced by a compile-time constant per MMA.  (Measured: an MMA still takes
